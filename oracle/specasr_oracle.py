@@ -1,0 +1,328 @@
+"""CPU fp64 oracle for the target decoder's tree-verification step.  TEST INFRASTRUCTURE ONLY.
+
+This is a plain, slow restatement of what one verification round computes
+(Section II-B: the target model checks every draft token at once, stops at the
+first token that fails, and the output is identical to non-speculative greedy
+decoding; Section II-B / Fig. 13 and Section IV-C: a draft token *tree* is
+verified in one pass with a 2-D attention mask so that every branch gets its own
+outcome).  It exists so that the CUDA path can be compared against it; only the
+tests, the smoke check and the benchmark's CPU-baseline leg may import it.  It
+shares no code with the CUDA path and never calls it.
+
+The paper has no equations for this step, so the definition used is the plain
+one the method must reproduce exactly:
+
+    logits[i] = Decoder(prefix ++ tokens on the root->i path)[-1]   (ordinary causal attention)
+    argmax[i] = lowest-id maximiser of logits[i]
+    node i != root matches   iff tokens[i] == argmax[parent[i]]
+    node i is accepted       iff every non-root node on its root path matches
+    result                   = deepest accepted node (lowest index among equals), its path,
+                               accept_len = its depth, bonus = its argmax
+
+`causal_forward` is that definition written out with no cache and no tree mask;
+`verify_tree` is the cached, tree-masked form and is trusted only because the
+tests show it equals the former node by node.
+
+Readings taken where the paper is silent (all from the workload description,
+none from the paper): pre-norm Llama block, RMSNorm eps 1e-6 with a learned
+gain, rotate-half RoPE (pairs (k, k + dh/2), theta_k = base^(-2k/dh)), SwiGLU,
+GQA with q-head h reading kv-head h // (Hq/Hkv), score scale 1/sqrt(dh), no
+biases, untied LM head; audio-embedding vectors enter layer 0 directly at
+positions 0..Ta-1 and are followed by text tokens; node 0 of a tree is the last
+committed token (never verified); tree node i sits at position L + depth[i];
+argmax ties go to the lowest token id.
+
+Parity pins (tests/test_oracle_*.py): an independent library decoder
+(transformers' Llama in fp64 with the same tensors) for the block wiring, RoPE
+pairing and GQA grouping; torch's scaled_dot_product_attention for the masked
+attention; closed forms for RMSNorm / softmax / SiLU / RoPE; brute force over
+root paths for the tree forward and for the accept rule; a plain prefill of the
+accepted path for the commit.  The paper prints no worked numbers for this step,
+so parity with numbers *in the paper* is unpinned; only its lossless property
+binds, and the tests check it.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+F64 = np.float64
+
+
+# --------------------------------------------------------------------------- storage widening
+
+def widen(a: np.ndarray) -> np.ndarray:
+    """uint16 arrays are bf16 bit patterns; everything is widened to fp64."""
+    a = np.asarray(a)
+    if a.dtype == np.uint16:
+        return (a.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(F64)
+    return a.astype(F64)
+
+
+class Weights:
+    """Adapter over any store with .layer(l) / .globals() -> dict of arrays.  Widens on access, one
+    layer at a time, so that a 7B-shape model never sits in memory in fp64."""
+
+    def __init__(self, store, cache_layers: bool = False):
+        self.store = store
+        self._cache = {} if cache_layers else None
+        self._globals = None
+
+    def layer(self, l: int) -> dict:
+        if self._cache is not None and l in self._cache:
+            return self._cache[l]
+        w = {k: widen(v) for k, v in self.store.layer(l).items()}
+        if self._cache is not None:
+            self._cache[l] = w
+        return w
+
+    def globals(self) -> dict:
+        if self._globals is None:
+            self._globals = {k: widen(v) for k, v in self.store.globals().items()}
+        return self._globals
+
+
+# --------------------------------------------------------------------------- elementwise pieces
+
+def rmsnorm(x: np.ndarray, g: np.ndarray, eps: float) -> np.ndarray:
+    """x / sqrt(mean(x^2) + eps) * g over the last axis."""
+    ms = np.mean(x * x, axis=-1, keepdims=True)
+    return x / np.sqrt(ms + eps) * g
+
+
+def silu(x: np.ndarray) -> np.ndarray:
+    return x / (1.0 + np.exp(-x))
+
+
+def rope(x: np.ndarray, pos: np.ndarray, base: float) -> np.ndarray:
+    """Rotate-half rotary embedding.  x: [T, H, dh]; pos: [T] integer positions."""
+    dh = x.shape[-1]
+    half = dh // 2
+    theta = base ** (-2.0 * np.arange(half, dtype=F64) / dh)
+    ang = np.asarray(pos, dtype=F64)[:, None] * theta[None, :]          # [T, half]
+    c = np.cos(ang)[:, None, :]
+    s = np.sin(ang)[:, None, :]
+    x1, x2 = x[..., :half], x[..., half:]
+    return np.concatenate([x1 * c - x2 * s, x2 * c + x1 * s], axis=-1)
+
+
+def masked_softmax(scores: np.ndarray, mask: np.ndarray) -> np.ndarray:
+    """Row softmax over the entries where mask is True (each row has at least one)."""
+    s = np.where(mask, scores, -np.inf)
+    s = s - np.max(s, axis=-1, keepdims=True)
+    e = np.exp(s)
+    return e / np.sum(e, axis=-1, keepdims=True)
+
+
+def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, mask: np.ndarray) -> np.ndarray:
+    """q: [T, Hq, dh]; k, v: [S, Hkv, dh]; mask: [T, S] bool (True = visible).  Returns [T, Hq, dh]."""
+    T, Hq, dh = q.shape
+    Hkv = k.shape[1]
+    group = Hq // Hkv
+    out = np.empty_like(q)
+    for h in range(Hq):
+        kv = h // group
+        scores = (q[:, h, :] @ k[:, kv, :].T) / np.sqrt(F64(dh))
+        out[:, h, :] = masked_softmax(scores, mask) @ v[:, kv, :]
+    return out
+
+
+# --------------------------------------------------------------------------- KV cache
+
+class KVCache:
+    """Per layer K and V of every committed position: lists of [L, Hkv, dh] fp64 arrays."""
+
+    def __init__(self, cfg):
+        self.cfg = cfg
+        self.K = [np.zeros((0, cfg.n_kv_heads, cfg.head_dim), F64) for _ in range(cfg.n_layers)]
+        self.V = [np.zeros((0, cfg.n_kv_heads, cfg.head_dim), F64) for _ in range(cfg.n_layers)]
+
+    @property
+    def length(self) -> int:
+        return self.K[0].shape[0]
+
+    def copy(self) -> "KVCache":
+        c = KVCache(self.cfg)
+        c.K = [a.copy() for a in self.K]
+        c.V = [a.copy() for a in self.V]
+        return c
+
+    def append(self, new_k, new_v):
+        for l in range(self.cfg.n_layers):
+            self.K[l] = np.concatenate([self.K[l], new_k[l]], axis=0)
+            self.V[l] = np.concatenate([self.V[l], new_v[l]], axis=0)
+
+
+# --------------------------------------------------------------------------- the decoder
+
+def embed(weights: Weights, tokens) -> np.ndarray:
+    return weights.globals()["embed"][np.asarray(tokens, dtype=np.int64)]
+
+
+def decoder_stack(cfg, weights: Weights, x: np.ndarray, pos: np.ndarray, mask_new: np.ndarray,
+                  cache: KVCache | None):
+    """Run all layers over T new rows.
+
+    x: [T, d] layer-0 inputs; pos: [T] positions; mask_new: [T, T] visibility among the new rows;
+    every cached position is visible to every new row.  Returns (final hidden [T, d] before the
+    final norm, list of new K per layer, list of new V per layer).
+    """
+    T = x.shape[0]
+    L = cache.length if cache is not None else 0
+    full_mask = np.concatenate([np.ones((T, L), dtype=bool), mask_new.astype(bool)], axis=1)
+    new_k, new_v = [], []
+    x = x.astype(F64)
+    for l in range(cfg.n_layers):
+        w = weights.layer(l)
+        h = rmsnorm(x, w["g_attn"], cfg.eps)
+        q = (h @ w["wq"].T).reshape(T, cfg.n_heads, cfg.head_dim)
+        k = (h @ w["wk"].T).reshape(T, cfg.n_kv_heads, cfg.head_dim)
+        v = (h @ w["wv"].T).reshape(T, cfg.n_kv_heads, cfg.head_dim)
+        q = rope(q, pos, cfg.rope_base)
+        k = rope(k, pos, cfg.rope_base)
+        new_k.append(k)
+        new_v.append(v)
+        if cache is not None:
+            k_all = np.concatenate([cache.K[l], k], axis=0)
+            v_all = np.concatenate([cache.V[l], v], axis=0)
+        else:
+            k_all, v_all = k, v
+        a = attention(q, k_all, v_all, full_mask).reshape(T, cfg.q_dim)
+        x = x + a @ w["wo"].T
+        h = rmsnorm(x, w["g_ffn"], cfg.eps)
+        x = x + (silu(h @ w["wg"].T) * (h @ w["wu"].T)) @ w["wd"].T
+    return x, new_k, new_v
+
+
+def lm_logits(cfg, weights: Weights, hidden: np.ndarray) -> np.ndarray:
+    g = weights.globals()
+    return rmsnorm(hidden, g["g_final"], cfg.eps) @ g["lm_head"].T
+
+
+def causal_forward(cfg, weights: Weights, inputs: np.ndarray) -> np.ndarray:
+    """The plain definition: ordinary causal decoder over a whole sequence of layer-0 input
+    vectors, no cache.  Returns logits [T, V]."""
+    T = inputs.shape[0]
+    mask = np.tril(np.ones((T, T), dtype=bool))
+    hidden, _, _ = decoder_stack(cfg, weights, inputs, np.arange(T), mask, None)
+    return lm_logits(cfg, weights, hidden)
+
+
+def prefill(cfg, weights: Weights, cache: KVCache, inputs: np.ndarray, want_logits: bool = False):
+    """Append T positions (audio vectors or embedded tokens) to the cache under causal attention."""
+    T = inputs.shape[0]
+    mask = np.tril(np.ones((T, T), dtype=bool))
+    pos = cache.length + np.arange(T)
+    hidden, nk, nv = decoder_stack(cfg, weights, inputs, pos, mask, cache)
+    cache.append(nk, nv)
+    if want_logits:
+        return lm_logits(cfg, weights, hidden)
+    return None
+
+
+# --------------------------------------------------------------------------- tree side
+
+class TreeError(ValueError):
+    pass
+
+
+def tree_prep(parent) -> tuple[np.ndarray, np.ndarray]:
+    """depth[n] (root = 0) and anc[n, n] with anc[i, j] = True iff j is i or an ancestor of i.
+    This matrix is the 2-D attention mask of a draft token tree (Fig. 13)."""
+    parent = np.asarray(parent, dtype=np.int64)
+    n = len(parent)
+    if n < 1 or parent[0] != -1:
+        raise TreeError("node 0 must be the root with parent -1")
+    depth = np.zeros(n, dtype=np.int64)
+    anc = np.zeros((n, n), dtype=bool)
+    anc[0, 0] = True
+    for i in range(1, n):
+        p = parent[i]
+        if p < 0 or p >= i:
+            raise TreeError(f"parent[{i}] = {p} must satisfy 0 <= parent < index")
+        depth[i] = depth[p] + 1
+        anc[i] = anc[p]
+        anc[i, i] = True
+    return depth, anc
+
+
+def top2_gap(logits: np.ndarray) -> np.ndarray:
+    part = np.partition(logits, -2, axis=-1)
+    return part[..., -1] - part[..., -2]
+
+
+def accept(tokens, parent, argmax) -> dict:
+    """Greedy acceptance: follow draft tokens while they equal the target's own next token and stop
+    at the first that does not (Section II-B), independently on every branch."""
+    tokens = np.asarray(tokens)
+    parent = np.asarray(parent, dtype=np.int64)
+    depth, _ = tree_prep(parent)
+    n = len(parent)
+    ok = np.zeros(n, dtype=bool)
+    ok[0] = True
+    for i in range(1, n):
+        ok[i] = ok[parent[i]] and (tokens[i] == argmax[parent[i]])
+    best = 0
+    for i in range(1, n):
+        if ok[i] and depth[i] > depth[best]:
+            best = i
+    path = []
+    j = best
+    while j >= 0:
+        path.append(j)
+        j = parent[j]
+    path = path[::-1]
+    return {
+        "accept_len": int(depth[best]),
+        "best": int(best),
+        "path": np.asarray(path, dtype=np.int32),
+        "bonus": int(argmax[best]),
+        "accepted_mask": ok,
+    }
+
+
+def verify_tree(cfg, weights: Weights, cache: KVCache, tokens, parent, decisive_gap: float = 1e-2) -> dict:
+    """One verification round over a draft token tree on top of `cache` (which is not modified)."""
+    tokens = np.asarray(tokens, dtype=np.int64)
+    depth, anc = tree_prep(parent)
+    if np.any(tokens < 0) or np.any(tokens >= cfg.vocab):
+        raise TreeError("token id out of range")
+    pos = cache.length + depth
+    hidden, tk, tv = decoder_stack(cfg, weights, embed(weights, tokens), pos, anc, cache)
+    logits = lm_logits(cfg, weights, hidden)
+    argmax = np.argmax(logits, axis=-1).astype(np.int32)
+    gap = top2_gap(logits)
+    res = accept(tokens, parent, argmax)
+    is_parent = np.zeros(len(tokens), dtype=bool)
+    is_parent[np.asarray(parent)[1:]] = True
+    consulted = is_parent.copy()
+    consulted[res["best"]] = True
+    res.update({
+        "logits": logits, "argmax": argmax, "gap": gap, "depth": depth, "pos": pos,
+        "tree_K": tk, "tree_V": tv,
+        # the accept result is unambiguous when every argmax it reads is decided by a clear margin
+        "decisive": bool(np.all(gap[consulted] > decisive_gap)),
+    })
+    return res
+
+
+def commit(cache: KVCache, result: dict) -> list[tuple[int, int]]:
+    """Keep the accepted path: cache slot L + j receives tree node path[j].  Returns the
+    (source slot, destination slot) pairs, slots counted from the start of the cache."""
+    L = cache.length
+    path = result["path"]
+    moves = [(L + int(p), L + j) for j, p in enumerate(path)]
+    cache.append([k[path] for k in result["tree_K"]], [v[path] for v in result["tree_V"]])
+    return moves
+
+
+def greedy_continuation(cfg, weights: Weights, cache: KVCache, root_token: int, k: int) -> list[int]:
+    """Ordinary autoregressive greedy decoding: feed root_token, then each emitted token, k times.
+    `cache` is left untouched."""
+    c = cache.copy()
+    out = []
+    tok = int(root_token)
+    for _ in range(k):
+        logits = prefill(cfg, weights, c, embed(weights, [tok]), want_logits=True)
+        tok = int(np.argmax(logits[-1]))
+        out.append(tok)
+    return out

@@ -1,0 +1,58 @@
+import numpy as np
+import torch
+
+import gen
+
+
+def test_bf16_rounding_matches_library_rne():
+    rng = np.random.default_rng(1)
+    x = np.concatenate([rng.standard_normal(4096).astype(np.float32) * 0.02,
+                        np.array([0.0, -0.0, 1.0, 1.00390625, 1.01171875, 3.0e38, 1e-40], np.float32)])
+    bits = gen.f32_to_bf16_bits(x)
+    ref = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(bits, ref)
+    back = gen.bf16_bits_to_f32(bits)
+    assert np.array_equal(back, torch.from_numpy(x).to(torch.bfloat16).float().numpy())
+
+
+def test_weights_are_reproducible_and_random_access():
+    cfg = gen.get_config("micro")
+    a = gen.WeightStore(cfg, 3)
+    b = gen.WeightStore(cfg, 3)
+    assert np.array_equal(a.tensor(1, "wd"), b.layer(1)["wd"])
+    assert not np.array_equal(a.tensor(0, "wq"), a.tensor(1, "wq"))
+    assert not np.array_equal(a.tensor(0, "wq"), gen.WeightStore(cfg, 4).tensor(0, "wq"))
+    w = gen.bf16_bits_to_f32(a.tensor(0, "wg"))
+    assert w.shape == (cfg.ffn, cfg.d_model)
+    assert abs(w.std() - 0.02) < 2e-3
+    g = a.tensor(0, "g_attn")
+    assert g.dtype == np.float32 and abs(g.mean() - 1.0) < 0.01
+    seen = {}
+    a.map_tensors(lambda l, n, arr: seen.__setitem__((l, n), arr.shape), a.all_keys(), threads=3)
+    assert len(seen) == 3 + 9 * cfg.n_layers
+
+
+def test_tree_generators():
+    p = gen.sparse_tree(64, seed=0, levels=12)
+    assert len(p) == 64 and p[0] == -1 and all(0 <= p[i] < i for i in range(1, 64))
+    assert list(p[1:5]) == [0, 0, 0, 0] and list(p[5:13]) == [1, 1, 2, 2, 3, 3, 4, 4]
+    depth = np.zeros(64, int)
+    for i in range(1, 64):
+        depth[i] = depth[p[i]] + 1
+    assert depth.max() == 11                       # 12 levels counting the root
+    mp = gen.main_path(p)
+    assert len(mp) == 12 and list(depth[mp]) == list(range(12))
+    for n in (16, 256):
+        q = gen.sparse_tree(n, seed=1)
+        assert len(q) == n and all(0 <= q[i] < i for i in range(1, n))
+    assert list(gen.chain_tree(3)) == [-1, 0, 1, 2]
+    assert list(gen.complete_binary_tree(7)) == [-1, 0, 0, 1, 1, 2, 2]
+    toks = gen.fill_tree_tokens(p, 50, seed=2, root_token=7, main_tokens=list(range(100, 111)), corrupt_p=0.0)
+    assert toks[0] == 7 and list(toks[mp[1:]]) == list(range(100, 111))
+    for i in range(64):
+        kids = [int(toks[j]) for j in range(1, 64) if p[j] == i]
+        assert len(kids) == len(set(kids))
+    p2, t2, old = gen.relabel_tree(p, toks, seed=5)
+    assert all(0 <= p2[i] < i for i in range(1, 64)) and sorted(old) == list(range(64))
+    for new in range(1, 64):
+        assert old[p2[new]] == p[old[new]] and t2[new] == toks[old[new]]

@@ -1,0 +1,134 @@
+"""Pins of the oracle's building blocks against things other than itself: closed forms,
+library routines, and an independent library decoder."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import gen
+from oracle import specasr_oracle as O
+from helpers import oracle_weights
+
+
+def test_widen_reads_bf16_bits():
+    x = np.array([1.0, -2.5, 0.0, 0.00390625], np.float32)
+    assert np.array_equal(O.widen(gen.f32_to_bf16_bits(x)), x.astype(np.float64))
+    # 0x3F80 is 1.0, 0xC000 is -2.0 in bf16
+    assert list(O.widen(np.array([0x3F80, 0xC000], np.uint16))) == [1.0, -2.0]
+
+
+def test_rmsnorm_closed_forms():
+    # constant row c: mean square c^2, so output = c / sqrt(c^2 + eps) * g
+    g = np.array([1.0, 2.0, -1.0, 0.5])
+    y = O.rmsnorm(np.full((1, 4), 3.0), g, 1e-6)
+    assert np.allclose(y[0], 3.0 / math.sqrt(9.0 + 1e-6) * g, rtol=0, atol=1e-15)
+    # (3,4,0,0): mean square 6.25 -> rms 2.5
+    y = O.rmsnorm(np.array([[3.0, 4.0, 0.0, 0.0]]), np.ones(4), 0.0)
+    assert np.allclose(y[0], [1.2, 1.6, 0.0, 0.0])
+    # eps matters for a zero row (no division by zero) and scale invariance holds without it
+    assert np.all(O.rmsnorm(np.zeros((1, 4)), np.ones(4), 1e-6) == 0.0)
+    x = np.random.default_rng(0).standard_normal((3, 16))
+    assert np.allclose(O.rmsnorm(x, g=np.ones(16), eps=0.0), O.rmsnorm(7.0 * x, np.ones(16), 0.0))
+    ref = torch.nn.functional.rms_norm(torch.from_numpy(x), (16,), eps=1e-6).numpy()
+    assert np.allclose(O.rmsnorm(x, np.ones(16), 1e-6), ref, atol=1e-14)
+
+
+def test_silu_and_softmax_closed_forms():
+    assert O.silu(np.array([0.0]))[0] == 0.0
+    assert np.allclose(O.silu(np.array([1.0, -1.0])), [1 / (1 + math.exp(-1)), -1 / (1 + math.e)])
+    x = np.linspace(-5, 5, 11)
+    assert np.allclose(O.silu(x), torch.nn.functional.silu(torch.from_numpy(x)).numpy(), atol=1e-15)
+    s = np.array([[0.0, math.log(2.0), math.log(5.0), 100.0]])
+    m = np.array([[True, True, True, False]])
+    p = O.masked_softmax(s, m)
+    assert np.allclose(p, [[1 / 8, 2 / 8, 5 / 8, 0.0]])
+    assert np.allclose(O.masked_softmax(s + 1234.5, m), p)          # shift invariance
+    assert np.allclose(O.masked_softmax(np.random.default_rng(0).standard_normal((5, 9)),
+                                        np.ones((5, 9), bool)).sum(-1), 1.0)
+
+
+def test_rope_closed_forms():
+    rng = np.random.default_rng(0)
+    dh, base = 8, 1e4
+    x = rng.standard_normal((1, 1, dh))
+    assert np.array_equal(O.rope(x, np.array([0]), base), x)                      # position 0 = identity
+    # pair (k, k + dh/2) is rotated by angle pos * base^(-2k/dh): check one pair by hand
+    pos, k = 3, 1
+    ang = pos * base ** (-2.0 * k / dh)
+    y = O.rope(x, np.array([pos]), base)[0, 0]
+    assert np.isclose(y[k], x[0, 0, k] * math.cos(ang) - x[0, 0, k + dh // 2] * math.sin(ang))
+    assert np.isclose(y[k + dh // 2], x[0, 0, k + dh // 2] * math.cos(ang) + x[0, 0, k] * math.sin(ang))
+    # pair 0 turns by exactly `pos` radians
+    y0 = O.rope(np.array([[[1.0, 0, 0, 0, 0.0, 0, 0, 0]]]), np.array([2]), base)[0, 0]
+    assert np.isclose(y0[0], math.cos(2.0)) and np.isclose(y0[4], math.sin(2.0))
+    # norms preserved; inner products depend on the position difference only
+    q = rng.standard_normal((1, 2, dh))
+    kk = rng.standard_normal((1, 2, dh))
+    assert np.isclose(np.linalg.norm(O.rope(q, np.array([17]), base)), np.linalg.norm(q))
+    d1 = np.sum(O.rope(q, np.array([9]), base) * O.rope(kk, np.array([4]), base))
+    d2 = np.sum(O.rope(q, np.array([1005]), base) * O.rope(kk, np.array([1000]), base))
+    assert np.isclose(d1, d2, atol=1e-11)
+
+
+@pytest.mark.parametrize("hq,hkv", [(4, 4), (4, 2), (8, 2)])
+def test_attention_matches_library_sdpa(hq, hkv):
+    rng = np.random.default_rng(hq * 10 + hkv)
+    T, S, dh = 5, 11, 16
+    q = rng.standard_normal((T, hq, dh))
+    k = rng.standard_normal((S, hkv, dh))
+    v = rng.standard_normal((S, hkv, dh))
+    mask = rng.random((T, S)) < 0.6
+    mask[:, 0] = True
+    out = O.attention(q, k, v, mask)
+    rep = hq // hkv
+    tq = torch.from_numpy(q).permute(1, 0, 2)[None]
+    tk = torch.from_numpy(k).permute(1, 0, 2).repeat_interleave(rep, dim=0)[None]
+    tv = torch.from_numpy(v).permute(1, 0, 2).repeat_interleave(rep, dim=0)[None]
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, attn_mask=torch.from_numpy(mask)[None, None])
+    assert np.allclose(out, ref[0].permute(1, 0, 2).numpy(), atol=1e-13)
+
+
+def _hf_model(cfg, W):
+    from transformers import LlamaConfig, LlamaForCausalLM
+    hc = LlamaConfig(vocab_size=cfg.vocab, hidden_size=cfg.d_model, intermediate_size=cfg.ffn,
+                     num_hidden_layers=cfg.n_layers, num_attention_heads=cfg.n_heads,
+                     num_key_value_heads=cfg.n_kv_heads, head_dim=cfg.head_dim, rms_norm_eps=cfg.eps,
+                     rope_theta=cfg.rope_base, attention_bias=False, mlp_bias=False,
+                     tie_word_embeddings=False, max_position_embeddings=4096)
+    model = LlamaForCausalLM(hc).double().eval()
+    g = W.globals()
+    sd = {"model.embed_tokens.weight": g["embed"], "lm_head.weight": g["lm_head"], "model.norm.weight": g["g_final"]}
+    names = {"wq": "self_attn.q_proj", "wk": "self_attn.k_proj", "wv": "self_attn.v_proj", "wo": "self_attn.o_proj",
+             "wg": "mlp.gate_proj", "wu": "mlp.up_proj", "wd": "mlp.down_proj",
+             "g_attn": "input_layernorm", "g_ffn": "post_attention_layernorm"}
+    for l in range(cfg.n_layers):
+        w = W.layer(l)
+        for k, v in names.items():
+            sd[f"model.layers.{l}.{v}.weight"] = w[k]
+    model.load_state_dict({k: torch.from_numpy(np.ascontiguousarray(v)) for k, v in sd.items()}, strict=True)
+    return model
+
+
+@pytest.mark.parametrize("name", ["micro", "tiny"])
+def test_causal_forward_matches_library_llama(name):
+    """Block wiring, RoPE pairing, GQA grouping, SwiGLU, norms, audio vectors as inputs_embeds:
+    an independent implementation fed the same tensors must give the same logits.  (The library
+    builds its rotary table in fp32, hence 1e-6 rather than 1e-12.)"""
+    pytest.importorskip("transformers")
+    cfg = gen.get_config(name)
+    W = oracle_weights(cfg, seed=1)
+    model = _hf_model(cfg, W)
+    audio = gen.audio_prefix(12, cfg.d_model, 1).astype(np.float64)
+    toks = gen.prompt_tokens(9, cfg.vocab, 1)
+    x = np.concatenate([audio, O.embed(W, toks)], axis=0)
+    ours = O.causal_forward(cfg, W, x)
+    with torch.no_grad():
+        ref = model(inputs_embeds=torch.from_numpy(x)[None]).logits[0].numpy()
+    assert np.abs(ours - ref).max() < 1e-6
+    assert np.array_equal(ours.argmax(-1), ref.argmax(-1))
+    # pure-token input goes through the embedding table on both sides
+    ours_t = O.causal_forward(cfg, W, O.embed(W, toks))
+    with torch.no_grad():
+        ref_t = model(input_ids=torch.from_numpy(toks.astype(np.int64))[None]).logits[0].numpy()
+    assert np.abs(ours_t - ref_t).max() < 1e-6
