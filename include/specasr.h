@@ -1,0 +1,178 @@
+/*
+ * specasr.h -- C ABI of the B200 tree-verification library.
+ *
+ * One verification round of speculative decoding for an LLM-based speech recogniser: the target
+ * decoder runs ONE forward pass over a draft token tree on top of a KV cache that already holds the
+ * audio-embedding prefix and the text decoded so far, the longest draft path whose tokens equal the
+ * target's own greedy tokens is selected, and the accepted nodes' K/V are compacted into contiguous
+ * cache slots.  (Draft-then-verify and its lossless property: paper Section II-B; verification of a
+ * token tree in one pass with a 2-D attention mask: Section II-B, Fig. 13, and Section IV-C.)
+ *
+ * Conventions
+ *  - Plain C.  No C++ exception crosses this boundary.  Every call returns a specasr_status;
+ *    specasr_last_error() gives a thread-local message for the last failure on this thread.
+ *  - Pointers marked [device] must be device-accessible on the CUDA device that was current when the
+ *    model was created; pointers marked [host] are ordinary host memory.  `stream` is a cudaStream_t
+ *    passed as void* (NULL = the legacy default stream).
+ *  - Ownership: the caller owns every device buffer (weights, KV pools, page table, workspace,
+ *    inputs, outputs).  Handles borrow them and never free them.  The library itself only allocates
+ *    the rotary table (device, once per model) and a few bytes of pinned host memory per KV handle.
+ *  - Calls are asynchronous on `stream`; outputs are valid once the stream reaches that point.
+ *  - Errors that the host can see (null pointer, n out of range, no pending verify, ...) are returned
+ *    before anything is enqueued and leave all state untouched.  Errors only the device can see
+ *    (malformed parent array, token id out of range, cache capacity exceeded with a length the host
+ *    does not know yet, a bounded wait that ran out) set the device status word: the remaining
+ *    kernels of that call do nothing, out_accept_len receives -1, and specasr_poll_status reports
+ *    the code.  Nothing traps, asserts or spins without a limit.
+ *
+ * Tree format: tokens[n] and parent_idx[n] with parent_idx[0] = -1 and 0 <= parent_idx[i] < i.
+ * Node 0 is the root: the last committed token, whose K/V is not in the cache yet; it is not
+ * verified.  Nodes 1..n-1 are draft tokens.  1 <= n <= SPECASR_MAX_NODES.
+ */
+#ifndef SPECASR_H_
+#define SPECASR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SPECASR_MAX_NODES 256
+
+typedef enum specasr_status {
+  SPECASR_OK = 0,
+  SPECASR_ERR_INVALID_ARG = 1,
+  SPECASR_ERR_INVALID_TREE = 2,
+  SPECASR_ERR_KV_CAPACITY = 3,
+  SPECASR_ERR_STATE = 4,
+  SPECASR_ERR_UNSUPPORTED = 5,
+  SPECASR_ERR_TIMEOUT = 6,
+  SPECASR_ERR_CUDA = 7
+} specasr_status;
+
+/* Decoder shape (pre-norm Llama block: RMSNorm, rotary GQA attention, SwiGLU; no biases). */
+typedef struct specasr_model_config {
+  int32_t n_layers;
+  int32_t d_model;
+  int32_t n_heads;      /* query heads */
+  int32_t n_kv_heads;   /* key/value heads; n_heads % n_kv_heads == 0 */
+  int32_t head_dim;     /* 32, 64 or 128 */
+  int32_t ffn;          /* SwiGLU inner width */
+  int32_t vocab;
+  int32_t page_size;    /* tokens per KV page; a multiple of 8 (16 in the reference workload) */
+  int32_t max_positions;/* length of the rotary table = largest position + 1 */
+  float rms_eps;
+  float rope_base;
+  int32_t gemm_path;    /* 0 = tcgen05 tensor-core projections (product path);
+                           1 = plain FMA projections, kept for cross-checking kernels on a GPU */
+  int32_t reserved[3];
+} specasr_model_config;
+
+/*
+ * Weights, all [device], all borrowed.  Matrices are bf16, row-major [out_features, in_features]
+ * with rows 16-byte aligned (in_features % 8 == 0).  Gains are fp32.
+ *   wqkv[l] : [(n_heads + 2 n_kv_heads) * head_dim, d_model]  rows = all Q heads, all K heads, all V heads
+ *   wo[l]   : [d_model, n_heads * head_dim]
+ *   wgu[l]  : [2 * ffn, d_model]   row 2f = gate row f, row 2f+1 = up row f (interleaved so that one
+ *             output tile holds both halves of a SwiGLU feature)
+ *   wd[l]   : [d_model, ffn]
+ * The per-layer arrays are [host] arrays of n_layers device pointers (copied at create time).
+ */
+typedef struct specasr_weight_ptrs {
+  const void* embed;            /* [vocab, d_model] bf16 */
+  const void* lm_head;          /* [vocab, d_model] bf16 */
+  const float* g_final;         /* [d_model] */
+  const void* const* wqkv;
+  const void* const* wo;
+  const void* const* wgu;
+  const void* const* wd;
+  const float* const* g_attn;
+  const float* const* g_ffn;
+} specasr_weight_ptrs;
+
+typedef struct specasr_model specasr_model;
+typedef struct specasr_kv specasr_kv;
+
+/* Creates a model handle on the current CUDA device.  Fails with SPECASR_ERR_UNSUPPORTED for shapes
+ * the kernels do not cover (head_dim not in {32,64,128}, d_model or ffn not a multiple of 8, ...). */
+specasr_status specasr_model_create(const specasr_model_config* cfg, const specasr_weight_ptrs* w,
+                                    specasr_model** out);
+void specasr_model_destroy(specasr_model* m);
+
+/* Bytes of [device] workspace a KV handle needs to verify trees of up to max_nodes nodes. */
+size_t specasr_workspace_bytes(const specasr_model* m, int32_t max_nodes);
+
+/* Bytes of ONE of the two KV pools (K and V have the same size) for n_pages pages.
+ * Pool layout: [n_layers][n_pages][n_kv_heads][2 planes][page_size][head_dim] bf16; plane 0 is the
+ * bf16 rounding of the value, plane 1 the bf16 rounding of the remainder (value ~ hi + lo). */
+size_t specasr_kv_pool_bytes(const specasr_model* m, int32_t n_pages);
+
+/*
+ * KV handle over caller-owned pools.  page_table [device] int32[max_pages] maps logical page ->
+ * physical page (< n_pages); slot s lives in page_table[s / page_size] at offset s % page_size.
+ * The capacity is max_pages * page_size slots.  The handle starts empty (length 0).
+ * `workspace` [device] of specasr_workspace_bytes(m, max_nodes) bytes, 256-byte aligned.
+ */
+specasr_status specasr_kv_create(const specasr_model* m, void* k_pool, void* v_pool, int32_t n_pages,
+                                 const int32_t* page_table, int32_t max_pages, void* workspace,
+                                 int32_t max_nodes, specasr_kv** out);
+void specasr_kv_destroy(specasr_kv* kv);
+
+/* Committed length in tokens, [host] out.  Synchronises `stream` if a commit is still in flight. */
+specasr_status specasr_kv_length(specasr_kv* kv, int32_t* out_len, void* stream);
+/* Rewinds (or empties) the cache to `len` <= current length.  Drops any pending verify. */
+specasr_status specasr_kv_truncate(specasr_kv* kv, int32_t len, void* stream);
+
+/* Context fill (the prefill of Section II-A: audio vectors "alongside text prompts"), causal
+ * attention, no logits.  embeds [device] fp32 [n, d_model] enter layer 0 directly; tokens [device]
+ * int32[n] go through the embedding table.  Any n >= 1 (processed in chunks); advances the length. */
+specasr_status specasr_prefill_embeds(specasr_model* m, specasr_kv* kv, const float* embeds, int32_t n, void* stream);
+specasr_status specasr_prefill_tokens(specasr_model* m, specasr_kv* kv, const int32_t* tokens, int32_t n, void* stream);
+
+/*
+ * Verify a draft token tree (Section II-B; tree mask per Fig. 13 / Section IV-C).
+ *   tokens, parent_idx : [device] int32[n_nodes]
+ *   out_argmax         : [device] int32[n_nodes]  target greedy token after each node (lowest id on ties)
+ *   out_accept_len     : [device] int32[1]        accepted draft nodes on the best path (-1 on device error)
+ *   out_path           : [device] int32[n_nodes]  node indices root..best, padded with -1
+ * Writes the tree's K/V to cache slots L..L+n-1 (L = committed length) and marks the handle
+ * "pending"; the committed length does not change.  Calling verify again without a commit simply
+ * overwrites those slots (that is how a round is abandoned).
+ */
+specasr_status specasr_verify_tree(specasr_model* m, specasr_kv* kv, const int32_t* tokens,
+                                   const int32_t* parent_idx, int32_t n_nodes, int32_t* out_argmax,
+                                   int32_t* out_accept_len, int32_t* out_path, void* stream);
+
+/* Same, plus optional outputs: out_logits [device] fp32 [n_nodes, vocab] (NULL to skip) and
+ * out_bonus [device] int32[1] = out_argmax[best] (the token emitted after the accepted path). */
+specasr_status specasr_verify_tree_ex(specasr_model* m, specasr_kv* kv, const int32_t* tokens,
+                                      const int32_t* parent_idx, int32_t n_nodes, int32_t* out_argmax,
+                                      int32_t* out_accept_len, int32_t* out_path, float* out_logits,
+                                      int32_t* out_bonus, void* stream);
+
+/*
+ * Keep the accepted path (the "revert to the draft model" step of Section II-B needs the cache to
+ * hold exactly prefix + accepted tokens): slot L+j <- slot L+path[j] for j = 0..accept_len, all
+ * layers, K and V; then L <- L + accept_len + 1.  path / accept_len are the [device] arrays a
+ * preceding verify wrote (or the caller's own choice of a root path of that tree).  Requires a
+ * pending verify (else SPECASR_ERR_STATE); clears it.  accept_len < 0 on the device (failed verify)
+ * makes the commit a no-op.
+ */
+specasr_status specasr_commit_kv(specasr_model* m, specasr_kv* kv, const int32_t* path,
+                                 const int32_t* accept_len, void* stream);
+
+/* Reads the device status word of the last verify/prefill on this handle ([host] out; synchronises
+ * `stream`).  SPECASR_OK, SPECASR_ERR_INVALID_TREE, SPECASR_ERR_KV_CAPACITY or SPECASR_ERR_TIMEOUT. */
+specasr_status specasr_poll_status(specasr_kv* kv, int32_t* out_device_status, void* stream);
+
+/* Number of kernels the library has launched on this handle so far (for launch accounting). */
+int64_t specasr_launch_count(const specasr_kv* kv);
+
+const char* specasr_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPECASR_H_ */

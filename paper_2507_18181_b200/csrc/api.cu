@@ -1,0 +1,498 @@
+// C ABI entry points: handle management, host-side validation and the kernel sequence of one
+// verification round.  See include/specasr.h for the contract of every call.
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+
+#include "internal.h"
+
+// ------------------------------------------------------------------------------------------------
+static thread_local char g_err[512] = "";
+
+void set_error(const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+}
+
+extern "C" const char* specasr_last_error(void) { return g_err; }
+
+#define CUDA_TRY(expr)                                                              \
+  do {                                                                              \
+    cudaError_t e__ = (expr);                                                       \
+    if (e__ != cudaSuccess) {                                                       \
+      set_error("%s failed: %s (%s:%d)", #expr, cudaGetErrorString(e__), __FILE__, __LINE__); \
+      return SPECASR_ERR_CUDA;                                                      \
+    }                                                                               \
+  } while (0)
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+static inline int round_up(int x, int a) { return (x + a - 1) / a * a; }
+
+int lm_tiles_of(const specasr_model* m) {
+  return m->cfg.gemm_path == 1 ? gemm_fma_tiles(m->cfg.vocab) : gemm_tc_tiles(m->cfg.vocab);
+}
+
+Workspace carve_workspace(const specasr_model* m, int n_alloc, void* base) {
+  const specasr_model_config& c = m->cfg;
+  Workspace w;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    char* p = base ? (char*)base + off : nullptr;
+    off += align_up(bytes, 256);
+    return (void*)p;
+  };
+  const size_t wide = (size_t)(c.d_model > m->qkv_dim ? c.d_model : m->qkv_dim);
+  w.ctl = (int32_t*)take(sizeof(int32_t) * kCtlWords);
+  w.depth = (int32_t*)take(sizeof(int32_t) * n_alloc);
+  w.pos = (int32_t*)take(sizeof(int32_t) * n_alloc);
+  w.anc = (unsigned long long*)take(sizeof(unsigned long long) * 4 * n_alloc);
+  w.X = (float*)take(sizeof(float) * n_alloc * c.d_model);
+  w.H = (bf16*)take(sizeof(bf16) * 2 * n_alloc * c.d_model);
+  w.P = (float*)take(sizeof(float) * kMaxSplitK * n_alloc * wide);
+  w.Q = (bf16*)take(sizeof(bf16) * 2 * n_alloc * m->q_dim);
+  w.AO = (bf16*)take(sizeof(bf16) * 2 * n_alloc * m->q_dim);
+  w.A = (bf16*)take(sizeof(bf16) * 2 * n_alloc * c.ffn);
+  w.attO = (float*)take(sizeof(float) * kMaxAttnSplits * n_alloc * c.n_heads * c.head_dim);
+  w.attML = (float2*)take(sizeof(float2) * kMaxAttnSplits * n_alloc * c.n_heads);
+  w.amax = (unsigned long long*)take(sizeof(unsigned long long) * lm_tiles_of(m) * n_alloc);
+  w.bytes = off;
+  return w;
+}
+
+// ------------------------------------------------------------------------------------------------
+extern "C" specasr_status specasr_model_create(const specasr_model_config* cfg, const specasr_weight_ptrs* w,
+                                               specasr_model** out) {
+  if (!cfg || !w || !out) {
+    set_error("specasr_model_create: null argument");
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  *out = nullptr;
+  const specasr_model_config& c = *cfg;
+  if (c.n_layers < 1 || c.d_model < 8 || c.n_heads < 1 || c.n_kv_heads < 1 || c.ffn < 8 || c.vocab < 1 ||
+      c.max_positions < 1 || c.page_size < 1) {
+    set_error("specasr_model_create: non-positive dimension");
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  if ((c.head_dim != 32 && c.head_dim != 64 && c.head_dim != 128) || c.n_heads % c.n_kv_heads != 0 ||
+      c.d_model % 8 != 0 || c.ffn % 8 != 0 || c.page_size % 8 != 0 || (c.gemm_path != 0 && c.gemm_path != 1)) {
+    set_error("specasr_model_create: unsupported shape (head_dim in {32,64,128}, d_model/ffn/page_size %% 8 == 0)");
+    return SPECASR_ERR_UNSUPPORTED;
+  }
+  if (!w->embed || !w->lm_head || !w->g_final || !w->wqkv || !w->wo || !w->wgu || !w->wd || !w->g_attn || !w->g_ffn) {
+    set_error("specasr_model_create: null weight pointer");
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  specasr_model* m = new (std::nothrow) specasr_model();
+  if (!m) {
+    set_error("out of host memory");
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  m->cfg = c;
+  m->q_dim = c.n_heads * c.head_dim;
+  m->kv_dim = c.n_kv_heads * c.head_dim;
+  m->qkv_dim = m->q_dim + 2 * m->kv_dim;
+  m->embed = (const bf16*)w->embed;
+  m->lm_head = (const bf16*)w->lm_head;
+  m->g_final = w->g_final;
+  m->rope_table = nullptr;
+  for (int l = 0; l < c.n_layers; ++l) {
+    if (!w->wqkv[l] || !w->wo[l] || !w->wgu[l] || !w->wd[l] || !w->g_attn[l] || !w->g_ffn[l]) {
+      delete m;
+      set_error("specasr_model_create: null weight pointer in layer %d", l);
+      return SPECASR_ERR_INVALID_ARG;
+    }
+    m->wqkv.push_back((const bf16*)w->wqkv[l]);
+    m->wo.push_back((const bf16*)w->wo[l]);
+    m->wgu.push_back((const bf16*)w->wgu[l]);
+    m->wd.push_back((const bf16*)w->wd[l]);
+    m->g_attn.push_back(w->g_attn[l]);
+    m->g_ffn.push_back(w->g_ffn[l]);
+  }
+  cudaError_t e = cudaGetDevice(&m->device);
+  cudaDeviceProp prop;
+  if (e == cudaSuccess) e = cudaGetDeviceProperties(&prop, m->device);
+  if (e != cudaSuccess) {
+    delete m;
+    set_error("no usable CUDA device: %s", cudaGetErrorString(e));
+    return SPECASR_ERR_CUDA;
+  }
+  m->n_sm = prop.multiProcessorCount;
+  if (c.gemm_path == 0 && prop.major != 10) {
+    delete m;
+    set_error("the tensor-core path needs an sm_100 device (found sm_%d%d)", prop.major, prop.minor);
+    return SPECASR_ERR_UNSUPPORTED;
+  }
+  // rotary table in fp64 on the host: angle = pos * base^(-2k/dh)
+  const int half = c.head_dim / 2;
+  std::vector<float2> tab((size_t)c.max_positions * half);
+  for (int k = 0; k < half; ++k) {
+    const double theta = pow((double)c.rope_base, -2.0 * k / c.head_dim);
+    for (int p = 0; p < c.max_positions; ++p) {
+      const double ang = (double)p * theta;
+      tab[(size_t)p * half + k] = make_float2((float)cos(ang), (float)sin(ang));
+    }
+  }
+  e = cudaMalloc(&m->rope_table, tab.size() * sizeof(float2));
+  if (e == cudaSuccess) e = cudaMemcpy(m->rope_table, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) {
+    if (m->rope_table) cudaFree(m->rope_table);
+    delete m;
+    set_error("rotary table upload failed: %s", cudaGetErrorString(e));
+    return SPECASR_ERR_CUDA;
+  }
+  if (c.gemm_path == 0) {
+    bool ok = true;
+    m->tm_wqkv.resize(c.n_layers);
+    m->tm_wo.resize(c.n_layers);
+    m->tm_wgu.resize(c.n_layers);
+    m->tm_wd.resize(c.n_layers);
+    for (int l = 0; l < c.n_layers && ok; ++l) {
+      ok = ok && make_tensor_map_2d(&m->tm_wqkv[l], m->wqkv[l], c.d_model, m->qkv_dim, 64, 128);
+      ok = ok && make_tensor_map_2d(&m->tm_wo[l], m->wo[l], m->q_dim, c.d_model, 64, 128);
+      ok = ok && make_tensor_map_2d(&m->tm_wgu[l], m->wgu[l], c.d_model, 2 * (uint64_t)c.ffn, 64, 128);
+      ok = ok && make_tensor_map_2d(&m->tm_wd[l], m->wd[l], c.ffn, c.d_model, 64, 128);
+    }
+    ok = ok && make_tensor_map_2d(&m->tm_lm, m->lm_head, c.d_model, c.vocab, 64, 128);
+    if (!ok) {
+      cudaFree(m->rope_table);
+      delete m;
+      return SPECASR_ERR_CUDA;   // message set by make_tensor_map_2d
+    }
+  }
+  *out = m;
+  return SPECASR_OK;
+}
+
+extern "C" void specasr_model_destroy(specasr_model* m) {
+  if (!m) return;
+  if (m->rope_table) cudaFree(m->rope_table);
+  delete m;
+}
+
+extern "C" size_t specasr_workspace_bytes(const specasr_model* m, int32_t max_nodes) {
+  if (!m || max_nodes < 1 || max_nodes > SPECASR_MAX_NODES) return 0;
+  return carve_workspace(m, round_up(max_nodes, 16), nullptr).bytes;
+}
+
+extern "C" size_t specasr_kv_pool_bytes(const specasr_model* m, int32_t n_pages) {
+  if (!m || n_pages < 1) return 0;
+  const specasr_model_config& c = m->cfg;
+  return (size_t)c.n_layers * n_pages * c.n_kv_heads * 2 * c.page_size * c.head_dim * sizeof(bf16);
+}
+
+extern "C" specasr_status specasr_kv_create(const specasr_model* m, void* k_pool, void* v_pool, int32_t n_pages,
+                                            const int32_t* page_table, int32_t max_pages, void* workspace,
+                                            int32_t max_nodes, specasr_kv** out) {
+  if (!m || !k_pool || !v_pool || !page_table || !workspace || !out) {
+    set_error("specasr_kv_create: null argument");
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  *out = nullptr;
+  if (n_pages < 1 || max_pages < 1 || max_nodes < 1 || max_nodes > SPECASR_MAX_NODES) {
+    set_error("specasr_kv_create: n_pages, max_pages >= 1 and 1 <= max_nodes <= %d required", SPECASR_MAX_NODES);
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  if (((uintptr_t)workspace & 255) || ((uintptr_t)k_pool & 15) || ((uintptr_t)v_pool & 15)) {
+    set_error("specasr_kv_create: workspace must be 256-byte aligned, pools 16-byte aligned");
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  specasr_kv* kv = new (std::nothrow) specasr_kv();
+  if (!kv) {
+    set_error("out of host memory");
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  kv->m = m;
+  kv->k_pool = (bf16*)k_pool;
+  kv->v_pool = (bf16*)v_pool;
+  kv->n_pages = n_pages;
+  kv->page_table = page_table;
+  kv->max_pages = max_pages;
+  kv->max_nodes = max_nodes;
+  kv->n_alloc = round_up(max_nodes, 16);
+  kv->ws = carve_workspace(m, kv->n_alloc, workspace);
+  kv->pending_n = 0;
+  kv->len_host = 0;
+  kv->len_exact = true;
+  kv->len_upper = 0;
+  kv->pinned = nullptr;
+  kv->len_event_pending = false;
+  kv->launches = 0;
+  cudaError_t e = cudaHostAlloc(&kv->pinned, 4 * sizeof(int32_t), cudaHostAllocDefault);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&kv->len_event, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaMemset(kv->ws.ctl, 0, sizeof(int32_t) * kCtlWords);
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) {
+    if (kv->pinned) cudaFreeHost(kv->pinned);
+    delete kv;
+    set_error("specasr_kv_create: %s", cudaGetErrorString(e));
+    return SPECASR_ERR_CUDA;
+  }
+  if (m->cfg.gemm_path == 0) {
+    const specasr_model_config& c = m->cfg;
+    bool ok = true;
+    for (int i = 0, b = 16; i < 5 && b <= kv->n_alloc && ok; ++i, b <<= 1) {
+      ok = make_act_map(&kv->tm_H[i], kv->ws.H, c.d_model, kv->n_alloc, b) &&
+           make_act_map(&kv->tm_AO[i], kv->ws.AO, m->q_dim, kv->n_alloc, b) &&
+           make_act_map(&kv->tm_A[i], kv->ws.A, c.ffn, kv->n_alloc, b);
+    }
+    if (!ok) {
+      cudaFreeHost(kv->pinned);
+      cudaEventDestroy(kv->len_event);
+      delete kv;
+      return SPECASR_ERR_CUDA;
+    }
+  }
+  *out = kv;
+  return SPECASR_OK;
+}
+
+extern "C" void specasr_kv_destroy(specasr_kv* kv) {
+  if (!kv) return;
+  if (kv->len_event_pending) cudaEventSynchronize(kv->len_event);
+  cudaEventDestroy(kv->len_event);
+  if (kv->pinned) cudaFreeHost(kv->pinned);
+  delete kv;
+}
+
+extern "C" int64_t specasr_launch_count(const specasr_kv* kv) { return kv ? kv->launches : 0; }
+
+// The host learns the committed length lazily: a commit enqueues a copy of the device length word
+// into pinned memory followed by an event.
+static void refresh_len(specasr_kv* kv, bool wait) {
+  if (!kv->len_event_pending) return;
+  cudaError_t q = wait ? cudaEventSynchronize(kv->len_event) : cudaEventQuery(kv->len_event);
+  if (q == cudaSuccess) {
+    kv->len_host = kv->pinned[0];
+    kv->len_upper = kv->len_host;
+    kv->len_exact = true;
+    kv->len_event_pending = false;
+  } else if (q != cudaErrorNotReady) {
+    cudaGetLastError();
+  }
+}
+
+extern "C" specasr_status specasr_kv_length(specasr_kv* kv, int32_t* out_len, void* stream) {
+  (void)stream;
+  if (!kv || !out_len) {
+    set_error("specasr_kv_length: null argument");
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  refresh_len(kv, true);
+  *out_len = kv->len_host;
+  return SPECASR_OK;
+}
+
+extern "C" specasr_status specasr_kv_truncate(specasr_kv* kv, int32_t len, void* stream) {
+  if (!kv) {
+    set_error("specasr_kv_truncate: null handle");
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  refresh_len(kv, true);
+  if (len < 0 || len > kv->len_host) {
+    set_error("specasr_kv_truncate: len %d outside [0, %d]", len, kv->len_host);
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  launch_set_len(kv, len, (cudaStream_t)stream);
+  kv->len_host = kv->len_upper = len;
+  kv->pending_n = 0;
+  CUDA_TRY(cudaGetLastError());
+  return SPECASR_OK;
+}
+
+extern "C" specasr_status specasr_poll_status(specasr_kv* kv, int32_t* out_device_status, void* stream) {
+  if (!kv || !out_device_status) {
+    set_error("specasr_poll_status: null argument");
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  cudaStream_t s = (cudaStream_t)stream;
+  CUDA_TRY(cudaMemcpyAsync(kv->pinned + 2, kv->ws.ctl + CTL_STATUS, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+  CUDA_TRY(cudaStreamSynchronize(s));
+  *out_device_status = kv->pinned[2];
+  return SPECASR_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+static void run_gemm(specasr_kv* kv, GemmArgs& a, cudaStream_t s) {
+  if (kv->m->cfg.gemm_path == 1) {
+    a.splits = 1;
+    launch_gemm_fma(kv, a, s);
+  } else {
+    launch_gemm_tc(kv, a, s);
+  }
+}
+
+static int attention_splits(const specasr_kv* kv, int n, int len_upper) {
+  const specasr_model_config& c = kv->m->cfg;
+  const int group = c.n_heads / c.n_kv_heads;
+  const int row_tiles = (n * group + 63) / 64;
+  const int ctas = c.n_kv_heads * row_tiles;
+  int splits = (kv->m->n_sm + ctas - 1) / ctas;
+  const int by_len = (len_upper + n + 63) / 64;
+  if (splits > by_len) splits = by_len;
+  if (splits > kMaxAttnSplits) splits = kMaxAttnSplits;
+  if (splits < 1) splits = 1;
+  return splits;
+}
+
+// The layer stack over n rows whose layer-0 inputs are already in ws.X.  With want_head the final
+// norm, the vocabulary projection and its fused per-tile argmax run as well.
+static void run_stack(specasr_model* m, specasr_kv* kv, int n, bool want_head, float* out_logits, cudaStream_t s) {
+  const specasr_model_config& c = m->cfg;
+  const int n_pad = round_up(n, 16);
+  const int att_splits = attention_splits(kv, n, kv->len_upper);
+  const bool tc = c.gemm_path == 0;
+  int down_splits = 0;
+  GemmArgs a;
+  memset(&a, 0, sizeof(a));
+  a.n = n;
+  a.n_pad = n_pad;
+  a.n_alloc = kv->n_alloc;
+  a.ctl = kv->ws.ctl;
+  for (int l = 0; l < c.n_layers; ++l) {
+    launch_rmsnorm_split(kv, m->g_attn[l], n, n_pad, down_splits, s);
+    a.W = m->wqkv[l]; a.tmW = tc ? &m->tm_wqkv[l] : nullptr; a.tmAct = kv->tm_H; a.act = kv->ws.H;
+    a.M = m->qkv_dim; a.K = c.d_model; a.epilogue = EPI_PARTIAL; a.P = kv->ws.P;
+    a.splits = tc ? gemm_tc_pick_splits(m, a.M, a.K) : 1;
+    run_gemm(kv, a, s);
+    launch_rope_append(kv, l, n, a.splits, s);
+    launch_tree_attention(kv, l, n, att_splits, s);
+    launch_attn_merge(kv, n, n_pad, att_splits, s);
+    a.W = m->wo[l]; a.tmW = tc ? &m->tm_wo[l] : nullptr; a.tmAct = kv->tm_AO; a.act = kv->ws.AO;
+    a.M = c.d_model; a.K = m->q_dim; a.epilogue = EPI_PARTIAL;
+    a.splits = tc ? gemm_tc_pick_splits(m, a.M, a.K) : 1;
+    run_gemm(kv, a, s);
+    launch_rmsnorm_split(kv, m->g_ffn[l], n, n_pad, a.splits, s);
+    a.W = m->wgu[l]; a.tmW = tc ? &m->tm_wgu[l] : nullptr; a.tmAct = kv->tm_H; a.act = kv->ws.H;
+    a.M = 2 * c.ffn; a.K = c.d_model; a.epilogue = EPI_SWIGLU; a.A = kv->ws.A; a.splits = 1;
+    run_gemm(kv, a, s);
+    a.W = m->wd[l]; a.tmW = tc ? &m->tm_wd[l] : nullptr; a.tmAct = kv->tm_A; a.act = kv->ws.A;
+    a.M = c.d_model; a.K = c.ffn; a.epilogue = EPI_PARTIAL;
+    a.splits = tc ? gemm_tc_pick_splits(m, a.M, a.K) : 1;
+    run_gemm(kv, a, s);
+    down_splits = a.splits;
+  }
+  if (!want_head) return;   // context fill: K/V of every layer are written, the last FFN output is not needed
+  launch_rmsnorm_split(kv, m->g_final, n, n_pad, down_splits, s);
+  a.W = m->lm_head; a.tmW = tc ? &m->tm_lm : nullptr; a.tmAct = kv->tm_H; a.act = kv->ws.H;
+  a.M = c.vocab; a.K = c.d_model; a.epilogue = EPI_ARGMAX; a.amax = kv->ws.amax; a.logits = out_logits; a.splits = 1;
+  run_gemm(kv, a, s);
+}
+
+static specasr_status prefill_common(specasr_model* m, specasr_kv* kv, const float* embeds, const int32_t* tokens,
+                                     int n, cudaStream_t s, const char* who) {
+  if (!m || !kv || (!embeds && !tokens)) {
+    set_error("%s: null argument", who);
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  if (kv->m != m) {
+    set_error("%s: KV handle belongs to another model", who);
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  if (n < 1) {
+    set_error("%s: n must be >= 1", who);
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  refresh_len(kv, true);
+  int cap = kv->max_pages * m->cfg.page_size;
+  if (m->cfg.max_positions < cap) cap = m->cfg.max_positions;
+  if (kv->len_host + n > cap) {
+    set_error("%s: %d + %d positions exceed the capacity of %d", who, kv->len_host, n, cap);
+    return SPECASR_ERR_KV_CAPACITY;
+  }
+  kv->pending_n = 0;
+  for (int done = 0; done < n;) {
+    const int chunk = n - done < kv->max_nodes ? n - done : kv->max_nodes;
+    launch_chain_prep(kv, chunk, s);
+    if (embeds) launch_copy_embeds(kv, embeds + (size_t)done * m->cfg.d_model, chunk, s);
+    else launch_embed_tokens(kv, tokens + done, chunk, s);
+    run_stack(m, kv, chunk, false, nullptr, s);
+    launch_advance_len(kv, chunk, s);
+    kv->len_host += chunk;
+    kv->len_upper = kv->len_host;
+    done += chunk;
+  }
+  CUDA_TRY(cudaGetLastError());
+  return SPECASR_OK;
+}
+
+extern "C" specasr_status specasr_prefill_embeds(specasr_model* m, specasr_kv* kv, const float* embeds, int32_t n,
+                                                 void* stream) {
+  return prefill_common(m, kv, embeds, nullptr, n, (cudaStream_t)stream, "specasr_prefill_embeds");
+}
+
+extern "C" specasr_status specasr_prefill_tokens(specasr_model* m, specasr_kv* kv, const int32_t* tokens, int32_t n,
+                                                 void* stream) {
+  return prefill_common(m, kv, nullptr, tokens, n, (cudaStream_t)stream, "specasr_prefill_tokens");
+}
+
+extern "C" specasr_status specasr_verify_tree_ex(specasr_model* m, specasr_kv* kv, const int32_t* tokens,
+                                                 const int32_t* parent_idx, int32_t n_nodes, int32_t* out_argmax,
+                                                 int32_t* out_accept_len, int32_t* out_path, float* out_logits,
+                                                 int32_t* out_bonus, void* stream) {
+  if (!m || !kv || !tokens || !parent_idx || !out_argmax || !out_accept_len || !out_path) {
+    set_error("specasr_verify_tree: null argument");
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  if (kv->m != m) {
+    set_error("specasr_verify_tree: KV handle belongs to another model");
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  if (n_nodes < 1 || n_nodes > kv->max_nodes) {
+    set_error("specasr_verify_tree: n_nodes = %d outside [1, %d]", n_nodes, kv->max_nodes);
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  refresh_len(kv, false);
+  int cap = kv->max_pages * m->cfg.page_size;
+  if (m->cfg.max_positions < cap) cap = m->cfg.max_positions;
+  if (kv->len_exact && kv->len_host + n_nodes > cap) {
+    set_error("specasr_verify_tree: %d committed + %d tree slots exceed the capacity of %d", kv->len_host, n_nodes, cap);
+    return SPECASR_ERR_KV_CAPACITY;
+  }
+  cudaStream_t s = (cudaStream_t)stream;
+  launch_tree_prep(kv, tokens, parent_idx, n_nodes, s);
+  launch_embed_tokens(kv, tokens, n_nodes, s);
+  run_stack(m, kv, n_nodes, true, out_logits, s);
+  launch_accept(kv, tokens, parent_idx, n_nodes, lm_tiles_of(m), out_argmax, out_accept_len, out_path, out_bonus, s);
+  kv->pending_n = n_nodes;
+  CUDA_TRY(cudaGetLastError());
+  return SPECASR_OK;
+}
+
+extern "C" specasr_status specasr_verify_tree(specasr_model* m, specasr_kv* kv, const int32_t* tokens,
+                                              const int32_t* parent_idx, int32_t n_nodes, int32_t* out_argmax,
+                                              int32_t* out_accept_len, int32_t* out_path, void* stream) {
+  return specasr_verify_tree_ex(m, kv, tokens, parent_idx, n_nodes, out_argmax, out_accept_len, out_path, nullptr,
+                                nullptr, stream);
+}
+
+extern "C" specasr_status specasr_commit_kv(specasr_model* m, specasr_kv* kv, const int32_t* path,
+                                            const int32_t* accept_len, void* stream) {
+  if (!m || !kv || !path || !accept_len) {
+    set_error("specasr_commit_kv: null argument");
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  if (kv->m != m) {
+    set_error("specasr_commit_kv: KV handle belongs to another model");
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  if (kv->pending_n == 0) {
+    set_error("specasr_commit_kv: no verify is pending on this handle");
+    return SPECASR_ERR_STATE;
+  }
+  cudaStream_t s = (cudaStream_t)stream;
+  refresh_len(kv, false);
+  launch_commit(kv, path, accept_len, s);
+  CUDA_TRY(cudaMemcpyAsync(kv->pinned, kv->ws.ctl + CTL_LEN, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+  CUDA_TRY(cudaEventRecord(kv->len_event, s));
+  kv->len_event_pending = true;
+  kv->len_exact = false;
+  kv->len_upper += kv->pending_n;
+  kv->pending_n = 0;
+  CUDA_TRY(cudaGetLastError());
+  return SPECASR_OK;
+}

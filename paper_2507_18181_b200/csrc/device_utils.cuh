@@ -1,0 +1,59 @@
+// Small device helpers shared by the kernels.
+#pragma once
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+__device__ __forceinline__ float bf16lo_to_f32(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16hi_to_f32(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+// x ~ hi + lo with hi = bf16(x), lo = bf16(x - hi): about 16 significant bits survive.
+__device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bfloat16& lo) {
+  hi = __float2bfloat16_rn(x);
+  lo = __float2bfloat16_rn(x - __bfloat162float(hi));
+}
+
+// Two values -> packed (hi0, hi1) and (lo0, lo1) words, element 0 in the low half.
+__device__ __forceinline__ void split2_pack(float a, float b, uint32_t& hi, uint32_t& lo) {
+  __nv_bfloat16 ha, la, hb, lb;
+  split_bf16(a, ha, la);
+  split_bf16(b, hb, lb);
+  hi = (uint32_t)__bfloat16_as_ushort(ha) | ((uint32_t)__bfloat16_as_ushort(hb) << 16);
+  lo = (uint32_t)__bfloat16_as_ushort(la) | ((uint32_t)__bfloat16_as_ushort(lb) << 16);
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+  return v;
+}
+
+// Sum over a 256-thread block; every thread receives the total.
+__device__ __forceinline__ float block_sum_256(float v) {
+  __shared__ float s_part[8];
+  __shared__ float s_total;
+  v = warp_sum(v);
+  if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = v;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    float t = threadIdx.x < 8 ? s_part[threadIdx.x] : 0.f;
+    t = warp_sum(t);
+    if (threadIdx.x == 0) s_total = t;
+  }
+  __syncthreads();
+  return s_total;
+}
+
+// Element offset of plane `plane` (0 = hi, 1 = lo) of (layer, physical page, kv head) in a KV pool
+// laid out [n_layers][n_pages][n_kv_heads][2][page_size][head_dim].
+__device__ __forceinline__ size_t kv_plane_offset(int layer, int n_pages, int Hkv, int page_size, int dh, int page,
+                                                  int kvh, int plane) {
+  return ((((size_t)layer * n_pages + page) * Hkv + kvh) * 2 + plane) * (size_t)page_size * dh;
+}
+
+// Order-preserving map of a float to an unsigned key, packed with the complement of an index so that
+// a plain unsigned max picks the largest value and, among equals, the lowest index.
+__device__ __forceinline__ unsigned long long pack_max_key(float v, uint32_t idx) {
+  uint32_t u = __float_as_uint(v);
+  u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+  return ((unsigned long long)u << 32) | (unsigned long long)(0xFFFFFFFFu - idx);
+}

@@ -1,0 +1,129 @@
+// Internal declarations of the tree-verification library (not part of the C ABI).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "specasr.h"
+
+typedef __nv_bfloat16 bf16;
+
+constexpr int kMaxSplitK = 8;      // split-K partial planes for the projections
+constexpr int kMaxAttnSplits = 32; // KV splits of the attention kernel
+constexpr int kCtlWords = 64;      // int32 control block at the start of the workspace
+
+// control block word indices
+enum { CTL_LEN = 0, CTL_STATUS = 1, CTL_N = 2 };
+
+struct GemmMaps {           // TMA descriptors of one weight matrix (tcgen05 path)
+  CUtensorMap w;
+};
+
+struct specasr_model {
+  specasr_model_config cfg;
+  int device;
+  int qkv_dim;              // (Hq + 2 Hkv) * dh
+  int q_dim;                // Hq * dh
+  int kv_dim;               // Hkv * dh
+  const bf16* embed;
+  const bf16* lm_head;
+  const float* g_final;
+  std::vector<const bf16*> wqkv, wo, wgu, wd;
+  std::vector<const float*> g_attn, g_ffn;
+  float2* rope_table;       // [max_positions][dh/2] (cos, sin), built in fp64 on the host
+  std::vector<CUtensorMap> tm_wqkv, tm_wo, tm_wgu, tm_wd;
+  CUtensorMap tm_lm;
+  int n_sm;
+};
+
+struct Workspace {
+  int32_t* ctl;             // [kCtlWords]
+  int32_t* depth;           // [n_alloc]
+  int32_t* pos;             // [n_alloc]
+  unsigned long long* anc;  // [n_alloc][4] ancestor-or-self bitmask over node indices
+  float* X;                 // [n_alloc][d] residual stream
+  bf16* H;                  // [2][n_alloc][d]      normed activations, hi / lo planes
+  float* P;                 // [kMaxSplitK][n_alloc][max(d, qkv_dim)] split-K partial sums
+  bf16* Q;                  // [2][n_alloc][q_dim]  rotated queries, hi / lo planes
+  bf16* AO;                 // [2][n_alloc][q_dim]  attention output, hi / lo planes
+  bf16* A;                  // [2][n_alloc][ffn]    SwiGLU output, hi / lo planes
+  float* attO;              // [kMaxAttnSplits][n_alloc * Hq][dh] unnormalised partial outputs
+  float2* attML;            // [kMaxAttnSplits][n_alloc * Hq]     (running max in log2 units, sum)
+  unsigned long long* amax; // [lm_tiles][n_alloc] packed (ordered logit, ~token id) per vocab tile
+  size_t bytes;
+};
+
+struct specasr_kv {
+  const specasr_model* m;
+  bf16* k_pool;
+  bf16* v_pool;
+  int n_pages;
+  const int32_t* page_table;
+  int max_pages;
+  int max_nodes;
+  int n_alloc;              // max_nodes rounded up to 16
+  Workspace ws;
+  // host-side state
+  int pending_n;            // nodes of the verify awaiting a commit, 0 = none
+  int len_host;             // last length the host knows exactly
+  bool len_exact;           // false while a commit's length has not been read back
+  int len_upper;            // upper bound of the length
+  int32_t* pinned;          // [2] pinned host words: length, status
+  cudaEvent_t len_event;
+  bool len_event_pending;
+  int64_t launches;
+  // activation TMA descriptors (tcgen05 path)
+  // activation TMA descriptors (tcgen05 path), one per box height 16 << i
+  CUtensorMap tm_H[5], tm_AO[5], tm_A[5];
+};
+
+void set_error(const char* fmt, ...);
+Workspace carve_workspace(const specasr_model* m, int n_alloc, void* base);
+int lm_tiles_of(const specasr_model* m);
+
+// ---- kernels_small.cu
+void launch_tree_prep(specasr_kv* kv, const int32_t* tokens, const int32_t* parent, int n, cudaStream_t s);
+void launch_chain_prep(specasr_kv* kv, int n, cudaStream_t s);
+void launch_embed_tokens(specasr_kv* kv, const int32_t* tokens, int n, cudaStream_t s);
+void launch_copy_embeds(specasr_kv* kv, const float* embeds, int n, cudaStream_t s);
+void launch_rmsnorm_split(specasr_kv* kv, const float* gain, int n, int n_pad, int n_partials, cudaStream_t s);
+void launch_rope_append(specasr_kv* kv, int layer, int n, int n_partials, cudaStream_t s);
+void launch_attn_merge(specasr_kv* kv, int n, int n_pad, int n_splits, cudaStream_t s);
+void launch_accept(specasr_kv* kv, const int32_t* tokens, const int32_t* parent, int n, int n_tiles,
+                   int32_t* out_argmax, int32_t* out_accept_len, int32_t* out_path, int32_t* out_bonus,
+                   cudaStream_t s);
+void launch_advance_len(specasr_kv* kv, int n, cudaStream_t s);
+void launch_set_len(specasr_kv* kv, int len, cudaStream_t s);
+void launch_commit(specasr_kv* kv, const int32_t* path, const int32_t* accept_len, cudaStream_t s);
+
+// ---- attention.cu
+void launch_tree_attention(specasr_kv* kv, int layer, int n, int n_splits, cudaStream_t s);
+
+// ---- gemm_fma.cu / gemm_tcgen05.cu
+enum GemmEpilogue { EPI_PARTIAL = 0, EPI_SWIGLU = 1, EPI_ARGMAX = 2 };
+struct GemmArgs {
+  const bf16* W;            // [M, K]
+  const CUtensorMap* tmW;   // tcgen05 path
+  const CUtensorMap* tmAct; // tcgen05 path: activation planes [2 * n_alloc, K]
+  const bf16* act;          // [2][n_alloc][K] hi / lo planes
+  int M, K, n, n_pad, n_alloc;
+  int epilogue;
+  int splits;               // EPI_PARTIAL only
+  float* P;                 // EPI_PARTIAL: [splits][n_alloc][M]
+  bf16* A;                  // EPI_SWIGLU: [2][n_alloc][M/2]
+  unsigned long long* amax; // EPI_ARGMAX: [tiles][n_alloc]
+  float* logits;            // EPI_ARGMAX: optional [n][M]
+  const int32_t* ctl;
+};
+int gemm_fma_tiles(int M);
+void launch_gemm_fma(specasr_kv* kv, const GemmArgs& a, cudaStream_t s);
+int gemm_tc_tiles(int M);
+int gemm_tc_pick_splits(const specasr_model* m, int M, int K);
+void launch_gemm_tc(specasr_kv* kv, const GemmArgs& a, cudaStream_t s);
+bool make_tensor_map_2d(CUtensorMap* out, const void* base, uint64_t inner, uint64_t outer,
+                        uint32_t box_inner, uint32_t box_outer);
+bool make_act_map(CUtensorMap* out, const void* base, uint64_t K, uint64_t n_alloc, uint32_t box_rows);

@@ -1,0 +1,170 @@
+"""Device-memory plumbing around the C ABI: torch allocates and owns every buffer, the library
+borrows them.  No arithmetic of the verification path lives here."""
+import ctypes as C
+
+import numpy as np
+import torch
+
+from . import binding as B
+
+
+def _bf16_from_bits(bits: np.ndarray, device) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(device).view(torch.bfloat16)
+
+
+class DeviceModel:
+    """Weights of one decoder on the GPU in the layouts include/specasr.h asks for.
+
+    `cfg` needs n_layers, d_model, n_heads, n_kv_heads, head_dim, ffn, vocab, eps, rope_base.
+    `store` needs tensor(layer, name) -> numpy array (uint16 bf16 bit patterns for matrices, fp32 for
+    gains; layer -1 = embed / lm_head / g_final) and optionally map_tensors(fn, keys) for threaded draws.
+    """
+
+    def __init__(self, cfg, store, page_size=16, max_positions=8192, gemm_path=0, device="cuda:0"):
+        self.cfg = cfg
+        self.device = torch.device(device)
+        torch.cuda.set_device(self.device)
+        self.page_size = page_size
+        L = cfg.n_layers
+        got = {}
+
+        def put(layer, name, arr):
+            if arr.dtype == np.uint16:
+                got[(layer, name)] = _bf16_from_bits(arr, self.device)
+            else:
+                got[(layer, name)] = torch.from_numpy(np.ascontiguousarray(arr, dtype=np.float32)).to(self.device)
+            if layer >= 0 and all((layer, k) in got for k in ("wq", "wk", "wv")):
+                got[(layer, "wqkv")] = torch.cat([got.pop((layer, k)) for k in ("wq", "wk", "wv")], dim=0).contiguous()
+            if layer >= 0 and all((layer, k) in got for k in ("wg", "wu")):
+                g, u = got.pop((layer, "wg")), got.pop((layer, "wu"))
+                got[(layer, "wgu")] = torch.stack([g, u], dim=1).reshape(2 * cfg.ffn, cfg.d_model).contiguous()
+
+        keys = [(-1, n) for n in ("embed", "lm_head", "g_final")]
+        for l in range(L):
+            keys += [(l, n) for n in ("wq", "wk", "wv", "wo", "wg", "wu", "wd", "g_attn", "g_ffn")]
+        if hasattr(store, "map_tensors"):
+            store.map_tensors(put, keys)
+        else:
+            for k in keys:
+                put(k[0], k[1], store.tensor(*k))
+        self.t = got
+        self._arrays = {}
+        wp = B.WeightPtrs()
+        wp.embed = got[(-1, "embed")].data_ptr()
+        wp.lm_head = got[(-1, "lm_head")].data_ptr()
+        wp.g_final = got[(-1, "g_final")].data_ptr()
+        for field in ("wqkv", "wo", "wgu", "wd", "g_attn", "g_ffn"):
+            arr = (C.c_void_p * L)(*[got[(l, field)].data_ptr() for l in range(L)])
+            self._arrays[field] = arr
+            setattr(wp, field, C.cast(arr, C.POINTER(C.c_void_p)))
+        mc = B.ModelConfig(n_layers=L, d_model=cfg.d_model, n_heads=cfg.n_heads, n_kv_heads=cfg.n_kv_heads,
+                           head_dim=cfg.head_dim, ffn=cfg.ffn, vocab=cfg.vocab, page_size=page_size,
+                           max_positions=max_positions, rms_eps=cfg.eps, rope_base=cfg.rope_base,
+                           gemm_path=gemm_path)
+        self.handle = B.specasr_model_create(mc, wp)
+
+    def weight_bytes(self) -> int:
+        return sum(v.numel() * v.element_size() for v in self.t.values())
+
+    def close(self):
+        if self.handle:
+            B.specasr_model_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class DeviceKV:
+    """Paged KV cache + workspace for one utterance."""
+
+    def __init__(self, model: DeviceModel, max_tokens: int, max_nodes: int = 256, shuffle_pages_seed=None):
+        self.model = model
+        cfg = model.cfg
+        dev = model.device
+        ps = model.page_size
+        self.max_pages = (max_tokens + ps - 1) // ps
+        self.n_pages = self.max_pages
+        self.max_nodes = max_nodes
+        pool_bytes = B.specasr_kv_pool_bytes(model.handle, self.n_pages)
+        self.k_pool = torch.zeros(pool_bytes // 2, dtype=torch.bfloat16, device=dev)
+        self.v_pool = torch.zeros(pool_bytes // 2, dtype=torch.bfloat16, device=dev)
+        if shuffle_pages_seed is None:
+            table = np.arange(self.max_pages, dtype=np.int32)
+        else:
+            table = np.random.default_rng(shuffle_pages_seed).permutation(self.max_pages).astype(np.int32)
+        self.page_table_host = table
+        self.page_table = torch.from_numpy(table).to(dev)
+        ws_bytes = B.specasr_workspace_bytes(model.handle, max_nodes)
+        self.workspace = torch.zeros(ws_bytes + 256, dtype=torch.uint8, device=dev)
+        ws_ptr = (self.workspace.data_ptr() + 255) // 256 * 256
+        self.handle = B.specasr_kv_create(model.handle, self.k_pool.data_ptr(), self.v_pool.data_ptr(), self.n_pages,
+                                          self.page_table.data_ptr(), self.max_pages, ws_ptr, max_nodes)
+        self.out_argmax = torch.empty(max_nodes, dtype=torch.int32, device=dev)
+        self.out_path = torch.empty(max_nodes, dtype=torch.int32, device=dev)
+        self.out_accept = torch.empty(1, dtype=torch.int32, device=dev)
+        self.out_bonus = torch.empty(1, dtype=torch.int32, device=dev)
+
+    @staticmethod
+    def _stream() -> int:
+        return torch.cuda.current_stream().cuda_stream
+
+    def length(self) -> int:
+        return B.specasr_kv_length(self.handle, self._stream())
+
+    def truncate(self, n: int):
+        B.specasr_kv_truncate(self.handle, n, self._stream())
+
+    def prefill_embeds(self, embeds: torch.Tensor):
+        assert embeds.dtype == torch.float32 and embeds.is_cuda and embeds.is_contiguous()
+        B.specasr_prefill_embeds(self.model.handle, self.handle, embeds.data_ptr(), embeds.shape[0], self._stream())
+
+    def prefill_tokens(self, tokens: torch.Tensor):
+        assert tokens.dtype == torch.int32 and tokens.is_cuda and tokens.is_contiguous()
+        B.specasr_prefill_tokens(self.model.handle, self.handle, tokens.data_ptr(), tokens.shape[0], self._stream())
+
+    def verify(self, tokens: torch.Tensor, parent: torch.Tensor, logits: torch.Tensor | None = None):
+        """Enqueues one verification round; results land in out_argmax / out_accept / out_path / out_bonus."""
+        n = tokens.shape[0]
+        B.specasr_verify_tree_ex(self.model.handle, self.handle, tokens.data_ptr(), parent.data_ptr(), n,
+                                 self.out_argmax.data_ptr(), self.out_accept.data_ptr(), self.out_path.data_ptr(),
+                                 logits.data_ptr() if logits is not None else 0, self.out_bonus.data_ptr(),
+                                 self._stream())
+
+    def commit(self):
+        B.specasr_commit_kv(self.model.handle, self.handle, self.out_path.data_ptr(), self.out_accept.data_ptr(),
+                            self._stream())
+
+    def status(self) -> int:
+        return B.specasr_poll_status(self.handle, self._stream())
+
+    def launches(self) -> int:
+        return B.specasr_launch_count(self.handle)
+
+    def read_kv(self, layer: int, n_slots: int):
+        """Host copy of K and V of slots [0, n_slots) of one layer as fp64 [n, Hkv, dh] (hi + lo)."""
+        cfg = self.model.cfg
+        ps = self.model.page_size
+        shape = (cfg.n_layers, self.n_pages, cfg.n_kv_heads, 2, ps, cfg.head_dim)
+        out = []
+        for pool in (self.k_pool, self.v_pool):
+            p = pool.view(shape)[layer].float().cpu().numpy().astype(np.float64)   # [pages, Hkv, 2, ps, dh]
+            logical = p[self.page_table_host]                                      # logical page order
+            val = logical[:, :, 0] + logical[:, :, 1]                              # [pages, Hkv, ps, dh]
+            val = val.transpose(0, 2, 1, 3).reshape(-1, cfg.n_kv_heads, cfg.head_dim)
+            out.append(val[:n_slots])
+        return out[0], out[1]
+
+    def close(self):
+        if self.handle:
+            B.specasr_kv_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,264 @@
+"""Parity of the CUDA path against the CPU oracle, through the C ABI, on seeded inputs.
+
+Bars: integer work (tree prep results visible through positions, accept length, path, committed
+length, compaction moves) bit-exact; logits within 2e-2 max-abs of the fp64 oracle on the same bf16
+weights; argmax / accept / path exact wherever the oracle's top-2 gap exceeds 1e-2 at every node the
+result reads, otherwise the GPU result must be self-consistent and its argmax within 2e-2 of the top.
+"""
+import numpy as np
+import pytest
+import torch
+
+import gen
+from oracle import specasr_oracle as O
+from helpers import oracle_weights
+
+pytestmark = pytest.mark.gpu
+
+LOGIT_TOL = 2e-2
+GAP = 1e-2
+
+
+def _gpu_stack(cfg_name, seed, gemm_path, max_tokens=512, max_nodes=64, shuffle=None):
+    from paper_2507_18181_b200.runtime import DeviceModel, DeviceKV
+    cfg = gen.get_config(cfg_name)
+    store = gen.WeightStore(cfg, seed)
+    model = DeviceModel(cfg, store, gemm_path=gemm_path)
+    kv = DeviceKV(model, max_tokens=max_tokens, max_nodes=max_nodes, shuffle_pages_seed=shuffle)
+    return cfg, store, model, kv
+
+
+def _fill_both(cfg, store, kv, n_audio, n_prompt, seed):
+    W = O.Weights(store, cache_layers=True)
+    audio = gen.audio_prefix(n_audio, cfg.d_model, seed)
+    prompt = gen.prompt_tokens(n_prompt, cfg.vocab, seed)
+    cache = O.KVCache(cfg)
+    O.prefill(cfg, W, cache, np.concatenate([audio.astype(np.float64), O.embed(W, prompt[:-1])], 0))
+    kv.prefill_embeds(torch.from_numpy(audio).cuda())
+    if n_prompt > 1:
+        kv.prefill_tokens(torch.from_numpy(prompt[:-1].copy()).cuda())
+    return W, cache, prompt
+
+
+def _verify_gpu(cfg, kv, tokens, parent):
+    n = len(tokens)
+    logits = torch.empty(n, cfg.vocab, dtype=torch.float32, device="cuda")
+    kv.verify(torch.from_numpy(np.asarray(tokens, np.int32)).cuda(), torch.from_numpy(np.asarray(parent, np.int32)).cuda(),
+              logits)
+    torch.cuda.synchronize()
+    assert kv.status() == 0
+    return {
+        "logits": logits.cpu().numpy().astype(np.float64),
+        "argmax": kv.out_argmax[:n].cpu().numpy(),
+        "accept_len": int(kv.out_accept.item()),
+        "path": kv.out_path[:n].cpu().numpy(),
+        "bonus": int(kv.out_bonus.item()),
+    }
+
+
+def _check_against_oracle(got, want, tokens, parent):
+    n = len(tokens)
+    err = np.abs(got["logits"] - want["logits"]).max()
+    assert err < LOGIT_TOL, f"max-abs logit error {err}"
+    clear = want["gap"] > GAP
+    assert np.array_equal(got["argmax"][clear], want["argmax"][clear])
+    # wherever the gap is small the GPU's pick must still be (numerically) a maximiser
+    top = want["logits"].max(-1)
+    picked = want["logits"][np.arange(n), got["argmax"]]
+    assert np.all(top - picked <= LOGIT_TOL)
+    # self-consistency: accept rule applied to the GPU's own argmax
+    mine = O.accept(tokens, parent, got["argmax"])
+    assert got["accept_len"] == mine["accept_len"] and got["bonus"] == mine["bonus"]
+    a = got["accept_len"]
+    assert list(got["path"][:a + 1]) == list(mine["path"]) and np.all(got["path"][a + 1:] == -1)
+    if want["decisive"]:
+        assert a == want["accept_len"] and list(got["path"][:a + 1]) == list(want["path"])
+        assert got["bonus"] == want["bonus"]
+    return err
+
+
+CASES = [
+    # cfg, gemm_path, n_audio, n_prompt, tree
+    ("tiny", 1, 64, 8, "binary15"),
+    ("tiny", 0, 64, 8, "binary15"),
+    ("micro", 1, 21, 6, "sparse24"),
+    ("micro", 0, 21, 6, "sparse24"),
+    ("small", 1, 150, 9, "sparse64"),
+    ("small", 0, 150, 9, "sparse64"),
+    ("small", 0, 37, 3, "chain8"),
+    ("small", 0, 100, 5, "sparse40"),     # n not a power of two: several activation boxes per stage
+]
+
+
+def _tree(kind, seed):
+    if kind == "binary15":
+        return gen.complete_binary_tree(15)
+    if kind.startswith("sparse"):
+        n = int(kind[6:])
+        return gen.sparse_tree(n, seed=seed, levels=12 if n == 64 else None)
+    return gen.chain_tree(int(kind[5:]))
+
+
+@pytest.mark.parametrize("cfg_name,gemm_path,n_audio,n_prompt,tree", CASES)
+def test_verify_matches_oracle(cfg_name, gemm_path, n_audio, n_prompt, tree):
+    cfg, store, model, kv = _gpu_stack(cfg_name, 0, gemm_path, shuffle=11)
+    W, cache, prompt = _fill_both(cfg, store, kv, n_audio, n_prompt, 0)
+    assert kv.length() == cache.length == n_audio + n_prompt - 1
+    # the filled cache itself
+    for layer in (0, cfg.n_layers - 1):
+        k, v = kv.read_kv(layer, cache.length)
+        assert np.abs(k - cache.K[layer]).max() < 2e-3 and np.abs(v - cache.V[layer]).max() < 2e-3
+    root = int(prompt[-1])
+    parent = _tree(tree, 0)
+    depth_main = len(gen.main_path(parent)) - 1
+    greedy = O.greedy_continuation(cfg, W, cache, root, depth_main)
+    tokens = gen.fill_tree_tokens(parent, cfg.vocab, seed=0, root_token=root, main_tokens=greedy,
+                                  corrupt_p=0.0 if tree == "binary15" else 0.2)
+    if tree == "binary15":
+        tokens = gen.fill_tree_tokens(parent, cfg.vocab, seed=0, root_token=root, main_tokens=greedy[:3])
+    want = O.verify_tree(cfg, W, cache, tokens, parent)
+    got = _verify_gpu(cfg, kv, tokens, parent)
+    _check_against_oracle(got, want, tokens, parent)
+    # verify does not move the committed length, and is repeatable
+    assert kv.length() == cache.length
+    again = _verify_gpu(cfg, kv, tokens, parent)
+    assert np.array_equal(again["logits"], got["logits"]) and again["accept_len"] == got["accept_len"]
+
+    # commit: compaction moves, new length, cache contents
+    L = cache.length
+    a = got["accept_len"]
+    before_k, before_v = kv.read_kv(cfg.n_layers - 1, L + len(tokens))
+    kv.commit()
+    assert kv.length() == L + a + 1
+    after_k, after_v = kv.read_kv(cfg.n_layers - 1, L + a + 1)
+    src = L + got["path"][:a + 1]
+    assert np.array_equal(after_k[L:], before_k[src]) and np.array_equal(after_v[L:], before_v[src])   # bitwise
+    assert np.array_equal(after_k[:L], before_k[:L])
+    if want["decisive"]:
+        moves = O.commit(cache, want)
+        assert moves == [(int(s), L + j) for j, s in enumerate(src)]
+        assert np.abs(after_k - cache.K[-1]).max() < 2e-3 and np.abs(after_v - cache.V[-1]).max() < 2e-3
+
+
+def test_tensor_core_and_fma_projections_agree():
+    """Same operands, two engines: the only difference allowed is fp32 summation order."""
+    outs = []
+    for path in (1, 0):
+        cfg, store, model, kv = _gpu_stack("small", 3, path)
+        W, cache, prompt = _fill_both(cfg, store, kv, 90, 4, 3)
+        parent = gen.sparse_tree(48, seed=3)
+        tokens = gen.fill_tree_tokens(parent, cfg.vocab, seed=3, root_token=int(prompt[-1]))
+        outs.append(_verify_gpu(cfg, kv, tokens, parent))
+    assert np.abs(outs[0]["logits"] - outs[1]["logits"]).max() < 2e-3
+
+
+def test_speculative_rounds_are_lossless_on_gpu():
+    """verify -> commit rounds with corrupted chain drafts and sparse trees reproduce the oracle's
+    autoregressive greedy transcript; every round is also checked against the oracle."""
+    cfg, store, model, kv = _gpu_stack("micro", 5, 0, shuffle=3)
+    W, cache, prompt = _fill_both(cfg, store, kv, 30, 5, 5)
+    root = int(prompt[-1])
+    total = 24
+    want = O.greedy_continuation(cfg, W, cache, root, total + 12)
+    rng = np.random.default_rng(5)
+    out = []
+    rounds = 0
+    while len(out) < total:
+        parent = gen.chain_tree(6) if rounds % 2 == 0 else gen.sparse_tree(20, seed=rounds)
+        k = len(gen.main_path(parent)) - 1
+        truth = want[len(out):len(out) + k]
+        tokens = gen.fill_tree_tokens(parent, cfg.vocab, seed=100 + rounds, root_token=root, main_tokens=truth,
+                                      corrupt_p=0.25)
+        ref = O.verify_tree(cfg, W, cache, tokens, parent)
+        got = _verify_gpu(cfg, kv, tokens, parent)
+        _check_against_oracle(got, ref, tokens, parent)
+        if not ref["decisive"]:
+            pytest.skip("near-tie in the seeded inputs")
+        kv.commit()
+        O.commit(cache, ref)
+        assert kv.length() == cache.length
+        a = got["accept_len"]
+        out += [int(t) for t in tokens[got["path"][1:a + 1]]] + [got["bonus"]]
+        root = got["bonus"]
+        rounds += 1
+    assert out[:total] == want[:total]
+
+
+def test_node_order_does_not_matter_on_gpu():
+    cfg, store, model, kv = _gpu_stack("micro", 2, 0)
+    W, cache, prompt = _fill_both(cfg, store, kv, 17, 4, 2)
+    parent = gen.sparse_tree(30, seed=2)
+    tokens = gen.fill_tree_tokens(parent, cfg.vocab, seed=2, root_token=int(prompt[-1]))
+    a = _verify_gpu(cfg, kv, tokens, parent)
+    p2, t2, old = gen.relabel_tree(parent, tokens, seed=4)
+    b = _verify_gpu(cfg, kv, t2, p2)
+    assert np.abs(b["logits"] - a["logits"][old]).max() < 1e-3
+    assert b["accept_len"] == a["accept_len"]
+
+
+def test_error_paths_leave_state_untouched():
+    from paper_2507_18181_b200 import binding as B
+    cfg, store, model, kv = _gpu_stack("micro", 0, 0, max_tokens=64, max_nodes=32)
+    W, cache, prompt = _fill_both(cfg, store, kv, 20, 3, 0)
+    L = kv.length()
+    dev = "cuda"
+    tok = torch.zeros(8, dtype=torch.int32, device=dev)
+    par = torch.tensor([-1, 0, 1, 2, 3, 4, 5, 6], dtype=torch.int32, device=dev)
+    # host-visible errors
+    with pytest.raises(B.SpecasrError) as e:
+        B.specasr_verify_tree(model.handle, kv.handle, tok.data_ptr(), par.data_ptr(), 0, kv.out_argmax.data_ptr(),
+                              kv.out_accept.data_ptr(), kv.out_path.data_ptr())
+    assert e.value.status == B.SPECASR_ERR_INVALID_ARG
+    with pytest.raises(B.SpecasrError) as e:
+        B.specasr_verify_tree(model.handle, kv.handle, tok.data_ptr(), par.data_ptr(), 33, kv.out_argmax.data_ptr(),
+                              kv.out_accept.data_ptr(), kv.out_path.data_ptr())
+    assert e.value.status == B.SPECASR_ERR_INVALID_ARG
+    with pytest.raises(B.SpecasrError) as e:
+        B.specasr_verify_tree(model.handle, kv.handle, 0, par.data_ptr(), 8, kv.out_argmax.data_ptr(),
+                              kv.out_accept.data_ptr(), kv.out_path.data_ptr())
+    assert e.value.status == B.SPECASR_ERR_INVALID_ARG
+    with pytest.raises(B.SpecasrError) as e:
+        kv.commit()                                     # nothing pending
+    assert e.value.status == B.SPECASR_ERR_STATE
+    # device-visible errors: cycle / forward parent, token out of range
+    for bad_par, bad_tok in (([-1, 0, 3, 2, 1, 1, 1, 1], None), ([0, 0, 1, 2, 3, 4, 5, 6], None),
+                             ([-1, 0, 1, 2, 3, 4, 5, 6], cfg.vocab)):
+        p = torch.tensor(bad_par, dtype=torch.int32, device=dev)
+        t = tok.clone()
+        if bad_tok is not None:
+            t[3] = bad_tok
+        kv.verify(t, p)
+        torch.cuda.synchronize()
+        assert kv.status() == B.SPECASR_ERR_INVALID_TREE
+        assert int(kv.out_accept.item()) == -1 and bool((kv.out_path[:8] == -1).all())
+        kv.commit()                                     # committing a failed verify is a no-op
+        assert kv.length() == L
+    # capacity: 22 committed + 32 tree slots fit in 64, a prefill that does not fit is refused
+    with pytest.raises(B.SpecasrError) as e:
+        kv.prefill_tokens(torch.zeros(60, dtype=torch.int32, device=dev))
+    assert e.value.status == B.SPECASR_ERR_KV_CAPACITY
+    assert kv.length() == L
+    # a good verify still works afterwards and gives the oracle's answer
+    parent = gen.chain_tree(7)
+    tokens = gen.fill_tree_tokens(parent, cfg.vocab, seed=1, root_token=int(prompt[-1]))
+    got = _verify_gpu(cfg, kv, tokens, parent)
+    _check_against_oracle(got, O.verify_tree(cfg, W, cache, tokens, parent), tokens, parent)
+    # abandoning a round: verify twice, commit once
+    kv.truncate(L)
+    assert kv.length() == L
+
+
+def test_single_node_tree_and_max_nodes():
+    cfg, store, model, kv = _gpu_stack("micro", 1, 0, max_tokens=600, max_nodes=256)
+    W, cache, prompt = _fill_both(cfg, store, kv, 10, 2, 1)
+    root = int(prompt[-1])
+    # n = 1: plain autoregressive step
+    got = _verify_gpu(cfg, kv, np.array([root], np.int32), np.array([-1], np.int32))
+    want = O.verify_tree(cfg, W, cache, [root], [-1])
+    _check_against_oracle(got, want, np.array([root]), np.array([-1]))
+    assert got["accept_len"] == 0 and got["path"][0] == 0
+    # n = 256: the largest tree the ancestor bitmask holds
+    parent = gen.sparse_tree(256, seed=1)
+    tokens = gen.fill_tree_tokens(parent, cfg.vocab, seed=1, root_token=root)
+    got = _verify_gpu(cfg, kv, tokens, parent)
+    _check_against_oracle(got, O.verify_tree(cfg, W, cache, tokens, parent), tokens, parent)
