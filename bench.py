@@ -1,0 +1,399 @@
+#!/usr/bin/env python
+"""Benchmark of the tree-verification step (verify + commit) on the 7B-shape, 64-node workload.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload config3]
+
+One step = one pass of the whole hot path: tree prep, embedding, 32 decoder layers over the tree
+(projections, rotary + KV append, tree attention, SwiGLU), vocabulary projection + argmax, accept,
+KV compaction.  Prints ONE JSON line on rank 0.  With --gpus N > 1 (under torchrun) every rank runs
+an independent replica (the path does not shard) and the value is the sum over ranks divided by the
+slowest rank's time.  `--impl reference` times the CPU oracle on a bounded sample instead.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import gen  # noqa: E402
+
+WORKLOADS = {
+    # name: (model, n_audio, n_text (decoded tokens incl. the root), n_nodes, tree kind, page size)
+    "config3": dict(model="7b", n_audio=1500, n_text=201, n_nodes=64, levels=12, chain=False),
+    "config2": dict(model="1b", n_audio=750, n_text=33, n_nodes=9, levels=None, chain=True),
+    "config1": dict(model="tiny", n_audio=64, n_text=8, n_nodes=15, levels=None, chain=False),
+    # config3 cut to two layers: same kernels and launch shapes, small enough for a profiler capture
+    "config3_2layers": dict(model="7b", n_layers=2, n_audio=1500, n_text=201, n_nodes=64, levels=12, chain=False),
+}
+METRIC = "tree_tokens_per_s"
+UNIT = "tree tokens/s"
+
+
+def model_config(wl):
+    over = {"n_layers": wl["n_layers"]} if "n_layers" in wl else {}
+    return gen.get_config(wl["model"], **over)
+
+
+def algorithmic_bytes(cfg, L, n):
+    w = 2 * (cfg.n_layers * (cfg.d_model * (cfg.q_dim + 2 * cfg.kv_dim) + cfg.q_dim * cfg.d_model
+                             + 3 * cfg.d_model * cfg.ffn) + cfg.d_model * cfg.vocab)
+    kv_row = cfg.n_layers * 2 * cfg.n_kv_heads * cfg.head_dim * 4          # K and V, hi + lo bf16 planes
+    return {"weights": w, "kv_read": (L + n) * kv_row, "kv_write": n * kv_row,
+            "total": w + (L + 2 * n) * kv_row}
+
+
+def gemm_weight_bytes(cfg):
+    d, F = cfg.d_model, cfg.ffn
+    return {"gemm_qkv": 2 * d * (cfg.q_dim + 2 * cfg.kv_dim), "gemm_o": 2 * cfg.q_dim * d, "gemm_gu": 4 * d * F,
+            "gemm_down": 2 * d * F, "gemm_lm": 2 * d * cfg.vocab}
+
+
+def algorithmic_flops(cfg, L, n):
+    params = cfg.n_layers * (cfg.d_model * (cfg.q_dim + 2 * cfg.kv_dim) + cfg.q_dim * cfg.d_model
+                             + 3 * cfg.d_model * cfg.ffn) + cfg.d_model * cfg.vocab
+    return 2 * n * params + 4 * n * cfg.q_dim * (L + n) * cfg.n_layers
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+        self.file = None
+
+    def start(self):
+        try:
+            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=self.file, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.file.flush()
+        rows = [r.strip().split(", ") for r in open(self.file.name) if r.strip()]
+        os.unlink(self.file.name)
+        rows = [r for r in rows if len(r) == 6 and r[0].replace(".", "").isdigit()]
+        if rows:
+            out["sm_mhz"] = float(np.median([float(r[0]) for r in rows]))
+            out["sm_max_mhz"] = float(rows[0][1])
+            names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+            out["reasons"] = [nm for j, nm in enumerate(names) if any(r[2 + j].strip() == "Active" for r in rows)]
+            out["samples"] = len(rows)
+        return out
+
+
+# ------------------------------------------------------------------------------------------------ CPU oracle leg
+
+class _DictStore:
+    def __init__(self, layers, glob):
+        self._layers, self._glob = layers, glob
+
+    def layer(self, l):
+        return self._layers[l]
+
+    def globals(self):
+        return self._glob
+
+
+def oracle_sample(wl, seed=1):
+    """Bounded sample of the workload for the CPU oracle: the oracle's own steps of the same verify
+    call (same tree, same KV length, same shapes) run over ONE of the model's layers plus the embedding
+    and vocabulary projection, each part timed; the full call is extrapolated as
+    t_globals + n_layers * t_layer + t_head.  Returns a closure that runs the sample once and returns the
+    extrapolated seconds per full call."""
+    from oracle import specasr_oracle as O
+    cfg_full = model_config(wl)
+    cfg = gen.get_config(wl["model"], n_layers=1)
+    store = gen.WeightStore(cfg_full, seed)
+    layers = [store.layer(0)]
+    glob = store.globals()
+    L = wl["n_audio"] + wl["n_text"] - 1
+    n = wl["n_nodes"]
+    parent = gen.chain_tree(n - 1) if wl["chain"] else gen.sparse_tree(n, seed=seed, levels=wl["levels"])
+    tokens = gen.fill_tree_tokens(parent, cfg_full.vocab, seed=seed, root_token=1)
+    rng = np.random.default_rng(seed)
+    cache = O.KVCache(cfg)
+    cache.K = [rng.standard_normal((L, cfg.n_kv_heads, cfg.head_dim))]
+    cache.V = [rng.standard_normal((L, cfg.n_kv_heads, cfg.head_dim))]
+
+    def run_once():
+        W = O.Weights(_DictStore(layers, glob))          # fresh: nothing widened ahead of the timed call
+        t0 = time.perf_counter()
+        depth, anc = O.tree_prep(parent)
+        x = O.embed(W, tokens)                           # widens embedding, vocabulary matrix, final gain
+        t1 = time.perf_counter()
+        hidden, _, _ = O.decoder_stack(cfg, W, x, cache.length + depth, anc, cache)
+        t2 = time.perf_counter()
+        logits = O.lm_logits(cfg, W, hidden)
+        O.accept(tokens, parent, np.argmax(logits, axis=-1))
+        t3 = time.perf_counter()
+        return (t1 - t0) + cfg_full.n_layers * (t2 - t1) + (t3 - t2)
+
+    desc = (f"oracle steps of verify_tree on the {wl['model']} shape, {n}-node tree, KV length {L} (seeded N(0,1) "
+            f"K/V): embedding + 1 of {cfg_full.n_layers} layers + vocabulary projection + accept, full call = "
+            f"t_embed + {cfg_full.n_layers} * t_layer + t_head")
+    return run_once, desc
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    run_once, desc = oracle_sample(wl)
+    for _ in range(args.warmup):
+        run_once()
+    secs = [run_once() for _ in range(args.steps)]
+    per_call = float(np.mean(secs))
+    n = wl["n_nodes"]
+    cores = len(os.sched_getaffinity(0))
+    value = n / per_call
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_call * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, **{k: v for k, v in wl.items()}},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------ CUDA leg
+
+def build_workload(wl, device, seed=1):
+    import torch
+    from paper_2507_18181_b200 import build as _build
+    from paper_2507_18181_b200.runtime import DeviceModel, DeviceKV
+    _build.build()
+    cfg = model_config(wl)
+    store = gen.WeightStore(cfg, seed)
+    model = DeviceModel(cfg, store, device=device)
+    L = wl["n_audio"] + wl["n_text"] - 1
+    n = wl["n_nodes"]
+    kv = DeviceKV(model, max_tokens=L + n + 64, max_nodes=max(n, 16))
+    audio = gen.audio_prefix(wl["n_audio"], cfg.d_model, seed)
+    text = gen.prompt_tokens(wl["n_text"], cfg.vocab, seed)
+    kv.prefill_embeds(torch.from_numpy(audio).to(device))
+    kv.prefill_tokens(torch.from_numpy(text[:-1].copy()).to(device))
+    assert kv.length() == L
+    root = int(text[-1])
+    parent = gen.chain_tree(n - 1) if wl["chain"] else gen.sparse_tree(n, seed=seed, levels=wl["levels"])
+    # the target's own greedy continuation (input construction: autoregressive single-node rounds)
+    k = len(gen.main_path(parent)) - 1
+    greedy = []
+    tok = root
+    one_p = torch.tensor([-1], dtype=torch.int32, device=device)
+    for _ in range(k):
+        kv.verify(torch.tensor([tok], dtype=torch.int32, device=device), one_p)
+        kv.commit()
+        tok = int(kv.out_bonus.item())
+        greedy.append(tok)
+    kv.truncate(L)
+    tokens = gen.fill_tree_tokens(parent, cfg.vocab, seed=seed, root_token=root, main_tokens=greedy, corrupt_p=0.2)
+    return cfg, model, kv, L, tokens, parent
+
+
+def run_ours(args, wl):
+    import torch
+    from paper_2507_18181_b200 import binding as B
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: there is no CPU fallback for the verification path")
+    device = f"cuda:{local}"
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(device))
+    cfg, model, kv, L, tokens, parent = build_workload(wl, device)
+    n = len(tokens)
+    d_tokens = torch.from_numpy(tokens).to(device)
+    d_parent = torch.from_numpy(parent).to(device)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        kv.verify(d_tokens, d_parent)
+        kv.commit()
+        kv.truncate(L)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    launches0 = kv.launches()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    step_events = []
+    barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        step()
+        b.record(stream)
+        step_events.append((a, b))
+    e1.record(stream)
+    barrier()
+    clocks = sampler.stop() if rank == 0 else {}
+    elapsed_ms = e0.elapsed_time(e1)
+    launches = kv.launches() - launches0
+    per_step = sorted(a.elapsed_time(b) for a, b in step_events)
+    accept_len = int(kv.out_accept.item())
+    if world > 1:
+        t = torch.tensor([elapsed_ms], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+
+    # end to end through the C ABI with host buffers: H2D of the tree, D2H of the results, every step
+    h_tokens = torch.from_numpy(tokens).pin_memory()
+    h_parent = torch.from_numpy(parent).pin_memory()
+    h_out = torch.empty(2 * n + 2, dtype=torch.int32).pin_memory()
+    dd_tokens, dd_parent = torch.empty_like(d_tokens), torch.empty_like(d_parent)
+
+    def e2e_step():
+        dd_tokens.copy_(h_tokens, non_blocking=True)
+        dd_parent.copy_(h_parent, non_blocking=True)
+        kv.verify(dd_tokens, dd_parent)
+        kv.commit()
+        h_out[:n].copy_(kv.out_argmax[:n], non_blocking=True)
+        h_out[n:2 * n].copy_(kv.out_path[:n], non_blocking=True)
+        h_out[2 * n:2 * n + 1].copy_(kv.out_accept, non_blocking=True)
+        h_out[2 * n + 1:].copy_(kv.out_bonus, non_blocking=True)
+        torch.cuda.synchronize()          # the caller needs accept_len and the bonus token to go on
+        kv.truncate(L)
+
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        e2e_step()
+    barrier()
+    e2e_s = time.perf_counter() - t0
+    if world > 1:
+        t = torch.tensor([e2e_s], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # per-kernel times with events around every launch (separate pass, same steps)
+    B.specasr_profile_enable(kv.handle, 1)
+    prof_steps = min(args.steps, 10)
+    for _ in range(prof_steps):
+        step()
+    ms, cnt = B.specasr_profile_read(kv.handle, stream.cuda_stream)
+    B.specasr_profile_enable(kv.handle, 0)
+    kernels = {k: {"launches_per_step": cnt[k] / prof_steps, "ms_per_step": ms[k] / prof_steps} for k in ms if cnt[k]}
+    gb = gemm_weight_bytes(cfg)
+    gemm_bytes_step = cfg.n_layers * (gb["gemm_qkv"] + gb["gemm_o"] + gb["gemm_gu"] + gb["gemm_down"]) + gb["gemm_lm"]
+    gemm_ms_step = sum(ms[k] for k in gb) / prof_steps
+    gemm_launches = sum(cnt[k] for k in gb) / prof_steps
+    peaks = measured_peaks()
+    achieved = gemm_bytes_step / (gemm_ms_step * 1e-3) / 1e9
+    for k in gb:
+        per = gb[k] * (cfg.n_layers if k != "gemm_lm" else 1)
+        kernels[k]["achieved_gbs"] = per / (ms[k] / prof_steps * 1e-3) / 1e9
+
+    ms_per_step = elapsed_ms / args.steps
+    value = world * n * args.steps / (elapsed_ms * 1e-3)
+    ab = algorithmic_bytes(cfg, L, n)
+    fl = algorithmic_flops(cfg, L, n)
+    t_roof_ms = max(ab["total"] / (peaks["hbm_gbs"] * 1e9), fl / (peaks["bf16_tflops"] * 1e12)) * 1e3
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, **wl, "kv_len": L, "page_size": model.page_size,
+                   "kv_storage": "bf16 hi+lo planes (4 bytes/element)", "l2": "inputs larger than L2 (weights "
+                   f"{ab['weights'] / 1e9:.2f} GB per step)", "parallelism": "replicas" if world > 1 else "single"},
+        "latency_ms": {"mean": ms_per_step, "median": per_step[len(per_step) // 2], "min": per_step[0]},
+        "accept_len": accept_len, "accepted_tokens_per_s": world * (accept_len + 1) * args.steps / (elapsed_ms * 1e-3),
+        "step_roofline": {"algorithmic_bytes": ab["total"], "algorithmic_flops": fl, "roof_ms": t_roof_ms,
+                          "frac_of_" + peaks["source"]: t_roof_ms / ms_per_step,
+                          "frac_of_nominal_8TBs": (ab["total"] / 8e12 * 1e3) / ms_per_step},
+        "roofline": {"kernel": "k_gemm_tc (all projections)", "bound": "hbm", "achieved": achieved,
+                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                     "peak_source": peaks["source"], "traffic": None,
+                     "algorithmic_bytes_per_launch": gemm_bytes_step / gemm_launches,
+                     "avg_launch_ms": gemm_ms_step / gemm_launches},
+        "kernels": kernels,
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "e2e": {"value": world * n * args.steps / e2e_s, "unit": UNIT, "ms_per_step": e2e_s / args.steps * 1e3,
+                "h2d_bytes_per_step": int(2 * n * 4), "d2h_bytes_per_step": int((2 * n + 2) * 4)},
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        run_once, desc = oracle_sample(wl)
+        run_once()
+        reps, t_start, secs = 0, time.perf_counter(), []
+        while reps < 3 and time.perf_counter() - t_start < 25:
+            secs.append(run_once())
+            reps += 1
+        per_call = float(np.mean(secs))
+        line["cpu_baseline"] = {"value": n / per_call, "unit": UNIT, "cores": len(os.sched_getaffinity(0)),
+                                "kind": "oracle", "sample": desc, "ms_per_step": per_call * 1e3}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="config3", choices=sorted(WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    wl = WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()

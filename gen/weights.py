@@ -12,6 +12,7 @@ and a gain of exactly one would hide a missing multiply).
 """
 from concurrent.futures import ThreadPoolExecutor
 import os
+import threading
 
 import numpy as np
 
@@ -19,6 +20,16 @@ from .bf16 import f32_to_bf16_bits
 from .configs import ModelConfig
 
 _STREAM_WEIGHTS = 0x5EC0
+_scratch = threading.local()
+
+
+def _scratch_f32(n: int) -> np.ndarray:
+    """Per-thread reusable fp32 buffer: large draws do not pay for fresh pages every time."""
+    buf = getattr(_scratch, "buf", None)
+    if buf is None or buf.size < n:
+        buf = np.empty(n, dtype=np.float32)
+        _scratch.buf = buf
+    return buf[:n]
 
 # name -> (code, shape function)
 LAYER_TENSORS = {
@@ -55,20 +66,22 @@ class WeightStore:
         table = GLOBAL_TENSORS if layer < 0 else LAYER_TENSORS
         code, shape_fn = table[name]
         shape = shape_fn(self.cfg)
-        z = self._rng(layer, code).standard_normal(shape, dtype=np.float32)
         if len(shape) == 1:
+            z = self._rng(layer, code).standard_normal(shape, dtype=np.float32)
             z *= np.float32(0.02)
             z += np.float32(1.0)
             return z
+        z = _scratch_f32(int(np.prod(shape))).reshape(shape)
+        self._rng(layer, code).standard_normal(dtype=np.float32, out=z)
         z *= np.float32(0.02)
-        return z
+        return z          # view of the thread's scratch buffer: consume before the next draw
 
     def tensor(self, layer: int, name: str) -> np.ndarray:
         """Matrix: uint16 bf16 bit patterns (or fp32 if round_bf16=False).  Gain vector: fp32.
         `layer` = -1 addresses the global tensors (embed, lm_head, g_final)."""
         z = self._draw(layer, name)
-        if z.ndim == 2 and self.round_bf16:
-            return f32_to_bf16_bits(z)
+        if z.ndim == 2:
+            return f32_to_bf16_bits(z) if self.round_bf16 else z.copy()
         return z
 
     def layer(self, layer: int) -> dict:

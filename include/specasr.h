@@ -170,6 +170,31 @@ specasr_status specasr_poll_status(specasr_kv* kv, int32_t* out_device_status, v
 /* Number of kernels the library has launched on this handle so far (for launch accounting). */
 int64_t specasr_launch_count(const specasr_kv* kv);
 
+/*
+ * Optional per-kernel timing for measurement (no counterpart in the paper, which reports only
+ * end-to-end latencies, Table 2).  While enabled, every kernel launch on this handle is bracketed by
+ * CUDA events on the launching stream.  specasr_profile_read synchronises `stream`, returns the
+ * milliseconds and launch counts accumulated per kernel kind since the last read (both [host] arrays
+ * of SPECASR_KIND_COUNT entries) and clears them.  Leave it disabled when timing whole calls.
+ */
+enum {
+  SPECASR_KIND_PREP = 0,        /* tree / chain preparation, layer-0 inputs */
+  SPECASR_KIND_NORM = 1,        /* RMSNorm + residual + operand split */
+  SPECASR_KIND_GEMM_QKV = 2,
+  SPECASR_KIND_ROPE = 3,        /* rotary embedding + KV append */
+  SPECASR_KIND_ATTN = 4,        /* tree-masked attention */
+  SPECASR_KIND_ATTN_MERGE = 5,
+  SPECASR_KIND_GEMM_O = 6,
+  SPECASR_KIND_GEMM_GU = 7,     /* gate/up projection + SwiGLU */
+  SPECASR_KIND_GEMM_DOWN = 8,
+  SPECASR_KIND_GEMM_LM = 9,     /* vocabulary projection + argmax */
+  SPECASR_KIND_ACCEPT = 10,
+  SPECASR_KIND_COMMIT = 11,     /* KV compaction and length bookkeeping */
+  SPECASR_KIND_COUNT = 12
+};
+specasr_status specasr_profile_enable(specasr_kv* kv, int32_t enable);
+specasr_status specasr_profile_read(specasr_kv* kv, double* out_ms, int64_t* out_launches, void* stream);
+
 const char* specasr_last_error(void);
 
 #ifdef __cplusplus

@@ -20,7 +20,10 @@ EXPORTS = [
     "specasr_kv_create", "specasr_kv_destroy", "specasr_kv_length", "specasr_kv_truncate",
     "specasr_prefill_embeds", "specasr_prefill_tokens", "specasr_verify_tree", "specasr_verify_tree_ex",
     "specasr_commit_kv", "specasr_poll_status", "specasr_launch_count", "specasr_last_error",
+    "specasr_profile_enable", "specasr_profile_read",
 ]
+KIND_NAMES = ["prep", "norm", "gemm_qkv", "rope", "attn", "attn_merge", "gemm_o", "gemm_gu", "gemm_down", "gemm_lm",
+              "accept", "commit"]
 
 
 class ModelConfig(C.Structure):
@@ -77,6 +80,10 @@ def lib() -> C.CDLL:
         L.specasr_poll_status.restype = st
         L.specasr_launch_count.argtypes = [vp]
         L.specasr_launch_count.restype = C.c_int64
+        L.specasr_profile_enable.argtypes = [vp, i32]
+        L.specasr_profile_enable.restype = st
+        L.specasr_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64), vp]
+        L.specasr_profile_read.restype = st
         L.specasr_last_error.argtypes = []
         L.specasr_last_error.restype = C.c_char_p
         _lib = L
@@ -171,3 +178,16 @@ def specasr_poll_status(kv: int, stream: int = 0) -> int:
 
 def specasr_launch_count(kv: int) -> int:
     return lib().specasr_launch_count(kv)
+
+
+def specasr_profile_enable(kv: int, enable: int) -> None:
+    _check(lib().specasr_profile_enable(kv, enable))
+
+
+def specasr_profile_read(kv: int, stream: int = 0):
+    """Returns ({kind name: ms}, {kind name: launches}) accumulated since the last read."""
+    n = len(KIND_NAMES)
+    ms = (C.c_double * n)()
+    cnt = (C.c_int64 * n)()
+    _check(lib().specasr_profile_read(kv, ms, cnt, stream))
+    return dict(zip(KIND_NAMES, list(ms))), dict(zip(KIND_NAMES, list(cnt)))

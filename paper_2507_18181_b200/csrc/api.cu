@@ -222,6 +222,8 @@ extern "C" specasr_status specasr_kv_create(const specasr_model* m, void* k_pool
   kv->pinned = nullptr;
   kv->len_event_pending = false;
   kv->launches = 0;
+  kv->prof_on = false;
+  kv->prof_used = 0;
   cudaError_t e = cudaHostAlloc(&kv->pinned, 4 * sizeof(int32_t), cudaHostAllocDefault);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&kv->len_event, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaMemset(kv->ws.ctl, 0, sizeof(int32_t) * kCtlWords);
@@ -254,12 +256,43 @@ extern "C" specasr_status specasr_kv_create(const specasr_model* m, void* k_pool
 extern "C" void specasr_kv_destroy(specasr_kv* kv) {
   if (!kv) return;
   if (kv->len_event_pending) cudaEventSynchronize(kv->len_event);
+  for (cudaEvent_t e : kv->prof_events) cudaEventDestroy(e);
   cudaEventDestroy(kv->len_event);
   if (kv->pinned) cudaFreeHost(kv->pinned);
   delete kv;
 }
 
 extern "C" int64_t specasr_launch_count(const specasr_kv* kv) { return kv ? kv->launches : 0; }
+
+extern "C" specasr_status specasr_profile_enable(specasr_kv* kv, int32_t enable) {
+  if (!kv) {
+    set_error("specasr_profile_enable: null handle");
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  kv->prof_on = enable != 0;
+  kv->prof_used = 0;
+  return SPECASR_OK;
+}
+
+extern "C" specasr_status specasr_profile_read(specasr_kv* kv, double* out_ms, int64_t* out_launches, void* stream) {
+  if (!kv || !out_ms || !out_launches) {
+    set_error("specasr_profile_read: null argument");
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+  for (int k = 0; k < SPECASR_KIND_COUNT; ++k) {
+    out_ms[k] = 0.0;
+    out_launches[k] = 0;
+  }
+  for (size_t i = 0; i < kv->prof_used; ++i) {
+    float ms = 0.f;
+    CUDA_TRY(cudaEventElapsedTime(&ms, kv->prof_events[2 * i], kv->prof_events[2 * i + 1]));
+    out_ms[kv->prof_kinds[i]] += ms;
+    out_launches[kv->prof_kinds[i]] += 1;
+  }
+  kv->prof_used = 0;
+  return SPECASR_OK;
+}
 
 // The host learns the committed length lazily: a commit enqueues a copy of the device length word
 // into pinned memory followed by an event.
@@ -317,12 +350,12 @@ extern "C" specasr_status specasr_poll_status(specasr_kv* kv, int32_t* out_devic
 }
 
 // ------------------------------------------------------------------------------------------------
-static void run_gemm(specasr_kv* kv, GemmArgs& a, cudaStream_t s) {
+static void run_gemm(specasr_kv* kv, GemmArgs& a, int kind, cudaStream_t s) {
   if (kv->m->cfg.gemm_path == 1) {
     a.splits = 1;
-    launch_gemm_fma(kv, a, s);
+    launch_gemm_fma(kv, a, kind, s);
   } else {
-    launch_gemm_tc(kv, a, s);
+    launch_gemm_tc(kv, a, kind, s);
   }
 }
 
@@ -358,29 +391,29 @@ static void run_stack(specasr_model* m, specasr_kv* kv, int n, bool want_head, f
     a.W = m->wqkv[l]; a.tmW = tc ? &m->tm_wqkv[l] : nullptr; a.tmAct = kv->tm_H; a.act = kv->ws.H;
     a.M = m->qkv_dim; a.K = c.d_model; a.epilogue = EPI_PARTIAL; a.P = kv->ws.P;
     a.splits = tc ? gemm_tc_pick_splits(m, a.M, a.K) : 1;
-    run_gemm(kv, a, s);
+    run_gemm(kv, a, SPECASR_KIND_GEMM_QKV, s);
     launch_rope_append(kv, l, n, a.splits, s);
     launch_tree_attention(kv, l, n, att_splits, s);
     launch_attn_merge(kv, n, n_pad, att_splits, s);
     a.W = m->wo[l]; a.tmW = tc ? &m->tm_wo[l] : nullptr; a.tmAct = kv->tm_AO; a.act = kv->ws.AO;
     a.M = c.d_model; a.K = m->q_dim; a.epilogue = EPI_PARTIAL;
     a.splits = tc ? gemm_tc_pick_splits(m, a.M, a.K) : 1;
-    run_gemm(kv, a, s);
+    run_gemm(kv, a, SPECASR_KIND_GEMM_O, s);
     launch_rmsnorm_split(kv, m->g_ffn[l], n, n_pad, a.splits, s);
     a.W = m->wgu[l]; a.tmW = tc ? &m->tm_wgu[l] : nullptr; a.tmAct = kv->tm_H; a.act = kv->ws.H;
     a.M = 2 * c.ffn; a.K = c.d_model; a.epilogue = EPI_SWIGLU; a.A = kv->ws.A; a.splits = 1;
-    run_gemm(kv, a, s);
+    run_gemm(kv, a, SPECASR_KIND_GEMM_GU, s);
     a.W = m->wd[l]; a.tmW = tc ? &m->tm_wd[l] : nullptr; a.tmAct = kv->tm_A; a.act = kv->ws.A;
     a.M = c.d_model; a.K = c.ffn; a.epilogue = EPI_PARTIAL;
     a.splits = tc ? gemm_tc_pick_splits(m, a.M, a.K) : 1;
-    run_gemm(kv, a, s);
+    run_gemm(kv, a, SPECASR_KIND_GEMM_DOWN, s);
     down_splits = a.splits;
   }
   if (!want_head) return;   // context fill: K/V of every layer are written, the last FFN output is not needed
   launch_rmsnorm_split(kv, m->g_final, n, n_pad, down_splits, s);
   a.W = m->lm_head; a.tmW = tc ? &m->tm_lm : nullptr; a.tmAct = kv->tm_H; a.act = kv->ws.H;
   a.M = c.vocab; a.K = c.d_model; a.epilogue = EPI_ARGMAX; a.amax = kv->ws.amax; a.logits = out_logits; a.splits = 1;
-  run_gemm(kv, a, s);
+  run_gemm(kv, a, SPECASR_KIND_GEMM_LM, s);
 }
 
 static specasr_status prefill_common(specasr_model* m, specasr_kv* kv, const float* embeds, const int32_t* tokens,

@@ -183,11 +183,11 @@ void launch_dh(specasr_kv* kv, int layer, int n, int n_splits, cudaStream_t s) {
   }
   dim3 grid(c.n_kv_heads, (n * group + ROWS - 1) / ROWS, n_splits);
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
+  LaunchScope scope(kv, SPECASR_KIND_ATTN, s);
   k_tree_attention<DH><<<grid, 256, smem, s>>>(kv->ws.ctl, kv->ws.Q, (size_t)kv->n_alloc * m->q_dim, kv->k_pool,
                                                kv->v_pool, kv->page_table, kv->n_pages, c.page_size, layer,
                                                c.n_heads, c.n_kv_heads, n, kv->ws.anc, n_splits, scale_log2,
                                                kv->ws.attO, kv->ws.attML, (size_t)kv->n_alloc * c.n_heads);
-  kv->launches++;
 }
 }  // namespace
 

@@ -106,10 +106,10 @@ __global__ void __launch_bounds__(256) k_gemm_fma(GemmArgs a) {
 
 int gemm_fma_tiles(int M) { return (M + BM - 1) / BM; }
 
-void launch_gemm_fma(specasr_kv* kv, const GemmArgs& a, cudaStream_t s) {
+void launch_gemm_fma(specasr_kv* kv, const GemmArgs& a, int kind, cudaStream_t s) {
+  LaunchScope scope(kv, kind, s);
   dim3 grid((a.M + BM - 1) / BM, (a.n + BN - 1) / BN);
   if (a.epilogue == EPI_PARTIAL) k_gemm_fma<EPI_PARTIAL><<<grid, 256, 0, s>>>(a);
   else if (a.epilogue == EPI_SWIGLU) k_gemm_fma<EPI_SWIGLU><<<grid, 256, 0, s>>>(a);
   else k_gemm_fma<EPI_ARGMAX><<<grid, 256, 0, s>>>(a);
-  kv->launches++;
 }

@@ -378,7 +378,7 @@ int gemm_tc_pick_splits(const specasr_model* m, int M, int K) {
   return s;
 }
 
-void launch_gemm_tc(specasr_kv* kv, const GemmArgs& a, cudaStream_t s) {
+void launch_gemm_tc(specasr_kv* kv, const GemmArgs& a, int kind, cudaStream_t s) {
   TcParams p;
   p.M = a.M; p.K = a.K; p.n = a.n; p.n_pad = a.n_pad; p.n_alloc = a.n_alloc;
   p.box_rows = pick_box_rows(a.n_pad);
@@ -406,8 +406,8 @@ void launch_gemm_tc(specasr_kv* kv, const GemmArgs& a, cudaStream_t s) {
   for (int b = 16; b < p.box_rows; b <<= 1) ++idx;
   act = &a.tmAct[idx];
   dim3 grid(gemm_tc_tiles(a.M), p.splits);
+  LaunchScope scope(kv, kind, s);
   if (a.epilogue == EPI_PARTIAL) k_gemm_tc<EPI_PARTIAL><<<grid, 192, smem, s>>>(*a.tmW, *act, p);
   else if (a.epilogue == EPI_SWIGLU) k_gemm_tc<EPI_SWIGLU><<<grid, 192, smem, s>>>(*a.tmW, *act, p);
   else k_gemm_tc<EPI_ARGMAX><<<grid, 192, smem, s>>>(*a.tmW, *act, p);
-  kv->launches++;
 }

@@ -76,9 +76,39 @@ struct specasr_kv {
   cudaEvent_t len_event;
   bool len_event_pending;
   int64_t launches;
+  // optional per-kernel timing (specasr_profile_*): event pairs recorded around every launch
+  bool prof_on;
+  std::vector<cudaEvent_t> prof_events;   // 2 per recorded launch
+  std::vector<int> prof_kinds;
+  size_t prof_used;                       // launches recorded since the last read
   // activation TMA descriptors (tcgen05 path)
   // activation TMA descriptors (tcgen05 path), one per box height 16 << i
   CUtensorMap tm_H[5], tm_AO[5], tm_A[5];
+};
+
+// Counts a launch and, when profiling is on, brackets it with events on the launching stream.
+struct LaunchScope {
+  specasr_kv* kv;
+  cudaStream_t s;
+  LaunchScope(specasr_kv* kv_, int kind, cudaStream_t s_) : kv(kv_), s(s_) {
+    kv->launches++;
+    if (!kv->prof_on) return;
+    if (kv->prof_events.size() < 2 * (kv->prof_used + 1)) {
+      cudaEvent_t a, b;
+      cudaEventCreate(&a);
+      cudaEventCreate(&b);
+      kv->prof_events.push_back(a);
+      kv->prof_events.push_back(b);
+      kv->prof_kinds.push_back(kind);
+    }
+    kv->prof_kinds[kv->prof_used] = kind;
+    cudaEventRecord(kv->prof_events[2 * kv->prof_used], s);
+  }
+  ~LaunchScope() {
+    if (!kv->prof_on) return;
+    cudaEventRecord(kv->prof_events[2 * kv->prof_used + 1], s);
+    kv->prof_used++;
+  }
 };
 
 void set_error(const char* fmt, ...);
@@ -120,10 +150,10 @@ struct GemmArgs {
   const int32_t* ctl;
 };
 int gemm_fma_tiles(int M);
-void launch_gemm_fma(specasr_kv* kv, const GemmArgs& a, cudaStream_t s);
+void launch_gemm_fma(specasr_kv* kv, const GemmArgs& a, int kind, cudaStream_t s);
 int gemm_tc_tiles(int M);
 int gemm_tc_pick_splits(const specasr_model* m, int M, int K);
-void launch_gemm_tc(specasr_kv* kv, const GemmArgs& a, cudaStream_t s);
+void launch_gemm_tc(specasr_kv* kv, const GemmArgs& a, int kind, cudaStream_t s);
 bool make_tensor_map_2d(CUtensorMap* out, const void* base, uint64_t inner, uint64_t outer,
                         uint32_t box_inner, uint32_t box_outer);
 bool make_act_map(CUtensorMap* out, const void* base, uint64_t K, uint64_t n_alloc, uint32_t box_rows);

@@ -80,17 +80,17 @@ void launch_tree_prep(specasr_kv* kv, const int32_t* tokens, const int32_t* pare
   const specasr_model* m = kv->m;
   int cap = kv->max_pages * m->cfg.page_size;
   if (m->cfg.max_positions < cap) cap = m->cfg.max_positions;
+  LaunchScope scope(kv, SPECASR_KIND_PREP, s);
   k_tree_prep<<<1, 256, 0, s>>>(kv->ws.ctl, tokens, parent, n, m->cfg.vocab, cap, kv->ws.depth, kv->ws.pos,
                                 kv->ws.anc);
-  kv->launches++;
 }
 
 void launch_chain_prep(specasr_kv* kv, int n, cudaStream_t s) {
   const specasr_model* m = kv->m;
   int cap = kv->max_pages * m->cfg.page_size;
   if (m->cfg.max_positions < cap) cap = m->cfg.max_positions;
+  LaunchScope scope(kv, SPECASR_KIND_PREP, s);
   k_chain_prep<<<1, 256, 0, s>>>(kv->ws.ctl, n, cap, kv->ws.depth, kv->ws.pos, kv->ws.anc);
-  kv->launches++;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -123,13 +123,13 @@ __global__ void k_copy_embeds(const int32_t* __restrict__ ctl, const float* __re
 }
 
 void launch_embed_tokens(specasr_kv* kv, const int32_t* tokens, int n, cudaStream_t s) {
+  LaunchScope scope(kv, SPECASR_KIND_PREP, s);
   k_embed_tokens<<<n, 128, 0, s>>>(kv->ws.ctl, tokens, kv->m->embed, kv->m->cfg.d_model, kv->ws.X);
-  kv->launches++;
 }
 
 void launch_copy_embeds(specasr_kv* kv, const float* embeds, int n, cudaStream_t s) {
+  LaunchScope scope(kv, SPECASR_KIND_PREP, s);
   k_copy_embeds<<<n, 128, 0, s>>>(kv->ws.ctl, embeds, kv->m->cfg.d_model, kv->ws.X);
-  kv->launches++;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -181,9 +181,9 @@ __global__ void __launch_bounds__(256) k_rmsnorm_split(const int32_t* __restrict
 void launch_rmsnorm_split(specasr_kv* kv, const float* gain, int n, int n_pad, int n_partials, cudaStream_t s) {
   const specasr_model* m = kv->m;
   const int d = m->cfg.d_model;
+  LaunchScope scope(kv, SPECASR_KIND_NORM, s);
   k_rmsnorm_split<<<n_pad, 256, 0, s>>>(kv->ws.ctl, kv->ws.X, kv->ws.P, n_partials, (size_t)kv->n_alloc * d, gain,
                                         d, m->cfg.rms_eps, n, (size_t)kv->n_alloc * d, kv->ws.H);
-  kv->launches++;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -246,11 +246,11 @@ void launch_rope_append(specasr_kv* kv, int layer, int n, int n_partials, cudaSt
   const specasr_model_config& c = m->cfg;
   dim3 grid(n, c.n_heads + 2 * c.n_kv_heads);
   const int threads = c.head_dim / 2 < 32 ? 32 : c.head_dim / 2;
+  LaunchScope scope(kv, SPECASR_KIND_ROPE, s);
   k_rope_append<<<grid, threads, 0, s>>>(kv->ws.ctl, kv->ws.P, n_partials, (size_t)kv->n_alloc * m->qkv_dim,
                                          m->qkv_dim, c.n_heads, c.n_kv_heads, c.head_dim, kv->ws.pos,
                                          m->rope_table, layer, kv->ws.Q, (size_t)kv->n_alloc * m->q_dim,
                                          kv->k_pool, kv->v_pool, kv->page_table, kv->n_pages, c.page_size);
-  kv->launches++;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -293,10 +293,10 @@ void launch_attn_merge(specasr_kv* kv, int n, int n_pad, int n_splits, cudaStrea
   const specasr_model_config& c = kv->m->cfg;
   dim3 grid(n_pad, c.n_heads);
   const int threads = c.head_dim < 32 ? 32 : c.head_dim;
+  LaunchScope scope(kv, SPECASR_KIND_ATTN_MERGE, s);
   k_attn_merge<<<grid, threads, 0, s>>>(kv->ws.ctl, kv->ws.attO, kv->ws.attML, n_splits,
                                         (size_t)kv->n_alloc * c.n_heads, c.n_heads, c.head_dim, n, kv->ws.AO,
                                         (size_t)kv->n_alloc * kv->m->q_dim);
-  kv->launches++;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -365,9 +365,9 @@ __global__ void __launch_bounds__(256) k_accept(const int32_t* __restrict__ ctl,
 void launch_accept(specasr_kv* kv, const int32_t* tokens, const int32_t* parent, int n, int n_tiles,
                    int32_t* out_argmax, int32_t* out_accept_len, int32_t* out_path, int32_t* out_bonus,
                    cudaStream_t s) {
+  LaunchScope scope(kv, SPECASR_KIND_ACCEPT, s);
   k_accept<<<1, 256, 0, s>>>(kv->ws.ctl, kv->ws.amax, n_tiles, kv->n_alloc, tokens, parent, kv->ws.depth, n,
                              out_argmax, out_accept_len, out_path, out_bonus);
-  kv->launches++;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -382,12 +382,12 @@ __global__ void k_set_len(int32_t* ctl, int len) {
   ctl[CTL_N] = 0;
 }
 void launch_advance_len(specasr_kv* kv, int n, cudaStream_t s) {
+  LaunchScope scope(kv, SPECASR_KIND_COMMIT, s);
   k_advance_len<<<1, 1, 0, s>>>(kv->ws.ctl, n);
-  kv->launches++;
 }
 void launch_set_len(specasr_kv* kv, int len, cudaStream_t s) {
+  LaunchScope scope(kv, SPECASR_KIND_COMMIT, s);
   k_set_len<<<1, 1, 0, s>>>(kv->ws.ctl, len);
-  kv->launches++;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -437,8 +437,9 @@ __global__ void k_commit_finish(int32_t* ctl, const int32_t* __restrict__ accept
 void launch_commit(specasr_kv* kv, const int32_t* path, const int32_t* accept_len, cudaStream_t s) {
   const specasr_model_config& c = kv->m->cfg;
   dim3 grid(c.n_layers, 2);
+  LaunchScope scope(kv, SPECASR_KIND_COMMIT, s);
   k_commit<<<grid, 256, 0, s>>>(kv->ws.ctl, path, accept_len, kv->k_pool, kv->v_pool, kv->page_table, kv->n_pages,
                                 c.n_kv_heads, c.page_size, c.head_dim);
   k_commit_finish<<<1, 1, 0, s>>>(kv->ws.ctl, accept_len);
-  kv->launches += 2;
+  kv->launches++;
 }
