@@ -224,6 +224,7 @@ extern "C" specasr_status specasr_kv_create(const specasr_model* m, void* k_pool
   kv->launches = 0;
   kv->prof_on = false;
   kv->prof_used = 0;
+  kv->attn_tc = false;
   cudaError_t e = cudaHostAlloc(&kv->pinned, 4 * sizeof(int32_t), cudaHostAllocDefault);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&kv->len_event, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaMemset(kv->ws.ctl, 0, sizeof(int32_t) * kCtlWords);
@@ -242,6 +243,8 @@ extern "C" specasr_status specasr_kv_create(const specasr_model* m, void* k_pool
            make_act_map(&kv->tm_AO[i], kv->ws.AO, m->q_dim, kv->n_alloc, b) &&
            make_act_map(&kv->tm_A[i], kv->ws.A, c.ffn, kv->n_alloc, b);
     }
+    kv->attn_tc = ok && attention_tc_supported(m);
+    if (kv->attn_tc) ok = attention_tc_make_maps(kv);
     if (!ok) {
       cudaFreeHost(kv->pinned);
       cudaEventDestroy(kv->len_event);
@@ -359,8 +362,16 @@ static void run_gemm(specasr_kv* kv, GemmArgs& a, int kind, cudaStream_t s) {
   }
 }
 
-static int attention_splits(const specasr_kv* kv, int n, int len_upper) {
+static int attention_splits(const specasr_kv* kv, int n, int len_upper, bool* use_tc) {
   const specasr_model_config& c = kv->m->cfg;
+  *use_tc = false;
+  if (kv->attn_tc) {
+    const int s = attention_tc_splits(len_upper + n);
+    if (s <= kMaxAttnSplits) {
+      *use_tc = true;
+      return s;
+    }
+  }
   const int group = c.n_heads / c.n_kv_heads;
   const int row_tiles = (n * group + 63) / 64;
   const int ctas = c.n_kv_heads * row_tiles;
@@ -377,7 +388,8 @@ static int attention_splits(const specasr_kv* kv, int n, int len_upper) {
 static void run_stack(specasr_model* m, specasr_kv* kv, int n, bool want_head, float* out_logits, cudaStream_t s) {
   const specasr_model_config& c = m->cfg;
   const int n_pad = round_up(n, 16);
-  const int att_splits = attention_splits(kv, n, kv->len_upper);
+  bool att_tc = false;
+  const int att_splits = attention_splits(kv, n, kv->len_upper, &att_tc);
   const bool tc = c.gemm_path == 0;
   int down_splits = 0;
   GemmArgs a;
@@ -393,7 +405,8 @@ static void run_stack(specasr_model* m, specasr_kv* kv, int n, bool want_head, f
     a.splits = tc ? gemm_tc_pick_splits(m, a.M, a.K) : 1;
     run_gemm(kv, a, SPECASR_KIND_GEMM_QKV, s);
     launch_rope_append(kv, l, n, a.splits, s);
-    launch_tree_attention(kv, l, n, att_splits, s);
+    if (att_tc) launch_tree_attention_tc(kv, l, n, att_splits, s);
+    else launch_tree_attention(kv, l, n, att_splits, s);
     launch_attn_merge(kv, n, n_pad, att_splits, s);
     a.W = m->wo[l]; a.tmW = tc ? &m->tm_wo[l] : nullptr; a.tmAct = kv->tm_AO; a.act = kv->ws.AO;
     a.M = c.d_model; a.K = m->q_dim; a.epilogue = EPI_PARTIAL;

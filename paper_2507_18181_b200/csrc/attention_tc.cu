@@ -1,0 +1,338 @@
+// Tree-masked grouped-query attention on the 5th-generation tensor cores (sm_100a).
+//
+// Node i sees every committed cache position [0, L) and the tree slots L + j for which j is i or an
+// ancestor of i (bit j of the node's ancestor mask): the 2-D mask of a draft token tree.
+//
+// One CTA owns one KV head, a tile of up to 128 query rows (row = node * group + head-in-group, so a
+// whole query group shares every K/V element that is staged) and one block of 128 cache positions:
+//   S = Q K^T      M = 128 rows, N = keys, K = head_dim        (both operands K-major)
+//   P = exp2(S * scale - rowmax), masked                         (one thread per row, fp32, from TMEM)
+//   O = P V        M = 128 rows, N = head_dim, K = keys          (V is the MN-major B operand)
+// Q, P, K and V are all carried as two bf16 planes (value ~ hi + lo); each product is three MMAs
+// (hi*hi + hi*lo + lo*hi) into the same fp32 accumulator, which keeps ~16 significant bits.
+// Pages of K and V arrive by TMA straight from the paged pool (one box per page, plane and 64-wide
+// half of the head), Q by one box per plane and half.  The CTA emits an unnormalised partial
+// (row max in log2 units, row sum, output) that k_attn_merge combines over the key blocks.
+//
+// Every mbarrier wait is bounded; on expiry the CTA records SPECASR_ERR_TIMEOUT, lets copies in
+// flight land, frees its TMEM and returns.
+#include "internal.h"
+#include "device_utils.cuh"
+#include "sm100_ptx.cuh"
+
+using namespace sm100;
+
+namespace {
+
+constexpr int KEYS = 128;                 // cache positions per CTA
+constexpr int SUB = 128 * 64 * 2;         // bytes of one [128 rows][64 bf16] swizzled sub-tile
+
+struct AttnCtl {
+  unsigned long long bar_qk, bar_v, bar_s, bar_p, bar_o;
+  uint32_t tmem_base;
+  int abort;
+};
+
+struct AttnParams {
+  int32_t* ctl;
+  const int32_t* page_table;
+  const unsigned long long* anc;
+  float* attO;
+  float2* attML;
+  size_t rows_alloc;      // n_alloc * Hq
+  int n_pages, page_size, layer, Hq, Hkv, group, nodes_per_tile, n;
+  float scale_log2;
+};
+
+template <int DH>
+__global__ void __launch_bounds__(192, 1) k_tree_attention_tc(const __grid_constant__ CUtensorMap tmQ,
+                                                              const __grid_constant__ CUtensorMap tmK,
+                                                              const __grid_constant__ CUtensorMap tmV, AttnParams p) {
+  constexpr int H = DH / 64;                               // 64-wide halves of the head
+  constexpr int A_BYTES = 2 * H * SUB < 4 * SUB ? 4 * SUB : 2 * H * SUB;   // Q planes, later the P planes
+  constexpr int KV_BYTES = 2 * H * SUB;
+  extern __shared__ uint8_t smem_raw[];
+  if (p.ctl[CTL_STATUS] != 0) return;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int kvh = blockIdx.x, split = blockIdx.z;
+  const int node0 = blockIdx.y * p.nodes_per_tile;
+  const int rows_used = p.nodes_per_tile * p.group;
+  const int L = p.ctl[CTL_LEN];
+  const int Ltot = L + p.n;
+  const int k_begin = split * KEYS;
+
+  // row owned by an epilogue thread (warps 2..5): TMEM lane = 32 * (warp % 4) + lane
+  const int r = ((warp & 3) << 5) | lane;
+  const int node = node0 + r / p.group;
+  const bool row_valid = warp >= 2 && r < rows_used && node < p.n;
+  const size_t out_row = (size_t)split * p.rows_alloc + (size_t)node * p.Hq + kvh * p.group + r % p.group;
+
+  if (k_begin >= Ltot) {             // this key block lies beyond the cache: an empty partial
+    if (row_valid) p.attML[out_row] = make_float2(-INFINITY, 0.f);
+    return;
+  }
+  const int kc = min(KEYS, Ltot - k_begin);
+  const int kc_pad = (kc + 15) & ~15;
+  const int pages = (kc + p.page_size - 1) / p.page_size;
+
+  uint8_t* As = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint8_t* Ks = As + A_BYTES;
+  uint8_t* Vs = Ks + KV_BYTES;
+  AttnCtl* sc = (AttnCtl*)(Vs + KV_BYTES);
+
+  if (threadIdx.x == 0) {
+    mbar_init(&sc->bar_qk, 1);
+    mbar_init(&sc->bar_v, 1);
+    mbar_init(&sc->bar_s, 1);
+    mbar_init(&sc->bar_p, 128);
+    mbar_init(&sc->bar_o, 1);
+    sc->abort = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&tmQ);
+    tma_prefetch_desc(&tmK);
+    tma_prefetch_desc(&tmV);
+  }
+  if (rows_used < 128) {             // query rows the TMA box does not cover must not hold garbage
+    const int chunks = (128 - rows_used) * 8;
+    for (int sub = 0; sub < 2 * H; ++sub)
+      for (int i = threadIdx.x; i < chunks; i += blockDim.x)
+        *reinterpret_cast<uint4*>(As + sub * SUB + rows_used * 128 + i * 16) = make_uint4(0, 0, 0, 0);
+    fence_proxy_async_smem();
+  }
+  if (warp == 1) tmem_alloc(&sc->tmem_base, 256);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_s = sc->tmem_base;           // S: columns [0, 128)
+  const uint32_t tmem_o = sc->tmem_base + 128;     // O: columns [128, 128 + DH)
+  volatile int* abort = &sc->abort;
+  int32_t* status = p.ctl + CTL_STATUS;
+
+  if (warp == 0) {
+    // ---------------- TMA producer: lane 0 fetches Q, lane j fetches page j of K and of V
+    const uint32_t q_bytes = 2 * H * rows_used * 128;
+    const uint32_t kv_bytes = 2 * H * pages * p.page_size * 128;
+    if (lane == 0) {
+      mbar_expect_tx(&sc->bar_qk, q_bytes + kv_bytes);
+      mbar_expect_tx(&sc->bar_v, kv_bytes);
+    }
+    __syncwarp();
+    if (lane == 0) {
+      for (int plane = 0; plane < 2; ++plane)
+        for (int h = 0; h < H; ++h)
+          tma_load_4d(As + (plane * H + h) * SUB, &tmQ, h * 64, kvh * p.group, node0, plane, &sc->bar_qk);
+    }
+    for (int j = lane; j < pages; j += 32) {
+      const int page = p.page_table[k_begin / p.page_size + j];
+      const int c4 = p.layer * p.n_pages + page;
+      const int off = j * p.page_size * 128;
+      for (int plane = 0; plane < 2; ++plane)
+        for (int h = 0; h < H; ++h)
+          tma_load_5d(Ks + (plane * H + h) * SUB + off, &tmK, h * 64, 0, plane, kvh, c4, &sc->bar_qk);
+      for (int plane = 0; plane < 2; ++plane)
+        for (int h = 0; h < H; ++h)
+          tma_load_5d(Vs + (plane * H + h) * SUB + off, &tmV, h * 64, 0, plane, kvh, c4, &sc->bar_v);
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ---------------- MMA issuer
+    bool ok = mbar_wait(&sc->bar_qk, 0u, abort, status);
+    if (ok) {
+      tc_fence_after();
+      const uint32_t idesc = make_idesc_bf16(kc_pad);
+      const uint32_t a0 = smem_u32(As), b0 = smem_u32(Ks);
+      uint32_t acc = 0u;
+#pragma unroll
+      for (int term = 0; term < 3; ++term) {
+        const int qp = term == 2 ? 1 : 0, kp = term == 1 ? 1 : 0;     // hi*hi, hi*lo, lo*hi
+        for (int h = 0; h < H; ++h) {
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            umma_bf16(tmem_s, make_smem_desc(a0 + (qp * H + h) * SUB + k * 32),
+                      make_smem_desc(b0 + (kp * H + h) * SUB + k * 32), idesc, acc);
+            acc = 1u;
+          }
+        }
+      }
+      umma_commit(&sc->bar_s);
+      ok = mbar_wait(&sc->bar_p, 0u, abort, status) && mbar_wait(&sc->bar_v, 0u, abort, status);
+    }
+    if (ok) {
+      tc_fence_after();
+      const uint32_t idesc = make_idesc_bf16(DH, true);
+      const uint32_t a0 = smem_u32(As), b0 = smem_u32(Vs);
+      uint32_t acc = 0u;
+#pragma unroll
+      for (int term = 0; term < 3; ++term) {
+        const int pp = term == 2 ? 1 : 0, vp = term == 1 ? 1 : 0;
+        for (int j = 0; j < kc_pad / 16; ++j) {
+          // A: P plane pp, 64-key block j / 4, 16 keys = 32 bytes along the row
+          // B: V plane vp, keys 16 j .. 16 j + 15 are rows of 128 bytes; the second half of the head is SUB further on
+          umma_bf16(tmem_o, make_smem_desc(a0 + (pp * 2 + (j >> 2)) * SUB + (j & 3) * 32),
+                    make_smem_desc(b0 + vp * H * SUB + j * 2048, SUB), idesc, acc);
+          acc = 1u;
+        }
+      }
+      umma_commit(&sc->bar_o);
+    }
+  } else if (warp >= 2) {
+    // ---------------- softmax and epilogue: one thread per query row
+    unsigned long long my_anc[4] = {0ull, 0ull, 0ull, 0ull};
+    if (row_valid) {
+#pragma unroll
+      for (int w = 0; w < 4; ++w) my_anc[w] = p.anc[node * 4 + w];
+    }
+    const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+    bool ok = mbar_wait(&sc->bar_s, 0u, abort, status);
+    float m_row = -INFINITY, l_row = 0.f;
+    if (ok) {
+      tc_fence_after();
+      float s[KEYS];
+#pragma unroll
+      for (int c0 = 0; c0 < KEYS; c0 += 32) {
+        if (c0 < kc_pad) tmem_ld32(tmem_s + lane_off + c0, s + c0);
+      }
+      const bool no_mask = k_begin + KEYS <= L;
+#pragma unroll
+      for (int c = 0; c < KEYS; ++c) {
+        bool vis = true;
+        if (!no_mask) {
+          const int kg = k_begin + c;
+          vis = kg < L;
+          if (!vis && kg < Ltot) {
+            const int t = kg - L;
+            vis = (my_anc[t >> 6] >> (t & 63)) & 1ull;
+          }
+        }
+        s[c] = vis ? s[c] * p.scale_log2 : -INFINITY;
+        m_row = fmaxf(m_row, s[c]);
+      }
+      const float m_use = m_row > -INFINITY ? m_row : 0.f;    // a fully masked row gives p = 0 everywhere
+#pragma unroll
+      for (int c8 = 0; c8 < KEYS / 8; ++c8) {
+        if (c8 * 8 < kc_pad) {
+          uint32_t hi[4], lo[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float p0 = exp2f(s[c8 * 8 + 2 * e] - m_use);
+            const float p1 = exp2f(s[c8 * 8 + 2 * e + 1] - m_use);
+            l_row += p0 + p1;
+            split2_pack(p0, p1, hi[e], lo[e]);
+          }
+          const int off = (c8 >> 3) * SUB + r * 128 + (((c8 & 7) ^ (r & 7)) << 4);
+          *reinterpret_cast<uint4*>(As + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+          *reinterpret_cast<uint4*>(As + 2 * SUB + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        }
+      }
+      if (kc < kc_pad) {
+        // value rows past the end of the cache meet p = 0, but 0 * garbage could still be NaN: clear them
+        ok = mbar_wait(&sc->bar_v, 0u, abort, status);
+        if (ok && r < kc_pad - kc) {
+          for (int sub = 0; sub < 2 * H; ++sub)
+            for (int i = 0; i < 8; ++i)
+              *reinterpret_cast<uint4*>(Vs + sub * SUB + (kc + r) * 128 + i * 16) = make_uint4(0, 0, 0, 0);
+        }
+      }
+    }
+    if (ok) {
+      fence_proxy_async_smem();
+      mbar_arrive(&sc->bar_p);
+      ok = mbar_wait(&sc->bar_o, 0u, abort, status);
+    }
+    if (ok) {
+      tc_fence_after();
+#pragma unroll
+      for (int c0 = 0; c0 < DH; c0 += 32) {
+        float o[32];
+        tmem_ld32(tmem_o + lane_off + c0, o);
+        if (row_valid) {
+          float4* dst = reinterpret_cast<float4*>(p.attO + out_row * DH + c0);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) dst[e] = make_float4(o[4 * e], o[4 * e + 1], o[4 * e + 2], o[4 * e + 3]);
+        }
+      }
+      if (row_valid) p.attML[out_row] = make_float2(m_row, l_row);
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (*abort) {
+    // give copies still in flight time to land before the shared memory is handed back
+    for (int i = 0; i < 64; ++i) __nanosleep(20000);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(sc->tmem_base, 256);
+  }
+}
+
+template <int DH>
+void launch_dh(specasr_kv* kv, int layer, int n, int n_splits, cudaStream_t s) {
+  const specasr_model* m = kv->m;
+  const specasr_model_config& c = m->cfg;
+  constexpr int H = DH / 64;
+  constexpr int A_BYTES = 2 * H * SUB < 4 * SUB ? 4 * SUB : 2 * H * SUB;
+  const size_t smem = A_BYTES + 2 * (2 * H * SUB) + sizeof(AttnCtl) + 1024;
+  static bool configured = false;
+  if (!configured) {
+    cudaFuncSetAttribute(k_tree_attention_tc<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    configured = true;
+  }
+  AttnParams p;
+  p.ctl = kv->ws.ctl;
+  p.page_table = kv->page_table;
+  p.anc = kv->ws.anc;
+  p.attO = kv->ws.attO;
+  p.attML = kv->ws.attML;
+  p.rows_alloc = (size_t)kv->n_alloc * c.n_heads;
+  p.n_pages = kv->n_pages;
+  p.page_size = c.page_size;
+  p.layer = layer;
+  p.Hq = c.n_heads;
+  p.Hkv = c.n_kv_heads;
+  p.group = c.n_heads / c.n_kv_heads;
+  p.nodes_per_tile = 128 / p.group;
+  p.n = n;
+  p.scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
+  dim3 grid(c.n_kv_heads, (n + p.nodes_per_tile - 1) / p.nodes_per_tile, n_splits);
+  LaunchScope scope(kv, SPECASR_KIND_ATTN, s);
+  k_tree_attention_tc<DH><<<grid, 192, smem, s>>>(kv->tm_Q, kv->tm_K, kv->tm_V, p);
+}
+
+}  // namespace
+
+bool attention_tc_supported(const specasr_model* m) {
+  const specasr_model_config& c = m->cfg;
+  const int group = c.n_heads / c.n_kv_heads;
+  return c.gemm_path == 0 && (c.head_dim == 64 || c.head_dim == 128) && c.page_size % 16 == 0 && c.page_size <= KEYS &&
+         KEYS % c.page_size == 0 && group <= 128;
+}
+
+int attention_tc_splits(int total_len) { return (total_len + KEYS - 1) / KEYS; }
+
+// Tensor maps of the rotated queries and of the two pools, as the kernel above walks them.
+bool attention_tc_make_maps(specasr_kv* kv) {
+  const specasr_model* m = kv->m;
+  const specasr_model_config& c = m->cfg;
+  const int group = c.n_heads / c.n_kv_heads;
+  const uint64_t dh = c.head_dim;
+  {  // Q: [plane][node][head][dh]; box = 64 of dh, the `group` heads of one KV head, 128 / group nodes
+    uint64_t dims[4] = {dh, (uint64_t)c.n_heads, (uint64_t)kv->n_alloc, 2};
+    uint64_t strides[3] = {dh * 2, (uint64_t)m->q_dim * 2, (uint64_t)kv->n_alloc * m->q_dim * 2};
+    uint32_t box[4] = {64, (uint32_t)group, (uint32_t)(128 / group), 1};
+    if (!make_tensor_map_nd(&kv->tm_Q, kv->ws.Q, 4, dims, strides, box)) return false;
+  }
+  const uint64_t ps = c.page_size;
+  uint64_t dims[5] = {dh, ps, 2, (uint64_t)c.n_kv_heads, (uint64_t)c.n_layers * kv->n_pages};
+  uint64_t strides[4] = {dh * 2, ps * dh * 2, 2 * ps * dh * 2, (uint64_t)c.n_kv_heads * 2 * ps * dh * 2};
+  uint32_t box[5] = {64, (uint32_t)ps, 1, 1, 1};
+  return make_tensor_map_nd(&kv->tm_K, kv->k_pool, 5, dims, strides, box) &&
+         make_tensor_map_nd(&kv->tm_V, kv->v_pool, 5, dims, strides, box);
+}
+
+void launch_tree_attention_tc(specasr_kv* kv, int layer, int n, int n_splits, cudaStream_t s) {
+  if (kv->m->cfg.head_dim == 64) launch_dh<64>(kv, layer, n, n_splits, s);
+  else launch_dh<128>(kv, layer, n, n_splits, s);
+}

@@ -13,7 +13,7 @@
 typedef __nv_bfloat16 bf16;
 
 constexpr int kMaxSplitK = 8;      // split-K partial planes for the projections
-constexpr int kMaxAttnSplits = 32; // KV splits of the attention kernel
+constexpr int kMaxAttnSplits = 40; // KV splits of the attention kernels
 constexpr int kCtlWords = 64;      // int32 control block at the start of the workspace
 
 // control block word indices
@@ -81,9 +81,11 @@ struct specasr_kv {
   std::vector<cudaEvent_t> prof_events;   // 2 per recorded launch
   std::vector<int> prof_kinds;
   size_t prof_used;                       // launches recorded since the last read
-  // activation TMA descriptors (tcgen05 path)
   // activation TMA descriptors (tcgen05 path), one per box height 16 << i
   CUtensorMap tm_H[5], tm_AO[5], tm_A[5];
+  // tensor-core attention: rotated queries and the two pools
+  bool attn_tc;
+  CUtensorMap tm_Q, tm_K, tm_V;
 };
 
 // Counts a launch and, when profiling is on, brackets it with events on the launching stream.
@@ -130,8 +132,12 @@ void launch_advance_len(specasr_kv* kv, int n, cudaStream_t s);
 void launch_set_len(specasr_kv* kv, int len, cudaStream_t s);
 void launch_commit(specasr_kv* kv, const int32_t* path, const int32_t* accept_len, cudaStream_t s);
 
-// ---- attention.cu
+// ---- attention.cu (plain FMA) / attention_tc.cu (tcgen05)
 void launch_tree_attention(specasr_kv* kv, int layer, int n, int n_splits, cudaStream_t s);
+bool attention_tc_supported(const specasr_model* m);
+int attention_tc_splits(int total_len);
+bool attention_tc_make_maps(specasr_kv* kv);
+void launch_tree_attention_tc(specasr_kv* kv, int layer, int n, int n_splits, cudaStream_t s);
 
 // ---- gemm_fma.cu / gemm_tcgen05.cu
 enum GemmEpilogue { EPI_PARTIAL = 0, EPI_SWIGLU = 1, EPI_ARGMAX = 2 };
@@ -157,3 +163,6 @@ void launch_gemm_tc(specasr_kv* kv, const GemmArgs& a, int kind, cudaStream_t s)
 bool make_tensor_map_2d(CUtensorMap* out, const void* base, uint64_t inner, uint64_t outer,
                         uint32_t box_inner, uint32_t box_outer);
 bool make_act_map(CUtensorMap* out, const void* base, uint64_t K, uint64_t n_alloc, uint32_t box_rows);
+// bf16 tensor map of any rank with 128-byte swizzle; strides[i] is the byte stride of dimension i + 1
+bool make_tensor_map_nd(CUtensorMap* out, const void* base, int rank, const uint64_t* dims, const uint64_t* strides,
+                        const uint32_t* box);
