@@ -176,52 +176,65 @@ __global__ void __launch_bounds__(192, 1) k_tree_attention_tc(const __grid_const
       umma_commit(&sc->bar_o);
     }
   } else if (warp >= 2) {
-    // ---------------- softmax and epilogue: one thread per query row
-    unsigned long long my_anc[4] = {0ull, 0ull, 0ull, 0ull};
+    // ---------------- softmax and epilogue: one thread per query row.  The loops over 32-column
+    // chunks are kept rolled on purpose: straight-line code that runs once is bound by instruction fetch.
+    unsigned long long anc0 = 0ull, anc1 = 0ull, anc2 = 0ull, anc3 = 0ull;
     if (row_valid) {
-#pragma unroll
-      for (int w = 0; w < 4; ++w) my_anc[w] = p.anc[node * 4 + w];
+      anc0 = p.anc[node * 4 + 0];
+      anc1 = p.anc[node * 4 + 1];
+      anc2 = p.anc[node * 4 + 2];
+      anc3 = p.anc[node * 4 + 3];
     }
+    // bit j of the result = key (base + j) is visible to this row
+    auto visible32 = [&](int base) -> uint32_t {
+      const int t0 = base - L;                      // tree slot of the chunk's first key
+      if (t0 <= -32) return 0xFFFFFFFFu;            // all 32 keys lie in the committed prefix
+      const int ts = t0 > 0 ? t0 : 0;
+      uint32_t win = 0u;                            // ancestor bits of tree slots ts .. ts + 31
+      if (ts < SPECASR_MAX_NODES) {
+        const int w = ts >> 6, sh = ts & 63;
+        const unsigned long long a = w == 0 ? anc0 : w == 1 ? anc1 : w == 2 ? anc2 : anc3;
+        const unsigned long long b = w == 0 ? anc1 : w == 1 ? anc2 : w == 2 ? anc3 : 0ull;
+        win = (uint32_t)(sh ? (a >> sh) | (b << (64 - sh)) : a);
+      }
+      return t0 < 0 ? ((1u << (-t0)) - 1u) | (win << (-t0)) : win;
+    };
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
     bool ok = mbar_wait(&sc->bar_s, 0u, abort, status);
     float m_row = -INFINITY, l_row = 0.f;
     if (ok) {
       tc_fence_after();
-      float s[KEYS];
+#pragma unroll 1
+      for (int c0 = 0; c0 < kc_pad; c0 += 32) {
+        float s[32];
+        tmem_ld32(tmem_s + lane_off + c0, s);
+        const uint32_t vis = visible32(k_begin + c0);
 #pragma unroll
-      for (int c0 = 0; c0 < KEYS; c0 += 32) {
-        if (c0 < kc_pad) tmem_ld32(tmem_s + lane_off + c0, s + c0);
-      }
-      const bool no_mask = k_begin + KEYS <= L;
-#pragma unroll
-      for (int c = 0; c < KEYS; ++c) {
-        bool vis = true;
-        if (!no_mask) {
-          const int kg = k_begin + c;
-          vis = kg < L;
-          if (!vis && kg < Ltot) {
-            const int t = kg - L;
-            vis = (my_anc[t >> 6] >> (t & 63)) & 1ull;
-          }
-        }
-        s[c] = vis ? s[c] * p.scale_log2 : -INFINITY;
-        m_row = fmaxf(m_row, s[c]);
+        for (int j = 0; j < 32; ++j) m_row = fmaxf(m_row, ((vis >> j) & 1u) ? s[j] * p.scale_log2 : -INFINITY);
       }
       const float m_use = m_row > -INFINITY ? m_row : 0.f;    // a fully masked row gives p = 0 everywhere
+#pragma unroll 1
+      for (int c0 = 0; c0 < kc_pad; c0 += 32) {
+        float s[32];
+        tmem_ld32(tmem_s + lane_off + c0, s);
+        const uint32_t vis = visible32(k_begin + c0);
 #pragma unroll
-      for (int c8 = 0; c8 < KEYS / 8; ++c8) {
-        if (c8 * 8 < kc_pad) {
+        for (int g = 0; g < 4; ++g) {
           uint32_t hi[4], lo[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            const float p0 = exp2f(s[c8 * 8 + 2 * e] - m_use);
-            const float p1 = exp2f(s[c8 * 8 + 2 * e + 1] - m_use);
+            const int j = g * 8 + 2 * e;
+            const float p0 = ((vis >> j) & 1u) ? exp2f(s[j] * p.scale_log2 - m_use) : 0.f;
+            const float p1 = ((vis >> (j + 1)) & 1u) ? exp2f(s[j + 1] * p.scale_log2 - m_use) : 0.f;
             l_row += p0 + p1;
             split2_pack(p0, p1, hi[e], lo[e]);
           }
-          const int off = (c8 >> 3) * SUB + r * 128 + (((c8 & 7) ^ (r & 7)) << 4);
-          *reinterpret_cast<uint4*>(As + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-          *reinterpret_cast<uint4*>(As + 2 * SUB + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+          const int c8 = (c0 >> 3) + g;                        // 8-key group within the block of 128
+          if (c8 * 8 < kc_pad) {
+            const int off = (c8 >> 3) * SUB + r * 128 + (((c8 & 7) ^ (r & 7)) << 4);
+            *reinterpret_cast<uint4*>(As + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+            *reinterpret_cast<uint4*>(As + 2 * SUB + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+          }
         }
       }
       if (kc < kc_pad) {
@@ -241,14 +254,30 @@ __global__ void __launch_bounds__(192, 1) k_tree_attention_tc(const __grid_const
     }
     if (ok) {
       tc_fence_after();
-#pragma unroll
+      // O leaves through the (now idle) K tile so that a warp writes whole 512-byte rows: thread r parks its
+      // row with the 16-byte columns rotated by r, then lane c of the warp reads column c of each of its 32 rows.
+      float4* stage = reinterpret_cast<float4*>(Ks);
+      constexpr int C4 = DH / 4;                             // float4 columns per row
+#pragma unroll 1
       for (int c0 = 0; c0 < DH; c0 += 32) {
         float o[32];
         tmem_ld32(tmem_o + lane_off + c0, o);
-        if (row_valid) {
-          float4* dst = reinterpret_cast<float4*>(p.attO + out_row * DH + c0);
 #pragma unroll
-          for (int e = 0; e < 8; ++e) dst[e] = make_float4(o[4 * e], o[4 * e + 1], o[4 * e + 2], o[4 * e + 3]);
+        for (int e = 0; e < 8; ++e) {
+          const int c4 = (c0 >> 2) + e;
+          stage[r * C4 + (c4 ^ (r & (C4 - 1)))] = make_float4(o[4 * e], o[4 * e + 1], o[4 * e + 2], o[4 * e + 3]);
+        }
+      }
+      __syncwarp();
+      const int r_base = (warp & 3) << 5;
+#pragma unroll 1
+      for (int i = 0; i < 32; ++i) {
+        const int rr = r_base + i;
+        const int nd = node0 + rr / p.group;
+        if (rr < rows_used && nd < p.n) {
+          const size_t orow = (size_t)split * p.rows_alloc + (size_t)nd * p.Hq + kvh * p.group + rr % p.group;
+          float4* dst = reinterpret_cast<float4*>(p.attO + orow * DH);
+          for (int c4 = lane; c4 < C4; c4 += 32) dst[c4] = stage[rr * C4 + (c4 ^ (rr & (C4 - 1)))];
         }
       }
       if (row_valid) p.attML[out_row] = make_float2(m_row, l_row);
