@@ -73,7 +73,10 @@ typedef struct specasr_model_config {
 /*
  * Weights, all [device], all borrowed.  Matrices are bf16, row-major [out_features, in_features]
  * with rows 16-byte aligned (in_features % 8 == 0).  Gains are fp32.
- *   wqkv[l] : [(n_heads + 2 n_kv_heads) * head_dim, d_model]  rows = all Q heads, all K heads, all V heads
+ *   wqkv[l] : [(n_heads + 2 n_kv_heads) * head_dim, d_model]  rows = all Q heads, all K heads, all V heads;
+ *             within every head the rows are in rotary-paired order: stored row 32 g + 16 h + j holds
+ *             feature 16 g + j + h * head_dim / 2 (0 <= j < 16, h in {0, 1}), so that a feature and its
+ *             rotation partner land in the same warp of the projection's epilogue
  *   wo[l]   : [d_model, n_heads * head_dim]
  *   wgu[l]  : [2 * ffn, d_model]   row 2f = gate row f, row 2f+1 = up row f (interleaved so that one
  *             output tile holds both halves of a SwiGLU feature)

@@ -54,6 +54,8 @@ Workspace carve_workspace(const specasr_model* m, int n_alloc, void* base) {
   w.X = (float*)take(sizeof(float) * n_alloc * c.d_model);
   w.H = (bf16*)take(sizeof(bf16) * 2 * n_alloc * c.d_model);
   w.P = (float*)take(sizeof(float) * kMaxSplitK * n_alloc * wide);
+  w.fixP = (float*)take(m->cfg.gemm_path == 0 ? gemm_tc_fixup_bytes(m, n_alloc) : 256);
+  w.fixFlag = (int32_t*)take(sizeof(int32_t) * (m->n_sm > 0 ? m->n_sm : 1));
   w.Q = (bf16*)take(sizeof(bf16) * 2 * n_alloc * m->q_dim);
   w.AO = (bf16*)take(sizeof(bf16) * 2 * n_alloc * m->q_dim);
   w.A = (bf16*)take(sizeof(bf16) * 2 * n_alloc * c.ffn);
@@ -222,12 +224,14 @@ extern "C" specasr_status specasr_kv_create(const specasr_model* m, void* k_pool
   kv->pinned = nullptr;
   kv->len_event_pending = false;
   kv->launches = 0;
+  kv->gemm_epoch = 0;
   kv->prof_on = false;
   kv->prof_used = 0;
   kv->attn_tc = false;
   cudaError_t e = cudaHostAlloc(&kv->pinned, 4 * sizeof(int32_t), cudaHostAllocDefault);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&kv->len_event, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaMemset(kv->ws.ctl, 0, sizeof(int32_t) * kCtlWords);
+  if (e == cudaSuccess) e = cudaMemset(kv->ws.fixFlag, 0, sizeof(int32_t) * m->n_sm);
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
     if (kv->pinned) cudaFreeHost(kv->pinned);
@@ -358,6 +362,7 @@ static void run_gemm(specasr_kv* kv, GemmArgs& a, int kind, cudaStream_t s) {
     a.splits = 1;
     launch_gemm_fma(kv, a, kind, s);
   } else {
+    a.splits = gemm_tc_pick_splits(kv->m, a.M, a.K, a.n_pad);
     launch_gemm_tc(kv, a, kind, s);
   }
 }
@@ -391,18 +396,18 @@ static void run_stack(specasr_model* m, specasr_kv* kv, int n, bool want_head, f
   bool att_tc = false;
   const int att_splits = attention_splits(kv, n, kv->len_upper, &att_tc);
   const bool tc = c.gemm_path == 0;
-  int down_splits = 0;
+  int pending = 0;               // partial planes of the last down projection still to be added to X
   GemmArgs a;
   memset(&a, 0, sizeof(a));
   a.n = n;
   a.n_pad = n_pad;
   a.n_alloc = kv->n_alloc;
   a.ctl = kv->ws.ctl;
+  a.P = kv->ws.P;
   for (int l = 0; l < c.n_layers; ++l) {
-    launch_rmsnorm_split(kv, m->g_attn[l], n, n_pad, down_splits, s);
+    launch_rmsnorm_split(kv, m->g_attn[l], n, n_pad, pending, s);
     a.W = m->wqkv[l]; a.tmW = tc ? &m->tm_wqkv[l] : nullptr; a.tmAct = kv->tm_H; a.act = kv->ws.H;
-    a.M = m->qkv_dim; a.K = c.d_model; a.epilogue = EPI_PARTIAL; a.P = kv->ws.P;
-    a.splits = tc ? gemm_tc_pick_splits(m, a.M, a.K) : 1;
+    a.M = m->qkv_dim; a.K = c.d_model; a.epilogue = EPI_PARTIAL;
     run_gemm(kv, a, SPECASR_KIND_GEMM_QKV, s);
     launch_rope_append(kv, l, n, a.splits, s);
     if (att_tc) launch_tree_attention_tc(kv, l, n, att_splits, s);
@@ -410,22 +415,20 @@ static void run_stack(specasr_model* m, specasr_kv* kv, int n, bool want_head, f
     launch_attn_merge(kv, n, n_pad, att_splits, s);
     a.W = m->wo[l]; a.tmW = tc ? &m->tm_wo[l] : nullptr; a.tmAct = kv->tm_AO; a.act = kv->ws.AO;
     a.M = c.d_model; a.K = m->q_dim; a.epilogue = EPI_PARTIAL;
-    a.splits = tc ? gemm_tc_pick_splits(m, a.M, a.K) : 1;
     run_gemm(kv, a, SPECASR_KIND_GEMM_O, s);
     launch_rmsnorm_split(kv, m->g_ffn[l], n, n_pad, a.splits, s);
     a.W = m->wgu[l]; a.tmW = tc ? &m->tm_wgu[l] : nullptr; a.tmAct = kv->tm_H; a.act = kv->ws.H;
-    a.M = 2 * c.ffn; a.K = c.d_model; a.epilogue = EPI_SWIGLU; a.A = kv->ws.A; a.splits = 1;
+    a.M = 2 * c.ffn; a.K = c.d_model; a.epilogue = EPI_SWIGLU; a.A = kv->ws.A;
     run_gemm(kv, a, SPECASR_KIND_GEMM_GU, s);
     a.W = m->wd[l]; a.tmW = tc ? &m->tm_wd[l] : nullptr; a.tmAct = kv->tm_A; a.act = kv->ws.A;
     a.M = c.d_model; a.K = c.ffn; a.epilogue = EPI_PARTIAL;
-    a.splits = tc ? gemm_tc_pick_splits(m, a.M, a.K) : 1;
     run_gemm(kv, a, SPECASR_KIND_GEMM_DOWN, s);
-    down_splits = a.splits;
+    pending = a.splits;
   }
   if (!want_head) return;   // context fill: K/V of every layer are written, the last FFN output is not needed
-  launch_rmsnorm_split(kv, m->g_final, n, n_pad, down_splits, s);
+  launch_rmsnorm_split(kv, m->g_final, n, n_pad, pending, s);
   a.W = m->lm_head; a.tmW = tc ? &m->tm_lm : nullptr; a.tmAct = kv->tm_H; a.act = kv->ws.H;
-  a.M = c.vocab; a.K = c.d_model; a.epilogue = EPI_ARGMAX; a.amax = kv->ws.amax; a.logits = out_logits; a.splits = 1;
+  a.M = c.vocab; a.K = c.d_model; a.epilogue = EPI_ARGMAX; a.amax = kv->ws.amax; a.logits = out_logits;
   run_gemm(kv, a, SPECASR_KIND_GEMM_LM, s);
 }
 

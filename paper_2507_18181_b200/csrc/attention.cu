@@ -22,6 +22,8 @@ __global__ void __launch_bounds__(256) k_tree_attention(const int32_t* __restric
                                                         const unsigned long long* __restrict__ anc, int n_splits,
                                                         float scale_log2, float* __restrict__ attO,
                                                         float2* __restrict__ attML, size_t rows_alloc) {
+  grid_dep_launch();
+  grid_dep_wait();
   if (ctl[CTL_STATUS] != 0) return;
   extern __shared__ float smem[];
   float* Qs = smem;                         // [ROWS][DH + 1]
@@ -184,7 +186,7 @@ void launch_dh(specasr_kv* kv, int layer, int n, int n_splits, cudaStream_t s) {
   dim3 grid(c.n_kv_heads, (n * group + ROWS - 1) / ROWS, n_splits);
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
   LaunchScope scope(kv, SPECASR_KIND_ATTN, s);
-  k_tree_attention<DH><<<grid, 256, smem, s>>>(kv->ws.ctl, kv->ws.Q, (size_t)kv->n_alloc * m->q_dim, kv->k_pool,
+  launch_pdl(k_tree_attention<DH>, grid, dim3(256), smem, s, kv->ws.ctl, kv->ws.Q, (size_t)kv->n_alloc * m->q_dim, kv->k_pool,
                                                kv->v_pool, kv->page_table, kv->n_pages, c.page_size, layer,
                                                c.n_heads, c.n_kv_heads, n, kv->ws.anc, n_splits, scale_log2,
                                                kv->ws.attO, kv->ws.attML, (size_t)kv->n_alloc * c.n_heads);

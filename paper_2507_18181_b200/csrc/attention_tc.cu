@@ -52,6 +52,8 @@ __global__ void __launch_bounds__(192, 1) k_tree_attention_tc(const __grid_const
   constexpr int A_BYTES = 2 * H * SUB < 4 * SUB ? 4 * SUB : 2 * H * SUB;   // Q planes, later the P planes
   constexpr int KV_BYTES = 2 * H * SUB;
   extern __shared__ uint8_t smem_raw[];
+  pdl_launch_dependents();
+  pdl_wait();
   if (p.ctl[CTL_STATUS] != 0) return;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -327,7 +329,7 @@ void launch_dh(specasr_kv* kv, int layer, int n, int n_splits, cudaStream_t s) {
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
   dim3 grid(c.n_kv_heads, (n + p.nodes_per_tile - 1) / p.nodes_per_tile, n_splits);
   LaunchScope scope(kv, SPECASR_KIND_ATTN, s);
-  k_tree_attention_tc<DH><<<grid, 192, smem, s>>>(kv->tm_Q, kv->tm_K, kv->tm_V, p);
+  launch_pdl(k_tree_attention_tc<DH>, grid, dim3(192), smem, s, kv->tm_Q, kv->tm_K, kv->tm_V, p);
 }
 
 }  // namespace

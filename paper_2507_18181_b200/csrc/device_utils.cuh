@@ -57,3 +57,16 @@ __device__ __forceinline__ unsigned long long pack_max_key(float v, uint32_t idx
   u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
   return ((unsigned long long)u << 32) | (unsigned long long)(0xFFFFFFFFu - idx);
 }
+
+// Programmatic dependent launch (see launch_pdl): wait for the previous kernel of the stream, and let
+// the next one begin its prologue.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Rows of the fused QKV weight are stored in rotary-paired order within each head: row 32 g + j holds
+// feature 16 g + j and row 32 g + 16 + j its rotation partner dh/2 further on (0 <= j < 16).
+__device__ __forceinline__ int qkv_row_of_feature(int e, int dh) {
+  const int half = dh >> 1;
+  const int k = e % half;
+  return ((k >> 4) << 5) | ((e / half) << 4) | (k & 15);
+}

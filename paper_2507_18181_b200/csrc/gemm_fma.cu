@@ -9,6 +9,8 @@ constexpr int BM = 64, BN = 64, BK = 16;
 
 template <int EPI>
 __global__ void __launch_bounds__(256) k_gemm_fma(GemmArgs a) {
+  grid_dep_launch();
+  grid_dep_wait();
   if (a.ctl[CTL_STATUS] != 0) return;
   __shared__ float Ws[BK][BM + 4];
   __shared__ float As[BK][BN + 4];
@@ -109,7 +111,7 @@ int gemm_fma_tiles(int M) { return (M + BM - 1) / BM; }
 void launch_gemm_fma(specasr_kv* kv, const GemmArgs& a, int kind, cudaStream_t s) {
   LaunchScope scope(kv, kind, s);
   dim3 grid((a.M + BM - 1) / BM, (a.n + BN - 1) / BN);
-  if (a.epilogue == EPI_PARTIAL) k_gemm_fma<EPI_PARTIAL><<<grid, 256, 0, s>>>(a);
-  else if (a.epilogue == EPI_SWIGLU) k_gemm_fma<EPI_SWIGLU><<<grid, 256, 0, s>>>(a);
-  else k_gemm_fma<EPI_ARGMAX><<<grid, 256, 0, s>>>(a);
+  if (a.epilogue == EPI_PARTIAL) launch_pdl(k_gemm_fma<EPI_PARTIAL>, grid, dim3(256), 0, s, a);
+  else if (a.epilogue == EPI_SWIGLU) launch_pdl(k_gemm_fma<EPI_SWIGLU>, grid, dim3(256), 0, s, a);
+  else launch_pdl(k_gemm_fma<EPI_ARGMAX>, grid, dim3(256), 0, s, a);
 }

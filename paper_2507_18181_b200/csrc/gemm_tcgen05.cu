@@ -2,194 +2,389 @@
 //
 //   D[m][t] = sum_k W[m][k] * (hi[t][k] + lo[t][k])        W: [M, K] bf16, activations: two bf16 planes
 //
-// The weight matrix is the MMA "A" operand (M = 128 rows per CTA tile), the tree tokens are the MMA
-// "N" dimension, so a 64-node tree costs one 128 x 64 accumulator per tile and every weight byte is
+// The weight matrix is the MMA "A" operand (128 rows per tile), the tree tokens are the MMA "N"
+// dimension, so a 64-node tree costs one 128 x 64 fp32 accumulator per tile and every weight byte is
 // read from HBM exactly once.  Both operands are K-major and arrive by TMA into 128-byte-swizzled
-// shared-memory tiles; the hi and lo activation planes are two MMAs into the same TMEM accumulator.
-// One warp issues TMA, one thread issues tcgen05.mma, four warps drain TMEM (tcgen05.ld) into the
-// fused epilogue.  Grid = (M tiles, K splits): split-K planes are summed by the consumer kernel in a
-// fixed order, which keeps the result deterministic.
+// shared-memory tiles.  The hi and lo activation planes sit back to back in shared memory and form ONE
+// MMA of N = 2 x tokens (the weight tile, the large operand, is fetched once for both); the epilogue
+// adds the two halves of the accumulator.
+// A pipeline stage holds one k-block of `tm` adjacent weight tiles and the matching activation block,
+// so with tm = 2 the activation bytes (which every CTA re-reads from L2) are half the weight bytes.
 //
-// Every mbarrier wait is bounded by wall-clock time; on expiry the CTA records SPECASR_ERR_TIMEOUT in
-// the status word, lets copies in flight land, frees its TMEM and returns.
+// Scheduling.  The kernel is persistent, at most one CTA per SM, over (tile group, k-block) units.
+//  - Linear outputs (QKV, O, down): the k-blocks of every tile group are cut into `splits` equal
+//    parts, one CTA each; a CTA writes its fp32 partial sums to plane `split` and the consumer kernel
+//    adds the planes in a fixed order.
+//  - Non-linear epilogues (gate/up with SiLU * up, LM head with arg-max): the units of the whole
+//    matrix are cut into equal contiguous ranges, one per CTA, so every SM streams the same number of
+//    weight bytes whatever the tile count.  A tile group whose k-blocks fall into two ranges is summed
+//    in a fixed order: the CTA holding its later k-blocks (which it processes first) parks its partial
+//    sums in a workspace slot and publishes a flag; the CTA holding k-block 0 (which it processes
+//    last) adds them in CTA order and runs the epilogue.  All CTAs are co-resident and every flag wait
+//    is bounded.
+//
+// Roles: warp 0 issues TMA, one thread of warp 1 issues tcgen05.mma, warps 2..5 drain TMEM
+// (tcgen05.ld) into the epilogue; two TMEM accumulator sets let the epilogue of one tile group overlap
+// the main loop of the next.
+//
+// Programmatic dependent launch: the weight tiles of the first pipeline stages are requested before
+// the kernel waits for its predecessor in the stream, since weights never change; only activation
+// loads and global writes come after that wait.
+//
+// Every mbarrier or flag wait is bounded by wall-clock time; on expiry the CTA records
+// SPECASR_ERR_TIMEOUT in the status word, lets copies in flight land, frees its TMEM and returns.
 #include "internal.h"
 #include "device_utils.cuh"
 #include "sm100_ptx.cuh"
-
-#include <stdio.h>
 
 using namespace sm100;
 
 namespace {
 
 constexpr int TILE_M = 128;
-constexpr int TILE_K = 64;            // bf16 elements = 128 bytes = one swizzle row
+constexpr int SUB_K = 64;             // bf16 elements = 128 bytes = one swizzle row
 constexpr int UMMA_K = 16;
-constexpr int W_TILE_BYTES = TILE_M * TILE_K * 2;
-constexpr int MAX_STAGES = 8;
-constexpr int SMEM_BUDGET = 200 * 1024;
+constexpr int W_SUB_BYTES = TILE_M * SUB_K * 2;
+constexpr int MAX_STAGES = 6;
+constexpr int SMEM_LIMIT = 227 * 1024;  // dynamic shared memory one CTA may ask for
 
-struct SharedCtl {
+struct alignas(16) SharedCtl {
   unsigned long long full[MAX_STAGES];
   unsigned long long empty[MAX_STAGES];
-  unsigned long long accum;
+  unsigned long long acc_full[2];
+  unsigned long long acc_empty[2];
   unsigned long long key[SPECASR_MAX_NODES];
   uint32_t tmem_base;
   int abort;
 };
 
 struct TcParams {
-  int M, K, n, n_pad, n_alloc, box_rows, stages, tmem_cols, splits;
-  float* P;
-  bf16* A;
-  unsigned long long* amax;
-  float* logits;
+  int M, K, n, n_pad, n_alloc, box_rows, stages, ksub, tm, n_buf, tmem_cols, KB, tiles, groups, splits, epoch;
   int32_t* ctl;
+  float* fixP;              // [grid][tm][n_pad][128] parked partial sums (hi + lo halves added) of split tile groups
+  int32_t* fixFlag;         // [grid] launch number of the partial sums each CTA parked last
+  float* P;                 // EPI_PARTIAL: [splits][n_alloc][M]
+  bf16* A;                  // EPI_SWIGLU: [2][n_alloc][M/2]
+  unsigned long long* amax; // EPI_ARGMAX: [tiles][n_alloc]
+  float* logits;            // EPI_ARGMAX: optional [n][M]
 };
 
+__device__ __forceinline__ int ld_acquire(const int32_t* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release(int32_t* p, int v) {
+  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
 template <int EPI>
-__global__ void __launch_bounds__(192, 1) k_gemm_tc(const __grid_constant__ CUtensorMap tmW,
-                                                    const __grid_constant__ CUtensorMap tmAct, TcParams p) {
+__global__ void __launch_bounds__(192, 1) k_proj(const __grid_constant__ CUtensorMap tmW,
+                                                 const __grid_constant__ CUtensorMap tmAct, TcParams p) {
   extern __shared__ uint8_t smem_raw[];
-  if (p.ctl[CTL_STATUS] != 0) return;
   uint8_t* tiles = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  const int act_bytes = p.n_pad * 2 * TILE_K * 2;     // both planes
-  const int stage_bytes = W_TILE_BYTES + act_bytes;
+  const int w_bytes = p.tm * p.ksub * W_SUB_BYTES;
+  const int act_sub = p.n_pad * 2 * SUB_K * 2;         // both planes of one 64-wide k sub-block
+  const int stage_bytes = w_bytes + p.ksub * act_sub;
   SharedCtl* sc = (SharedCtl*)(tiles + (size_t)p.stages * stage_bytes);
+  bf16* epi_stage = (bf16*)(sc + 1);                    // EPI_SWIGLU: [2 planes][n_pad][64] output tile
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tile = blockIdx.x, split = blockIdx.y;
-  const int KB = (p.K + TILE_K - 1) / TILE_K;
-  const int kb0 = (int)(((long long)split * KB) / p.splits);
-  const int kb1 = (int)(((long long)(split + 1) * KB) / p.splits);
+  const int G = gridDim.x, cta = blockIdx.x;
+  const int KB = p.KB;
+  const long long U = (long long)p.groups * KB;
+  long long u0, u1;
+  if (EPI == EPI_PARTIAL) {           // one tile group, one part of its k-blocks
+    const int group = cta / p.splits, split = cta % p.splits;
+    u0 = (long long)group * KB + (long long)split * KB / p.splits;
+    u1 = (long long)group * KB + (long long)(split + 1) * KB / p.splits;
+  } else {                            // equal contiguous ranges of the whole unit list
+    u0 = cta * U / G;
+    u1 = (cta + 1) * U / G;
+  }
   const int n_blocks = p.n_pad / p.box_rows;
+  const int acc_cols = p.tm * 2 * p.n_pad;              // TMEM columns of one accumulator set (hi | lo halves)
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) {
       mbar_init(&sc->full[s], 1);
       mbar_init(&sc->empty[s], 1);
     }
-    mbar_init(&sc->accum, 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&sc->acc_full[b], 1);
+      mbar_init(&sc->acc_empty[b], 128);
+    }
     sc->abort = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_fence_init();
+    tma_prefetch_desc(&tmW);
+    tma_prefetch_desc(&tmAct);
   }
-  if (EPI == EPI_ARGMAX)
-    for (int t = threadIdx.x; t < SPECASR_MAX_NODES; t += blockDim.x) sc->key[t] = 0ull;
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sc->tmem_base)),
-                 "r"((uint32_t)p.tmem_cols)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  if (warp == 1) tmem_alloc(&sc->tmem_base, (uint32_t)p.tmem_cols);
+  tc_fence_before();
   __syncthreads();
-  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  tc_fence_after();
+  pdl_launch_dependents();
   const uint32_t tmem_base = sc->tmem_base;
   volatile int* abort = &sc->abort;
   int32_t* status = p.ctl + CTL_STATUS;
 
   if (warp == 0 && lane == 0) {
     // ---------------- TMA producer
-    int it = 0;
-    for (int kb = kb0; kb < kb1; ++kb, ++it) {
-      const int s = it % p.stages;
-      const uint32_t ph = (uint32_t)(it / p.stages) & 1u;
-      if (!mbar_wait(&sc->empty[s], ph ^ 1u, abort, status)) break;
+    const int total = (int)(u1 - u0);
+    auto load_w = [&](int i) {
+      const long long u = u0 + i;
+      const int group = (int)(u / KB), kb = (int)(u % KB), s = i % p.stages;
       uint8_t* st = tiles + (size_t)s * stage_bytes;
-      mbar_expect_tx(&sc->full[s], (uint32_t)stage_bytes);
-      tma_load_2d(st, &tmW, kb * TILE_K, tile * TILE_M, &sc->full[s]);
-      for (int jb = 0; jb < n_blocks; ++jb)
-        tma_load_3d(st + W_TILE_BYTES + (size_t)jb * p.box_rows * 2 * TILE_K * 2, &tmAct, kb * TILE_K,
-                    jb * p.box_rows, 0, &sc->full[s]);
+      for (int t = 0; t < p.tm; ++t)       // rows past M read as zeros
+        for (int q = 0; q < p.ksub; ++q)
+          tma_load_2d(st + (t * p.ksub + q) * W_SUB_BYTES, &tmW, (kb * p.ksub + q) * SUB_K,
+                      (group * p.tm + t) * TILE_M, &sc->full[s]);
+    };
+    auto load_act = [&](int i) {
+      const int kb = (int)((u0 + i) % KB), s = i % p.stages;
+      uint8_t* st = tiles + (size_t)s * stage_bytes + w_bytes;
+      for (int q = 0; q < p.ksub; ++q)
+        for (int jb = 0; jb < n_blocks; ++jb)
+          tma_load_3d(st + q * act_sub + (size_t)jb * p.box_rows * 2 * SUB_K * 2, &tmAct, (kb * p.ksub + q) * SUB_K,
+                      jb * p.box_rows, 0, &sc->full[s]);
+    };
+    // weights never change: request the first stages before waiting for the previous kernel
+    const int pre = total < p.stages ? total : p.stages;
+    for (int i = 0; i < pre; ++i) {
+      mbar_expect_tx(&sc->full[i], (uint32_t)stage_bytes);
+      load_w(i);
+    }
+    pdl_wait();
+    if (*(volatile int32_t*)status != 0) {
+      if (pre > 0) *abort = 1;       // weight tiles are in flight: hold the shared memory until they land
+    } else {
+      for (int i = 0; i < pre; ++i) load_act(i);
+      for (int i = pre; i < total; ++i) {
+        const int s = i % p.stages;
+        const uint32_t ph = (uint32_t)(i / p.stages) & 1u;
+        if (!mbar_wait(&sc->empty[s], ph ^ 1u, abort, status)) break;
+        mbar_expect_tx(&sc->full[s], (uint32_t)stage_bytes);
+        load_w(i);
+        load_act(i);
+      }
     }
   } else if (warp == 1 && lane == 0) {
     // ---------------- MMA issuer
-    const uint32_t idesc = make_idesc_bf16(p.box_rows);
-    int it = 0;
-    bool ok = true;
-    for (int kb = kb0; kb < kb1; ++kb, ++it) {
-      const int s = it % p.stages;
-      const uint32_t ph = (uint32_t)(it / p.stages) & 1u;
-      if (!mbar_wait(&sc->full[s], ph, abort, status)) {
-        ok = false;
-        break;
-      }
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t w_addr = smem_u32(tiles + (size_t)s * stage_bytes);
-      const uint32_t act_addr = w_addr + W_TILE_BYTES;
-      for (int jb = 0; jb < n_blocks; ++jb) {
-        for (int plane = 0; plane < 2; ++plane) {
-          const uint32_t b_addr = act_addr + (uint32_t)((jb * 2 + plane) * p.box_rows * TILE_K * 2);
-#pragma unroll
-          for (int k = 0; k < TILE_K / UMMA_K; ++k) {
-            const uint64_t ad = make_smem_desc(w_addr + k * UMMA_K * 2);
-            const uint64_t bd = make_smem_desc(b_addr + k * UMMA_K * 2);
-            const uint32_t acc = (kb > kb0 || plane > 0 || k > 0) ? 1u : 0u;
-            umma_bf16(tmem_base + (uint32_t)(jb * p.box_rows), ad, bd, idesc, acc);
+    pdl_wait();
+    if (*(volatile int32_t*)status == 0) {
+      const uint32_t idesc = make_idesc_bf16(2 * p.box_rows);      // both planes of a token block in one MMA
+      int i = 0, seg = 0;
+      bool ok = true;
+      for (long long u = u0; u < u1 && ok; ++seg) {
+        const int kb0 = (int)(u % KB);
+        const int kb1 = (int)((u1 - u) < (long long)(KB - kb0) ? kb0 + (u1 - u) : KB);
+        const int b = seg % p.n_buf;
+        if (!mbar_wait(&sc->acc_empty[b], (uint32_t)((seg / p.n_buf) & 1) ^ 1u, abort, status)) break;
+        tc_fence_after();
+        const uint32_t d_base = tmem_base + (uint32_t)(b * acc_cols);
+        for (int kb = kb0; kb < kb1; ++kb, ++i) {
+          const int s = i % p.stages;
+          const uint32_t ph = (uint32_t)(i / p.stages) & 1u;
+          if (!mbar_wait(&sc->full[s], ph, abort, status)) {
+            ok = false;
+            break;
           }
+          tc_fence_after();
+          const uint32_t w_addr = smem_u32(tiles + (size_t)s * stage_bytes);
+          const uint32_t act_addr = w_addr + w_bytes;
+          for (int t = 0; t < p.tm; ++t) {
+            for (int q = 0; q < p.ksub; ++q) {
+              const uint32_t a_addr = w_addr + (t * p.ksub + q) * W_SUB_BYTES;
+              for (int jb = 0; jb < n_blocks; ++jb) {
+                const uint32_t b_addr = act_addr + q * act_sub + (uint32_t)(jb * 2 * p.box_rows * SUB_K * 2);
+                const uint32_t d_addr = d_base + (uint32_t)(t * 2 * p.n_pad + jb * 2 * p.box_rows);
+#pragma unroll
+                for (int k = 0; k < SUB_K / UMMA_K; ++k) {
+                  const uint32_t acc = (kb > kb0 || q > 0 || k > 0) ? 1u : 0u;
+                  umma_bf16(d_addr, make_smem_desc(a_addr + k * UMMA_K * 2), make_smem_desc(b_addr + k * UMMA_K * 2),
+                            idesc, acc);
+                }
+              }
+            }
+          }
+          umma_commit(&sc->empty[s]);   // arrives once these MMAs have read the stage
         }
+        if (ok) umma_commit(&sc->acc_full[b]);
+        u += kb1 - kb0;
       }
-      umma_commit(&sc->empty[s]);   // arrives once these MMAs have read the stage
     }
-    if (ok) umma_commit(&sc->accum);
   } else if (warp >= 2) {
     // ---------------- epilogue: TMEM lane = output row of the tile
+    pdl_wait();
     const int quad = warp & 3;
-    const int m = tile * TILE_M + quad * 32 + lane;
-    const bool row_ok = m < p.M;
-    if (mbar_wait(&sc->accum, 0u, abort, status)) {
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
-      for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
-        float v[16];
-        tmem_ld16(lane_addr + (uint32_t)c0, v);
-        if (EPI == EPI_PARTIAL) {
-          float* out = p.P + (size_t)split * p.n_alloc * p.M;
+    const int row = quad * 32 + lane;
+    const int etid = threadIdx.x - 64;
+    bool ok = *(volatile int32_t*)status == 0;
+    int seg = 0;
+    // value of token block [c0, c0 + 16) of tile t2: hi half + lo half of the accumulator
+    auto load16 = [&](uint32_t lane_addr, int t2, int c0, float* v) {
+      const uint32_t col = (uint32_t)(t2 * 2 * p.n_pad + (c0 / p.box_rows) * 2 * p.box_rows + c0 % p.box_rows);
+      float lo[16];
+      tmem_ld16(lane_addr + col, v);
+      tmem_ld16(lane_addr + col + (uint32_t)p.box_rows, lo);
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const int t = c0 + j;
-            if (t < p.n && row_ok) out[(size_t)t * p.M + m] = v[j];
-          }
-        } else if (EPI == EPI_SWIGLU) {
-          const int F = p.M >> 1;
+      for (int j = 0; j < 16; ++j) v[j] += lo[j];
+    };
+    for (long long u = u0; u < u1; ++seg) {
+      const int group = (int)(u / KB);
+      const int kb0 = (int)(u % KB);
+      const int kb1 = (int)((u1 - u) < (long long)(KB - kb0) ? kb0 + (u1 - u) : KB);
+      u += kb1 - kb0;
+      const int b = seg % p.n_buf;
+      if (ok) ok = mbar_wait(&sc->acc_full[b], (uint32_t)((seg / p.n_buf) & 1), abort, status);
+      tc_fence_after();
+      const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(b * acc_cols);
+
+      if (EPI == EPI_PARTIAL) {
+        if (ok) {
+          float* out = p.P + (size_t)(cta % p.splits) * p.n_alloc * p.M;
+          for (int t2 = 0; t2 < p.tm; ++t2) {
+            const int m = (group * p.tm + t2) * TILE_M + row;
+            for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
+              float v[16];
+              load16(lane_addr, t2, c0, v);
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const int t = c0 + j;
-            const float other = __shfl_xor_sync(0xFFFFFFFFu, v[j], 1);
-            const float g = (lane & 1) ? other : v[j];
-            const float u = (lane & 1) ? v[j] : other;
-            const float a = g / (1.f + expf(-g)) * u;
-            bf16 hi, lo;
-            split_bf16(a, hi, lo);
-            if (t < p.n && row_ok) {
-              const size_t o = (size_t)t * F + (m >> 1);
-              if (lane & 1) p.A[(size_t)p.n_alloc * F + o] = lo;
-              else p.A[o] = hi;
+              for (int j = 0; j < 16; ++j)
+                if (c0 + j < p.n && m < p.M) out[(size_t)(c0 + j) * p.M + m] = v[j];
             }
           }
-        } else {
+          tc_fence_before();
+          mbar_arrive(&sc->acc_empty[b]);
+        }
+        continue;
+      }
+
+      if (kb0 != 0) {
+        // later k-blocks of a tile group whose first k-blocks belong to an earlier CTA: park the partial sums
+        float* dst = p.fixP + (size_t)cta * p.tm * p.n_pad * TILE_M;
+        if (ok) {
+          for (int t2 = 0; t2 < p.tm; ++t2)
+            for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
+              float v[16];
+              load16(lane_addr, t2, c0, v);
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const int t = c0 + j;
-            if (p.logits && t < p.n && row_ok) p.logits[(size_t)t * p.M + m] = v[j];
-            unsigned long long key = row_ok ? pack_max_key(v[j], (uint32_t)m) : 0ull;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-              const unsigned long long other = __shfl_xor_sync(0xFFFFFFFFu, key, o);
-              key = other > key ? other : key;
+              for (int j = 0; j < 16; ++j) dst[(size_t)(t2 * p.n_pad + c0 + j) * TILE_M + row] = v[j];
             }
-            if (lane == 0 && t < p.n) atomicMax(&sc->key[t], key);
+          tc_fence_before();
+          mbar_arrive(&sc->acc_empty[b]);
+          __threadfence();
+        }
+        epi_bar();
+        if (ok && threadIdx.x == 64) st_release(p.fixFlag + cta, p.epoch);
+        continue;
+      }
+
+      // first k-blocks of the tile group: collect the partial sums of the CTAs that hold the rest
+      int last = cta;
+      if (kb1 != KB)
+        while (last + 1 < G && (last + 1) * U / G < (long long)(group + 1) * KB) ++last;
+      if (last > cta) {
+        if (ok && threadIdx.x == 64) {
+          const unsigned long long t0 = global_ns();
+          for (int cc = cta + 1; cc <= last && !*abort; ++cc) {
+            while (ld_acquire(p.fixFlag + cc) != p.epoch) {
+              if (*abort) break;
+              if (global_ns() - t0 > WAIT_LIMIT_NS) {
+                *abort = 1;
+                atomicExch(status, (int32_t)SPECASR_ERR_TIMEOUT);
+                break;
+              }
+              __nanosleep(64);
+            }
           }
         }
+        epi_bar();
+        if (*abort) ok = false;
       }
-      if (EPI == EPI_ARGMAX) {
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        for (int t = threadIdx.x - 64; t < p.n; t += 128) p.amax[(size_t)tile * p.n_alloc + t] = sc->key[t];
+      for (int t2 = 0; t2 < p.tm; ++t2) {
+        const int tile = group * p.tm + t2;
+        if (tile >= p.tiles) break;
+        const int m = tile * TILE_M + row;
+        const bool row_ok = m < p.M;
+        if (EPI == EPI_ARGMAX) {
+          for (int t = etid; t < SPECASR_MAX_NODES; t += 128) sc->key[t] = 0ull;
+          epi_bar();
+        }
+        if (ok) {
+          for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
+            float v[16];
+            load16(lane_addr, t2, c0, v);
+            for (int cc = cta + 1; cc <= last; ++cc) {
+              const float* src = p.fixP + ((size_t)(cc * p.tm + t2) * p.n_pad + c0) * TILE_M + row;
+#pragma unroll
+              for (int j = 0; j < 16; ++j) v[j] += __ldcg(src + j * TILE_M);
+            }
+            if (EPI == EPI_SWIGLU) {
+              // rows 2f / 2f + 1 of the tile are gate / up of feature f: the even lane keeps the hi plane of
+              // the product, the odd lane the lo plane, staged in shared memory for 16-byte global stores
+              float a[16];
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                const float other = __shfl_xor_sync(0xFFFFFFFFu, v[j], 1);
+                const float g = (lane & 1) ? other : v[j];
+                const float up = (lane & 1) ? v[j] : other;
+                a[j] = __fdividef(g, 1.f + __expf(-g)) * up;
+              }
+              bf16* st = epi_stage + (size_t)(lane & 1) * p.n_pad * 64 + (size_t)c0 * 64 + (row >> 1);
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                bf16 hi, lo;
+                split_bf16(a[j], hi, lo);
+                st[j * 64] = (lane & 1) ? lo : hi;
+              }
+            } else if (EPI == EPI_ARGMAX) {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                const int t = c0 + j;
+                if (p.logits && t < p.n && row_ok) p.logits[(size_t)t * p.M + m] = v[j];
+                // warp arg-max: largest ordered key, then the lowest row among its holders
+                uint32_t key = __float_as_uint(v[j]);
+                key = (key & 0x80000000u) ? ~key : (key | 0x80000000u);
+                if (!row_ok) key = 0u;
+                const uint32_t best = __reduce_max_sync(0xFFFFFFFFu, key);
+                const uint32_t who = __reduce_min_sync(0xFFFFFFFFu, key == best ? (uint32_t)m : 0xFFFFFFFFu);
+                if (lane == 0 && t < p.n && best != 0u)
+                  atomicMax(&sc->key[t], ((unsigned long long)best << 32) | (unsigned long long)(0xFFFFFFFFu - who));
+              }
+            }
+          }
+        }
+        if (EPI == EPI_SWIGLU) {
+          epi_bar();
+          if (ok) {
+            const int F = p.M >> 1;
+            const int f0 = tile * 64;
+            const int chunks = 2 * p.n * 8;                 // 16-byte pieces of the [2][n][64] tile
+            for (int idx = etid; idx < chunks; idx += 128) {
+              const int plane = idx / (p.n * 8), rem = idx % (p.n * 8);
+              const int t = rem >> 3, ch = rem & 7;
+              if (f0 + ch * 8 < F)
+                *reinterpret_cast<uint4*>(p.A + (size_t)plane * p.n_alloc * F + (size_t)t * F + f0 + ch * 8) =
+                    *reinterpret_cast<const uint4*>(epi_stage + (size_t)plane * p.n_pad * 64 + t * 64 + ch * 8);
+            }
+          }
+          epi_bar();
+        }
+        if (EPI == EPI_ARGMAX) {
+          epi_bar();
+          if (ok)
+            for (int t = etid; t < p.n; t += 128) p.amax[(size_t)tile * p.n_alloc + t] = sc->key[t];
+        }
+      }
+      if (ok) {
+        tc_fence_before();
+        mbar_arrive(&sc->acc_empty[b]);
       }
     }
   }
 
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  tc_fence_before();
   __syncthreads();
   if (*abort) {
     // give copies still in flight time to land before the shared memory is handed back
@@ -197,9 +392,8 @@ __global__ void __launch_bounds__(192, 1) k_gemm_tc(const __grid_constant__ CUte
     __syncthreads();
   }
   if (warp == 1) {
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols)
-                 : "memory");
+    tc_fence_after();
+    tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
   }
 }
 
@@ -219,10 +413,23 @@ EncodeTiledFn get_encode() {
   return fn;
 }
 
+
+
 int pick_box_rows(int n_pad) {
-  int b = 256;
+  int b = 128;      // one MMA spans both planes of a box: N = 2 * box rows <= 256
   while (b > 16 && (n_pad % b) != 0) b >>= 1;
   return b;
+}
+
+template <int EPI>
+void launch_epi(const CUtensorMap& tmW, const CUtensorMap& tmAct, const TcParams& p, int grid, size_t smem,
+                cudaStream_t s) {
+  static bool configured = false;
+  if (!configured) {
+    cudaFuncSetAttribute(k_proj<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);
+    configured = true;
+  }
+  launch_pdl(k_proj<EPI>, dim3(grid), dim3(192), smem, s, tmW, tmAct, p);
 }
 
 }  // namespace
@@ -297,46 +504,66 @@ bool make_act_map(CUtensorMap* out, const void* base, uint64_t K, uint64_t n_all
 
 int gemm_tc_tiles(int M) { return (M + TILE_M - 1) / TILE_M; }
 
-int gemm_tc_pick_splits(const specasr_model* m, int M, int K) {
-  const int tiles = gemm_tc_tiles(M);
-  const int KB = (K + TILE_K - 1) / TILE_K;
-  int s = m->n_sm / tiles;
+// Tile groups per stage and k sub-blocks per stage for trees padded to n_pad nodes.
+static void tc_shape(int n_pad, int* tm, int* ksub) {
+  *tm = (n_pad >= 48 && n_pad <= 64) ? 2 : 1;     // two sets of tm * 2 * n_pad TMEM columns must fit in 512
+  *ksub = n_pad <= 64 ? 2 : 1;                    // 256 contiguous bytes per weight row keep DRAM pages busy
+}
+
+// Number of k parts of the linear projections: tile groups * parts should just fill the SMs.
+int gemm_tc_pick_splits(const specasr_model* m, int M, int K, int n_pad) {
+  int tm, ksub;
+  tc_shape(n_pad, &tm, &ksub);
+  const int groups = (gemm_tc_tiles(M) + tm - 1) / tm;
+  const int KB = (K + ksub * SUB_K - 1) / (ksub * SUB_K);
+  int s = m->n_sm / groups;
   if (s > kMaxSplitK) s = kMaxSplitK;
   if (s > KB) s = KB;
   if (s < 1) s = 1;
   return s;
 }
 
+// Bytes of the parked-partial workspace for trees of up to n_alloc nodes.
+size_t gemm_tc_fixup_bytes(const specasr_model* m, int n_alloc) {
+  return (size_t)m->n_sm * 2 * n_alloc * TILE_M * sizeof(float);
+}
+
 void launch_gemm_tc(specasr_kv* kv, const GemmArgs& a, int kind, cudaStream_t s) {
+  const specasr_model* m = kv->m;
   TcParams p;
+  memset(&p, 0, sizeof(p));
   p.M = a.M; p.K = a.K; p.n = a.n; p.n_pad = a.n_pad; p.n_alloc = a.n_alloc;
   p.box_rows = pick_box_rows(a.n_pad);
-  const int stage_bytes = W_TILE_BYTES + a.n_pad * 2 * TILE_K * 2;
-  int stages = (SMEM_BUDGET - (int)sizeof(SharedCtl) - 1024) / stage_bytes;
+  tc_shape(a.n_pad, &p.tm, &p.ksub);
+  const int stage_bytes = p.ksub * (p.tm * W_SUB_BYTES + a.n_pad * 2 * SUB_K * 2);
+  const int epi_bytes = a.epilogue == EPI_SWIGLU ? 2 * a.n_pad * 64 * 2 : 0;     // staged output tile
+  int stages = (SMEM_LIMIT - (int)sizeof(SharedCtl) - epi_bytes - 1024) / stage_bytes;
   if (stages > MAX_STAGES) stages = MAX_STAGES;
   p.stages = stages;
+  const int acc_cols = p.tm * 2 * a.n_pad;
+  p.n_buf = 2 * acc_cols <= 512 ? 2 : 1;
   int cols = 32;
-  while (cols < a.n_pad) cols <<= 1;
+  while (cols < p.n_buf * acc_cols) cols <<= 1;
   p.tmem_cols = cols;
-  p.splits = a.epilogue == EPI_PARTIAL ? a.splits : 1;
+  p.KB = (a.K + p.ksub * SUB_K - 1) / (p.ksub * SUB_K);
+  p.tiles = gemm_tc_tiles(a.M);
+  p.groups = (p.tiles + p.tm - 1) / p.tm;
+  p.splits = a.epilogue == EPI_PARTIAL ? a.splits : 0;
+  p.epoch = ++kv->gemm_epoch;
+  p.ctl = kv->ws.ctl;
+  p.fixP = kv->ws.fixP;
+  p.fixFlag = kv->ws.fixFlag;
   p.P = a.P; p.A = a.A; p.amax = a.amax; p.logits = a.logits;
-  p.ctl = const_cast<int32_t*>(a.ctl);
-  const size_t smem = (size_t)stages * stage_bytes + sizeof(SharedCtl) + 1024;
-  static bool configured = false;
-  if (!configured) {
-    cudaFuncSetAttribute(k_gemm_tc<EPI_PARTIAL>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET);
-    cudaFuncSetAttribute(k_gemm_tc<EPI_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET);
-    cudaFuncSetAttribute(k_gemm_tc<EPI_ARGMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET);
-    configured = true;
-  }
-  const CUtensorMap* act = &a.tmAct[0];
-  // a.tmAct points at an array of maps indexed by log2(box_rows / 16)
-  int idx = 0;
+  const long long units = (long long)p.groups * p.KB;
+  const int grid = a.epilogue == EPI_PARTIAL ? p.groups * p.splits : (int)(units < m->n_sm ? units : m->n_sm);
+  const size_t smem = (size_t)stages * stage_bytes + sizeof(SharedCtl) + epi_bytes + 1024;
+  int idx = 0;      // a.tmAct is an array of maps indexed by log2(box_rows / 16)
   for (int b = 16; b < p.box_rows; b <<= 1) ++idx;
-  act = &a.tmAct[idx];
-  dim3 grid(gemm_tc_tiles(a.M), p.splits);
+  const CUtensorMap& act = a.tmAct[idx];
   LaunchScope scope(kv, kind, s);
-  if (a.epilogue == EPI_PARTIAL) k_gemm_tc<EPI_PARTIAL><<<grid, 192, smem, s>>>(*a.tmW, *act, p);
-  else if (a.epilogue == EPI_SWIGLU) k_gemm_tc<EPI_SWIGLU><<<grid, 192, smem, s>>>(*a.tmW, *act, p);
-  else k_gemm_tc<EPI_ARGMAX><<<grid, 192, smem, s>>>(*a.tmW, *act, p);
+  switch (a.epilogue) {
+    case EPI_PARTIAL: launch_epi<EPI_PARTIAL>(*a.tmW, act, p, grid, smem, s); break;
+    case EPI_SWIGLU: launch_epi<EPI_SWIGLU>(*a.tmW, act, p, grid, smem, s); break;
+    default: launch_epi<EPI_ARGMAX>(*a.tmW, act, p, grid, smem, s); break;
+  }
 }

@@ -5,6 +5,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <string.h>
 
 #include <vector>
 
@@ -12,7 +13,7 @@
 
 typedef __nv_bfloat16 bf16;
 
-constexpr int kMaxSplitK = 8;      // split-K partial planes for the projections
+constexpr int kMaxSplitK = 12;     // partial planes of the linear projections
 constexpr int kMaxAttnSplits = 40; // KV splits of the attention kernels
 constexpr int kCtlWords = 64;      // int32 control block at the start of the workspace
 
@@ -47,7 +48,9 @@ struct Workspace {
   unsigned long long* anc;  // [n_alloc][4] ancestor-or-self bitmask over node indices
   float* X;                 // [n_alloc][d] residual stream
   bf16* H;                  // [2][n_alloc][d]      normed activations, hi / lo planes
-  float* P;                 // [kMaxSplitK][n_alloc][max(d, qkv_dim)] split-K partial sums
+  float* P;                 // [kMaxSplitK][n_alloc][max(d, qkv_dim)] partial sums of the linear projections
+  float* fixP;              // [n_sm][n_alloc][128] partial tiles of the persistent tensor-core projections
+  int32_t* fixFlag;         // [n_sm] launch number of the partial tile each CTA published last
   bf16* Q;                  // [2][n_alloc][q_dim]  rotated queries, hi / lo planes
   bf16* AO;                 // [2][n_alloc][q_dim]  attention output, hi / lo planes
   bf16* A;                  // [2][n_alloc][ffn]    SwiGLU output, hi / lo planes
@@ -76,6 +79,7 @@ struct specasr_kv {
   cudaEvent_t len_event;
   bool len_event_pending;
   int64_t launches;
+  int gemm_epoch;           // number of tensor-core projection launches so far (tags the fixup flags)
   // optional per-kernel timing (specasr_profile_*): event pairs recorded around every launch
   bool prof_on;
   std::vector<cudaEvent_t> prof_events;   // 2 per recorded launch
@@ -113,6 +117,25 @@ struct LaunchScope {
   }
 };
 
+// Launch with programmatic stream serialization: the kernel may start while its predecessor in the
+// stream is still running and must call griddepcontrol.wait before it touches anything the predecessor
+// writes (every kernel of this library does, whether or not it is launched this way).
+template <typename... KArgs, typename... Args>
+inline void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 void set_error(const char* fmt, ...);
 Workspace carve_workspace(const specasr_model* m, int n_alloc, void* base);
 int lm_tiles_of(const specasr_model* m);
@@ -140,7 +163,11 @@ bool attention_tc_make_maps(specasr_kv* kv);
 void launch_tree_attention_tc(specasr_kv* kv, int layer, int n, int n_splits, cudaStream_t s);
 
 // ---- gemm_fma.cu / gemm_tcgen05.cu
-enum GemmEpilogue { EPI_PARTIAL = 0, EPI_SWIGLU = 1, EPI_ARGMAX = 2 };
+enum GemmEpilogue {
+  EPI_PARTIAL = 0,   // fp32 partial sums [splits][n][M], added up by the consumer kernel
+  EPI_SWIGLU = 1,    // SiLU(gate) * up -> hi / lo planes
+  EPI_ARGMAX = 2     // per-tile arg-max candidates (+ optional logits)
+};
 struct GemmArgs {
   const bf16* W;            // [M, K]
   const CUtensorMap* tmW;   // tcgen05 path
@@ -158,7 +185,8 @@ struct GemmArgs {
 int gemm_fma_tiles(int M);
 void launch_gemm_fma(specasr_kv* kv, const GemmArgs& a, int kind, cudaStream_t s);
 int gemm_tc_tiles(int M);
-int gemm_tc_pick_splits(const specasr_model* m, int M, int K);
+size_t gemm_tc_fixup_bytes(const specasr_model* m, int n_alloc);
+int gemm_tc_pick_splits(const specasr_model* m, int M, int K, int n_pad);
 void launch_gemm_tc(specasr_kv* kv, const GemmArgs& a, int kind, cudaStream_t s);
 bool make_tensor_map_2d(CUtensorMap* out, const void* base, uint64_t inner, uint64_t outer,
                         uint32_t box_inner, uint32_t box_outer);

@@ -13,6 +13,8 @@ __global__ void k_tree_prep(int32_t* __restrict__ ctl, const int32_t* __restrict
                             unsigned long long* __restrict__ anc) {
   __shared__ int s_bad;
   const int i = threadIdx.x;
+  grid_dep_launch();
+  grid_dep_wait();
   if (i == 0) s_bad = 0;
   __syncthreads();
   const int L = ctl[CTL_LEN];
@@ -53,6 +55,8 @@ __global__ void k_tree_prep(int32_t* __restrict__ ctl, const int32_t* __restrict
 __global__ void k_chain_prep(int32_t* __restrict__ ctl, int n, int capacity, int32_t* __restrict__ depth,
                              int32_t* __restrict__ pos, unsigned long long* __restrict__ anc) {
   const int i = threadIdx.x;
+  grid_dep_launch();
+  grid_dep_wait();
   const int L = ctl[CTL_LEN];
   if (L < 0 || L + n > capacity) {
     if (i == 0) ctl[CTL_STATUS] = SPECASR_ERR_KV_CAPACITY;
@@ -81,7 +85,7 @@ void launch_tree_prep(specasr_kv* kv, const int32_t* tokens, const int32_t* pare
   int cap = kv->max_pages * m->cfg.page_size;
   if (m->cfg.max_positions < cap) cap = m->cfg.max_positions;
   LaunchScope scope(kv, SPECASR_KIND_PREP, s);
-  k_tree_prep<<<1, 256, 0, s>>>(kv->ws.ctl, tokens, parent, n, m->cfg.vocab, cap, kv->ws.depth, kv->ws.pos,
+  launch_pdl(k_tree_prep, dim3(1), dim3(256), 0, s, kv->ws.ctl, tokens, parent, n, m->cfg.vocab, cap, kv->ws.depth, kv->ws.pos,
                                 kv->ws.anc);
 }
 
@@ -90,13 +94,15 @@ void launch_chain_prep(specasr_kv* kv, int n, cudaStream_t s) {
   int cap = kv->max_pages * m->cfg.page_size;
   if (m->cfg.max_positions < cap) cap = m->cfg.max_positions;
   LaunchScope scope(kv, SPECASR_KIND_PREP, s);
-  k_chain_prep<<<1, 256, 0, s>>>(kv->ws.ctl, n, cap, kv->ws.depth, kv->ws.pos, kv->ws.anc);
+  launch_pdl(k_chain_prep, dim3(1), dim3(256), 0, s, kv->ws.ctl, n, cap, kv->ws.depth, kv->ws.pos, kv->ws.anc);
 }
 
 // ------------------------------------------------------------------------------------------------
 // Layer-0 inputs: embedding rows (bf16 -> fp32 residual stream), or caller-provided vectors.
 __global__ void k_embed_tokens(const int32_t* __restrict__ ctl, const int32_t* __restrict__ tokens,
                                const bf16* __restrict__ E, int d, float* __restrict__ X) {
+  grid_dep_launch();
+  grid_dep_wait();
   if (ctl[CTL_STATUS] != 0) return;
   const int i = blockIdx.x;
   const bf16* row = E + (size_t)tokens[i] * d;
@@ -116,6 +122,8 @@ __global__ void k_embed_tokens(const int32_t* __restrict__ ctl, const int32_t* _
 
 __global__ void k_copy_embeds(const int32_t* __restrict__ ctl, const float* __restrict__ src, int d,
                               float* __restrict__ X) {
+  grid_dep_launch();
+  grid_dep_wait();
   if (ctl[CTL_STATUS] != 0) return;
   const int i = blockIdx.x;
   for (int k = threadIdx.x * 4; k < d; k += blockDim.x * 4)
@@ -124,24 +132,25 @@ __global__ void k_copy_embeds(const int32_t* __restrict__ ctl, const float* __re
 
 void launch_embed_tokens(specasr_kv* kv, const int32_t* tokens, int n, cudaStream_t s) {
   LaunchScope scope(kv, SPECASR_KIND_PREP, s);
-  k_embed_tokens<<<n, 128, 0, s>>>(kv->ws.ctl, tokens, kv->m->embed, kv->m->cfg.d_model, kv->ws.X);
+  launch_pdl(k_embed_tokens, dim3(n), dim3(128), 0, s, kv->ws.ctl, tokens, kv->m->embed, kv->m->cfg.d_model, kv->ws.X);
 }
 
 void launch_copy_embeds(specasr_kv* kv, const float* embeds, int n, cudaStream_t s) {
   LaunchScope scope(kv, SPECASR_KIND_PREP, s);
-  k_copy_embeds<<<n, 128, 0, s>>>(kv->ws.ctl, embeds, kv->m->cfg.d_model, kv->ws.X);
+  launch_pdl(k_copy_embeds, dim3(n), dim3(128), 0, s, kv->ws.ctl, embeds, kv->m->cfg.d_model, kv->ws.X);
 }
 
 // ------------------------------------------------------------------------------------------------
-// RMSNorm with the residual update folded in: x <- x + sum of the previous projection's split-K
-// partial planes (fixed order, hence deterministic), h = x * rsqrt(mean(x^2) + eps) * g, emitted as
-// two bf16 planes hi = bf16(h), lo = bf16(h - hi) so that the tensor-core projections see ~16
-// significant bits of every activation.  Rows n..n_pad-1 of both planes are zeroed.
+// RMSNorm with the residual update folded in: x <- x + sum of the previous projection's partial planes
+// (fixed order, hence deterministic), h = x * rsqrt(mean(x^2) + eps) * g, emitted as two bf16 planes
+// hi = bf16(h), lo = bf16(h - hi) so that the tensor-core projections see ~16 significant bits of every
+// activation.  Rows n..n_pad-1 of both planes are zeroed.
 __global__ void __launch_bounds__(256) k_rmsnorm_split(const int32_t* __restrict__ ctl, float* __restrict__ X,
                                                        const float* __restrict__ P, int n_partials,
-                                                       size_t partial_stride, const float* __restrict__ gain,
-                                                       int d, float eps, int n, size_t plane_stride,
-                                                       bf16* __restrict__ H) {
+                                                       size_t partial_stride, const float* __restrict__ gain, int d, float eps, int n,
+                                                       size_t plane_stride, bf16* __restrict__ H) {
+  grid_dep_launch();
+  grid_dep_wait();
   if (ctl[CTL_STATUS] != 0) return;
   const int row = blockIdx.x;
   bf16* hi = H + (size_t)row * d;
@@ -158,7 +167,7 @@ __global__ void __launch_bounds__(256) k_rmsnorm_split(const int32_t* __restrict
   for (int k = threadIdx.x * 4; k < d; k += blockDim.x * 4) {
     float4 v = *reinterpret_cast<const float4*>(x + k);
     for (int s = 0; s < n_partials; ++s) {
-      const float4 p = *reinterpret_cast<const float4*>(P + s * partial_stride + (size_t)row * d + k);
+      const float4 p = __ldcg(reinterpret_cast<const float4*>(P + s * partial_stride + (size_t)row * d + k));
       v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
     }
     if (n_partials > 0) *reinterpret_cast<float4*>(x + k) = v;
@@ -182,21 +191,23 @@ void launch_rmsnorm_split(specasr_kv* kv, const float* gain, int n, int n_pad, i
   const specasr_model* m = kv->m;
   const int d = m->cfg.d_model;
   LaunchScope scope(kv, SPECASR_KIND_NORM, s);
-  k_rmsnorm_split<<<n_pad, 256, 0, s>>>(kv->ws.ctl, kv->ws.X, kv->ws.P, n_partials, (size_t)kv->n_alloc * d, gain,
-                                        d, m->cfg.rms_eps, n, (size_t)kv->n_alloc * d, kv->ws.H);
+  launch_pdl(k_rmsnorm_split, dim3(n_pad), dim3(256), 0, s, kv->ws.ctl, kv->ws.X, kv->ws.P, n_partials, (size_t)kv->n_alloc * d, gain,
+             d, m->cfg.rms_eps, n, (size_t)kv->n_alloc * d, kv->ws.H);
 }
 
 // ------------------------------------------------------------------------------------------------
 // Rotary embedding at tree positions + KV append.  One block per (node, head of the fused QKV row).
-// Sums the QKV projection's split-K partials, rotates Q and K heads by the angle of the node's
-// position (rotate-half pairing, table built in fp64 on the host), writes Q as hi/lo planes and K,V
-// as hi/lo planes into cache slot L + node.
+// Sums the QKV projection's partial planes (their columns follow the rotary-paired row order of Wqkv),
+// rotates Q and K heads by the angle of
+// the node's position (rotate-half pairing, table built in fp64 on the host), writes Q as hi/lo planes
+// and K,V as hi/lo planes into cache slot L + node.
 __global__ void k_rope_append(const int32_t* __restrict__ ctl, const float* __restrict__ P, int n_partials,
-                              size_t partial_stride, int qkv_dim, int Hq, int Hkv, int dh,
-                              const int32_t* __restrict__ pos, const float2* __restrict__ rope, int layer,
-                              bf16* __restrict__ Q, size_t q_plane_stride, bf16* __restrict__ k_pool,
+                              size_t partial_stride, int qkv_dim, int Hq, int Hkv, int dh, const int32_t* __restrict__ pos, const float2* __restrict__ rope,
+                              int layer, bf16* __restrict__ Q, size_t q_plane_stride, bf16* __restrict__ k_pool,
                               bf16* __restrict__ v_pool, const int32_t* __restrict__ page_table, int n_pages,
                               int page_size) {
+  grid_dep_launch();
+  grid_dep_wait();
   if (ctl[CTL_STATUS] != 0) return;
   const int i = blockIdx.x;
   const int head = blockIdx.y;
@@ -204,10 +215,11 @@ __global__ void k_rope_append(const int32_t* __restrict__ ctl, const float* __re
   const int k = threadIdx.x;
   if (k >= half) return;
   const size_t col = (size_t)i * qkv_dim + (size_t)head * dh;
+  const size_t c1 = col + qkv_row_of_feature(k, dh), c2 = col + qkv_row_of_feature(k + half, dh);
   float x1 = 0.f, x2 = 0.f;
   for (int s = 0; s < n_partials; ++s) {
-    x1 += P[s * partial_stride + col + k];
-    x2 += P[s * partial_stride + col + k + half];
+    x1 += __ldcg(P + s * partial_stride + c1);
+    x2 += __ldcg(P + s * partial_stride + c2);
   }
   const bool is_v = head >= Hq + Hkv;
   if (!is_v) {
@@ -247,10 +259,9 @@ void launch_rope_append(specasr_kv* kv, int layer, int n, int n_partials, cudaSt
   dim3 grid(n, c.n_heads + 2 * c.n_kv_heads);
   const int threads = c.head_dim / 2 < 32 ? 32 : c.head_dim / 2;
   LaunchScope scope(kv, SPECASR_KIND_ROPE, s);
-  k_rope_append<<<grid, threads, 0, s>>>(kv->ws.ctl, kv->ws.P, n_partials, (size_t)kv->n_alloc * m->qkv_dim,
-                                         m->qkv_dim, c.n_heads, c.n_kv_heads, c.head_dim, kv->ws.pos,
-                                         m->rope_table, layer, kv->ws.Q, (size_t)kv->n_alloc * m->q_dim,
-                                         kv->k_pool, kv->v_pool, kv->page_table, kv->n_pages, c.page_size);
+  launch_pdl(k_rope_append, grid, dim3(threads), 0, s, kv->ws.ctl, kv->ws.P, n_partials, (size_t)kv->n_alloc * m->qkv_dim, m->qkv_dim, c.n_heads, c.n_kv_heads,
+             c.head_dim, kv->ws.pos, m->rope_table, layer, kv->ws.Q, (size_t)kv->n_alloc * m->q_dim, kv->k_pool,
+             kv->v_pool, kv->page_table, kv->n_pages, c.page_size);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -259,6 +270,8 @@ void launch_rope_append(specasr_kv* kv, int layer, int n, int n_partials, cudaSt
 __global__ void k_attn_merge(const int32_t* __restrict__ ctl, const float* __restrict__ attO,
                              const float2* __restrict__ attML, int n_splits, size_t rows_alloc, int Hq, int dh,
                              int n, bf16* __restrict__ AO, size_t plane_stride) {
+  grid_dep_launch();
+  grid_dep_wait();
   if (ctl[CTL_STATUS] != 0) return;
   const int i = blockIdx.x;
   const int h = blockIdx.y;
@@ -294,7 +307,7 @@ void launch_attn_merge(specasr_kv* kv, int n, int n_pad, int n_splits, cudaStrea
   dim3 grid(n_pad, c.n_heads);
   const int threads = c.head_dim < 32 ? 32 : c.head_dim;
   LaunchScope scope(kv, SPECASR_KIND_ATTN_MERGE, s);
-  k_attn_merge<<<grid, threads, 0, s>>>(kv->ws.ctl, kv->ws.attO, kv->ws.attML, n_splits,
+  launch_pdl(k_attn_merge, grid, dim3(threads), 0, s, kv->ws.ctl, kv->ws.attO, kv->ws.attML, n_splits,
                                         (size_t)kv->n_alloc * c.n_heads, c.n_heads, c.head_dim, n, kv->ws.AO,
                                         (size_t)kv->n_alloc * kv->m->q_dim);
 }
@@ -312,6 +325,8 @@ __global__ void __launch_bounds__(256) k_accept(const int32_t* __restrict__ ctl,
   __shared__ int s_arg[SPECASR_MAX_NODES];
   __shared__ unsigned int s_best;
   const int i = threadIdx.x;
+  grid_dep_launch();
+  grid_dep_wait();
   if (ctl[CTL_STATUS] != 0) {
     if (i < n) {
       out_path[i] = -1;
@@ -366,28 +381,32 @@ void launch_accept(specasr_kv* kv, const int32_t* tokens, const int32_t* parent,
                    int32_t* out_argmax, int32_t* out_accept_len, int32_t* out_path, int32_t* out_bonus,
                    cudaStream_t s) {
   LaunchScope scope(kv, SPECASR_KIND_ACCEPT, s);
-  k_accept<<<1, 256, 0, s>>>(kv->ws.ctl, kv->ws.amax, n_tiles, kv->n_alloc, tokens, parent, kv->ws.depth, n,
+  launch_pdl(k_accept, dim3(1), dim3(256), 0, s, kv->ws.ctl, kv->ws.amax, n_tiles, kv->n_alloc, tokens, parent, kv->ws.depth, n,
                              out_argmax, out_accept_len, out_path, out_bonus);
 }
 
 // ------------------------------------------------------------------------------------------------
 // Cache length bookkeeping.
 __global__ void k_advance_len(int32_t* ctl, int n) {
+  grid_dep_launch();
+  grid_dep_wait();
   if (ctl[CTL_STATUS] != 0) return;
   ctl[CTL_LEN] += n;
 }
 __global__ void k_set_len(int32_t* ctl, int len) {
+  grid_dep_launch();
+  grid_dep_wait();
   ctl[CTL_LEN] = len;
   ctl[CTL_STATUS] = 0;
   ctl[CTL_N] = 0;
 }
 void launch_advance_len(specasr_kv* kv, int n, cudaStream_t s) {
   LaunchScope scope(kv, SPECASR_KIND_COMMIT, s);
-  k_advance_len<<<1, 1, 0, s>>>(kv->ws.ctl, n);
+  launch_pdl(k_advance_len, dim3(1), dim3(1), 0, s, kv->ws.ctl, n);
 }
 void launch_set_len(specasr_kv* kv, int len, cudaStream_t s) {
   LaunchScope scope(kv, SPECASR_KIND_COMMIT, s);
-  k_set_len<<<1, 1, 0, s>>>(kv->ws.ctl, len);
+  launch_pdl(k_set_len, dim3(1), dim3(1), 0, s, kv->ws.ctl, len);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -398,6 +417,8 @@ __global__ void __launch_bounds__(256) k_commit(const int32_t* __restrict__ ctl,
                                                 const int32_t* __restrict__ accept_len, bf16* __restrict__ k_pool,
                                                 bf16* __restrict__ v_pool, const int32_t* __restrict__ page_table,
                                                 int n_pages, int Hkv, int page_size, int dh) {
+  grid_dep_launch();
+  grid_dep_wait();
   const int a = accept_len[0];
   const int n = ctl[CTL_N];
   if (ctl[CTL_STATUS] != 0 || a < 0 || a >= n) return;
@@ -427,6 +448,8 @@ __global__ void __launch_bounds__(256) k_commit(const int32_t* __restrict__ ctl,
 }
 
 __global__ void k_commit_finish(int32_t* ctl, const int32_t* __restrict__ accept_len) {
+  grid_dep_launch();
+  grid_dep_wait();
   const int a = accept_len[0];
   const int n = ctl[CTL_N];
   if (ctl[CTL_STATUS] != 0 || a < 0 || a >= n) return;
@@ -438,8 +461,8 @@ void launch_commit(specasr_kv* kv, const int32_t* path, const int32_t* accept_le
   const specasr_model_config& c = kv->m->cfg;
   dim3 grid(c.n_layers, 2);
   LaunchScope scope(kv, SPECASR_KIND_COMMIT, s);
-  k_commit<<<grid, 256, 0, s>>>(kv->ws.ctl, path, accept_len, kv->k_pool, kv->v_pool, kv->page_table, kv->n_pages,
+  launch_pdl(k_commit, grid, dim3(256), 0, s, kv->ws.ctl, path, accept_len, kv->k_pool, kv->v_pool, kv->page_table, kv->n_pages,
                                 c.n_kv_heads, c.page_size, c.head_dim);
-  k_commit_finish<<<1, 1, 0, s>>>(kv->ws.ctl, accept_len);
+  launch_pdl(k_commit_finish, dim3(1), dim3(1), 0, s, kv->ws.ctl, accept_len);
   kv->launches++;
 }

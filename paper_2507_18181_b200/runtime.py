@@ -27,6 +27,13 @@ class DeviceModel:
         self.page_size = page_size
         L = cfg.n_layers
         got = {}
+        # rotary-paired row order of the fused QKV matrix (see include/specasr.h): within every head,
+        # stored row 32 g + 16 h + j holds feature 16 g + j + h * head_dim / 2
+        dh = cfg.head_dim
+        rho = np.arange(dh)
+        feat = (rho // 32) * 16 + rho % 16 + ((rho % 32) // 16) * (dh // 2)
+        n_heads_all = cfg.n_heads + 2 * cfg.n_kv_heads
+        self._qkv_rows = torch.from_numpy((np.arange(n_heads_all)[:, None] * dh + feat[None, :]).reshape(-1)).to(self.device)
 
         def put(layer, name, arr):
             if arr.dtype == np.uint16:
@@ -34,7 +41,8 @@ class DeviceModel:
             else:
                 got[(layer, name)] = torch.from_numpy(np.ascontiguousarray(arr, dtype=np.float32)).to(self.device)
             if layer >= 0 and all((layer, k) in got for k in ("wq", "wk", "wv")):
-                got[(layer, "wqkv")] = torch.cat([got.pop((layer, k)) for k in ("wq", "wk", "wv")], dim=0).contiguous()
+                fused = torch.cat([got.pop((layer, k)) for k in ("wq", "wk", "wv")], dim=0)
+                got[(layer, "wqkv")] = fused[self._qkv_rows].contiguous()
             if layer >= 0 and all((layer, k) in got for k in ("wg", "wu")):
                 g, u = got.pop((layer, "wg")), got.pop((layer, "wu"))
                 got[(layer, "wgu")] = torch.stack([g, u], dim=1).reshape(2 * cfg.ffn, cfg.d_model).contiguous()
