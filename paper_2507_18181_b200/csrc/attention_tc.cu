@@ -27,11 +27,16 @@ namespace {
 constexpr int KEYS = 128;                 // cache positions per CTA
 constexpr int SUB = 128 * 64 * 2;         // bytes of one [128 rows][64 bf16] swizzled sub-tile
 
+constexpr int SOFTMAX_THREADS = 256;      // warps 2..9; warps w and w + 4 share a TMEM lane quadrant
+
 struct AttnCtl {
   unsigned long long bar_qk, bar_v, bar_s, bar_p, bar_o;
+  float red_max[2][128];      // per-row partial maxima / sums of the two warps that share a row
+  float red_sum[2][128];
   uint32_t tmem_base;
   int abort;
 };
+__device__ __forceinline__ void softmax_bar() { asm volatile("bar.sync 2, 256;" ::: "memory"); }
 
 struct AttnParams {
   int32_t* ctl;
@@ -45,7 +50,7 @@ struct AttnParams {
 };
 
 template <int DH>
-__global__ void __launch_bounds__(192, 1) k_tree_attention_tc(const __grid_constant__ CUtensorMap tmQ,
+__global__ void __launch_bounds__(64 + SOFTMAX_THREADS, 1) k_tree_attention_tc(const __grid_constant__ CUtensorMap tmQ,
                                                               const __grid_constant__ CUtensorMap tmK,
                                                               const __grid_constant__ CUtensorMap tmV, AttnParams p) {
   constexpr int H = DH / 64;                               // 64-wide halves of the head
@@ -64,7 +69,7 @@ __global__ void __launch_bounds__(192, 1) k_tree_attention_tc(const __grid_const
   const int Ltot = L + p.n;
   const int k_begin = split * KEYS;
 
-  // row owned by an epilogue thread (warps 2..5): TMEM lane = 32 * (warp % 4) + lane
+  // row owned by a softmax thread (warps 2..9): TMEM lane = 32 * (warp % 4) + lane
   const int r = ((warp & 3) << 5) | lane;
   const int node = node0 + r / p.group;
   const bool row_valid = warp >= 2 && r < rows_used && node < p.n;
@@ -87,7 +92,7 @@ __global__ void __launch_bounds__(192, 1) k_tree_attention_tc(const __grid_const
     mbar_init(&sc->bar_qk, 1);
     mbar_init(&sc->bar_v, 1);
     mbar_init(&sc->bar_s, 1);
-    mbar_init(&sc->bar_p, 128);
+    mbar_init(&sc->bar_p, SOFTMAX_THREADS);
     mbar_init(&sc->bar_o, 1);
     sc->abort = 0;
     mbar_fence_init();
@@ -178,8 +183,10 @@ __global__ void __launch_bounds__(192, 1) k_tree_attention_tc(const __grid_const
       umma_commit(&sc->bar_o);
     }
   } else if (warp >= 2) {
-    // ---------------- softmax and epilogue: one thread per query row.  The loops over 32-column
-    // chunks are kept rolled on purpose: straight-line code that runs once is bound by instruction fetch.
+    // ---------------- softmax and epilogue: two threads per query row (warps w and w + 4), each taking
+    // alternate 32-key chunks.  The chunk loops are kept rolled on purpose: straight-line code that runs
+    // once is bound by instruction fetch.
+    const int eg = (warp - 2) >> 2;
     unsigned long long anc0 = 0ull, anc1 = 0ull, anc2 = 0ull, anc3 = 0ull;
     if (row_valid) {
       anc0 = p.anc[node * 4 + 0];
@@ -203,33 +210,41 @@ __global__ void __launch_bounds__(192, 1) k_tree_attention_tc(const __grid_const
     };
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
     bool ok = mbar_wait(&sc->bar_s, 0u, abort, status);
-    float m_row = -INFINITY, l_row = 0.f;
+    float m_row = -INFINITY, l_part = 0.f;
     if (ok) {
       tc_fence_after();
+      float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll 1
-      for (int c0 = 0; c0 < kc_pad; c0 += 32) {
+      for (int c0 = eg * 32; c0 < kc_pad; c0 += 64) {
         float s[32];
         tmem_ld32(tmem_s + lane_off + c0, s);
         const uint32_t vis = visible32(k_begin + c0);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) m_row = fmaxf(m_row, ((vis >> j) & 1u) ? s[j] * p.scale_log2 : -INFINITY);
+        for (int j = 0; j < 32; ++j) m4[j & 3] = fmaxf(m4[j & 3], ((vis >> j) & 1u) ? s[j] * p.scale_log2 : -INFINITY);
       }
+      m_row = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+    }
+    sc->red_max[eg][r] = m_row;
+    softmax_bar();
+    m_row = fmaxf(sc->red_max[0][r], sc->red_max[1][r]);
+    if (ok) {
       const float m_use = m_row > -INFINITY ? m_row : 0.f;    // a fully masked row gives p = 0 everywhere
+      float l2[2] = {0.f, 0.f};
 #pragma unroll 1
-      for (int c0 = 0; c0 < kc_pad; c0 += 32) {
+      for (int c0 = eg * 32; c0 < kc_pad; c0 += 64) {
         float s[32];
         tmem_ld32(tmem_s + lane_off + c0, s);
         const uint32_t vis = visible32(k_begin + c0);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) s[j] = ((vis >> j) & 1u) ? exp2f(s[j] * p.scale_log2 - m_use) : 0.f;
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
           uint32_t hi[4], lo[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const int j = g * 8 + 2 * e;
-            const float p0 = ((vis >> j) & 1u) ? exp2f(s[j] * p.scale_log2 - m_use) : 0.f;
-            const float p1 = ((vis >> (j + 1)) & 1u) ? exp2f(s[j + 1] * p.scale_log2 - m_use) : 0.f;
-            l_row += p0 + p1;
-            split2_pack(p0, p1, hi[e], lo[e]);
+            l2[e & 1] += s[j] + s[j + 1];
+            split2_pack(s[j], s[j + 1], hi[e], lo[e]);
           }
           const int c8 = (c0 >> 3) + g;                        // 8-key group within the block of 128
           if (c8 * 8 < kc_pad) {
@@ -239,29 +254,31 @@ __global__ void __launch_bounds__(192, 1) k_tree_attention_tc(const __grid_const
           }
         }
       }
+      l_part = l2[0] + l2[1];
       if (kc < kc_pad) {
         // value rows past the end of the cache meet p = 0, but 0 * garbage could still be NaN: clear them
         ok = mbar_wait(&sc->bar_v, 0u, abort, status);
-        if (ok && r < kc_pad - kc) {
+        if (ok && eg == 0 && r < kc_pad - kc) {
           for (int sub = 0; sub < 2 * H; ++sub)
             for (int i = 0; i < 8; ++i)
               *reinterpret_cast<uint4*>(Vs + sub * SUB + (kc + r) * 128 + i * 16) = make_uint4(0, 0, 0, 0);
         }
       }
     }
+    sc->red_sum[eg][r] = l_part;
     if (ok) {
       fence_proxy_async_smem();
       mbar_arrive(&sc->bar_p);
       ok = mbar_wait(&sc->bar_o, 0u, abort, status);
     }
+    // O leaves through the (now idle) K tile so that a warp writes whole rows: each thread parks its part of
+    // its row with the 16-byte columns rotated by the row number, then lane c reads column c of a row.
+    float4* stage = reinterpret_cast<float4*>(Ks);
+    constexpr int C4 = DH / 4;                               // float4 columns per row
     if (ok) {
       tc_fence_after();
-      // O leaves through the (now idle) K tile so that a warp writes whole 512-byte rows: thread r parks its
-      // row with the 16-byte columns rotated by r, then lane c of the warp reads column c of each of its 32 rows.
-      float4* stage = reinterpret_cast<float4*>(Ks);
-      constexpr int C4 = DH / 4;                             // float4 columns per row
 #pragma unroll 1
-      for (int c0 = 0; c0 < DH; c0 += 32) {
+      for (int c0 = eg * 32; c0 < DH; c0 += 64) {
         float o[32];
         tmem_ld32(tmem_o + lane_off + c0, o);
 #pragma unroll
@@ -270,10 +287,12 @@ __global__ void __launch_bounds__(192, 1) k_tree_attention_tc(const __grid_const
           stage[r * C4 + (c4 ^ (r & (C4 - 1)))] = make_float4(o[4 * e], o[4 * e + 1], o[4 * e + 2], o[4 * e + 3]);
         }
       }
-      __syncwarp();
-      const int r_base = (warp & 3) << 5;
+    }
+    softmax_bar();
+    if (ok) {
+      const int r_base = (warp - 2) * 16;                    // eight warps, sixteen rows each
 #pragma unroll 1
-      for (int i = 0; i < 32; ++i) {
+      for (int i = 0; i < 16; ++i) {
         const int rr = r_base + i;
         const int nd = node0 + rr / p.group;
         if (rr < rows_used && nd < p.n) {
@@ -282,7 +301,7 @@ __global__ void __launch_bounds__(192, 1) k_tree_attention_tc(const __grid_const
           for (int c4 = lane; c4 < C4; c4 += 32) dst[c4] = stage[rr * C4 + (c4 ^ (rr & (C4 - 1)))];
         }
       }
-      if (row_valid) p.attML[out_row] = make_float2(m_row, l_row);
+      if (row_valid && eg == 0) p.attML[out_row] = make_float2(m_row, sc->red_sum[0][r] + sc->red_sum[1][r]);
     }
   }
 
@@ -329,7 +348,7 @@ void launch_dh(specasr_kv* kv, int layer, int n, int n_splits, cudaStream_t s) {
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
   dim3 grid(c.n_kv_heads, (n + p.nodes_per_tile - 1) / p.nodes_per_tile, n_splits);
   LaunchScope scope(kv, SPECASR_KIND_ATTN, s);
-  launch_pdl(k_tree_attention_tc<DH>, grid, dim3(192), smem, s, kv->tm_Q, kv->tm_K, kv->tm_V, p);
+  launch_pdl(k_tree_attention_tc<DH>, grid, dim3(64 + SOFTMAX_THREADS), smem, s, kv->tm_Q, kv->tm_K, kv->tm_V, p);
 }
 
 }  // namespace

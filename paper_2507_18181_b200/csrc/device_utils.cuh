@@ -12,13 +12,13 @@ __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bflo
   lo = __float2bfloat16_rn(x - __bfloat162float(hi));
 }
 
-// Two values -> packed (hi0, hi1) and (lo0, lo1) words, element 0 in the low half.
+// Two values -> packed (hi0, hi1) and (lo0, lo1) words, element 0 in the low half; one packed
+// conversion per plane.
 __device__ __forceinline__ void split2_pack(float a, float b, uint32_t& hi, uint32_t& lo) {
-  __nv_bfloat16 ha, la, hb, lb;
-  split_bf16(a, ha, la);
-  split_bf16(b, hb, lb);
-  hi = (uint32_t)__bfloat16_as_ushort(ha) | ((uint32_t)__bfloat16_as_ushort(hb) << 16);
-  lo = (uint32_t)__bfloat16_as_ushort(la) | ((uint32_t)__bfloat16_as_ushort(lb) << 16);
+  const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+  hi = *reinterpret_cast<const uint32_t*>(&h);
+  const __nv_bfloat162 l = __floats2bfloat162_rn(a - bf16lo_to_f32(hi), b - bf16hi_to_f32(hi));
+  lo = *reinterpret_cast<const uint32_t*>(&l);
 }
 
 __device__ __forceinline__ float warp_sum(float v) {

@@ -23,8 +23,8 @@
 //    last) adds them in CTA order and runs the epilogue.  All CTAs are co-resident and every flag wait
 //    is bounded.
 //
-// Roles: warp 0 issues TMA, one thread of warp 1 issues tcgen05.mma, warps 2..5 drain TMEM
-// (tcgen05.ld) into the epilogue; two TMEM accumulator sets let the epilogue of one tile group overlap
+// Roles: warp 0 issues TMA, one thread of warp 1 issues tcgen05.mma, warps 2..9 drain TMEM
+// (tcgen05.ld; warps w and w + 4 share a lane quadrant and take alternate 16-token blocks) into the epilogue; two TMEM accumulator sets let the epilogue of one tile group overlap
 // the main loop of the next.
 //
 // Programmatic dependent launch: the weight tiles of the first pipeline stages are requested before
@@ -77,10 +77,11 @@ __device__ __forceinline__ int ld_acquire(const int32_t* p) {
 __device__ __forceinline__ void st_release(int32_t* p, int v) {
   asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
-__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+constexpr int EPI_THREADS = 256;      // warps 2..9
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 template <int EPI>
-__global__ void __launch_bounds__(192, 1) k_proj(const __grid_constant__ CUtensorMap tmW,
+__global__ void __launch_bounds__(64 + EPI_THREADS, 1) k_proj(const __grid_constant__ CUtensorMap tmW,
                                                  const __grid_constant__ CUtensorMap tmAct, TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -113,7 +114,7 @@ __global__ void __launch_bounds__(192, 1) k_proj(const __grid_constant__ CUtenso
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&sc->acc_full[b], 1);
-      mbar_init(&sc->acc_empty[b], 128);
+      mbar_init(&sc->acc_empty[b], EPI_THREADS);
     }
     sc->abort = 0;
     mbar_fence_init();
@@ -220,14 +221,14 @@ __global__ void __launch_bounds__(192, 1) k_proj(const __grid_constant__ CUtenso
     const int quad = warp & 3;
     const int row = quad * 32 + lane;
     const int etid = threadIdx.x - 64;
+    const int c_first = ((warp - 2) >> 2) * 16;          // this warp's first 16-token block; the stride is 32
     bool ok = *(volatile int32_t*)status == 0;
     int seg = 0;
     // value of token block [c0, c0 + 16) of tile t2: hi half + lo half of the accumulator
     auto load16 = [&](uint32_t lane_addr, int t2, int c0, float* v) {
       const uint32_t col = (uint32_t)(t2 * 2 * p.n_pad + (c0 / p.box_rows) * 2 * p.box_rows + c0 % p.box_rows);
       float lo[16];
-      tmem_ld16(lane_addr + col, v);
-      tmem_ld16(lane_addr + col + (uint32_t)p.box_rows, lo);
+      tmem_ld16x2(lane_addr + col, lane_addr + col + (uint32_t)p.box_rows, v, lo);
 #pragma unroll
       for (int j = 0; j < 16; ++j) v[j] += lo[j];
     };
@@ -246,7 +247,7 @@ __global__ void __launch_bounds__(192, 1) k_proj(const __grid_constant__ CUtenso
           float* out = p.P + (size_t)(cta % p.splits) * p.n_alloc * p.M;
           for (int t2 = 0; t2 < p.tm; ++t2) {
             const int m = (group * p.tm + t2) * TILE_M + row;
-            for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
+            for (int c0 = c_first; c0 < p.n_pad; c0 += 32) {
               float v[16];
               load16(lane_addr, t2, c0, v);
 #pragma unroll
@@ -265,7 +266,7 @@ __global__ void __launch_bounds__(192, 1) k_proj(const __grid_constant__ CUtenso
         float* dst = p.fixP + (size_t)cta * p.tm * p.n_pad * TILE_M;
         if (ok) {
           for (int t2 = 0; t2 < p.tm; ++t2)
-            for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
+            for (int c0 = c_first; c0 < p.n_pad; c0 += 32) {
               float v[16];
               load16(lane_addr, t2, c0, v);
 #pragma unroll
@@ -308,11 +309,11 @@ __global__ void __launch_bounds__(192, 1) k_proj(const __grid_constant__ CUtenso
         const int m = tile * TILE_M + row;
         const bool row_ok = m < p.M;
         if (EPI == EPI_ARGMAX) {
-          for (int t = etid; t < SPECASR_MAX_NODES; t += 128) sc->key[t] = 0ull;
+          for (int t = etid; t < SPECASR_MAX_NODES; t += EPI_THREADS) sc->key[t] = 0ull;
           epi_bar();
         }
         if (ok) {
-          for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
+          for (int c0 = c_first; c0 < p.n_pad; c0 += 32) {
             float v[16];
             load16(lane_addr, t2, c0, v);
             for (int cc = cta + 1; cc <= last; ++cc) {
@@ -361,7 +362,7 @@ __global__ void __launch_bounds__(192, 1) k_proj(const __grid_constant__ CUtenso
             const int F = p.M >> 1;
             const int f0 = tile * 64;
             const int chunks = 2 * p.n * 8;                 // 16-byte pieces of the [2][n][64] tile
-            for (int idx = etid; idx < chunks; idx += 128) {
+            for (int idx = etid; idx < chunks; idx += EPI_THREADS) {
               const int plane = idx / (p.n * 8), rem = idx % (p.n * 8);
               const int t = rem >> 3, ch = rem & 7;
               if (f0 + ch * 8 < F)
@@ -374,7 +375,7 @@ __global__ void __launch_bounds__(192, 1) k_proj(const __grid_constant__ CUtenso
         if (EPI == EPI_ARGMAX) {
           epi_bar();
           if (ok)
-            for (int t = etid; t < p.n; t += 128) p.amax[(size_t)tile * p.n_alloc + t] = sc->key[t];
+            for (int t = etid; t < p.n; t += EPI_THREADS) p.amax[(size_t)tile * p.n_alloc + t] = sc->key[t];
         }
       }
       if (ok) {
@@ -429,7 +430,7 @@ void launch_epi(const CUtensorMap& tmW, const CUtensorMap& tmAct, const TcParams
     cudaFuncSetAttribute(k_proj<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);
     configured = true;
   }
-  launch_pdl(k_proj<EPI>, dim3(grid), dim3(192), smem, s, tmW, tmAct, p);
+  launch_pdl(k_proj<EPI>, dim3(grid), dim3(64 + EPI_THREADS), smem, s, tmW, tmAct, p);
 }
 
 }  // namespace
