@@ -144,55 +144,96 @@ void launch_copy_embeds(specasr_kv* kv, const float* embeds, int n, cudaStream_t
 // RMSNorm with the residual update folded in: x <- x + sum of the previous projection's partial planes
 // (fixed order, hence deterministic), h = x * rsqrt(mean(x^2) + eps) * g, emitted as two bf16 planes
 // hi = bf16(h), lo = bf16(h - hi) so that the tensor-core projections see ~16 significant bits of every
-// activation.  Rows n..n_pad-1 of both planes are zeroed.
+// activation.  Rows n..n_pad-1 of both planes are zeroed.  One CTA per row; a thread keeps its ITER
+// float4 pieces of the row in registers, and the loads of up to four planes are issued together (an
+// in-order core would otherwise pay one L2 round trip per plane).
+template <int ITER>
 __global__ void __launch_bounds__(256) k_rmsnorm_split(const int32_t* __restrict__ ctl, float* __restrict__ X,
                                                        const float* __restrict__ P, int n_partials,
-                                                       size_t partial_stride, const float* __restrict__ gain, int d, float eps, int n,
-                                                       size_t plane_stride, bf16* __restrict__ H) {
+                                                       size_t partial_stride, const float* __restrict__ gain,
+                                                       int d, float eps, int n, size_t plane_stride,
+                                                       bf16* __restrict__ H) {
   grid_dep_launch();
+  const int row = blockIdx.x;
+  const int tid = threadIdx.x;
+  float4 g[ITER];
+#pragma unroll
+  for (int it = 0; it < ITER; ++it) {        // gains never change: fetch them before waiting
+    const int k = (it * 256 + tid) * 4;
+    g[it] = k < d ? *reinterpret_cast<const float4*>(gain + k) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
   grid_dep_wait();
   if (ctl[CTL_STATUS] != 0) return;
-  const int row = blockIdx.x;
   bf16* hi = H + (size_t)row * d;
   bf16* lo = hi + plane_stride;
   if (row >= n) {
-    for (int k = threadIdx.x * 8; k < d; k += blockDim.x * 8) {
+    for (int k = tid * 8; k < d; k += 256 * 8) {
       *reinterpret_cast<uint4*>(hi + k) = make_uint4(0, 0, 0, 0);
       *reinterpret_cast<uint4*>(lo + k) = make_uint4(0, 0, 0, 0);
     }
     return;
   }
   float* x = X + (size_t)row * d;
+  float4 v[ITER];
+#pragma unroll
+  for (int it = 0; it < ITER; ++it) {
+    const int k = (it * 256 + tid) * 4;
+    v[it] = k < d ? *reinterpret_cast<const float4*>(x + k) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  for (int s0 = 0; s0 < n_partials; s0 += 4) {
+    float4 q[4][ITER];
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+      for (int it = 0; it < ITER; ++it) {
+        const int k = (it * 256 + tid) * 4;
+        q[u][it] = (s0 + u < n_partials && k < d)
+                       ? __ldcg(reinterpret_cast<const float4*>(P + (s0 + u) * partial_stride + (size_t)row * d + k))
+                       : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+      for (int it = 0; it < ITER; ++it) {
+        v[it].x += q[u][it].x; v[it].y += q[u][it].y; v[it].z += q[u][it].z; v[it].w += q[u][it].w;
+      }
+  }
   float ss = 0.f;
-  for (int k = threadIdx.x * 4; k < d; k += blockDim.x * 4) {
-    float4 v = *reinterpret_cast<const float4*>(x + k);
-    for (int s = 0; s < n_partials; ++s) {
-      const float4 p = __ldcg(reinterpret_cast<const float4*>(P + s * partial_stride + (size_t)row * d + k));
-      v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
-    }
-    if (n_partials > 0) *reinterpret_cast<float4*>(x + k) = v;
-    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+#pragma unroll
+  for (int it = 0; it < ITER; ++it) {
+    const int k = (it * 256 + tid) * 4;
+    if (n_partials > 0 && k < d) *reinterpret_cast<float4*>(x + k) = v[it];
+    ss += v[it].x * v[it].x + v[it].y * v[it].y + v[it].z * v[it].z + v[it].w * v[it].w;
   }
   ss = block_sum_256(ss);
   const float inv = rsqrtf(ss / (float)d + eps);
-  for (int k = threadIdx.x * 4; k < d; k += blockDim.x * 4) {
-    const float4 v = *reinterpret_cast<const float4*>(x + k);
-    const float4 g = *reinterpret_cast<const float4*>(gain + k);
-    const float h[4] = {v.x * inv * g.x, v.y * inv * g.y, v.z * inv * g.z, v.w * inv * g.w};
-    uint32_t ph[2], pl[2];
-    split2_pack(h[0], h[1], ph[0], pl[0]);
-    split2_pack(h[2], h[3], ph[1], pl[1]);
-    *reinterpret_cast<uint2*>(hi + k) = make_uint2(ph[0], ph[1]);
-    *reinterpret_cast<uint2*>(lo + k) = make_uint2(pl[0], pl[1]);
+#pragma unroll
+  for (int it = 0; it < ITER; ++it) {
+    const int k = (it * 256 + tid) * 4;
+    if (k < d) {
+      uint32_t ph[2], pl[2];
+      split2_pack(v[it].x * inv * g[it].x, v[it].y * inv * g[it].y, ph[0], pl[0]);
+      split2_pack(v[it].z * inv * g[it].z, v[it].w * inv * g[it].w, ph[1], pl[1]);
+      *reinterpret_cast<uint2*>(hi + k) = make_uint2(ph[0], ph[1]);
+      *reinterpret_cast<uint2*>(lo + k) = make_uint2(pl[0], pl[1]);
+    }
   }
 }
 
 void launch_rmsnorm_split(specasr_kv* kv, const float* gain, int n, int n_pad, int n_partials, cudaStream_t s) {
   const specasr_model* m = kv->m;
   const int d = m->cfg.d_model;
+  const size_t stride = (size_t)kv->n_alloc * d;
   LaunchScope scope(kv, SPECASR_KIND_NORM, s);
-  launch_pdl(k_rmsnorm_split, dim3(n_pad), dim3(256), 0, s, kv->ws.ctl, kv->ws.X, kv->ws.P, n_partials, (size_t)kv->n_alloc * d, gain,
-             d, m->cfg.rms_eps, n, (size_t)kv->n_alloc * d, kv->ws.H);
+#define NORM_LAUNCH(I)                                                                                              \
+  launch_pdl(k_rmsnorm_split<I>, dim3(n_pad), dim3(256), 0, s, kv->ws.ctl, kv->ws.X, kv->ws.P, n_partials, stride, \
+             gain, d, m->cfg.rms_eps, n, stride, kv->ws.H)
+  if (d <= 1024) NORM_LAUNCH(1);
+  else if (d <= 2048) NORM_LAUNCH(2);
+  else if (d <= 4096) NORM_LAUNCH(4);
+  else if (d <= 8192) NORM_LAUNCH(8);
+  else NORM_LAUNCH(16);
+#undef NORM_LAUNCH
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -216,10 +257,17 @@ __global__ void k_rope_append(const int32_t* __restrict__ ctl, const float* __re
   if (k >= half) return;
   const size_t col = (size_t)i * qkv_dim + (size_t)head * dh;
   const size_t c1 = col + qkv_row_of_feature(k, dh), c2 = col + qkv_row_of_feature(k + half, dh);
+  float a1[kMaxSplitK], a2[kMaxSplitK];      // all plane loads in flight together, summed in plane order
+#pragma unroll
+  for (int s = 0; s < kMaxSplitK; ++s) {
+    a1[s] = s < n_partials ? __ldcg(P + s * partial_stride + c1) : 0.f;
+    a2[s] = s < n_partials ? __ldcg(P + s * partial_stride + c2) : 0.f;
+  }
   float x1 = 0.f, x2 = 0.f;
-  for (int s = 0; s < n_partials; ++s) {
-    x1 += __ldcg(P + s * partial_stride + c1);
-    x2 += __ldcg(P + s * partial_stride + c2);
+#pragma unroll
+  for (int s = 0; s < kMaxSplitK; ++s) {
+    x1 += a1[s];
+    x2 += a2[s];
   }
   const bool is_v = head >= Hq + Hkv;
   if (!is_v) {
@@ -266,50 +314,73 @@ void launch_rope_append(specasr_kv* kv, int layer, int n, int n_partials, cudaSt
 
 // ------------------------------------------------------------------------------------------------
 // Merge of the attention kernel's KV splits (log-sum-exp combination in base 2), normalisation and
-// hi/lo split of the result for the O projection.  Rows n..n_pad-1 are zeroed.
-__global__ void k_attn_merge(const int32_t* __restrict__ ctl, const float* __restrict__ attO,
-                             const float2* __restrict__ attML, int n_splits, size_t rows_alloc, int Hq, int dh,
-                             int n, bf16* __restrict__ AO, size_t plane_stride) {
+// hi/lo split of the result for the O projection.  One warp per (node, head) row: lane s holds the
+// (max, sum) of splits s and s + 32, lane c the output columns 4c .. 4c + 3; the partial outputs of
+// eight splits are requested together.  Rows n..n_pad-1 are zeroed.
+__global__ void __launch_bounds__(128) k_attn_merge(const int32_t* __restrict__ ctl, const float* __restrict__ attO,
+                                                    const float2* __restrict__ attML, int n_splits, size_t rows_alloc,
+                                                    int Hq, int dh, int n, int rows_total, bf16* __restrict__ AO,
+                                                    size_t plane_stride) {
   grid_dep_launch();
   grid_dep_wait();
   if (ctl[CTL_STATUS] != 0) return;
-  const int i = blockIdx.x;
-  const int h = blockIdx.y;
-  const int d = threadIdx.x;
-  if (d >= dh) return;
-  bf16* out = AO + (size_t)i * Hq * dh + (size_t)h * dh + d;
-  if (i >= n) {
-    out[0] = __float2bfloat16_rn(0.f);
-    out[plane_stride] = __float2bfloat16_rn(0.f);
+  const int lane = threadIdx.x & 31;
+  const int row = blockIdx.x * 4 + (threadIdx.x >> 5);       // = node * Hq + head
+  if (row >= rows_total) return;
+  const int c = lane * 4;
+  bf16* out = AO + (size_t)row * dh + c;
+  if (row / Hq >= n) {
+    if (c < dh) {
+      *reinterpret_cast<uint2*>(out) = make_uint2(0, 0);
+      *reinterpret_cast<uint2*>(out + plane_stride) = make_uint2(0, 0);
+    }
     return;
   }
-  const size_t row = (size_t)i * Hq + h;
-  float mx = -INFINITY;
-  for (int s = 0; s < n_splits; ++s) mx = fmaxf(mx, attML[s * rows_alloc + row].x);
-  float num = 0.f, den = 0.f;
-  for (int s = 0; s < n_splits; ++s) {
-    const float2 ml = attML[s * rows_alloc + row];
-    if (ml.y > 0.f) {
-      const float w = exp2f(ml.x - mx);
-      den += ml.y * w;
-      num += attO[(s * rows_alloc + row) * dh + d] * w;
+  const float2 none = make_float2(-INFINITY, 0.f);
+  const float2 ml0 = lane < n_splits ? __ldcg(attML + (size_t)lane * rows_alloc + row) : none;
+  const float2 ml1 = lane + 32 < n_splits ? __ldcg(attML + (size_t)(lane + 32) * rows_alloc + row) : none;
+  float mx = fmaxf(ml0.y > 0.f ? ml0.x : -INFINITY, ml1.y > 0.f ? ml1.x : -INFINITY);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+  const float w0 = ml0.y > 0.f ? exp2f(ml0.x - mx) : 0.f;
+  const float w1 = ml1.y > 0.f ? exp2f(ml1.x - mx) : 0.f;
+  // denominator: the terms are added one by one in split order, so the result does not depend on timing
+  float den = 0.f;
+  for (int s = 0; s < n_splits; ++s) den += __shfl_sync(0xFFFFFFFFu, s < 32 ? ml0.y * w0 : ml1.y * w1, s & 31);
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int s0 = 0; s0 < n_splits; s0 += 8) {
+    float4 o[8];
+    float w[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int s = s0 + u;
+      w[u] = __shfl_sync(0xFFFFFFFFu, s < 32 ? w0 : w1, s & 31);
+      if (s >= n_splits) w[u] = 0.f;
+      o[u] = (w[u] > 0.f && c < dh) ? __ldcg(reinterpret_cast<const float4*>(attO + ((size_t)s * rows_alloc + row) * dh + c))
+                                    : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      acc.x += o[u].x * w[u]; acc.y += o[u].y * w[u]; acc.z += o[u].z * w[u]; acc.w += o[u].w * w[u];
     }
   }
-  const float o = num / den;
-  bf16 hi, lo;
-  split_bf16(o, hi, lo);
-  out[0] = hi;
-  out[plane_stride] = lo;
+  if (c < dh) {
+    const float r = 1.f / den;
+    uint32_t ph[2], pl[2];
+    split2_pack(acc.x * r, acc.y * r, ph[0], pl[0]);
+    split2_pack(acc.z * r, acc.w * r, ph[1], pl[1]);
+    *reinterpret_cast<uint2*>(out) = make_uint2(ph[0], ph[1]);
+    *reinterpret_cast<uint2*>(out + plane_stride) = make_uint2(pl[0], pl[1]);
+  }
 }
 
 void launch_attn_merge(specasr_kv* kv, int n, int n_pad, int n_splits, cudaStream_t s) {
   const specasr_model_config& c = kv->m->cfg;
-  dim3 grid(n_pad, c.n_heads);
-  const int threads = c.head_dim < 32 ? 32 : c.head_dim;
+  const int rows_total = n_pad * c.n_heads;
   LaunchScope scope(kv, SPECASR_KIND_ATTN_MERGE, s);
-  launch_pdl(k_attn_merge, grid, dim3(threads), 0, s, kv->ws.ctl, kv->ws.attO, kv->ws.attML, n_splits,
-                                        (size_t)kv->n_alloc * c.n_heads, c.n_heads, c.head_dim, n, kv->ws.AO,
-                                        (size_t)kv->n_alloc * kv->m->q_dim);
+  launch_pdl(k_attn_merge, dim3((rows_total + 3) / 4), dim3(128), 0, s, kv->ws.ctl, kv->ws.attO, kv->ws.attML, n_splits,
+             (size_t)kv->n_alloc * c.n_heads, c.n_heads, c.head_dim, n, rows_total, kv->ws.AO,
+             (size_t)kv->n_alloc * kv->m->q_dim);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -339,16 +410,31 @@ __global__ void __launch_bounds__(256) k_accept(const int32_t* __restrict__ ctl,
     return;
   }
   if (i == 0) s_best = 0u;
-  if (i < n) {
+  // arg-max over the vocabulary tiles: one warp per node, lanes stride over the tiles, eight loads in flight
+  for (int node = i >> 5; node < n; node += 8) {
+    const int lane = i & 31;
     unsigned long long best = 0ull;
-    for (int t = 0; t < n_tiles; ++t) {
-      const unsigned long long v = amax[(size_t)t * n_alloc + i];
-      best = v > best ? v : best;
+    for (int t0 = 0; t0 < n_tiles; t0 += 256) {
+      unsigned long long v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int t = t0 + u * 32 + lane;
+        v[u] = t < n_tiles ? __ldcg(amax + (size_t)t * n_alloc + node) : 0ull;
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) best = v[u] > best ? v[u] : best;
     }
-    const int tok = (int)(0xFFFFFFFFu - (unsigned int)(best & 0xFFFFFFFFull));
-    s_arg[i] = tok;
-    out_argmax[i] = tok;
-    out_path[i] = -1;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const unsigned long long other = __shfl_xor_sync(0xFFFFFFFFu, best, o);
+      best = other > best ? other : best;
+    }
+    if (lane == 0) {
+      const int tok = (int)(0xFFFFFFFFu - (unsigned int)(best & 0xFFFFFFFFull));
+      s_arg[node] = tok;
+      out_argmax[node] = tok;
+      out_path[node] = -1;
+    }
   }
   __syncthreads();
   if (i < n) {
