@@ -198,6 +198,44 @@ enum {
 specasr_status specasr_profile_enable(specasr_kv* kv, int32_t enable);
 specasr_status specasr_profile_read(specasr_kv* kv, double* out_ms, int64_t* out_launches, void* stream);
 
+/*
+ * Accept step on its own, for callers that may not allocate.  (The paper has no counterpart: this is a
+ * packaging of the accept rule of Section II-B for hosts with a frozen memory plan.)
+ *
+ * Some users of this library are handed buffers but have no way to get device memory themselves: a
+ * plug-in running inside a serving process that reserved all of its device memory at start-up and
+ * forbids cudaMalloc afterwards, or a component that scores logits produced elsewhere (another
+ * decoder, a replayed trace) and owns nothing but its inputs and outputs.  This call gives them the
+ * arg-max + longest-accepted-path step without a model, a KV handle or a workspace.  It calls no
+ * cudaMalloc / cudaFree / cudaHostAlloc and no routine that allocates; the only memory it uses besides
+ * the arguments is one fixed array of 131328 bytes inside the library image, which every GPU that loads
+ * the library holds until the process exits.
+ *
+ *   logits             : [device] fp32 [n_nodes, vocab], row-major; row i = target logits after node i
+ *   tokens, parent_idx : [device] int32[n_nodes], the tree format described at the top of this file
+ *   out_argmax         : [device] int32[n_nodes]  arg-max token of every row (lowest id on ties)
+ *   out_accept_len     : [device] int32[1]        accepted draft nodes on the best path
+ *   out_path           : [device] int32[n_nodes]  node indices root..best, padded with -1
+ *   out_bonus          : [device] int32[1] or NULL, out_argmax[best]
+ * Same rule and same tie-breaks as specasr_verify_tree, so feeding it the logits of
+ * specasr_verify_tree_ex reproduces that call's out_argmax / out_accept_len / out_path / out_bonus.
+ *
+ * Limits and errors: 1 <= n_nodes <= SPECASR_MAX_NODES (the fixed array has room for exactly that many
+ * nodes; larger trees are refused with SPECASR_ERR_INVALID_ARG and a message that says so), vocab >= 1.
+ * A malformed parent array or a token id outside [0, vocab) is found on the device: out_accept_len
+ * receives -1 and out_argmax / out_path are filled with -1.
+ *
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that
+ * device current); make that first call outside any stream capture.  Asynchronous on `stream`.
+ * All calls on one device share the array, and it keeps what the last call left in it (the call clears
+ * the part that has to start at zero): two calls that overlap on the GPU, e.g. on different streams,
+ * race on it and may both return wrong results.  Issue them on one stream or order them with events.
+ */
+specasr_status specasr_accept_logits_static(const float* logits, int32_t vocab, const int32_t* tokens,
+                                            const int32_t* parent_idx, int32_t n_nodes, int32_t* out_argmax,
+                                            int32_t* out_accept_len, int32_t* out_path, int32_t* out_bonus,
+                                            void* stream);
+
 const char* specasr_last_error(void);
 
 #ifdef __cplusplus

@@ -20,7 +20,7 @@ EXPORTS = [
     "specasr_kv_create", "specasr_kv_destroy", "specasr_kv_length", "specasr_kv_truncate",
     "specasr_prefill_embeds", "specasr_prefill_tokens", "specasr_verify_tree", "specasr_verify_tree_ex",
     "specasr_commit_kv", "specasr_poll_status", "specasr_launch_count", "specasr_last_error",
-    "specasr_profile_enable", "specasr_profile_read",
+    "specasr_profile_enable", "specasr_profile_read", "specasr_accept_logits_static",
 ]
 KIND_NAMES = ["prep", "norm", "gemm_qkv", "rope", "attn", "attn_merge", "gemm_o", "gemm_gu", "gemm_down", "gemm_lm",
               "accept", "commit"]
@@ -84,6 +84,8 @@ def lib() -> C.CDLL:
         L.specasr_profile_enable.restype = st
         L.specasr_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64), vp]
         L.specasr_profile_read.restype = st
+        L.specasr_accept_logits_static.argtypes = [vp, i32, vp, vp, i32, vp, vp, vp, vp, vp]
+        L.specasr_accept_logits_static.restype = st
         L.specasr_last_error.argtypes = []
         L.specasr_last_error.restype = C.c_char_p
         _lib = L
@@ -168,6 +170,14 @@ def specasr_verify_tree_ex(model: int, kv: int, tokens: int, parent_idx: int, n_
 
 def specasr_commit_kv(model: int, kv: int, path: int, accept_len: int, stream: int = 0) -> None:
     _check(lib().specasr_commit_kv(model, kv, path, accept_len, stream))
+
+
+def specasr_accept_logits_static(logits: int, vocab: int, tokens: int, parent_idx: int, n_nodes: int, out_argmax: int,
+                                 out_accept_len: int, out_path: int, out_bonus: int = 0, stream: int = 0) -> None:
+    """Accept step from a logits matrix for callers that cannot allocate device memory (see the header):
+    all arguments are device addresses of caller-owned buffers; the library's built-in array is the only scratch."""
+    _check(lib().specasr_accept_logits_static(logits, vocab, tokens, parent_idx, n_nodes, out_argmax, out_accept_len,
+                                              out_path, out_bonus or None, stream))
 
 
 def specasr_poll_status(kv: int, stream: int = 0) -> int:
