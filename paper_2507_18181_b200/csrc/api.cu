@@ -367,12 +367,13 @@ static void run_gemm(specasr_kv* kv, GemmArgs& a, int kind, cudaStream_t s) {
   }
 }
 
-static int attention_splits(const specasr_kv* kv, int n, int len_upper, bool* use_tc) {
+static int attention_splits(const specasr_kv* kv, int n, int len_upper, bool* use_tc, int* chunk) {
   const specasr_model_config& c = kv->m->cfg;
   *use_tc = false;
+  *chunk = 0;
   if (kv->attn_tc) {
-    const int s = attention_tc_splits(len_upper + n);
-    if (s <= kMaxAttnSplits) {
+    int s = 0;
+    if (attention_tc_plan(kv->m, n, len_upper + n, kMaxAttnSplits, &s, chunk)) {
       *use_tc = true;
       return s;
     }
@@ -394,7 +395,8 @@ static void run_stack(specasr_model* m, specasr_kv* kv, int n, bool want_head, f
   const specasr_model_config& c = m->cfg;
   const int n_pad = round_up(n, 16);
   bool att_tc = false;
-  const int att_splits = attention_splits(kv, n, kv->len_upper, &att_tc);
+  int att_chunk = 0;
+  const int att_splits = attention_splits(kv, n, kv->len_upper, &att_tc, &att_chunk);
   const bool tc = c.gemm_path == 0;
   int pending = 0;               // partial planes of the last down projection still to be added to X
   GemmArgs a;
@@ -410,7 +412,7 @@ static void run_stack(specasr_model* m, specasr_kv* kv, int n, bool want_head, f
     a.M = m->qkv_dim; a.K = c.d_model; a.epilogue = EPI_PARTIAL;
     run_gemm(kv, a, SPECASR_KIND_GEMM_QKV, s);
     launch_rope_append(kv, l, n, a.splits, s);
-    if (att_tc) launch_tree_attention_tc(kv, l, n, att_splits, s);
+    if (att_tc) launch_tree_attention_tc(kv, l, n, att_splits, att_chunk, s);
     else launch_tree_attention(kv, l, n, att_splits, s);
     launch_attn_merge(kv, n, n_pad, att_splits, s);
     a.W = m->wo[l]; a.tmW = tc ? &m->tm_wo[l] : nullptr; a.tmAct = kv->tm_AO; a.act = kv->ws.AO;

@@ -4,15 +4,19 @@
 // ancestor of i (bit j of the node's ancestor mask): the 2-D mask of a draft token tree.
 //
 // One CTA owns one KV head, a tile of up to 128 query rows (row = node * group + head-in-group, so a
-// whole query group shares every K/V element that is staged) and one block of 128 cache positions:
+// whole query group shares every K/V element that is staged) and one block of up to 208 cache positions,
+// sized by the host so that the whole launch is one wave of CTAs:
 //   S = Q K^T      M = 128 rows, N = keys, K = head_dim        (both operands K-major)
-//   P = exp2(S * scale - rowmax), masked                         (one thread per row, fp32, from TMEM)
+//   P = exp2(S * scale - rowmax), masked                         (two threads per row, fp32, from TMEM)
 //   O = P V        M = 128 rows, N = head_dim, K = keys          (V is the MN-major B operand)
 // Q, P, K and V are all carried as two bf16 planes (value ~ hi + lo); each product is three MMAs
 // (hi*hi + hi*lo + lo*hi) into the same fp32 accumulator, which keeps ~16 significant bits.
 // Pages of K and V arrive by TMA straight from the paged pool (one box per page, plane and 64-wide
-// half of the head), Q by one box per plane and half.  The CTA emits an unnormalised partial
-// (row max in log2 units, row sum, output) that k_attn_merge combines over the key blocks.
+// half of the head), Q by one box per plane and half.  Shared memory holds two regions: Q, later
+// overwritten by P (in rounds of 128 keys, S stays in TMEM meanwhile), and K, later overwritten by V
+// (requested as soon as the S MMAs have finished reading K), later by the output tile on its way out.
+// The CTA emits an unnormalised partial (row max in log2 units, row sum, output) that k_attn_merge
+// combines over the key blocks.
 //
 // Every mbarrier wait is bounded; on expiry the CTA records SPECASR_ERR_TIMEOUT, lets copies in
 // flight land, frees its TMEM and returns.
@@ -24,13 +28,14 @@ using namespace sm100;
 
 namespace {
 
-constexpr int KEYS = 128;                 // cache positions per CTA
-constexpr int SUB = 128 * 64 * 2;         // bytes of one [128 rows][64 bf16] swizzled sub-tile
-
+constexpr int KEYS_MAX = 208;             // cache positions per CTA (13 pages of 16)
+constexpr int ROUND = 128;                // keys whose probabilities fit the P buffer at once
+constexpr int SUB = 128 * 64 * 2;         // bytes of one [128 rows][64 bf16] swizzled sub-tile (Q, P)
+constexpr int KVSUB = KEYS_MAX * 64 * 2;  // bytes of one [208 keys][64 bf16] swizzled sub-tile (K, V)
 constexpr int SOFTMAX_THREADS = 256;      // warps 2..9; warps w and w + 4 share a TMEM lane quadrant
 
 struct AttnCtl {
-  unsigned long long bar_qk, bar_v, bar_s, bar_p, bar_o;
+  unsigned long long bar_qk, bar_v, bar_s, bar_p[2], bar_o[2];
   float red_max[2][128];      // per-row partial maxima / sums of the two warps that share a row
   float red_sum[2][128];
   uint32_t tmem_base;
@@ -45,7 +50,7 @@ struct AttnParams {
   float* attO;
   float2* attML;
   size_t rows_alloc;      // n_alloc * Hq
-  int n_pages, page_size, layer, Hq, Hkv, group, nodes_per_tile, n;
+  int n_pages, page_size, layer, Hq, Hkv, group, nodes_per_tile, n, chunk;
   float scale_log2;
 };
 
@@ -54,8 +59,8 @@ __global__ void __launch_bounds__(64 + SOFTMAX_THREADS, 1) k_tree_attention_tc(c
                                                               const __grid_constant__ CUtensorMap tmK,
                                                               const __grid_constant__ CUtensorMap tmV, AttnParams p) {
   constexpr int H = DH / 64;                               // 64-wide halves of the head
-  constexpr int A_BYTES = 2 * H * SUB < 4 * SUB ? 4 * SUB : 2 * H * SUB;   // Q planes, later the P planes
-  constexpr int KV_BYTES = 2 * H * SUB;
+  constexpr int A_BYTES = 4 * SUB;                         // Q planes (2 H sub-tiles), later two P planes of 128 keys
+  constexpr int KV_BYTES = 2 * H * KVSUB;
   extern __shared__ uint8_t smem_raw[];
   pdl_launch_dependents();
   pdl_wait();
@@ -67,7 +72,7 @@ __global__ void __launch_bounds__(64 + SOFTMAX_THREADS, 1) k_tree_attention_tc(c
   const int rows_used = p.nodes_per_tile * p.group;
   const int L = p.ctl[CTL_LEN];
   const int Ltot = L + p.n;
-  const int k_begin = split * KEYS;
+  const int k_begin = split * p.chunk;
 
   // row owned by a softmax thread (warps 2..9): TMEM lane = 32 * (warp % 4) + lane
   const int r = ((warp & 3) << 5) | lane;
@@ -79,21 +84,23 @@ __global__ void __launch_bounds__(64 + SOFTMAX_THREADS, 1) k_tree_attention_tc(c
     if (row_valid) p.attML[out_row] = make_float2(-INFINITY, 0.f);
     return;
   }
-  const int kc = min(KEYS, Ltot - k_begin);
+  const int kc = min(p.chunk, Ltot - k_begin);
   const int kc_pad = (kc + 15) & ~15;
   const int pages = (kc + p.page_size - 1) / p.page_size;
+  const int rounds = (kc_pad + ROUND - 1) / ROUND;          // 1 or 2
 
   uint8_t* As = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  uint8_t* Ks = As + A_BYTES;
-  uint8_t* Vs = Ks + KV_BYTES;
-  AttnCtl* sc = (AttnCtl*)(Vs + KV_BYTES);
+  uint8_t* KVs = As + A_BYTES;
+  AttnCtl* sc = (AttnCtl*)(KVs + KV_BYTES);
 
   if (threadIdx.x == 0) {
     mbar_init(&sc->bar_qk, 1);
     mbar_init(&sc->bar_v, 1);
     mbar_init(&sc->bar_s, 1);
-    mbar_init(&sc->bar_p, SOFTMAX_THREADS);
-    mbar_init(&sc->bar_o, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&sc->bar_p[i], SOFTMAX_THREADS);
+      mbar_init(&sc->bar_o[i], 1);
+    }
     sc->abort = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tmQ);
@@ -107,17 +114,17 @@ __global__ void __launch_bounds__(64 + SOFTMAX_THREADS, 1) k_tree_attention_tc(c
         *reinterpret_cast<uint4*>(As + sub * SUB + rows_used * 128 + i * 16) = make_uint4(0, 0, 0, 0);
     fence_proxy_async_smem();
   }
-  if (warp == 1) tmem_alloc(&sc->tmem_base, 256);
+  if (warp == 1) tmem_alloc(&sc->tmem_base, 512);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem_s = sc->tmem_base;           // S: columns [0, 128)
-  const uint32_t tmem_o = sc->tmem_base + 128;     // O: columns [128, 128 + DH)
+  const uint32_t tmem_s = sc->tmem_base;           // S: columns [0, 208)
+  const uint32_t tmem_o = sc->tmem_base + 256;     // O: columns [256, 256 + DH)
   volatile int* abort = &sc->abort;
   int32_t* status = p.ctl + CTL_STATUS;
 
   if (warp == 0) {
-    // ---------------- TMA producer: lane 0 fetches Q, lane j fetches page j of K and of V
+    // ---------------- TMA producer: lane 0 fetches Q, lane j fetches page j of K and later of V
     const uint32_t q_bytes = 2 * H * rows_used * 128;
     const uint32_t kv_bytes = 2 * H * pages * p.page_size * 128;
     if (lane == 0) {
@@ -130,16 +137,20 @@ __global__ void __launch_bounds__(64 + SOFTMAX_THREADS, 1) k_tree_attention_tc(c
         for (int h = 0; h < H; ++h)
           tma_load_4d(As + (plane * H + h) * SUB, &tmQ, h * 64, kvh * p.group, node0, plane, &sc->bar_qk);
     }
-    for (int j = lane; j < pages; j += 32) {
-      const int page = p.page_table[k_begin / p.page_size + j];
-      const int c4 = p.layer * p.n_pages + page;
-      const int off = j * p.page_size * 128;
+    int c4 = 0;
+    const int off = lane * p.page_size * 128;
+    if (lane < pages) {
+      c4 = p.layer * p.n_pages + p.page_table[k_begin / p.page_size + lane];
       for (int plane = 0; plane < 2; ++plane)
         for (int h = 0; h < H; ++h)
-          tma_load_5d(Ks + (plane * H + h) * SUB + off, &tmK, h * 64, 0, plane, kvh, c4, &sc->bar_qk);
+          tma_load_5d(KVs + (plane * H + h) * KVSUB + off, &tmK, h * 64, 0, plane, kvh, c4, &sc->bar_qk);
+    }
+    // V takes K's place once the S MMAs have read K
+    const bool ok = mbar_wait(&sc->bar_s, 0u, abort, status);
+    if (ok && lane < pages) {
       for (int plane = 0; plane < 2; ++plane)
         for (int h = 0; h < H; ++h)
-          tma_load_5d(Vs + (plane * H + h) * SUB + off, &tmV, h * 64, 0, plane, kvh, c4, &sc->bar_v);
+          tma_load_5d(KVs + (plane * H + h) * KVSUB + off, &tmV, h * 64, 0, plane, kvh, c4, &sc->bar_v);
     }
   } else if (warp == 1 && lane == 0) {
     // ---------------- MMA issuer
@@ -147,7 +158,7 @@ __global__ void __launch_bounds__(64 + SOFTMAX_THREADS, 1) k_tree_attention_tc(c
     if (ok) {
       tc_fence_after();
       const uint32_t idesc = make_idesc_bf16(kc_pad);
-      const uint32_t a0 = smem_u32(As), b0 = smem_u32(Ks);
+      const uint32_t a0 = smem_u32(As), b0 = smem_u32(KVs);
       uint32_t acc = 0u;
 #pragma unroll
       for (int term = 0; term < 3; ++term) {
@@ -156,31 +167,34 @@ __global__ void __launch_bounds__(64 + SOFTMAX_THREADS, 1) k_tree_attention_tc(c
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
             umma_bf16(tmem_s, make_smem_desc(a0 + (qp * H + h) * SUB + k * 32),
-                      make_smem_desc(b0 + (kp * H + h) * SUB + k * 32), idesc, acc);
+                      make_smem_desc(b0 + (kp * H + h) * KVSUB + k * 32), idesc, acc);
             acc = 1u;
           }
         }
       }
       umma_commit(&sc->bar_s);
-      ok = mbar_wait(&sc->bar_p, 0u, abort, status) && mbar_wait(&sc->bar_v, 0u, abort, status);
+      ok = mbar_wait(&sc->bar_v, 0u, abort, status);
     }
-    if (ok) {
+    const uint32_t idesc2 = make_idesc_bf16(DH, true);
+    uint32_t acc = 0u;
+    for (int rd = 0; rd < rounds && ok; ++rd) {
+      ok = mbar_wait(&sc->bar_p[rd], 0u, abort, status);
+      if (!ok) break;
       tc_fence_after();
-      const uint32_t idesc = make_idesc_bf16(DH, true);
-      const uint32_t a0 = smem_u32(As), b0 = smem_u32(Vs);
-      uint32_t acc = 0u;
+      const uint32_t a0 = smem_u32(As), b0 = smem_u32(KVs);
+      const int j_end = min(kc_pad - rd * ROUND, ROUND) / 16;
 #pragma unroll
       for (int term = 0; term < 3; ++term) {
         const int pp = term == 2 ? 1 : 0, vp = term == 1 ? 1 : 0;
-        for (int j = 0; j < kc_pad / 16; ++j) {
-          // A: P plane pp, 64-key block j / 4, 16 keys = 32 bytes along the row
-          // B: V plane vp, keys 16 j .. 16 j + 15 are rows of 128 bytes; the second half of the head is SUB further on
+        for (int j = 0; j < j_end; ++j) {
+          // A: P plane pp, 64-key block j / 4 of this round, 16 keys = 32 bytes along the row
+          // B: V plane vp, keys of this step are rows of 128 bytes; the second half of the head is KVSUB further on
           umma_bf16(tmem_o, make_smem_desc(a0 + (pp * 2 + (j >> 2)) * SUB + (j & 3) * 32),
-                    make_smem_desc(b0 + vp * H * SUB + j * 2048, SUB), idesc, acc);
+                    make_smem_desc(b0 + vp * H * KVSUB + (rd * (ROUND / 16) + j) * 2048, KVSUB), idesc2, acc);
           acc = 1u;
         }
       }
-      umma_commit(&sc->bar_o);
+      umma_commit(&sc->bar_o[rd]);
     }
   } else if (warp >= 2) {
     // ---------------- softmax and epilogue: two threads per query row (warps w and w + 4), each taking
@@ -194,8 +208,7 @@ __global__ void __launch_bounds__(64 + SOFTMAX_THREADS, 1) k_tree_attention_tc(c
       anc2 = p.anc[node * 4 + 2];
       anc3 = p.anc[node * 4 + 3];
     }
-    // bit j of the result = key (base + j) is visible to this row
-    auto visible32 = [&](int base) -> uint32_t {
+    auto visible_keys = [&](int base) -> uint32_t {
       const int t0 = base - L;                      // tree slot of the chunk's first key
       if (t0 <= -32) return 0xFFFFFFFFu;            // all 32 keys lie in the committed prefix
       const int ts = t0 > 0 ? t0 : 0;
@@ -208,9 +221,14 @@ __global__ void __launch_bounds__(64 + SOFTMAX_THREADS, 1) k_tree_attention_tc(c
       }
       return t0 < 0 ? ((1u << (-t0)) - 1u) | (win << (-t0)) : win;
     };
+    // bit j of the result = key (k_begin + c0 + j) belongs to this CTA's block and is visible to this row
+    auto visible32 = [&](int c0) -> uint32_t {
+      const uint32_t mine = kc - c0 >= 32 ? 0xFFFFFFFFu : (1u << (kc - c0)) - 1u;   // c0 < kc always
+      return mine & visible_keys(k_begin + c0);
+    };
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
     bool ok = mbar_wait(&sc->bar_s, 0u, abort, status);
-    float m_row = -INFINITY, l_part = 0.f;
+    float m_row = -INFINITY;
     if (ok) {
       tc_fence_after();
       float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
@@ -218,7 +236,7 @@ __global__ void __launch_bounds__(64 + SOFTMAX_THREADS, 1) k_tree_attention_tc(c
       for (int c0 = eg * 32; c0 < kc_pad; c0 += 64) {
         float s[32];
         tmem_ld32(tmem_s + lane_off + c0, s);
-        const uint32_t vis = visible32(k_begin + c0);
+        const uint32_t vis = visible32(c0);
 #pragma unroll
         for (int j = 0; j < 32; ++j) m4[j & 3] = fmaxf(m4[j & 3], ((vis >> j) & 1u) ? s[j] * p.scale_log2 : -INFINITY);
       }
@@ -227,14 +245,18 @@ __global__ void __launch_bounds__(64 + SOFTMAX_THREADS, 1) k_tree_attention_tc(c
     sc->red_max[eg][r] = m_row;
     softmax_bar();
     m_row = fmaxf(sc->red_max[0][r], sc->red_max[1][r]);
-    if (ok) {
-      const float m_use = m_row > -INFINITY ? m_row : 0.f;    // a fully masked row gives p = 0 everywhere
-      float l2[2] = {0.f, 0.f};
+    const float m_use = m_row > -INFINITY ? m_row : 0.f;      // a fully masked row gives p = 0 everywhere
+    float l2[2] = {0.f, 0.f};
+    for (int rd = 0; rd < rounds && ok; ++rd) {
+      // the P buffer holds 128 keys: the second round waits until the first round's MMAs have read it
+      if (rd > 0) ok = mbar_wait(&sc->bar_o[rd - 1], 0u, abort, status);
+      if (!ok) break;
+      const int c_end = min(kc_pad, (rd + 1) * ROUND);
 #pragma unroll 1
-      for (int c0 = eg * 32; c0 < kc_pad; c0 += 64) {
+      for (int c0 = rd * ROUND + eg * 32; c0 < c_end; c0 += 64) {
         float s[32];
         tmem_ld32(tmem_s + lane_off + c0, s);
-        const uint32_t vis = visible32(k_begin + c0);
+        const uint32_t vis = visible32(c0);
 #pragma unroll
         for (int j = 0; j < 32; ++j) s[j] = ((vis >> j) & 1u) ? exp2f(s[j] * p.scale_log2 - m_use) : 0.f;
 #pragma unroll
@@ -246,34 +268,33 @@ __global__ void __launch_bounds__(64 + SOFTMAX_THREADS, 1) k_tree_attention_tc(c
             l2[e & 1] += s[j] + s[j + 1];
             split2_pack(s[j], s[j + 1], hi[e], lo[e]);
           }
-          const int c8 = (c0 >> 3) + g;                        // 8-key group within the block of 128
-          if (c8 * 8 < kc_pad) {
+          const int c8 = ((c0 - rd * ROUND) >> 3) + g;         // 8-key group within this round's 128 keys
+          if (rd * ROUND + c8 * 8 < kc_pad) {
             const int off = (c8 >> 3) * SUB + r * 128 + (((c8 & 7) ^ (r & 7)) << 4);
             *reinterpret_cast<uint4*>(As + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
             *reinterpret_cast<uint4*>(As + 2 * SUB + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
           }
         }
       }
-      l_part = l2[0] + l2[1];
-      if (kc < kc_pad) {
+      if (rd == rounds - 1 && kc < kc_pad) {
         // value rows past the end of the cache meet p = 0, but 0 * garbage could still be NaN: clear them
         ok = mbar_wait(&sc->bar_v, 0u, abort, status);
         if (ok && eg == 0 && r < kc_pad - kc) {
           for (int sub = 0; sub < 2 * H; ++sub)
             for (int i = 0; i < 8; ++i)
-              *reinterpret_cast<uint4*>(Vs + sub * SUB + (kc + r) * 128 + i * 16) = make_uint4(0, 0, 0, 0);
+              *reinterpret_cast<uint4*>(KVs + sub * KVSUB + (kc + r) * 128 + i * 16) = make_uint4(0, 0, 0, 0);
         }
       }
+      if (ok) {
+        fence_proxy_async_smem();
+        mbar_arrive(&sc->bar_p[rd]);
+      }
     }
-    sc->red_sum[eg][r] = l_part;
-    if (ok) {
-      fence_proxy_async_smem();
-      mbar_arrive(&sc->bar_p);
-      ok = mbar_wait(&sc->bar_o, 0u, abort, status);
-    }
-    // O leaves through the (now idle) K tile so that a warp writes whole rows: each thread parks its part of
+    sc->red_sum[eg][r] = l2[0] + l2[1];
+    if (ok) ok = mbar_wait(&sc->bar_o[rounds - 1], 0u, abort, status);
+    // O leaves through the (now idle) K/V region so that a warp writes whole rows: each thread parks its part of
     // its row with the 16-byte columns rotated by the row number, then lane c reads column c of a row.
-    float4* stage = reinterpret_cast<float4*>(Ks);
+    float4* stage = reinterpret_cast<float4*>(KVs);
     constexpr int C4 = DH / 4;                               // float4 columns per row
     if (ok) {
       tc_fence_after();
@@ -314,17 +335,16 @@ __global__ void __launch_bounds__(64 + SOFTMAX_THREADS, 1) k_tree_attention_tc(c
   }
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(sc->tmem_base, 256);
+    tmem_dealloc(sc->tmem_base, 512);
   }
 }
 
 template <int DH>
-void launch_dh(specasr_kv* kv, int layer, int n, int n_splits, cudaStream_t s) {
+void launch_dh(specasr_kv* kv, int layer, int n, int n_splits, int chunk, cudaStream_t s) {
   const specasr_model* m = kv->m;
   const specasr_model_config& c = m->cfg;
   constexpr int H = DH / 64;
-  constexpr int A_BYTES = 2 * H * SUB < 4 * SUB ? 4 * SUB : 2 * H * SUB;
-  const size_t smem = A_BYTES + 2 * (2 * H * SUB) + sizeof(AttnCtl) + 1024;
+  const size_t smem = 4 * SUB + 2 * H * KVSUB + sizeof(AttnCtl) + 1024;
   static bool configured = false;
   if (!configured) {
     cudaFuncSetAttribute(k_tree_attention_tc<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -345,6 +365,7 @@ void launch_dh(specasr_kv* kv, int layer, int n, int n_splits, cudaStream_t s) {
   p.group = c.n_heads / c.n_kv_heads;
   p.nodes_per_tile = 128 / p.group;
   p.n = n;
+  p.chunk = chunk;
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
   dim3 grid(c.n_kv_heads, (n + p.nodes_per_tile - 1) / p.nodes_per_tile, n_splits);
   LaunchScope scope(kv, SPECASR_KIND_ATTN, s);
@@ -356,11 +377,32 @@ void launch_dh(specasr_kv* kv, int layer, int n, int n_splits, cudaStream_t s) {
 bool attention_tc_supported(const specasr_model* m) {
   const specasr_model_config& c = m->cfg;
   const int group = c.n_heads / c.n_kv_heads;
-  return c.gemm_path == 0 && (c.head_dim == 64 || c.head_dim == 128) && c.page_size % 16 == 0 && c.page_size <= KEYS &&
-         KEYS % c.page_size == 0 && group <= 128;
+  return c.gemm_path == 0 && (c.head_dim == 64 || c.head_dim == 128) && c.page_size % 16 == 0 &&
+         c.page_size <= KEYS_MAX && group <= 128;
 }
 
-int attention_tc_splits(int total_len) { return (total_len + KEYS - 1) / KEYS; }
+// Keys per CTA and number of key blocks for `total_len` positions seen by `n` nodes: as few blocks as the
+// shared-memory tile allows, but enough to give every SM a CTA.  Returns false if they exceed `max_splits`.
+bool attention_tc_plan(const specasr_model* m, int n, int total_len, int max_splits, int* n_splits, int* chunk) {
+  const specasr_model_config& c = m->cfg;
+  const int group = c.n_heads / c.n_kv_heads;
+  const int nodes_per_tile = 128 / group;
+  const int ctas = c.n_kv_heads * ((n + nodes_per_tile - 1) / nodes_per_tile);
+  const int keys_max = KEYS_MAX / c.page_size * c.page_size;
+  int splits = (total_len + keys_max - 1) / keys_max;
+  const int fill = m->n_sm / ctas;                       // blocks that still fit in one wave
+  if (fill > splits) splits = fill;
+  if (splits > max_splits) splits = max_splits;
+  int per = (total_len + splits - 1) / splits;
+  per = (per + c.page_size - 1) / c.page_size * c.page_size;
+  if (per < c.page_size) per = c.page_size;
+  if (per > keys_max) per = keys_max;
+  splits = (total_len + per - 1) / per;
+  if (splits < 1) splits = 1;
+  *n_splits = splits;
+  *chunk = per;
+  return splits <= max_splits;
+}
 
 // Tensor maps of the rotated queries and of the two pools, as the kernel above walks them.
 bool attention_tc_make_maps(specasr_kv* kv) {
@@ -382,7 +424,7 @@ bool attention_tc_make_maps(specasr_kv* kv) {
          make_tensor_map_nd(&kv->tm_V, kv->v_pool, 5, dims, strides, box);
 }
 
-void launch_tree_attention_tc(specasr_kv* kv, int layer, int n, int n_splits, cudaStream_t s) {
-  if (kv->m->cfg.head_dim == 64) launch_dh<64>(kv, layer, n, n_splits, s);
-  else launch_dh<128>(kv, layer, n, n_splits, s);
+void launch_tree_attention_tc(specasr_kv* kv, int layer, int n, int n_splits, int chunk, cudaStream_t s) {
+  if (kv->m->cfg.head_dim == 64) launch_dh<64>(kv, layer, n, n_splits, chunk, s);
+  else launch_dh<128>(kv, layer, n, n_splits, chunk, s);
 }

@@ -313,13 +313,29 @@ __global__ void __launch_bounds__(64 + EPI_THREADS, 1) k_proj(const __grid_const
           epi_bar();
         }
         if (ok) {
-          for (int c0 = c_first; c0 < p.n_pad; c0 += 32) {
-            float v[16];
-            load16(lane_addr, t2, c0, v);
+          // parked partial sums of the CTAs that hold the rest of this tile group, added in CTA order; the
+          // loads for the next token block are in flight while the current one is processed
+          auto load_parked = [&](int c0, float* f) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) f[j] = 0.f;
             for (int cc = cta + 1; cc <= last; ++cc) {
               const float* src = p.fixP + ((size_t)(cc * p.tm + t2) * p.n_pad + c0) * TILE_M + row;
 #pragma unroll
-              for (int j = 0; j < 16; ++j) v[j] += __ldcg(src + j * TILE_M);
+              for (int j = 0; j < 16; ++j) f[j] += __ldcg(src + j * TILE_M);
+            }
+          };
+          float parked[16], parked_next[16];
+          if (last > cta && c_first < p.n_pad) load_parked(c_first, parked);
+          for (int c0 = c_first; c0 < p.n_pad; c0 += 32) {
+            float v[16];
+            load16(lane_addr, t2, c0, v);
+            if (last > cta) {
+              if (c0 + 32 < p.n_pad) load_parked(c0 + 32, parked_next);
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                v[j] += parked[j];
+                parked[j] = parked_next[j];
+              }
             }
             if (EPI == EPI_SWIGLU) {
               // rows 2f / 2f + 1 of the tile are gate / up of feature f: the even lane keeps the hi plane of

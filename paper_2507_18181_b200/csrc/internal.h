@@ -136,6 +136,28 @@ inline void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
   cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// Same, for a kernel whose CTAs form clusters of `cluster_x` along x.
+template <typename... KArgs, typename... Args>
+inline void launch_pdl_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, int cluster_x, cudaStream_t s,
+                               Args&&... args) {
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = cluster_x;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 void set_error(const char* fmt, ...);
 Workspace carve_workspace(const specasr_model* m, int n_alloc, void* base);
 int lm_tiles_of(const specasr_model* m);
@@ -158,9 +180,9 @@ void launch_commit(specasr_kv* kv, const int32_t* path, const int32_t* accept_le
 // ---- attention.cu (plain FMA) / attention_tc.cu (tcgen05)
 void launch_tree_attention(specasr_kv* kv, int layer, int n, int n_splits, cudaStream_t s);
 bool attention_tc_supported(const specasr_model* m);
-int attention_tc_splits(int total_len);
+bool attention_tc_plan(const specasr_model* m, int n, int total_len, int max_splits, int* n_splits, int* chunk);
 bool attention_tc_make_maps(specasr_kv* kv);
-void launch_tree_attention_tc(specasr_kv* kv, int layer, int n, int n_splits, cudaStream_t s);
+void launch_tree_attention_tc(specasr_kv* kv, int layer, int n, int n_splits, int chunk, cudaStream_t s);
 
 // ---- gemm_fma.cu / gemm_tcgen05.cu
 enum GemmEpilogue {

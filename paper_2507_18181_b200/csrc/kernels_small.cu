@@ -1,5 +1,7 @@
 // Integer and element-wise kernels of the verification step: tree preparation, embedding gather,
 // RMSNorm with operand split, rotary embedding + KV append, attention merge, accept, commit.
+#include <cooperative_groups.h>
+
 #include "internal.h"
 #include "device_utils.cuh"
 
@@ -144,55 +146,64 @@ void launch_copy_embeds(specasr_kv* kv, const float* embeds, int n, cudaStream_t
 // RMSNorm with the residual update folded in: x <- x + sum of the previous projection's partial planes
 // (fixed order, hence deterministic), h = x * rsqrt(mean(x^2) + eps) * g, emitted as two bf16 planes
 // hi = bf16(h), lo = bf16(h - hi) so that the tensor-core projections see ~16 significant bits of every
-// activation.  Rows n..n_pad-1 of both planes are zeroed.  One CTA per row; a thread keeps its ITER
-// float4 pieces of the row in registers, and the loads of up to four planes are issued together (an
-// in-order core would otherwise pay one L2 round trip per plane).
+// activation.  Rows n..n_pad-1 of both planes are zeroed.
+// A cluster of four CTAs owns a row, one quarter each, so that the few megabytes of partial planes are
+// pulled through 4 x n SMs at once and every thread has all its loads (x and up to 12 planes) in flight
+// together: an in-order core would otherwise pay one L2 round trip per plane.  The four partial sums of
+// squares meet through distributed shared memory and are added in rank order.
+constexpr int kNormCluster = 4;
+
 template <int ITER>
 __global__ void __launch_bounds__(256) k_rmsnorm_split(const int32_t* __restrict__ ctl, float* __restrict__ X,
                                                        const float* __restrict__ P, int n_partials,
                                                        size_t partial_stride, const float* __restrict__ gain,
-                                                       int d, float eps, int n, size_t plane_stride,
+                                                       int d, int d_part, float eps, int n, size_t plane_stride,
                                                        bf16* __restrict__ H) {
+  namespace cg = cooperative_groups;
+  __shared__ float s_ss;
   grid_dep_launch();
-  const int row = blockIdx.x;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int rank = (int)cluster.block_rank();
+  const int row = blockIdx.x / kNormCluster;
   const int tid = threadIdx.x;
+  const int k_end = min(d, (rank + 1) * d_part);
+  int kk[ITER];
   float4 g[ITER];
 #pragma unroll
   for (int it = 0; it < ITER; ++it) {        // gains never change: fetch them before waiting
-    const int k = (it * 256 + tid) * 4;
-    g[it] = k < d ? *reinterpret_cast<const float4*>(gain + k) : make_float4(0.f, 0.f, 0.f, 0.f);
+    kk[it] = rank * d_part + (it * 256 + tid) * 4;
+    g[it] = kk[it] < k_end ? *reinterpret_cast<const float4*>(gain + kk[it]) : make_float4(0.f, 0.f, 0.f, 0.f);
   }
   grid_dep_wait();
-  if (ctl[CTL_STATUS] != 0) return;
+  if (ctl[CTL_STATUS] != 0) return;          // same for the whole cluster
   bf16* hi = H + (size_t)row * d;
   bf16* lo = hi + plane_stride;
-  if (row >= n) {
-    for (int k = tid * 8; k < d; k += 256 * 8) {
-      *reinterpret_cast<uint4*>(hi + k) = make_uint4(0, 0, 0, 0);
-      *reinterpret_cast<uint4*>(lo + k) = make_uint4(0, 0, 0, 0);
-    }
+  if (row >= n) {                            // same for the whole cluster
+#pragma unroll
+    for (int it = 0; it < ITER; ++it)
+      if (kk[it] < k_end) {
+        *reinterpret_cast<uint2*>(hi + kk[it]) = make_uint2(0, 0);
+        *reinterpret_cast<uint2*>(lo + kk[it]) = make_uint2(0, 0);
+      }
     return;
   }
   float* x = X + (size_t)row * d;
   float4 v[ITER];
 #pragma unroll
-  for (int it = 0; it < ITER; ++it) {
-    const int k = (it * 256 + tid) * 4;
-    v[it] = k < d ? *reinterpret_cast<const float4*>(x + k) : make_float4(0.f, 0.f, 0.f, 0.f);
-  }
-  for (int s0 = 0; s0 < n_partials; s0 += 4) {
-    float4 q[4][ITER];
+  for (int it = 0; it < ITER; ++it)
+    v[it] = kk[it] < k_end ? *reinterpret_cast<const float4*>(x + kk[it]) : make_float4(0.f, 0.f, 0.f, 0.f);
+  constexpr int BATCH = ITER == 1 ? kMaxSplitK : (ITER == 2 ? 6 : 3);
+  for (int s0 = 0; s0 < n_partials; s0 += BATCH) {
+    float4 q[BATCH][ITER];
 #pragma unroll
-    for (int u = 0; u < 4; ++u)
+    for (int u = 0; u < BATCH; ++u)
 #pragma unroll
-      for (int it = 0; it < ITER; ++it) {
-        const int k = (it * 256 + tid) * 4;
-        q[u][it] = (s0 + u < n_partials && k < d)
-                       ? __ldcg(reinterpret_cast<const float4*>(P + (s0 + u) * partial_stride + (size_t)row * d + k))
+      for (int it = 0; it < ITER; ++it)
+        q[u][it] = (s0 + u < n_partials && kk[it] < k_end)
+                       ? __ldcg(reinterpret_cast<const float4*>(P + (s0 + u) * partial_stride + (size_t)row * d + kk[it]))
                        : make_float4(0.f, 0.f, 0.f, 0.f);
-      }
 #pragma unroll
-    for (int u = 0; u < 4; ++u)
+    for (int u = 0; u < BATCH; ++u)
 #pragma unroll
       for (int it = 0; it < ITER; ++it) {
         v[it].x += q[u][it].x; v[it].y += q[u][it].y; v[it].z += q[u][it].z; v[it].w += q[u][it].w;
@@ -201,21 +212,25 @@ __global__ void __launch_bounds__(256) k_rmsnorm_split(const int32_t* __restrict
   float ss = 0.f;
 #pragma unroll
   for (int it = 0; it < ITER; ++it) {
-    const int k = (it * 256 + tid) * 4;
-    if (n_partials > 0 && k < d) *reinterpret_cast<float4*>(x + k) = v[it];
+    if (n_partials > 0 && kk[it] < k_end) *reinterpret_cast<float4*>(x + kk[it]) = v[it];
     ss += v[it].x * v[it].x + v[it].y * v[it].y + v[it].z * v[it].z + v[it].w * v[it].w;
   }
   ss = block_sum_256(ss);
-  const float inv = rsqrtf(ss / (float)d + eps);
+  if (tid == 0) s_ss = ss;
+  cluster.sync();
+  float total = 0.f;
+#pragma unroll
+  for (int r = 0; r < kNormCluster; ++r) total += *cluster.map_shared_rank(&s_ss, r);
+  cluster.sync();                            // nobody leaves while a peer may still read its sum
+  const float inv = rsqrtf(total / (float)d + eps);
 #pragma unroll
   for (int it = 0; it < ITER; ++it) {
-    const int k = (it * 256 + tid) * 4;
-    if (k < d) {
+    if (kk[it] < k_end) {
       uint32_t ph[2], pl[2];
       split2_pack(v[it].x * inv * g[it].x, v[it].y * inv * g[it].y, ph[0], pl[0]);
       split2_pack(v[it].z * inv * g[it].z, v[it].w * inv * g[it].w, ph[1], pl[1]);
-      *reinterpret_cast<uint2*>(hi + k) = make_uint2(ph[0], ph[1]);
-      *reinterpret_cast<uint2*>(lo + k) = make_uint2(pl[0], pl[1]);
+      *reinterpret_cast<uint2*>(hi + kk[it]) = make_uint2(ph[0], ph[1]);
+      *reinterpret_cast<uint2*>(lo + kk[it]) = make_uint2(pl[0], pl[1]);
     }
   }
 }
@@ -223,16 +238,16 @@ __global__ void __launch_bounds__(256) k_rmsnorm_split(const int32_t* __restrict
 void launch_rmsnorm_split(specasr_kv* kv, const float* gain, int n, int n_pad, int n_partials, cudaStream_t s) {
   const specasr_model* m = kv->m;
   const int d = m->cfg.d_model;
+  const int d_part = (d + 4 * kNormCluster - 1) / (4 * kNormCluster) * 4;      // columns per CTA, a multiple of 4
   const size_t stride = (size_t)kv->n_alloc * d;
   LaunchScope scope(kv, SPECASR_KIND_NORM, s);
-#define NORM_LAUNCH(I)                                                                                              \
-  launch_pdl(k_rmsnorm_split<I>, dim3(n_pad), dim3(256), 0, s, kv->ws.ctl, kv->ws.X, kv->ws.P, n_partials, stride, \
-             gain, d, m->cfg.rms_eps, n, stride, kv->ws.H)
-  if (d <= 1024) NORM_LAUNCH(1);
-  else if (d <= 2048) NORM_LAUNCH(2);
-  else if (d <= 4096) NORM_LAUNCH(4);
-  else if (d <= 8192) NORM_LAUNCH(8);
-  else NORM_LAUNCH(16);
+#define NORM_LAUNCH(I)                                                                                           \
+  launch_pdl_cluster(k_rmsnorm_split<I>, dim3(kNormCluster * n_pad), dim3(256), kNormCluster, s, kv->ws.ctl,   \
+                     kv->ws.X, kv->ws.P, n_partials, stride, gain, d, d_part, m->cfg.rms_eps, n, stride, kv->ws.H)
+  if (d_part <= 1024) NORM_LAUNCH(1);
+  else if (d_part <= 2048) NORM_LAUNCH(2);
+  else if (d_part <= 4096) NORM_LAUNCH(4);
+  else NORM_LAUNCH(8);
 #undef NORM_LAUNCH
 }
 
