@@ -238,7 +238,47 @@ __global__ void __launch_bounds__(64 + EPI_THREADS, 1) k_proj(const __grid_const
       const int kb1 = (int)((u1 - u) < (long long)(KB - kb0) ? kb0 + (u1 - u) : KB);
       u += kb1 - kb0;
       const int b = seg % p.n_buf;
-      if (ok) ok = mbar_wait(&sc->acc_full[b], (uint32_t)((seg / p.n_buf) & 1), abort, status);
+      // A CTA that holds the first k-blocks of a split tile group adds the partial sums parked by the CTAs
+      // that hold the rest.  Those were parked early in their run, so their flags are polled and the first
+      // tile's parked sums are requested here, while this segment's MMAs are still running.
+      int last = cta;
+      if (EPI != EPI_PARTIAL && kb0 == 0 && kb1 != KB)
+        while (last + 1 < G && (last + 1) * U / G < (long long)(group + 1) * KB) ++last;
+      const bool quick = p.n_pad <= 64;          // at most two 16-token blocks per warp and tile: keep them in registers
+      float pk0[16], pk1[16];
+      auto load_parked = [&](int t2, int c0, float* f) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) f[j] = 0.f;
+        if (c0 < p.n_pad)
+          for (int cc = cta + 1; cc <= last; ++cc) {
+            const float* src = p.fixP + ((size_t)(cc * p.tm + t2) * p.n_pad + c0) * TILE_M + row;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) f[j] += __ldcg(src + j * TILE_M);
+          }
+      };
+      if (last > cta) {
+        if (ok && threadIdx.x == 64) {
+          const unsigned long long t0 = global_ns();
+          for (int cc = cta + 1; cc <= last && !*abort; ++cc) {
+            while (ld_acquire(p.fixFlag + cc) != p.epoch) {
+              if (*abort) break;
+              if (global_ns() - t0 > WAIT_LIMIT_NS) {
+                *abort = 1;
+                atomicExch(status, (int32_t)SPECASR_ERR_TIMEOUT);
+                break;
+              }
+              __nanosleep(64);
+            }
+          }
+        }
+        epi_bar();
+        if (*abort) ok = false;
+        if (ok && quick) {
+          load_parked(0, c_first, pk0);
+          load_parked(0, c_first + 32, pk1);
+        }
+      }
+      if (ok) ok = mbar_wait_relaxed(&sc->acc_full[b], (uint32_t)((seg / p.n_buf) & 1), abort, status);
       tc_fence_after();
       const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(b * acc_cols);
 
@@ -281,28 +321,7 @@ __global__ void __launch_bounds__(64 + EPI_THREADS, 1) k_proj(const __grid_const
         continue;
       }
 
-      // first k-blocks of the tile group: collect the partial sums of the CTAs that hold the rest
-      int last = cta;
-      if (kb1 != KB)
-        while (last + 1 < G && (last + 1) * U / G < (long long)(group + 1) * KB) ++last;
-      if (last > cta) {
-        if (ok && threadIdx.x == 64) {
-          const unsigned long long t0 = global_ns();
-          for (int cc = cta + 1; cc <= last && !*abort; ++cc) {
-            while (ld_acquire(p.fixFlag + cc) != p.epoch) {
-              if (*abort) break;
-              if (global_ns() - t0 > WAIT_LIMIT_NS) {
-                *abort = 1;
-                atomicExch(status, (int32_t)SPECASR_ERR_TIMEOUT);
-                break;
-              }
-              __nanosleep(64);
-            }
-          }
-        }
-        epi_bar();
-        if (*abort) ok = false;
-      }
+      // first k-blocks of the tile group (or all of them): run the epilogue on the complete sums
       for (int t2 = 0; t2 < p.tm; ++t2) {
         const int tile = group * p.tm + t2;
         if (tile >= p.tiles) break;
@@ -313,28 +332,32 @@ __global__ void __launch_bounds__(64 + EPI_THREADS, 1) k_proj(const __grid_const
           epi_bar();
         }
         if (ok) {
-          // parked partial sums of the CTAs that hold the rest of this tile group, added in CTA order; the
-          // loads for the next token block are in flight while the current one is processed
-          auto load_parked = [&](int c0, float* f) {
+          // parked sums of this tile (requested a tile ahead); the next tile's are requested now
+          float cur0[16], cur1[16];
+          if (last > cta && quick) {
 #pragma unroll
-            for (int j = 0; j < 16; ++j) f[j] = 0.f;
-            for (int cc = cta + 1; cc <= last; ++cc) {
-              const float* src = p.fixP + ((size_t)(cc * p.tm + t2) * p.n_pad + c0) * TILE_M + row;
-#pragma unroll
-              for (int j = 0; j < 16; ++j) f[j] += __ldcg(src + j * TILE_M);
+            for (int j = 0; j < 16; ++j) {
+              cur0[j] = pk0[j];
+              cur1[j] = pk1[j];
             }
-          };
-          float parked[16], parked_next[16];
-          if (last > cta && c_first < p.n_pad) load_parked(c_first, parked);
+            if (t2 + 1 < p.tm) {
+              load_parked(t2 + 1, c_first, pk0);
+              load_parked(t2 + 1, c_first + 32, pk1);
+            }
+          }
           for (int c0 = c_first; c0 < p.n_pad; c0 += 32) {
             float v[16];
             load16(lane_addr, t2, c0, v);
             if (last > cta) {
-              if (c0 + 32 < p.n_pad) load_parked(c0 + 32, parked_next);
+              if (quick) {
+                const bool first = c0 == c_first;
 #pragma unroll
-              for (int j = 0; j < 16; ++j) {
-                v[j] += parked[j];
-                parked[j] = parked_next[j];
+                for (int j = 0; j < 16; ++j) v[j] += first ? cur0[j] : cur1[j];
+              } else {
+                float f[16];
+                load_parked(t2, c0, f);
+#pragma unroll
+                for (int j = 0; j < 16; ++j) v[j] += f[j];
               }
             }
             if (EPI == EPI_SWIGLU) {

@@ -57,6 +57,25 @@ __device__ __forceinline__ bool mbar_wait(void* bar, uint32_t parity, volatile i
   }
 }
 
+// The same for waits that are expected to last long and are not latency critical (epilogue warps waiting
+// for a whole main loop): sleeping between polls leaves the issue slots to the warps that feed the pipeline.
+__device__ __forceinline__ bool mbar_wait_relaxed(void* bar, uint32_t parity, volatile int* abort, int32_t* status) {
+  if (mbar_try(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (uint32_t it = 1;; ++it) {
+    __nanosleep(200);
+    if (mbar_try(bar, parity)) return true;
+    if ((it & 63u) == 0u) {
+      if (*abort) return false;
+      if (global_ns() - t0 > WAIT_LIMIT_NS) {
+        *abort = 1;
+        atomicExch(status, (int32_t)SPECASR_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+
 // generic-proxy writes to shared memory -> visible to the async proxy (TMA, tcgen05.mma operands)
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
