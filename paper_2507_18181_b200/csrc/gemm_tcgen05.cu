@@ -546,7 +546,10 @@ int gemm_tc_tiles(int M) { return (M + TILE_M - 1) / TILE_M; }
 
 // Tile groups per stage and k sub-blocks per stage for trees padded to n_pad nodes.
 static void tc_shape(int n_pad, int* tm, int* ksub) {
-  *tm = (n_pad >= 48 && n_pad <= 64) ? 2 : 1;     // two sets of tm * 2 * n_pad TMEM columns must fit in 512
+  // One weight tile per stage: with 64 tokens a stage is 64 KB and three stages fit, which measured faster
+  // than two stages of a tile pair (tm = 2, activation block shared by both tiles) although the pair halves
+  // the activation traffic; the kernel keeps tm as a parameter.
+  *tm = 1;
   *ksub = n_pad <= 64 ? 2 : 1;                    // 256 contiguous bytes per weight row keep DRAM pages busy
 }
 
