@@ -191,6 +191,22 @@ def run_reference(args, wl):
 
 # ------------------------------------------------------------------------------------------------ CUDA leg
 
+def slowest_rank(elapsed, world, device):
+    """Replicas do not exchange data: the job's time is the slowest rank's (max over ranks)."""
+    if world <= 1:
+        return float(elapsed)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([elapsed], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(units_per_rank_step, steps, world, elapsed_s):
+    """Aggregate throughput of `world` independent replicas that each did `steps` steps in `elapsed_s`."""
+    return world * units_per_rank_step * steps / elapsed_s
+
+
 def build_workload(wl, device, seed=1):
     import torch
     from paper_2507_18181_b200 import build as _build
@@ -277,10 +293,7 @@ def run_ours(args, wl):
     launches = kv.launches() - launches0
     per_step = sorted(a.elapsed_time(b) for a, b in step_events)
     accept_len = int(kv.out_accept.item())
-    if world > 1:
-        t = torch.tensor([elapsed_ms], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+    elapsed_ms = slowest_rank(elapsed_ms, world, device)
 
     # end to end through the C ABI with host buffers: H2D of the tree, D2H of the results, every step
     h_tokens = torch.from_numpy(tokens).pin_memory()
@@ -308,10 +321,7 @@ def run_ours(args, wl):
         e2e_step()
     barrier()
     e2e_s = time.perf_counter() - t0
-    if world > 1:
-        t = torch.tensor([e2e_s], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    e2e_s = slowest_rank(e2e_s, world, device)
 
     if rank != 0:
         if world > 1:
@@ -337,7 +347,7 @@ def run_ours(args, wl):
         kernels[k]["achieved_gbs"] = per / (ms[k] / prof_steps * 1e-3) / 1e9
 
     ms_per_step = elapsed_ms / args.steps
-    value = world * n * args.steps / (elapsed_ms * 1e-3)
+    value = whole_job_rate(n, args.steps, world, elapsed_ms * 1e-3)
     ab = algorithmic_bytes(cfg, L, n)
     fl = algorithmic_flops(cfg, L, n)
     t_roof_ms = max(ab["total"] / (peaks["hbm_gbs"] * 1e9), fl / (peaks["bf16_tflops"] * 1e12)) * 1e3

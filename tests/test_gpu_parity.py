@@ -262,3 +262,112 @@ def test_single_node_tree_and_max_nodes():
     tokens = gen.fill_tree_tokens(parent, cfg.vocab, seed=1, root_token=root)
     got = _verify_gpu(cfg, kv, tokens, parent)
     _check_against_oracle(got, O.verify_tree(cfg, W, cache, tokens, parent), tokens, parent)
+
+
+def _bench_shape_case(cfg, n_audio, n_text, parent, seed, max_nodes):
+    """Same launch configuration as bench.py for that shape: prefill in chunks of max_nodes, page size 16,
+    tensor-core path; the oracle runs the same seeded inputs in fp64."""
+    from paper_2507_18181_b200.runtime import DeviceModel, DeviceKV
+    store = gen.WeightStore(cfg, seed)
+    model = DeviceModel(cfg, store)
+    L = n_audio + n_text - 1
+    n = len(parent)
+    kv = DeviceKV(model, max_tokens=L + n + 64, max_nodes=max_nodes)
+    W = O.Weights(store, cache_layers=True)
+    audio = gen.audio_prefix(n_audio, cfg.d_model, seed)
+    text = gen.prompt_tokens(n_text, cfg.vocab, seed)
+    cache = O.KVCache(cfg)
+    O.prefill(cfg, W, cache, np.concatenate([audio.astype(np.float64), O.embed(W, text[:-1])], 0))
+    kv.prefill_embeds(torch.from_numpy(audio).cuda())
+    kv.prefill_tokens(torch.from_numpy(text[:-1].copy()).cuda())
+    assert kv.length() == cache.length == L
+    root = int(text[-1])
+    k = len(gen.main_path(parent)) - 1
+    greedy = O.greedy_continuation(cfg, W, cache, root, k)
+    tokens = gen.fill_tree_tokens(parent, cfg.vocab, seed=seed, root_token=root, main_tokens=greedy, corrupt_p=0.2)
+    want = O.verify_tree(cfg, W, cache, tokens, parent)
+    got = _verify_gpu(cfg, kv, tokens, parent)
+    err = _check_against_oracle(got, want, tokens, parent)
+    # cache rows of the tree itself (last layer), then the commit
+    kk, vv = kv.read_kv(cfg.n_layers - 1, L + n)
+    assert np.abs(kk[L:] - want["tree_K"][-1]).max() < 2e-3 and np.abs(vv[L:] - want["tree_V"][-1]).max() < 2e-3
+    kv.commit()
+    assert kv.length() == L + got["accept_len"] + 1
+    return err, got, want
+
+
+def test_7b_shape_two_layers_in_the_benchmarked_launch_configuration():
+    """Config 3 with the layer count cut to two (the per-layer kernels, tile counts, split counts and the
+    1700 + 64 position attention are exactly those of the 32-layer benchmark run)."""
+    cfg = gen.get_config("7b", n_layers=2)
+    parent = gen.sparse_tree(64, seed=1, levels=12)
+    err, got, want = _bench_shape_case(cfg, 1500, 201, parent, seed=1, max_nodes=64)
+    assert err < LOGIT_TOL
+
+
+def test_1b_shape_chain_draft_full_size():
+    """Config 2 at full size: 16 layers, d 2048, 32 / 8 heads of 64, KV prefix 750 + 32, chain of 8 drafts."""
+    cfg = gen.get_config("1b")
+    parent = gen.chain_tree(8)
+    err, got, want = _bench_shape_case(cfg, 750, 33, parent, seed=2, max_nodes=16)
+    assert err < LOGIT_TOL
+    assert got["accept_len"] <= 8
+
+
+def test_7b_full_size_properties():
+    """Config 3 at full size (32 layers, 14 GB of weights), where the fp64 oracle would need minutes: properties
+    that hold at any size.  Determinism, the accept rule applied to the GPU's own arg-max, invariance under
+    renumbering of the tree, agreement of a node with the same node verified as a chain (its root path), and
+    the cache after commit."""
+    from paper_2507_18181_b200.runtime import DeviceModel, DeviceKV
+    cfg = gen.get_config("7b")
+    store = gen.WeightStore(cfg, 1)
+    model = DeviceModel(cfg, store)
+    L, n = 1700, 64
+    kv = DeviceKV(model, max_tokens=L + n + 64, max_nodes=64)
+    kv.prefill_embeds(torch.from_numpy(gen.audio_prefix(1500, cfg.d_model, 1)).cuda())
+    text = gen.prompt_tokens(201, cfg.vocab, 1)
+    kv.prefill_tokens(torch.from_numpy(text[:-1].copy()).cuda())
+    assert kv.length() == L
+    root = int(text[-1])
+    parent = gen.sparse_tree(n, seed=1, levels=12)
+    # the target's own greedy continuation, by single-node rounds of the library itself
+    greedy, tok = [], root
+    for _ in range(11):
+        kv.verify(torch.tensor([tok], dtype=torch.int32, device="cuda"), torch.tensor([-1], dtype=torch.int32, device="cuda"))
+        kv.commit()
+        tok = int(kv.out_bonus.item())
+        greedy.append(tok)
+    kv.truncate(L)
+    tokens = gen.fill_tree_tokens(parent, cfg.vocab, seed=1, root_token=root, main_tokens=greedy, corrupt_p=0.2)
+    a = _verify_gpu(cfg, kv, tokens, parent)
+    b = _verify_gpu(cfg, kv, tokens, parent)
+    assert np.array_equal(a["logits"], b["logits"]) and np.array_equal(a["path"], b["path"])
+    assert np.isfinite(a["logits"]).all()
+    mine = O.accept(tokens, parent, a["argmax"])
+    assert a["accept_len"] == mine["accept_len"] and a["bonus"] == mine["bonus"]
+    assert list(a["path"][:a["accept_len"] + 1]) == list(mine["path"])
+    assert np.array_equal(a["argmax"], a["logits"].argmax(-1))
+    # greedy drafts up to the first corrupted position are accepted (lossless acceptance of the target's own tokens)
+    mp = gen.main_path(parent)
+    k_ok = 0
+    while k_ok < 11 and tokens[mp[k_ok + 1]] == greedy[k_ok]:
+        k_ok += 1
+    assert a["accept_len"] >= k_ok
+    # renumbering
+    p2, t2, old = gen.relabel_tree(parent, tokens, seed=3)
+    c = _verify_gpu(cfg, kv, t2, p2)
+    assert np.abs(c["logits"] - a["logits"][old]).max() < 2e-3
+    assert c["accept_len"] == a["accept_len"]
+    # the deepest node of the main path, verified as a plain chain (= causal decoding of its root path)
+    chain_tokens = tokens[mp].astype(np.int32)
+    d = _verify_gpu(cfg, kv, chain_tokens, gen.chain_tree(len(mp) - 1))
+    assert np.abs(d["logits"] - a["logits"][mp]).max() < 2e-3
+    # commit of the tree result
+    res = _verify_gpu(cfg, kv, tokens, parent)
+    k_before, v_before = kv.read_kv(31, L + n)
+    kv.commit()
+    al = res["accept_len"]
+    assert kv.length() == L + al + 1
+    k_after, _ = kv.read_kv(31, L + al + 1)
+    assert np.array_equal(k_after[L:], k_before[L + res["path"][:al + 1]])
