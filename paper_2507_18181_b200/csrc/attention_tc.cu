@@ -63,31 +63,12 @@ __global__ void __launch_bounds__(64 + SOFTMAX_THREADS, 1) k_tree_attention_tc(c
   constexpr int KV_BYTES = 2 * H * KVSUB;
   extern __shared__ uint8_t smem_raw[];
   pdl_launch_dependents();
-  pdl_wait();
-  if (p.ctl[CTL_STATUS] != 0) return;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int kvh = blockIdx.x, split = blockIdx.z;
   const int node0 = blockIdx.y * p.nodes_per_tile;
   const int rows_used = p.nodes_per_tile * p.group;
-  const int L = p.ctl[CTL_LEN];
-  const int Ltot = L + p.n;
   const int k_begin = split * p.chunk;
-
-  // row owned by a softmax thread (warps 2..9): TMEM lane = 32 * (warp % 4) + lane
-  const int r = ((warp & 3) << 5) | lane;
-  const int node = node0 + r / p.group;
-  const bool row_valid = warp >= 2 && r < rows_used && node < p.n;
-  const size_t out_row = (size_t)split * p.rows_alloc + (size_t)node * p.Hq + kvh * p.group + r % p.group;
-
-  if (k_begin >= Ltot) {             // this key block lies beyond the cache: an empty partial
-    if (row_valid) p.attML[out_row] = make_float2(-INFINITY, 0.f);
-    return;
-  }
-  const int kc = min(p.chunk, Ltot - k_begin);
-  const int kc_pad = (kc + 15) & ~15;
-  const int pages = (kc + p.page_size - 1) / p.page_size;
-  const int rounds = (kc_pad + ROUND - 1) / ROUND;          // 1 or 2
 
   uint8_t* As = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* KVs = As + A_BYTES;
@@ -118,12 +99,32 @@ __global__ void __launch_bounds__(64 + SOFTMAX_THREADS, 1) k_tree_attention_tc(c
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  // everything above is independent of the previous kernel; its results are read from here on
+  pdl_wait();
+  const bool live = p.ctl[CTL_STATUS] == 0;
+  const int L = p.ctl[CTL_LEN];
+  const int Ltot = L + p.n;
+  // row owned by a softmax thread (warps 2..9): TMEM lane = 32 * (warp % 4) + lane
+  const int r = ((warp & 3) << 5) | lane;
+  const int node = node0 + r / p.group;
+  const bool row_valid = warp >= 2 && r < rows_used && node < p.n;
+  const size_t out_row = (size_t)split * p.rows_alloc + (size_t)node * p.Hq + kvh * p.group + r % p.group;
+
+  const bool active = live && k_begin < Ltot;
+  if (live && !active && row_valid) p.attML[out_row] = make_float2(-INFINITY, 0.f);   // key block beyond the cache: an empty partial
+  const int kc = min(p.chunk, Ltot - k_begin);
+  const int kc_pad = (kc + 15) & ~15;
+  const int pages = (kc + p.page_size - 1) / p.page_size;
+  const int rounds = (kc_pad + ROUND - 1) / ROUND;          // 1 or 2
+
   const uint32_t tmem_s = sc->tmem_base;           // S: columns [0, 208)
   const uint32_t tmem_o = sc->tmem_base + 256;     // O: columns [256, 256 + DH)
   volatile int* abort = &sc->abort;
   int32_t* status = p.ctl + CTL_STATUS;
 
-  if (warp == 0) {
+  if (!active) {
+    // nothing to do for this CTA
+  } else if (warp == 0) {
     // ---------------- TMA producer: lane 0 fetches Q, lane j fetches page j of K and later of V
     const uint32_t q_bytes = 2 * H * rows_used * 128;
     const uint32_t kv_bytes = 2 * H * pages * p.page_size * 128;

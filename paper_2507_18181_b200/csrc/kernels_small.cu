@@ -252,7 +252,7 @@ void launch_rmsnorm_split(specasr_kv* kv, const float* gain, int n, int n_pad, i
 }
 
 // ------------------------------------------------------------------------------------------------
-// Rotary embedding at tree positions + KV append.  One block per (node, head of the fused QKV row).
+// Rotary embedding at tree positions + KV append.  One thread per (node, head of the fused QKV row, rotation pair).
 // Sums the QKV projection's partial planes (their columns follow the rotary-paired row order of Wqkv),
 // rotates Q and K heads by the angle of
 // the node's position (rotate-half pairing, table built in fp64 on the host), writes Q as hi/lo planes
@@ -266,10 +266,10 @@ __global__ void k_rope_append(const int32_t* __restrict__ ctl, const float* __re
   grid_dep_wait();
   if (ctl[CTL_STATUS] != 0) return;
   const int i = blockIdx.x;
-  const int head = blockIdx.y;
   const int half = dh >> 1;
-  const int k = threadIdx.x;
-  if (k >= half) return;
+  const int head = blockIdx.y * (blockDim.x / half) + threadIdx.x / half;     // several heads per block
+  const int k = threadIdx.x % half;
+  if (head >= Hq + 2 * Hkv) return;
   const size_t col = (size_t)i * qkv_dim + (size_t)head * dh;
   const size_t c1 = col + qkv_row_of_feature(k, dh), c2 = col + qkv_row_of_feature(k + half, dh);
   float a1[kMaxSplitK], a2[kMaxSplitK];      // all plane loads in flight together, summed in plane order
@@ -319,8 +319,9 @@ __global__ void k_rope_append(const int32_t* __restrict__ ctl, const float* __re
 void launch_rope_append(specasr_kv* kv, int layer, int n, int n_partials, cudaStream_t s) {
   const specasr_model* m = kv->m;
   const specasr_model_config& c = m->cfg;
-  dim3 grid(n, c.n_heads + 2 * c.n_kv_heads);
-  const int threads = c.head_dim / 2 < 32 ? 32 : c.head_dim / 2;
+  const int heads_per_block = 256 / (c.head_dim / 2);
+  dim3 grid(n, (c.n_heads + 2 * c.n_kv_heads + heads_per_block - 1) / heads_per_block);
+  const int threads = 256;
   LaunchScope scope(kv, SPECASR_KIND_ROPE, s);
   launch_pdl(k_rope_append, grid, dim3(threads), 0, s, kv->ws.ctl, kv->ws.P, n_partials, (size_t)kv->n_alloc * m->qkv_dim, m->qkv_dim, c.n_heads, c.n_kv_heads,
              c.head_dim, kv->ws.pos, m->rope_table, layer, kv->ws.Q, (size_t)kv->n_alloc * m->q_dim, kv->k_pool,
