@@ -389,6 +389,72 @@ def run_ours(args, wl):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """Verify-cost sweep (draft / target latency balance): the 7B shape, chain drafts of 4 / 8 / 16 / 32 tokens and
+    sparse trees of 16 / 64 / 256 nodes at KV lengths 512 .. 4096.  One JSON line per point, the model is built
+    once.  Latency is the CUDA-event time of verify + commit (+ length reset) averaged over --steps rounds."""
+    import torch
+    from paper_2507_18181_b200 import build as _build
+    from paper_2507_18181_b200.runtime import DeviceModel, DeviceKV
+    _build.build()
+    device = "cuda:0"
+    torch.cuda.set_device(0)
+    seed = 1
+    cfg = gen.get_config("7b")
+    model = DeviceModel(cfg, gen.WeightStore(cfg, seed), device=device)
+    peaks = measured_peaks()
+    stream = torch.cuda.current_stream()
+    shapes = [("chain", k + 1) for k in (4, 8, 16, 32)] + [("tree", n) for n in (16, 64, 256)]
+    for L in (512, 1024, 2048, 4096):
+        kv = DeviceKV(model, max_tokens=L + 256 + 64, max_nodes=256)
+        n_text = 200
+        kv.prefill_embeds(torch.from_numpy(gen.audio_prefix(L - n_text + 1, cfg.d_model, seed)).to(device))
+        text = gen.prompt_tokens(n_text, cfg.vocab, seed)
+        kv.prefill_tokens(torch.from_numpy(text[:-1].copy()).to(device))
+        assert kv.length() == L
+        root = int(text[-1])
+        one_p = torch.tensor([-1], dtype=torch.int32, device=device)
+        greedy, tok = [], root
+        for _ in range(32):
+            kv.verify(torch.tensor([tok], dtype=torch.int32, device=device), one_p)
+            kv.commit()
+            tok = int(kv.out_bonus.item())
+            greedy.append(tok)
+        kv.truncate(L)
+        for kind, n in shapes:
+            parent = gen.chain_tree(n - 1) if kind == "chain" else gen.sparse_tree(n, seed=seed)
+            tokens = gen.fill_tree_tokens(parent, cfg.vocab, seed=seed, root_token=root, main_tokens=greedy, corrupt_p=0.2)
+            d_tokens, d_parent = torch.from_numpy(tokens).to(device), torch.from_numpy(parent).to(device)
+
+            def step():
+                kv.verify(d_tokens, d_parent)
+                kv.commit()
+                kv.truncate(L)
+
+            for _ in range(max(args.warmup, 3)):
+                step()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(args.steps):
+                step()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / args.steps
+            ab, fl = algorithmic_bytes(cfg, L, n), algorithmic_flops(cfg, L, n)
+            t_hbm = ab["total"] / (peaks["hbm_gbs"] * 1e9) * 1e3
+            t_tc = fl / (peaks["bf16_tflops"] * 1e12) * 1e3
+            print(json.dumps({
+                "workload": f"config4 {kind} n_nodes={n} kv_len={L}", "ms_per_step": ms, "tree_tokens_per_s": n / (ms * 1e-3),
+                "accept_len": int(kv.out_accept.item()), "algorithmic_bytes": ab["total"], "algorithmic_flops": fl,
+                "roof_ms": max(t_hbm, t_tc), "bound": "hbm" if t_hbm >= t_tc else "tensor",
+                "frac_of_" + peaks["source"]: max(t_hbm, t_tc) / ms,
+                "frac_of_nominal_8TBs": (ab["total"] / 8e12 * 1e3) / ms}), flush=True)
+        kv.close()
+        del kv
+        torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -397,7 +463,11 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="config3", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="config 4: one JSON line per (draft shape, KV length) point")
     args = ap.parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     wl = WORKLOADS[args.workload]
     if args.impl == "reference":
         run_reference(args, wl)

@@ -31,7 +31,13 @@ extern "C" const char* specasr_last_error(void) { return g_err; }
   } while (0)
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
-static inline int round_up(int x, int a) { return (x + a - 1) / a * a; }
+// Token counts are padded to 16, 32, 64, 128 or 256 so that the activation block of a projection is one TMA box
+// and one MMA (a padded count like 48 would need three narrow MMAs per k-step).
+static inline int pad_tokens(int n) {
+  int p = 16;
+  while (p < n) p <<= 1;
+  return p;
+}
 
 int lm_tiles_of(const specasr_model* m) {
   return m->cfg.gemm_path == 1 ? gemm_fma_tiles(m->cfg.vocab) : gemm_tc_tiles(m->cfg.vocab);
@@ -178,7 +184,7 @@ extern "C" void specasr_model_destroy(specasr_model* m) {
 
 extern "C" size_t specasr_workspace_bytes(const specasr_model* m, int32_t max_nodes) {
   if (!m || max_nodes < 1 || max_nodes > SPECASR_MAX_NODES) return 0;
-  return carve_workspace(m, round_up(max_nodes, 16), nullptr).bytes;
+  return carve_workspace(m, pad_tokens(max_nodes), nullptr).bytes;
 }
 
 extern "C" size_t specasr_kv_pool_bytes(const specasr_model* m, int32_t n_pages) {
@@ -215,7 +221,7 @@ extern "C" specasr_status specasr_kv_create(const specasr_model* m, void* k_pool
   kv->page_table = page_table;
   kv->max_pages = max_pages;
   kv->max_nodes = max_nodes;
-  kv->n_alloc = round_up(max_nodes, 16);
+  kv->n_alloc = pad_tokens(max_nodes);
   kv->ws = carve_workspace(m, kv->n_alloc, workspace);
   kv->pending_n = 0;
   kv->len_host = 0;
@@ -393,7 +399,7 @@ static int attention_splits(const specasr_kv* kv, int n, int len_upper, bool* us
 // norm, the vocabulary projection and its fused per-tile argmax run as well.
 static void run_stack(specasr_model* m, specasr_kv* kv, int n, bool want_head, float* out_logits, cudaStream_t s) {
   const specasr_model_config& c = m->cfg;
-  const int n_pad = round_up(n, 16);
+  const int n_pad = pad_tokens(n);
   bool att_tc = false;
   int att_chunk = 0;
   const int att_splits = attention_splits(kv, n, kv->len_upper, &att_tc, &att_chunk);
