@@ -40,6 +40,7 @@ extern "C" {
 #endif
 
 #define SPECASR_MAX_NODES 256
+#define SPECASR_MAX_BATCH 32
 
 typedef enum specasr_status {
   SPECASR_OK = 0,
@@ -154,6 +155,38 @@ specasr_status specasr_verify_tree_ex(specasr_model* m, specasr_kv* kv, const in
                                       const int32_t* parent_idx, int32_t n_nodes, int32_t* out_argmax,
                                       int32_t* out_accept_len, int32_t* out_path, float* out_logits,
                                       int32_t* out_bonus, void* stream);
+
+/*
+ * Verify the draft trees of several utterances in one pass over the weights.  Section II-B defines the
+ * verification of one draft (all of its tokens checked by the target model at once); the paper decodes one
+ * utterance at a time and has no batched form.  This call applies that same definition to several
+ * utterances side by side so that they share one stream of the weights: every utterance keeps its own
+ * cache, committed length and tree, and the results are those of `batch` separate specasr_verify_tree calls.
+ *   batch              : 1 .. SPECASR_MAX_BATCH
+ *   kv                 : [host] `batch` distinct handles of model `m`, all on the tensor-core attention path
+ *                        (head_dim 64 or 128, page_size a multiple of 16).  The workspace of kv[0] carries the
+ *                        rows of all utterances, so node_offsets[batch] <= max_nodes of kv[0]; it also
+ *                        receives the launch counts and profile records of the call.
+ *   node_offsets       : [host] int32[batch + 1], node_offsets[0] = 0, strictly increasing; utterance b owns
+ *                        nodes node_offsets[b] .. node_offsets[b+1]-1 of the arrays below
+ *   tokens, parent_idx : [device] int32[node_offsets[batch]]; parent_idx is local to the utterance
+ *                        (-1 for its root, otherwise 0 <= parent < index within the utterance)
+ *   out_argmax, out_path : [device] int32[node_offsets[batch]], per utterance as in specasr_verify_tree
+ *                        (path entries are local node indices)
+ *   out_accept_len     : [device] int32[batch]
+ *   out_bonus          : [device] int32[batch] or NULL
+ * Each handle becomes "pending" and is committed on its own:
+ *   specasr_commit_kv(m, kv[b], out_path + node_offsets[b], out_accept_len + b, stream).
+ * Errors: host-visible ones (null, batch or offsets out of range, a handle twice, a cache that would
+ * overflow, SPECASR_ERR_UNSUPPORTED for a handle without the tensor-core attention path) return before
+ * anything is enqueued.  A malformed tree fails only its own utterance (its out_accept_len is -1 and its
+ * handle's status word is set); a bounded wait that runs out in a kernel shared by all utterances fails
+ * every one of them.
+ */
+specasr_status specasr_verify_tree_batch(specasr_model* m, int32_t batch, specasr_kv* const* kv,
+                                         const int32_t* tokens, const int32_t* parent_idx,
+                                         const int32_t* node_offsets, int32_t* out_argmax, int32_t* out_accept_len,
+                                         int32_t* out_path, int32_t* out_bonus, void* stream);
 
 /*
  * Keep the accepted path (the "revert to the draft model" step of Section II-B needs the cache to

@@ -11,6 +11,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libspecasr.so")
 
 SPECASR_MAX_NODES = 256
+SPECASR_MAX_BATCH = 32
 (SPECASR_OK, SPECASR_ERR_INVALID_ARG, SPECASR_ERR_INVALID_TREE, SPECASR_ERR_KV_CAPACITY, SPECASR_ERR_STATE,
  SPECASR_ERR_UNSUPPORTED, SPECASR_ERR_TIMEOUT, SPECASR_ERR_CUDA) = range(8)
 STATUS_NAMES = ["OK", "INVALID_ARG", "INVALID_TREE", "KV_CAPACITY", "STATE", "UNSUPPORTED", "TIMEOUT", "CUDA"]
@@ -19,7 +20,7 @@ EXPORTS = [
     "specasr_model_create", "specasr_model_destroy", "specasr_workspace_bytes", "specasr_kv_pool_bytes",
     "specasr_kv_create", "specasr_kv_destroy", "specasr_kv_length", "specasr_kv_truncate",
     "specasr_prefill_embeds", "specasr_prefill_tokens", "specasr_verify_tree", "specasr_verify_tree_ex",
-    "specasr_commit_kv", "specasr_poll_status", "specasr_launch_count", "specasr_last_error",
+    "specasr_verify_tree_batch", "specasr_commit_kv", "specasr_poll_status", "specasr_launch_count", "specasr_last_error",
     "specasr_profile_enable", "specasr_profile_read", "specasr_accept_logits_static",
 ]
 KIND_NAMES = ["prep", "norm", "gemm_qkv", "rope", "attn", "attn_merge", "gemm_o", "gemm_gu", "gemm_down", "gemm_lm",
@@ -74,6 +75,8 @@ def lib() -> C.CDLL:
         L.specasr_verify_tree.restype = st
         L.specasr_verify_tree_ex.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp]
         L.specasr_verify_tree_ex.restype = st
+        L.specasr_verify_tree_batch.argtypes = [vp, i32, C.POINTER(vp), vp, vp, C.POINTER(i32), vp, vp, vp, vp, vp]
+        L.specasr_verify_tree_batch.restype = st
         L.specasr_commit_kv.argtypes = [vp, vp, vp, vp, vp]
         L.specasr_commit_kv.restype = st
         L.specasr_poll_status.argtypes = [vp, C.POINTER(i32), vp]
@@ -166,6 +169,19 @@ def specasr_verify_tree_ex(model: int, kv: int, tokens: int, parent_idx: int, n_
                            stream: int = 0) -> None:
     _check(lib().specasr_verify_tree_ex(model, kv, tokens, parent_idx, n_nodes, out_argmax, out_accept_len, out_path,
                                         out_logits or None, out_bonus or None, stream))
+
+
+def specasr_verify_tree_batch(model: int, kv_handles, tokens: int, parent_idx: int, node_offsets, out_argmax: int,
+                              out_accept_len: int, out_path: int, out_bonus: int = 0, stream: int = 0) -> None:
+    """kv_handles: sequence of handles; node_offsets: sequence of batch + 1 ints (both host side);
+    the other arguments are device addresses covering all utterances back to back."""
+    batch = len(kv_handles)
+    handles = (C.c_void_p * batch)(*kv_handles)
+    offsets = (C.c_int32 * len(node_offsets))(*node_offsets)
+    if len(node_offsets) != batch + 1:
+        raise ValueError("node_offsets needs batch + 1 entries")
+    _check(lib().specasr_verify_tree_batch(model, batch, handles, tokens, parent_idx, offsets, out_argmax,
+                                           out_accept_len, out_path, out_bonus or None, stream))
 
 
 def specasr_commit_kv(model: int, kv: int, path: int, accept_len: int, stream: int = 0) -> None:

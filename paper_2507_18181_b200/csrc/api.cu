@@ -373,13 +373,15 @@ static void run_gemm(specasr_kv* kv, GemmArgs& a, int kind, cudaStream_t s) {
   }
 }
 
-static int attention_splits(const specasr_kv* kv, int n, int len_upper, bool* use_tc, int* chunk) {
+// Key blocks of the attention over `n` nodes of one utterance; `sm_budget` is the number of SMs the launch
+// should fill (all of them for a plain call, a share of them when several utterances launch back to back).
+static int attention_splits(const specasr_kv* kv, int n, int len_upper, int sm_budget, bool* use_tc, int* chunk) {
   const specasr_model_config& c = kv->m->cfg;
   *use_tc = false;
   *chunk = 0;
   if (kv->attn_tc) {
     int s = 0;
-    if (attention_tc_plan(kv->m, n, len_upper + n, kMaxAttnSplits, &s, chunk)) {
+    if (attention_tc_plan(kv->m, n, len_upper + n, sm_budget, kMaxAttnSplits, &s, chunk)) {
       *use_tc = true;
       return s;
     }
@@ -387,7 +389,7 @@ static int attention_splits(const specasr_kv* kv, int n, int len_upper, bool* us
   const int group = c.n_heads / c.n_kv_heads;
   const int row_tiles = (n * group + 63) / 64;
   const int ctas = c.n_kv_heads * row_tiles;
-  int splits = (kv->m->n_sm + ctas - 1) / ctas;
+  int splits = (sm_budget + ctas - 1) / ctas;
   const int by_len = (len_upper + n + 63) / 64;
   if (splits > by_len) splits = by_len;
   if (splits > kMaxAttnSplits) splits = kMaxAttnSplits;
@@ -395,49 +397,69 @@ static int attention_splits(const specasr_kv* kv, int n, int len_upper, bool* us
   return splits;
 }
 
-// The layer stack over n rows whose layer-0 inputs are already in ws.X.  With want_head the final
-// norm, the vocabulary projection and its fused per-tile argmax run as well.
-static void run_stack(specasr_model* m, specasr_kv* kv, int n, bool want_head, float* out_logits, cudaStream_t s) {
+struct AttnPlan {
+  bool tc;
+  int splits;      // grid depth of every utterance's launch (the largest any of them needs)
+  int chunk[SPECASR_MAX_BATCH];
+};
+
+// The layer stack over the rows of `nseg` utterances laid out back to back in the workspace of `wk`
+// (n_total rows, layer-0 inputs already in ws.X).  Norms, projections and the attention merge run once over
+// all rows and look at the control block `ctl_shared`; the rotary/append and attention kernels run per
+// utterance against its own cache and control block.  With want_head the final norm, the vocabulary projection
+// and its fused per-tile argmax run as well.
+static void run_stack(specasr_model* m, specasr_kv* wk, const Rows* segs, int nseg, int n_total,
+                      const int32_t* ctl_shared, const AttnPlan& plan, bool want_head, float* out_logits,
+                      cudaStream_t s) {
   const specasr_model_config& c = m->cfg;
+  const int n = n_total;
   const int n_pad = pad_tokens(n);
-  bool att_tc = false;
-  int att_chunk = 0;
-  const int att_splits = attention_splits(kv, n, kv->len_upper, &att_tc, &att_chunk);
   const bool tc = c.gemm_path == 0;
   int pending = 0;               // partial planes of the last down projection still to be added to X
   GemmArgs a;
   memset(&a, 0, sizeof(a));
   a.n = n;
   a.n_pad = n_pad;
-  a.n_alloc = kv->n_alloc;
-  a.ctl = kv->ws.ctl;
-  a.P = kv->ws.P;
+  a.n_alloc = wk->n_alloc;
+  a.ctl = ctl_shared;
+  a.P = wk->ws.P;
   for (int l = 0; l < c.n_layers; ++l) {
-    launch_rmsnorm_split(kv, m->g_attn[l], n, n_pad, pending, s);
-    a.W = m->wqkv[l]; a.tmW = tc ? &m->tm_wqkv[l] : nullptr; a.tmAct = kv->tm_H; a.act = kv->ws.H;
+    launch_rmsnorm_split(wk, ctl_shared, m->g_attn[l], n, n_pad, pending, s);
+    a.W = m->wqkv[l]; a.tmW = tc ? &m->tm_wqkv[l] : nullptr; a.tmAct = wk->tm_H; a.act = wk->ws.H;
     a.M = m->qkv_dim; a.K = c.d_model; a.epilogue = EPI_PARTIAL;
-    run_gemm(kv, a, SPECASR_KIND_GEMM_QKV, s);
-    launch_rope_append(kv, l, n, a.splits, s);
-    if (att_tc) launch_tree_attention_tc(kv, l, n, att_splits, att_chunk, s);
-    else launch_tree_attention(kv, l, n, att_splits, s);
-    launch_attn_merge(kv, n, n_pad, att_splits, s);
-    a.W = m->wo[l]; a.tmW = tc ? &m->tm_wo[l] : nullptr; a.tmAct = kv->tm_AO; a.act = kv->ws.AO;
+    run_gemm(wk, a, SPECASR_KIND_GEMM_QKV, s);
+    for (int b = 0; b < nseg; ++b) launch_rope_append(wk, segs[b], l, a.splits, s);
+    for (int b = 0; b < nseg; ++b) {
+      if (plan.tc) launch_tree_attention_tc(wk, segs[b], l, plan.splits, plan.chunk[b], s);
+      else launch_tree_attention(wk, l, n, plan.splits, s);      // single utterance only
+    }
+    launch_attn_merge(wk, ctl_shared, n, n_pad, plan.splits, s);
+    a.W = m->wo[l]; a.tmW = tc ? &m->tm_wo[l] : nullptr; a.tmAct = wk->tm_AO; a.act = wk->ws.AO;
     a.M = c.d_model; a.K = m->q_dim; a.epilogue = EPI_PARTIAL;
-    run_gemm(kv, a, SPECASR_KIND_GEMM_O, s);
-    launch_rmsnorm_split(kv, m->g_ffn[l], n, n_pad, a.splits, s);
-    a.W = m->wgu[l]; a.tmW = tc ? &m->tm_wgu[l] : nullptr; a.tmAct = kv->tm_H; a.act = kv->ws.H;
-    a.M = 2 * c.ffn; a.K = c.d_model; a.epilogue = EPI_SWIGLU; a.A = kv->ws.A;
-    run_gemm(kv, a, SPECASR_KIND_GEMM_GU, s);
-    a.W = m->wd[l]; a.tmW = tc ? &m->tm_wd[l] : nullptr; a.tmAct = kv->tm_A; a.act = kv->ws.A;
+    run_gemm(wk, a, SPECASR_KIND_GEMM_O, s);
+    launch_rmsnorm_split(wk, ctl_shared, m->g_ffn[l], n, n_pad, a.splits, s);
+    a.W = m->wgu[l]; a.tmW = tc ? &m->tm_wgu[l] : nullptr; a.tmAct = wk->tm_H; a.act = wk->ws.H;
+    a.M = 2 * c.ffn; a.K = c.d_model; a.epilogue = EPI_SWIGLU; a.A = wk->ws.A;
+    run_gemm(wk, a, SPECASR_KIND_GEMM_GU, s);
+    a.W = m->wd[l]; a.tmW = tc ? &m->tm_wd[l] : nullptr; a.tmAct = wk->tm_A; a.act = wk->ws.A;
     a.M = c.d_model; a.K = c.ffn; a.epilogue = EPI_PARTIAL;
-    run_gemm(kv, a, SPECASR_KIND_GEMM_DOWN, s);
+    run_gemm(wk, a, SPECASR_KIND_GEMM_DOWN, s);
     pending = a.splits;
   }
   if (!want_head) return;   // context fill: K/V of every layer are written, the last FFN output is not needed
-  launch_rmsnorm_split(kv, m->g_final, n, n_pad, pending, s);
-  a.W = m->lm_head; a.tmW = tc ? &m->tm_lm : nullptr; a.tmAct = kv->tm_H; a.act = kv->ws.H;
-  a.M = c.vocab; a.K = c.d_model; a.epilogue = EPI_ARGMAX; a.amax = kv->ws.amax; a.logits = out_logits;
-  run_gemm(kv, a, SPECASR_KIND_GEMM_LM, s);
+  launch_rmsnorm_split(wk, ctl_shared, m->g_final, n, n_pad, pending, s);
+  a.W = m->lm_head; a.tmW = tc ? &m->tm_lm : nullptr; a.tmAct = wk->tm_H; a.act = wk->ws.H;
+  a.M = c.vocab; a.K = c.d_model; a.epilogue = EPI_ARGMAX; a.amax = wk->ws.amax; a.logits = out_logits;
+  run_gemm(wk, a, SPECASR_KIND_GEMM_LM, s);
+}
+
+// One utterance in its own workspace: the plain calls.
+static void run_stack_single(specasr_model* m, specasr_kv* kv, int n, bool want_head, float* out_logits,
+                             cudaStream_t s) {
+  AttnPlan plan;
+  plan.splits = attention_splits(kv, n, kv->len_upper, m->n_sm, &plan.tc, &plan.chunk[0]);
+  const Rows seg{kv, 0, n};
+  run_stack(m, kv, &seg, 1, n, kv->ws.ctl, plan, want_head, out_logits, s);
 }
 
 static specasr_status prefill_common(specasr_model* m, specasr_kv* kv, const float* embeds, const int32_t* tokens,
@@ -466,8 +488,8 @@ static specasr_status prefill_common(specasr_model* m, specasr_kv* kv, const flo
     const int chunk = n - done < kv->max_nodes ? n - done : kv->max_nodes;
     launch_chain_prep(kv, chunk, s);
     if (embeds) launch_copy_embeds(kv, embeds + (size_t)done * m->cfg.d_model, chunk, s);
-    else launch_embed_tokens(kv, tokens + done, chunk, s);
-    run_stack(m, kv, chunk, false, nullptr, s);
+    else launch_embed_tokens(kv, Rows{kv, 0, chunk}, tokens + done, s);
+    run_stack_single(m, kv, chunk, false, nullptr, s);
     launch_advance_len(kv, chunk, s);
     kv->len_host += chunk;
     kv->len_upper = kv->len_host;
@@ -511,10 +533,11 @@ extern "C" specasr_status specasr_verify_tree_ex(specasr_model* m, specasr_kv* k
     return SPECASR_ERR_KV_CAPACITY;
   }
   cudaStream_t s = (cudaStream_t)stream;
-  launch_tree_prep(kv, tokens, parent_idx, n_nodes, s);
-  launch_embed_tokens(kv, tokens, n_nodes, s);
-  run_stack(m, kv, n_nodes, true, out_logits, s);
-  launch_accept(kv, tokens, parent_idx, n_nodes, lm_tiles_of(m), out_argmax, out_accept_len, out_path, out_bonus, s);
+  const Rows seg{kv, 0, n_nodes};
+  launch_tree_prep(kv, seg, tokens, parent_idx, s);
+  launch_embed_tokens(kv, seg, tokens, s);
+  run_stack_single(m, kv, n_nodes, true, out_logits, s);
+  launch_accept(kv, seg, nullptr, tokens, parent_idx, lm_tiles_of(m), out_argmax, out_accept_len, out_path, out_bonus, s);
   kv->pending_n = n_nodes;
   CUDA_TRY(cudaGetLastError());
   return SPECASR_OK;
@@ -525,6 +548,95 @@ extern "C" specasr_status specasr_verify_tree(specasr_model* m, specasr_kv* kv, 
                                               int32_t* out_accept_len, int32_t* out_path, void* stream) {
   return specasr_verify_tree_ex(m, kv, tokens, parent_idx, n_nodes, out_argmax, out_accept_len, out_path, nullptr,
                                 nullptr, stream);
+}
+
+// Several utterances in one pass over the weights: the verification of Section II-B applied to each utterance,
+// with the norms and projections run once over all rows.
+extern "C" specasr_status specasr_verify_tree_batch(specasr_model* m, int32_t batch, specasr_kv* const* kv,
+                                                    const int32_t* tokens, const int32_t* parent_idx,
+                                                    const int32_t* node_offsets, int32_t* out_argmax,
+                                                    int32_t* out_accept_len, int32_t* out_path, int32_t* out_bonus,
+                                                    void* stream) {
+  const char* who = "specasr_verify_tree_batch";
+  if (!m || !kv || !tokens || !parent_idx || !node_offsets || !out_argmax || !out_accept_len || !out_path) {
+    set_error("%s: null argument", who);
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  if (batch < 1 || batch > SPECASR_MAX_BATCH) {
+    set_error("%s: batch = %d outside [1, %d]", who, batch, SPECASR_MAX_BATCH);
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  if (node_offsets[0] != 0) {
+    set_error("%s: node_offsets[0] must be 0", who);
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  for (int b = 0; b < batch; ++b) {
+    if (!kv[b] || kv[b]->m != m) {
+      set_error("%s: handle %d is null or belongs to another model", who, b);
+      return SPECASR_ERR_INVALID_ARG;
+    }
+    for (int j = 0; j < b; ++j)
+      if (kv[j] == kv[b]) {
+        set_error("%s: handle %d appears twice", who, b);
+        return SPECASR_ERR_INVALID_ARG;
+      }
+    if (node_offsets[b + 1] <= node_offsets[b]) {
+      set_error("%s: utterance %d has no nodes (node_offsets must increase)", who, b);
+      return SPECASR_ERR_INVALID_ARG;
+    }
+  }
+  specasr_kv* wk = kv[0];
+  const int total = node_offsets[batch];
+  if (total > wk->max_nodes) {
+    set_error("%s: %d nodes in all exceed the %d rows of the first handle's workspace", who, total, wk->max_nodes);
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  int cap = m->cfg.max_positions;
+  AttnPlan plan;
+  plan.tc = true;
+  plan.splits = 1;
+  int budget = m->n_sm / batch;
+  if (budget < 1) budget = 1;
+  for (int b = 0; b < batch; ++b) {
+    specasr_kv* u = kv[b];
+    const int n_b = node_offsets[b + 1] - node_offsets[b];
+    if (!u->attn_tc) {
+      set_error("%s: needs the tensor-core attention path (head_dim 64 or 128, page_size %% 16 == 0)", who);
+      return SPECASR_ERR_UNSUPPORTED;
+    }
+    refresh_len(u, false);
+    int cap_b = u->max_pages * m->cfg.page_size;
+    if (cap < cap_b) cap_b = cap;
+    if (u->len_exact && u->len_host + n_b > cap_b) {
+      set_error("%s: utterance %d: %d committed + %d tree slots exceed the capacity of %d", who, b, u->len_host, n_b,
+                cap_b);
+      return SPECASR_ERR_KV_CAPACITY;
+    }
+    bool use_tc = false;
+    const int sp = attention_splits(u, n_b, u->len_upper, budget, &use_tc, &plan.chunk[b]);
+    if (!use_tc) {
+      set_error("%s: utterance %d: cache of up to %d positions needs more key blocks than the workspace holds", who, b,
+                u->len_upper + n_b);
+      return SPECASR_ERR_UNSUPPORTED;
+    }
+    if (sp > plan.splits) plan.splits = sp;
+  }
+  cudaStream_t s = (cudaStream_t)stream;
+  int32_t* ctl_shared = wk->ws.ctl + kCtlBatch;
+  CUDA_TRY(cudaMemsetAsync(ctl_shared, 0, sizeof(int32_t) * 4, s));
+  Rows segs[SPECASR_MAX_BATCH];
+  for (int b = 0; b < batch; ++b) segs[b] = Rows{kv[b], node_offsets[b], node_offsets[b + 1] - node_offsets[b]};
+  for (int b = 0; b < batch; ++b) launch_tree_prep(wk, segs[b], tokens + segs[b].row0, parent_idx + segs[b].row0, s);
+  for (int b = 0; b < batch; ++b) launch_embed_tokens(wk, segs[b], tokens + segs[b].row0, s);
+  run_stack(m, wk, segs, batch, total, ctl_shared, plan, true, nullptr, s);
+  for (int b = 0; b < batch; ++b) {
+    const int o = segs[b].row0;
+    launch_accept(wk, segs[b], ctl_shared, tokens + o, parent_idx + o, lm_tiles_of(m), out_argmax + o,
+                  out_accept_len + b, out_path + o, out_bonus ? out_bonus + b : nullptr, s);
+    kv[b]->pending_n = segs[b].n;
+  }
+  CUDA_TRY(cudaGetLastError());
+  return SPECASR_OK;
 }
 
 extern "C" specasr_status specasr_commit_kv(specasr_model* m, specasr_kv* kv, const int32_t* path,

@@ -50,7 +50,7 @@ struct AttnParams {
   float* attO;
   float2* attML;
   size_t rows_alloc;      // n_alloc * Hq
-  int n_pages, page_size, layer, Hq, Hkv, group, nodes_per_tile, n, chunk;
+  int n_pages, page_size, layer, Hq, Hkv, group, nodes_per_tile, n, chunk, row0;
   float scale_log2;
 };
 
@@ -136,7 +136,7 @@ __global__ void __launch_bounds__(64 + SOFTMAX_THREADS, 1) k_tree_attention_tc(c
     if (lane == 0) {
       for (int plane = 0; plane < 2; ++plane)
         for (int h = 0; h < H; ++h)
-          tma_load_4d(As + (plane * H + h) * SUB, &tmQ, h * 64, kvh * p.group, node0, plane, &sc->bar_qk);
+          tma_load_4d(As + (plane * H + h) * SUB, &tmQ, h * 64, kvh * p.group, p.row0 + node0, plane, &sc->bar_qk);
     }
     int c4 = 0;
     const int off = lane * p.page_size * 128;
@@ -341,8 +341,10 @@ __global__ void __launch_bounds__(64 + SOFTMAX_THREADS, 1) k_tree_attention_tc(c
 }
 
 template <int DH>
-void launch_dh(specasr_kv* kv, int layer, int n, int n_splits, int chunk, cudaStream_t s) {
-  const specasr_model* m = kv->m;
+void launch_dh(specasr_kv* wk, const Rows& r, int layer, int n_splits, int chunk, cudaStream_t s) {
+  const specasr_model* m = wk->m;
+  specasr_kv* kv = r.kv;
+  const int n = r.n;
   const specasr_model_config& c = m->cfg;
   constexpr int H = DH / 64;
   const size_t smem = 4 * SUB + 2 * H * KVSUB + sizeof(AttnCtl) + 1024;
@@ -354,10 +356,11 @@ void launch_dh(specasr_kv* kv, int layer, int n, int n_splits, int chunk, cudaSt
   AttnParams p;
   p.ctl = kv->ws.ctl;
   p.page_table = kv->page_table;
-  p.anc = kv->ws.anc;
-  p.attO = kv->ws.attO;
-  p.attML = kv->ws.attML;
-  p.rows_alloc = (size_t)kv->n_alloc * c.n_heads;
+  p.anc = wk->ws.anc + (size_t)r.row0 * 4;
+  p.attO = wk->ws.attO + (size_t)r.row0 * c.n_heads * DH;
+  p.attML = wk->ws.attML + (size_t)r.row0 * c.n_heads;
+  p.rows_alloc = (size_t)wk->n_alloc * c.n_heads;
+  p.row0 = r.row0;
   p.n_pages = kv->n_pages;
   p.page_size = c.page_size;
   p.layer = layer;
@@ -369,8 +372,8 @@ void launch_dh(specasr_kv* kv, int layer, int n, int n_splits, int chunk, cudaSt
   p.chunk = chunk;
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
   dim3 grid(c.n_kv_heads, (n + p.nodes_per_tile - 1) / p.nodes_per_tile, n_splits);
-  LaunchScope scope(kv, SPECASR_KIND_ATTN, s);
-  launch_pdl(k_tree_attention_tc<DH>, grid, dim3(64 + SOFTMAX_THREADS), smem, s, kv->tm_Q, kv->tm_K, kv->tm_V, p);
+  LaunchScope scope(wk, SPECASR_KIND_ATTN, s);
+  launch_pdl(k_tree_attention_tc<DH>, grid, dim3(64 + SOFTMAX_THREADS), smem, s, wk->tm_Q, kv->tm_K, kv->tm_V, p);
 }
 
 }  // namespace
@@ -383,15 +386,17 @@ bool attention_tc_supported(const specasr_model* m) {
 }
 
 // Keys per CTA and number of key blocks for `total_len` positions seen by `n` nodes: as few blocks as the
-// shared-memory tile allows, but enough to give every SM a CTA.  Returns false if they exceed `max_splits`.
-bool attention_tc_plan(const specasr_model* m, int n, int total_len, int max_splits, int* n_splits, int* chunk) {
+// shared-memory tile allows, but enough to give each of `sm_budget` SMs a CTA.  Returns false if they exceed
+// `max_splits`.
+bool attention_tc_plan(const specasr_model* m, int n, int total_len, int sm_budget, int max_splits, int* n_splits,
+                       int* chunk) {
   const specasr_model_config& c = m->cfg;
   const int group = c.n_heads / c.n_kv_heads;
   const int nodes_per_tile = 128 / group;
   const int ctas = c.n_kv_heads * ((n + nodes_per_tile - 1) / nodes_per_tile);
   const int keys_max = KEYS_MAX / c.page_size * c.page_size;
   int splits = (total_len + keys_max - 1) / keys_max;
-  const int fill = m->n_sm / ctas;                       // blocks that still fit in one wave
+  const int fill = sm_budget / ctas;                      // blocks that still fit in one wave
   if (fill > splits) splits = fill;
   if (splits > max_splits) splits = max_splits;
   int per = (total_len + splits - 1) / splits;
@@ -425,7 +430,7 @@ bool attention_tc_make_maps(specasr_kv* kv) {
          make_tensor_map_nd(&kv->tm_V, kv->v_pool, 5, dims, strides, box);
 }
 
-void launch_tree_attention_tc(specasr_kv* kv, int layer, int n, int n_splits, int chunk, cudaStream_t s) {
-  if (kv->m->cfg.head_dim == 64) launch_dh<64>(kv, layer, n, n_splits, chunk, s);
-  else launch_dh<128>(kv, layer, n, n_splits, chunk, s);
+void launch_tree_attention_tc(specasr_kv* wk, const Rows& r, int layer, int n_splits, int chunk, cudaStream_t s) {
+  if (wk->m->cfg.head_dim == 64) launch_dh<64>(wk, r, layer, n_splits, chunk, s);
+  else launch_dh<128>(wk, r, layer, n_splits, chunk, s);
 }

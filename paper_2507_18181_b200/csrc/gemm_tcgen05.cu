@@ -593,7 +593,7 @@ void launch_gemm_tc(specasr_kv* kv, const GemmArgs& a, int kind, cudaStream_t s)
   p.groups = (p.tiles + p.tm - 1) / p.tm;
   p.splits = a.epilogue == EPI_PARTIAL ? a.splits : 0;
   p.epoch = ++kv->gemm_epoch;
-  p.ctl = kv->ws.ctl;
+  p.ctl = const_cast<int32_t*>(a.ctl);
   p.fixP = kv->ws.fixP;
   p.fixFlag = kv->ws.fixFlag;
   p.P = a.P; p.A = a.A; p.amax = a.amax; p.logits = a.logits;

@@ -19,6 +19,9 @@ constexpr int kCtlWords = 64;      // int32 control block at the start of the wo
 
 // control block word indices
 enum { CTL_LEN = 0, CTL_STATUS = 1, CTL_N = 2 };
+// A second control block (same word layout) at this offset serves the kernels that a batched call runs once
+// over all utterances: its status word only ever records a bounded wait that ran out.
+constexpr int kCtlBatch = 16;
 
 struct GemmMaps {           // TMA descriptors of one weight matrix (tcgen05 path)
   CUtensorMap w;
@@ -158,19 +161,29 @@ inline void launch_pdl_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, 
   cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// The rows of one utterance in a (possibly batched) call: its handle (control words, pools, page table),
+// the first workspace row it occupies and its number of rows.  A plain call is one such segment at row 0
+// of its own workspace.
+struct Rows {
+  specasr_kv* kv;
+  int row0;
+  int n;
+};
+
 void set_error(const char* fmt, ...);
 Workspace carve_workspace(const specasr_model* m, int n_alloc, void* base);
 int lm_tiles_of(const specasr_model* m);
 
 // ---- kernels_small.cu
-void launch_tree_prep(specasr_kv* kv, const int32_t* tokens, const int32_t* parent, int n, cudaStream_t s);
+void launch_tree_prep(specasr_kv* wk, const Rows& r, const int32_t* tokens, const int32_t* parent, cudaStream_t s);
 void launch_chain_prep(specasr_kv* kv, int n, cudaStream_t s);
-void launch_embed_tokens(specasr_kv* kv, const int32_t* tokens, int n, cudaStream_t s);
+void launch_embed_tokens(specasr_kv* wk, const Rows& r, const int32_t* tokens, cudaStream_t s);
 void launch_copy_embeds(specasr_kv* kv, const float* embeds, int n, cudaStream_t s);
-void launch_rmsnorm_split(specasr_kv* kv, const float* gain, int n, int n_pad, int n_partials, cudaStream_t s);
-void launch_rope_append(specasr_kv* kv, int layer, int n, int n_partials, cudaStream_t s);
-void launch_attn_merge(specasr_kv* kv, int n, int n_pad, int n_splits, cudaStream_t s);
-void launch_accept(specasr_kv* kv, const int32_t* tokens, const int32_t* parent, int n, int n_tiles,
+void launch_rmsnorm_split(specasr_kv* wk, const int32_t* ctl, const float* gain, int n, int n_pad, int n_partials,
+                          cudaStream_t s);
+void launch_rope_append(specasr_kv* wk, const Rows& r, int layer, int n_partials, cudaStream_t s);
+void launch_attn_merge(specasr_kv* wk, const int32_t* ctl, int n, int n_pad, int n_splits, cudaStream_t s);
+void launch_accept(specasr_kv* wk, const Rows& r, const int32_t* ctl_shared, const int32_t* tokens, const int32_t* parent, int n_tiles,
                    int32_t* out_argmax, int32_t* out_accept_len, int32_t* out_path, int32_t* out_bonus,
                    cudaStream_t s);
 void launch_advance_len(specasr_kv* kv, int n, cudaStream_t s);
@@ -180,9 +193,10 @@ void launch_commit(specasr_kv* kv, const int32_t* path, const int32_t* accept_le
 // ---- attention.cu (plain FMA) / attention_tc.cu (tcgen05)
 void launch_tree_attention(specasr_kv* kv, int layer, int n, int n_splits, cudaStream_t s);
 bool attention_tc_supported(const specasr_model* m);
-bool attention_tc_plan(const specasr_model* m, int n, int total_len, int max_splits, int* n_splits, int* chunk);
+bool attention_tc_plan(const specasr_model* m, int n, int total_len, int sm_budget, int max_splits, int* n_splits,
+                       int* chunk);
 bool attention_tc_make_maps(specasr_kv* kv);
-void launch_tree_attention_tc(specasr_kv* kv, int layer, int n, int n_splits, int chunk, cudaStream_t s);
+void launch_tree_attention_tc(specasr_kv* wk, const Rows& r, int layer, int n_splits, int chunk, cudaStream_t s);
 
 // ---- gemm_fma.cu / gemm_tcgen05.cu
 enum GemmEpilogue {
@@ -209,7 +223,7 @@ void launch_gemm_fma(specasr_kv* kv, const GemmArgs& a, int kind, cudaStream_t s
 int gemm_tc_tiles(int M);
 size_t gemm_tc_fixup_bytes(const specasr_model* m, int n_alloc);
 int gemm_tc_pick_splits(const specasr_model* m, int M, int K, int n_pad);
-void launch_gemm_tc(specasr_kv* kv, const GemmArgs& a, int kind, cudaStream_t s);
+void launch_gemm_tc(specasr_kv* kv, const GemmArgs& a, int kind, cudaStream_t s);   // a.ctl = control block to check
 bool make_tensor_map_2d(CUtensorMap* out, const void* base, uint64_t inner, uint64_t outer,
                         uint32_t box_inner, uint32_t box_outer);
 bool make_act_map(CUtensorMap* out, const void* base, uint64_t K, uint64_t n_alloc, uint32_t box_rows);

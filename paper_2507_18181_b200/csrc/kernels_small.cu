@@ -82,13 +82,13 @@ __global__ void k_chain_prep(int32_t* __restrict__ ctl, int n, int capacity, int
   }
 }
 
-void launch_tree_prep(specasr_kv* kv, const int32_t* tokens, const int32_t* parent, int n, cudaStream_t s) {
-  const specasr_model* m = kv->m;
-  int cap = kv->max_pages * m->cfg.page_size;
+void launch_tree_prep(specasr_kv* wk, const Rows& r, const int32_t* tokens, const int32_t* parent, cudaStream_t s) {
+  const specasr_model* m = wk->m;
+  int cap = r.kv->max_pages * m->cfg.page_size;
   if (m->cfg.max_positions < cap) cap = m->cfg.max_positions;
-  LaunchScope scope(kv, SPECASR_KIND_PREP, s);
-  launch_pdl(k_tree_prep, dim3(1), dim3(256), 0, s, kv->ws.ctl, tokens, parent, n, m->cfg.vocab, cap, kv->ws.depth, kv->ws.pos,
-                                kv->ws.anc);
+  LaunchScope scope(wk, SPECASR_KIND_PREP, s);
+  launch_pdl(k_tree_prep, dim3(1), dim3(256), 0, s, r.kv->ws.ctl, tokens, parent, r.n, m->cfg.vocab, cap,
+             wk->ws.depth + r.row0, wk->ws.pos + r.row0, wk->ws.anc + (size_t)r.row0 * 4);
 }
 
 void launch_chain_prep(specasr_kv* kv, int n, cudaStream_t s) {
@@ -132,9 +132,11 @@ __global__ void k_copy_embeds(const int32_t* __restrict__ ctl, const float* __re
     *reinterpret_cast<float4*>(X + (size_t)i * d + k) = *reinterpret_cast<const float4*>(src + (size_t)i * d + k);
 }
 
-void launch_embed_tokens(specasr_kv* kv, const int32_t* tokens, int n, cudaStream_t s) {
-  LaunchScope scope(kv, SPECASR_KIND_PREP, s);
-  launch_pdl(k_embed_tokens, dim3(n), dim3(128), 0, s, kv->ws.ctl, tokens, kv->m->embed, kv->m->cfg.d_model, kv->ws.X);
+void launch_embed_tokens(specasr_kv* wk, const Rows& r, const int32_t* tokens, cudaStream_t s) {
+  const int d = wk->m->cfg.d_model;
+  LaunchScope scope(wk, SPECASR_KIND_PREP, s);
+  launch_pdl(k_embed_tokens, dim3(r.n), dim3(128), 0, s, r.kv->ws.ctl, tokens, wk->m->embed, d,
+             wk->ws.X + (size_t)r.row0 * d);
 }
 
 void launch_copy_embeds(specasr_kv* kv, const float* embeds, int n, cudaStream_t s) {
@@ -235,14 +237,15 @@ __global__ void __launch_bounds__(256) k_rmsnorm_split(const int32_t* __restrict
   }
 }
 
-void launch_rmsnorm_split(specasr_kv* kv, const float* gain, int n, int n_pad, int n_partials, cudaStream_t s) {
+void launch_rmsnorm_split(specasr_kv* kv, const int32_t* ctl, const float* gain, int n, int n_pad, int n_partials,
+                          cudaStream_t s) {
   const specasr_model* m = kv->m;
   const int d = m->cfg.d_model;
   const int d_part = (d + 4 * kNormCluster - 1) / (4 * kNormCluster) * 4;      // columns per CTA, a multiple of 4
   const size_t stride = (size_t)kv->n_alloc * d;
   LaunchScope scope(kv, SPECASR_KIND_NORM, s);
 #define NORM_LAUNCH(I)                                                                                           \
-  launch_pdl_cluster(k_rmsnorm_split<I>, dim3(kNormCluster * n_pad), dim3(256), kNormCluster, s, kv->ws.ctl,   \
+  launch_pdl_cluster(k_rmsnorm_split<I>, dim3(kNormCluster * n_pad), dim3(256), kNormCluster, s, ctl,          \
                      kv->ws.X, kv->ws.P, n_partials, stride, gain, d, d_part, m->cfg.rms_eps, n, stride, kv->ws.H)
   if (d_part <= 1024) NORM_LAUNCH(1);
   else if (d_part <= 2048) NORM_LAUNCH(2);
@@ -316,16 +319,16 @@ __global__ void k_rope_append(const int32_t* __restrict__ ctl, const float* __re
   }
 }
 
-void launch_rope_append(specasr_kv* kv, int layer, int n, int n_partials, cudaStream_t s) {
-  const specasr_model* m = kv->m;
+void launch_rope_append(specasr_kv* wk, const Rows& r, int layer, int n_partials, cudaStream_t s) {
+  const specasr_model* m = wk->m;
   const specasr_model_config& c = m->cfg;
   const int heads_per_block = 256 / (c.head_dim / 2);
-  dim3 grid(n, (c.n_heads + 2 * c.n_kv_heads + heads_per_block - 1) / heads_per_block);
-  const int threads = 256;
-  LaunchScope scope(kv, SPECASR_KIND_ROPE, s);
-  launch_pdl(k_rope_append, grid, dim3(threads), 0, s, kv->ws.ctl, kv->ws.P, n_partials, (size_t)kv->n_alloc * m->qkv_dim, m->qkv_dim, c.n_heads, c.n_kv_heads,
-             c.head_dim, kv->ws.pos, m->rope_table, layer, kv->ws.Q, (size_t)kv->n_alloc * m->q_dim, kv->k_pool,
-             kv->v_pool, kv->page_table, kv->n_pages, c.page_size);
+  dim3 grid(r.n, (c.n_heads + 2 * c.n_kv_heads + heads_per_block - 1) / heads_per_block);
+  LaunchScope scope(wk, SPECASR_KIND_ROPE, s);
+  launch_pdl(k_rope_append, grid, dim3(256), 0, s, r.kv->ws.ctl, wk->ws.P + (size_t)r.row0 * m->qkv_dim, n_partials,
+             (size_t)wk->n_alloc * m->qkv_dim, m->qkv_dim, c.n_heads, c.n_kv_heads, c.head_dim, wk->ws.pos + r.row0,
+             m->rope_table, layer, wk->ws.Q + (size_t)r.row0 * m->q_dim, (size_t)wk->n_alloc * m->q_dim, r.kv->k_pool,
+             r.kv->v_pool, r.kv->page_table, r.kv->n_pages, c.page_size);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -390,11 +393,11 @@ __global__ void __launch_bounds__(128) k_attn_merge(const int32_t* __restrict__ 
   }
 }
 
-void launch_attn_merge(specasr_kv* kv, int n, int n_pad, int n_splits, cudaStream_t s) {
+void launch_attn_merge(specasr_kv* kv, const int32_t* ctl, int n, int n_pad, int n_splits, cudaStream_t s) {
   const specasr_model_config& c = kv->m->cfg;
   const int rows_total = n_pad * c.n_heads;
   LaunchScope scope(kv, SPECASR_KIND_ATTN_MERGE, s);
-  launch_pdl(k_attn_merge, dim3((rows_total + 3) / 4), dim3(128), 0, s, kv->ws.ctl, kv->ws.attO, kv->ws.attML, n_splits,
+  launch_pdl(k_attn_merge, dim3((rows_total + 3) / 4), dim3(128), 0, s, ctl, kv->ws.attO, kv->ws.attML, n_splits,
              (size_t)kv->n_alloc * c.n_heads, c.n_heads, c.head_dim, n, rows_total, kv->ws.AO,
              (size_t)kv->n_alloc * kv->m->q_dim);
 }
@@ -402,7 +405,7 @@ void launch_attn_merge(specasr_kv* kv, int n, int n_pad, int n_splits, cudaStrea
 // ------------------------------------------------------------------------------------------------
 // Accept: reduce the per-vocab-tile argmax candidates, then follow draft tokens while they equal the
 // target's greedy token at their parent; the deepest such node (lowest index among equals) wins.
-__global__ void __launch_bounds__(256) k_accept(const int32_t* __restrict__ ctl,
+__global__ void __launch_bounds__(256) k_accept(int32_t* __restrict__ ctl, const int32_t* __restrict__ ctl_shared,
                                                 const unsigned long long* __restrict__ amax, int n_tiles,
                                                 int n_alloc, const int32_t* __restrict__ tokens,
                                                 const int32_t* __restrict__ parent,
@@ -414,7 +417,10 @@ __global__ void __launch_bounds__(256) k_accept(const int32_t* __restrict__ ctl,
   const int i = threadIdx.x;
   grid_dep_launch();
   grid_dep_wait();
-  if (ctl[CTL_STATUS] != 0) {
+  // a failure of the kernels shared by a whole batch (a bounded wait that ran out) fails every utterance
+  const int shared_status = ctl_shared ? ctl_shared[CTL_STATUS] : 0;
+  if (ctl[CTL_STATUS] != 0 || shared_status != 0) {
+    if (i == 0 && ctl[CTL_STATUS] == 0) ctl[CTL_STATUS] = shared_status;
     if (i < n) {
       out_path[i] = -1;
       out_argmax[i] = -1;
@@ -479,12 +485,12 @@ __global__ void __launch_bounds__(256) k_accept(const int32_t* __restrict__ ctl,
   }
 }
 
-void launch_accept(specasr_kv* kv, const int32_t* tokens, const int32_t* parent, int n, int n_tiles,
+void launch_accept(specasr_kv* wk, const Rows& r, const int32_t* ctl_shared, const int32_t* tokens, const int32_t* parent, int n_tiles,
                    int32_t* out_argmax, int32_t* out_accept_len, int32_t* out_path, int32_t* out_bonus,
                    cudaStream_t s) {
-  LaunchScope scope(kv, SPECASR_KIND_ACCEPT, s);
-  launch_pdl(k_accept, dim3(1), dim3(256), 0, s, kv->ws.ctl, kv->ws.amax, n_tiles, kv->n_alloc, tokens, parent, kv->ws.depth, n,
-                             out_argmax, out_accept_len, out_path, out_bonus);
+  LaunchScope scope(wk, SPECASR_KIND_ACCEPT, s);
+  launch_pdl(k_accept, dim3(1), dim3(256), 0, s, r.kv->ws.ctl, ctl_shared, wk->ws.amax + r.row0, n_tiles, wk->n_alloc, tokens,
+             parent, wk->ws.depth + r.row0, r.n, out_argmax, out_accept_len, out_path, out_bonus);
 }
 
 // ------------------------------------------------------------------------------------------------

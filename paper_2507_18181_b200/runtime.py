@@ -176,3 +176,34 @@ class DeviceKV:
             self.close()
         except Exception:
             pass
+
+
+class BatchVerifier:
+    """Output buffers for specasr_verify_tree_batch over a fixed list of utterances.  The first
+    utterance's workspace carries the rows of all of them, so its max_nodes bounds the total."""
+
+    def __init__(self, kvs):
+        self.kvs = list(kvs)
+        self.model = self.kvs[0].model
+        dev = self.model.device
+        total = self.kvs[0].max_nodes
+        self.out_argmax = torch.empty(total, dtype=torch.int32, device=dev)
+        self.out_path = torch.empty(total, dtype=torch.int32, device=dev)
+        self.out_accept = torch.empty(len(self.kvs), dtype=torch.int32, device=dev)
+        self.out_bonus = torch.empty(len(self.kvs), dtype=torch.int32, device=dev)
+        self.offsets = [0] * (len(self.kvs) + 1)
+
+    def verify(self, tokens: torch.Tensor, parent: torch.Tensor, node_offsets):
+        """tokens / parent: int32 device tensors over all utterances back to back (parents local to the
+        utterance); node_offsets: batch + 1 host ints."""
+        self.offsets = [int(o) for o in node_offsets]
+        B.specasr_verify_tree_batch(self.model.handle, [kv.handle for kv in self.kvs], tokens.data_ptr(),
+                                    parent.data_ptr(), self.offsets, self.out_argmax.data_ptr(),
+                                    self.out_accept.data_ptr(), self.out_path.data_ptr(), self.out_bonus.data_ptr(),
+                                    DeviceKV._stream())
+
+    def commit(self):
+        item = self.out_path.element_size()
+        for b, kv in enumerate(self.kvs):
+            B.specasr_commit_kv(self.model.handle, kv.handle, self.out_path.data_ptr() + item * self.offsets[b],
+                                self.out_accept.data_ptr() + item * b, DeviceKV._stream())
