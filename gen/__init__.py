@@ -9,10 +9,12 @@ from .configs import ModelConfig, CONFIGS, get_config
 from .bf16 import f32_to_bf16_bits, bf16_bits_to_f32, bf16_bits_to_f64
 from .weights import WeightStore, LAYER_TENSORS, GLOBAL_TENSORS
 from .inputs import audio_prefix, prompt_tokens, uniform_tokens
+from .proposals import CorruptedGreedyProposer
 from .trees import (
     chain_tree,
     complete_binary_tree,
     sparse_tree,
+    trunk_tree,
     main_path,
     fill_tree_tokens,
     relabel_tree,
@@ -23,6 +25,7 @@ __all__ = [
     "f32_to_bf16_bits", "bf16_bits_to_f32", "bf16_bits_to_f64",
     "WeightStore", "LAYER_TENSORS", "GLOBAL_TENSORS",
     "audio_prefix", "prompt_tokens", "uniform_tokens",
-    "chain_tree", "complete_binary_tree", "sparse_tree",
+    "chain_tree", "complete_binary_tree", "sparse_tree", "trunk_tree",
     "main_path", "fill_tree_tokens", "relabel_tree",
+    "CorruptedGreedyProposer",
 ]

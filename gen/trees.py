@@ -82,6 +82,24 @@ def sparse_tree(n_nodes: int, seed: int = 0, root_fanout: int = 4, level2_fanout
     return np.asarray(parent, dtype=np.int32)
 
 
+def trunk_tree(n_nodes: int, trunk_len: int, seed: int = 0, max_branch: int = 3) -> np.ndarray:
+    """Root, a trunk (chain) of `trunk_len` draft nodes numbered 1..trunk_len, and the remaining nodes as short
+    side branches: each is a chain of 1..max_branch nodes hanging off a seeded trunk node (or the root) as a
+    sibling of the next trunk node -- the long-trunk / few-short-branches shape of a sparse draft tree
+    (Section IV-C).  The trunk is the main path (its nodes are the lowest-numbered children)."""
+    if trunk_len < 1 or trunk_len + 1 > n_nodes:
+        raise ValueError("trunk does not fit")
+    rng = _rng(seed, _STREAM_TREE)
+    parent = [-1] + list(range(trunk_len))
+    while len(parent) < n_nodes:
+        length = int(min(rng.integers(1, max_branch + 1), n_nodes - len(parent)))
+        prev = int(rng.integers(0, trunk_len))          # branches off below trunk node `prev` (0 = root)
+        for _ in range(length):
+            parent.append(prev)
+            prev = len(parent) - 1
+    return np.asarray(parent, dtype=np.int32)
+
+
 def main_path(parent: np.ndarray) -> np.ndarray:
     """Node indices root -> leaf obtained by always stepping to the lowest-numbered child."""
     n = len(parent)
