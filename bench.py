@@ -455,18 +455,155 @@ def run_sweep(args):
         torch.cuda.empty_cache()
 
 
+def run_loop(args):
+    """Config 5: the batched draft-then-verify loop end to end.  8 utterances with audio prefixes of 300..1500
+    frames decode 200 tokens each: per round the 0.5B-shape draft model is stepped autoregressively (all
+    utterances per step in one batched call), the 7B-shape target verifies one 32-node sparse tree per utterance
+    in one batched call, accepted paths are committed, and accept lengths / bonus tokens go back to the host.
+    Proposals are the target's greedy transcript (computed beforehand, untimed, by the library itself running
+    autoregressively) corrupted per position with p = 0.2, with the tail past a rejection recycled.  A step is
+    one full decode of the batch; the transcript of every step is checked token for token against the
+    autoregressive one.  One JSON line: emitted tokens per second, host control and copies included."""
+    import torch
+    from paper_2507_18181_b200 import build as _build
+    from paper_2507_18181_b200.loop import SpeculativeBatchLoop
+    from paper_2507_18181_b200.runtime import BatchVerifier, DeviceModel, DeviceKV
+    _build.build()
+    device = "cuda:0"
+    torch.cuda.set_device(0)
+    seed, B, n_tokens, n_nodes, k_max, n_prompt = 1, 8, 200, 32, 16, 8
+    small = args.workload == "config5_small"       # same loop on 2-layer cuts, for a quick functional run
+    cfg = gen.get_config("7b", **({"n_layers": 2} if small else {}))
+    dcfg = gen.get_config("0.5b", **({"n_layers": 2} if small else {}))
+    target = DeviceModel(cfg, gen.WeightStore(cfg, seed), device=device)
+    draft = DeviceModel(dcfg, gen.WeightStore(dcfg, seed + 1), device=device)
+    frames = np.random.Generator(np.random.PCG64(np.random.SeedSequence([seed, 0x5E55]))).integers(300, 1501, size=B)
+    margin = n_tokens + 2 * k_max + n_nodes + 64
+    need = n_tokens + 2 * k_max + 2
+    min_gap = 3e-4
+    kvs, dkvs, roots, L0, truth, redrawn = [], [], [], [], [], 0
+    one_p = torch.tensor([-1], dtype=torch.int32, device=device)
+    logits = torch.empty(1, cfg.vocab, dtype=torch.float32, device=device)
+    utt = 0
+    while len(kvs) < B:
+        # the target's autoregressive greedy transcript of this utterance (input construction and the reference
+        # of the check).  Token-for-token equality is only defined away from ties (two computation orders of
+        # the same fp32 sums differ by ~1e-5 in a logit), so an utterance whose transcript has a top-2 logit
+        # gap below min_gap anywhere is redrawn.
+        b = len(kvs)
+        prompt = gen.prompt_tokens(n_prompt, cfg.vocab, seed, utterance=utt)
+        kv = DeviceKV(target, max_tokens=int(frames[b]) + n_prompt + margin, max_nodes=B * n_nodes)
+        kv.prefill_embeds(torch.from_numpy(gen.audio_prefix(int(frames[b]), cfg.d_model, seed, utterance=utt)).to(device))
+        kv.prefill_tokens(torch.from_numpy(prompt[:-1].copy()).to(device))
+        L = int(frames[b]) + n_prompt - 1
+        tok, seq, gap = int(prompt[-1]), [], float("inf")
+        for _ in range(need):
+            kv.verify(torch.tensor([tok], dtype=torch.int32, device=device), one_p, logits)
+            kv.commit()
+            top = torch.topk(logits[0], 2).values
+            gap = min(gap, float(top[0] - top[1]))
+            tok = int(kv.out_bonus.item())
+            seq.append(tok)
+            if gap < min_gap:
+                break
+        if gap < min_gap:
+            redrawn += 1
+            utt += 1
+            kv.close()
+            continue
+        kv.truncate(L)
+        dkv = DeviceKV(draft, max_tokens=int(frames[b]) + n_prompt + margin, max_nodes=B * n_nodes)
+        dkv.prefill_embeds(torch.from_numpy(gen.audio_prefix(int(frames[b]), dcfg.d_model, seed, utterance=utt)).to(device))
+        dkv.prefill_tokens(torch.from_numpy(prompt[:-1].copy()).to(device))
+        kvs.append(kv)
+        dkvs.append(dkv)
+        roots.append(int(prompt[-1]))
+        L0.append(L)
+        truth.append(seq)
+        utt += 1
+    # batched one-token-per-step decoding with the same library, as the autoregressive baseline of the loop
+    bv = BatchVerifier(kvs)
+    toks = torch.tensor(roots, dtype=torch.int32, device=device)
+    minus = torch.full((B,), -1, dtype=torch.int32, device=device)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(n_tokens):
+        bv.verify(toks, minus, list(range(B + 1)))
+        bv.commit()
+        toks = bv.out_bonus.clone()
+        toks.cpu()
+    autoregressive_s = time.perf_counter() - t0
+
+    def reset():
+        for b in range(B):
+            kvs[b].truncate(L0[b])
+            dkvs[b].truncate(L0[b])
+
+    def one_decode():
+        reset()
+        proposer = gen.CorruptedGreedyProposer(truth, roots, cfg.vocab, seed=seed, n_nodes=n_nodes, k_min=4,
+                                               k_max=k_max, corrupt_p=0.2)
+        loop = SpeculativeBatchLoop(kvs, dkvs)
+        out = loop.decode(roots, n_tokens, proposer)
+        torch.cuda.synchronize()
+        return loop, out
+
+    warm = max(1, min(args.warmup, 2))
+    steps = max(1, min(args.steps, 5))
+    for _ in range(warm):
+        one_decode()
+    launches0 = sum(kv.launches() for kv in kvs + dkvs)
+    sampler = ClockSampler(0)
+    sampler.start()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        loop, out = one_decode()
+    elapsed = time.perf_counter() - t0
+    clocks = sampler.stop()
+    launches = sum(kv.launches() for kv in kvs + dkvs) - launches0
+    lossless = all(out[b] == truth[b][:n_tokens] for b in range(B))
+    per = elapsed / steps
+    line = {
+        "metric": "end_to_end_tokens_per_s", "value": B * n_tokens / per, "unit": "emitted tokens/s", "n_gpus": 1,
+        "steps": steps, "warmup": warm, "ms_per_step": per * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "target": cfg.name, "target_layers": cfg.n_layers, "draft": dcfg.name,
+                   "draft_layers": dcfg.n_layers, "utterances": B, "audio_frames": [int(f) for f in frames],
+                   "tokens_per_utterance": n_tokens, "tree_nodes": n_nodes, "draft_len": [4, k_max], "corrupt_p": 0.2,
+                   "utterances_redrawn_for_near_ties": redrawn, "min_top2_gap": min_gap,
+                   "timing": "host wall clock around the whole decode (host control, H2D of trees, D2H of results)"},
+        "lossless": lossless, "rounds_per_decode": loop.rounds, "draft_steps_per_decode": loop.draft_steps,
+        "tokens_per_tree": sum(len(o) for o in out) / max(1, loop.utterance_rounds),
+        "autoregressive_batched_tokens_per_s": B * n_tokens / autoregressive_s,
+        "speedup_over_autoregressive": autoregressive_s / per,
+        "gpu_launches": int(launches // steps), "clocks": clocks,
+    }
+    print(json.dumps(line))
+    if not lossless:
+        for b in range(B):
+            d = [i for i in range(n_tokens) if out[b][i] != truth[b][i]]
+            if d:
+                print(f"utterance {b}: first difference at token {d[0]}: {out[b][d[0]]} vs {truth[b][d[0]]}", file=sys.stderr)
+        raise SystemExit("speculative transcript differs from the autoregressive one")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="config3", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="config3", choices=sorted(WORKLOADS) + ["config5", "config5_small"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="config 4: one JSON line per (draft shape, KV length) point")
     args = ap.parse_args()
     if args.sweep:
         run_sweep(args)
+        return
+    if args.workload.startswith("config5"):
+        if args.impl == "reference" or args.gpus != 1:
+            raise SystemExit("config5 runs the CUDA loop on one GPU only")
+        run_loop(args)
         return
     wl = WORKLOADS[args.workload]
     if args.impl == "reference":

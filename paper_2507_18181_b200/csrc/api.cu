@@ -68,6 +68,7 @@ Workspace carve_workspace(const specasr_model* m, int n_alloc, void* base) {
   w.attO = (float*)take(sizeof(float) * kMaxAttnSplits * n_alloc * c.n_heads * c.head_dim);
   w.attML = (float2*)take(sizeof(float2) * kMaxAttnSplits * n_alloc * c.n_heads);
   w.amax = (unsigned long long*)take(sizeof(unsigned long long) * lm_tiles_of(m) * n_alloc);
+  w.tmKV = (CUtensorMap*)take(sizeof(CUtensorMap) * 2);
   w.bytes = off;
   return w;
 }
@@ -397,20 +398,32 @@ static int attention_splits(const specasr_kv* kv, int n, int len_upper, int sm_b
   return splits;
 }
 
-struct AttnPlan {
-  bool tc;
-  int splits;      // grid depth of every utterance's launch (the largest any of them needs)
-  int chunk[SPECASR_MAX_BATCH];
-};
+// Table entry of one utterance (everything but the attention plan).
+static SegDev seg_entry(const specasr_kv* u, int row0, int n) {
+  SegDev d;
+  memset(&d, 0, sizeof(d));
+  d.ctl = u->ws.ctl;
+  d.page_table = u->page_table;
+  d.k_pool = u->k_pool;
+  d.v_pool = u->v_pool;
+  d.tmK = u->attn_tc ? u->ws.tmKV : nullptr;
+  d.tmV = u->attn_tc ? u->ws.tmKV + 1 : nullptr;
+  d.n_pages = u->n_pages;
+  d.row0 = row0;
+  d.n = n;
+  int cap = u->max_pages * u->m->cfg.page_size;
+  if (u->m->cfg.max_positions < cap) cap = u->m->cfg.max_positions;
+  d.capacity = cap;
+  return d;
+}
 
-// The layer stack over the rows of `nseg` utterances laid out back to back in the workspace of `wk`
-// (n_total rows, layer-0 inputs already in ws.X).  Norms, projections and the attention merge run once over
-// all rows and look at the control block `ctl_shared`; the rotary/append and attention kernels run per
-// utterance against its own cache and control block.  With want_head the final norm, the vocabulary projection
+// The layer stack over the rows of the utterances in `tab`, laid out back to back in the workspace of `wk`
+// (n_total rows, layer-0 inputs already in ws.X).  Norms, projections and the attention merge look at the
+// control block `ctl_shared`; the rotary/append and attention kernels look up each row's utterance in the table
+// and work against its cache and control block.  With want_head the final norm, the vocabulary projection
 // and its fused per-tile argmax run as well.
-static void run_stack(specasr_model* m, specasr_kv* wk, const Rows* segs, int nseg, int n_total,
-                      const int32_t* ctl_shared, const AttnPlan& plan, bool want_head, float* out_logits,
-                      cudaStream_t s) {
+static void run_stack(specasr_model* m, specasr_kv* wk, const SegTable& tab, int n_total, int n_max, bool att_tc,
+                      const int32_t* ctl_shared, bool want_head, float* out_logits, cudaStream_t s) {
   const specasr_model_config& c = m->cfg;
   const int n = n_total;
   const int n_pad = pad_tokens(n);
@@ -428,12 +441,10 @@ static void run_stack(specasr_model* m, specasr_kv* wk, const Rows* segs, int ns
     a.W = m->wqkv[l]; a.tmW = tc ? &m->tm_wqkv[l] : nullptr; a.tmAct = wk->tm_H; a.act = wk->ws.H;
     a.M = m->qkv_dim; a.K = c.d_model; a.epilogue = EPI_PARTIAL;
     run_gemm(wk, a, SPECASR_KIND_GEMM_QKV, s);
-    for (int b = 0; b < nseg; ++b) launch_rope_append(wk, segs[b], l, a.splits, s);
-    for (int b = 0; b < nseg; ++b) {
-      if (plan.tc) launch_tree_attention_tc(wk, segs[b], l, plan.splits, plan.chunk[b], s);
-      else launch_tree_attention(wk, l, n, plan.splits, s);      // single utterance only
-    }
-    launch_attn_merge(wk, ctl_shared, n, n_pad, plan.splits, s);
+    launch_rope_append(wk, tab, n, l, a.splits, s);
+    if (att_tc) launch_tree_attention_tc(wk, tab, n_max, l, s);
+    else launch_tree_attention(wk, l, n, tab.splits, s);      // single utterance only
+    launch_attn_merge(wk, ctl_shared, n, n_pad, tab.splits, s);
     a.W = m->wo[l]; a.tmW = tc ? &m->tm_wo[l] : nullptr; a.tmAct = wk->tm_AO; a.act = wk->ws.AO;
     a.M = c.d_model; a.K = m->q_dim; a.epilogue = EPI_PARTIAL;
     run_gemm(wk, a, SPECASR_KIND_GEMM_O, s);
@@ -453,13 +464,14 @@ static void run_stack(specasr_model* m, specasr_kv* wk, const Rows* segs, int ns
   run_gemm(wk, a, SPECASR_KIND_GEMM_LM, s);
 }
 
-// One utterance in its own workspace: the plain calls.
-static void run_stack_single(specasr_model* m, specasr_kv* kv, int n, bool want_head, float* out_logits,
-                             cudaStream_t s) {
-  AttnPlan plan;
-  plan.splits = attention_splits(kv, n, kv->len_upper, m->n_sm, &plan.tc, &plan.chunk[0]);
-  const Rows seg{kv, 0, n};
-  run_stack(m, kv, &seg, 1, n, kv->ws.ctl, plan, want_head, out_logits, s);
+// The table of a plain call: one utterance at row 0 of its own workspace, attention planned for the whole GPU.
+static SegTable single_table(specasr_kv* kv, int n, bool* att_tc) {
+  SegTable t;
+  memset(&t, 0, sizeof(t));
+  t.count = 1;
+  t.seg[0] = seg_entry(kv, 0, n);
+  t.splits = attention_splits(kv, n, kv->len_upper, kv->m->n_sm, att_tc, &t.seg[0].chunk);
+  return t;
 }
 
 static specasr_status prefill_common(specasr_model* m, specasr_kv* kv, const float* embeds, const int32_t* tokens,
@@ -487,9 +499,11 @@ static specasr_status prefill_common(specasr_model* m, specasr_kv* kv, const flo
   for (int done = 0; done < n;) {
     const int chunk = n - done < kv->max_nodes ? n - done : kv->max_nodes;
     launch_chain_prep(kv, chunk, s);
+    bool att_tc = false;
+    const SegTable tab = single_table(kv, chunk, &att_tc);
     if (embeds) launch_copy_embeds(kv, embeds + (size_t)done * m->cfg.d_model, chunk, s);
-    else launch_embed_tokens(kv, Rows{kv, 0, chunk}, tokens + done, s);
-    run_stack_single(m, kv, chunk, false, nullptr, s);
+    else launch_embed_tokens(kv, tab, chunk, tokens + done, s);
+    run_stack(m, kv, tab, chunk, chunk, att_tc, kv->ws.ctl, false, nullptr, s);
     launch_advance_len(kv, chunk, s);
     kv->len_host += chunk;
     kv->len_upper = kv->len_host;
@@ -533,11 +547,12 @@ extern "C" specasr_status specasr_verify_tree_ex(specasr_model* m, specasr_kv* k
     return SPECASR_ERR_KV_CAPACITY;
   }
   cudaStream_t s = (cudaStream_t)stream;
-  const Rows seg{kv, 0, n_nodes};
-  launch_tree_prep(kv, seg, tokens, parent_idx, s);
-  launch_embed_tokens(kv, seg, tokens, s);
-  run_stack_single(m, kv, n_nodes, true, out_logits, s);
-  launch_accept(kv, seg, nullptr, tokens, parent_idx, lm_tiles_of(m), out_argmax, out_accept_len, out_path, out_bonus, s);
+  bool att_tc = false;
+  const SegTable tab = single_table(kv, n_nodes, &att_tc);
+  launch_tree_prep(kv, tab, tokens, parent_idx, s);
+  launch_embed_tokens(kv, tab, n_nodes, tokens, s);
+  run_stack(m, kv, tab, n_nodes, n_nodes, att_tc, kv->ws.ctl, true, out_logits, s);
+  launch_accept(kv, tab, nullptr, tokens, parent_idx, lm_tiles_of(m), out_argmax, out_accept_len, out_path, out_bonus, s);
   kv->pending_n = n_nodes;
   CUDA_TRY(cudaGetLastError());
   return SPECASR_OK;
@@ -591,12 +606,13 @@ extern "C" specasr_status specasr_verify_tree_batch(specasr_model* m, int32_t ba
     set_error("%s: %d nodes in all exceed the %d rows of the first handle's workspace", who, total, wk->max_nodes);
     return SPECASR_ERR_INVALID_ARG;
   }
-  int cap = m->cfg.max_positions;
-  AttnPlan plan;
-  plan.tc = true;
-  plan.splits = 1;
+  SegTable tab;
+  memset(&tab, 0, sizeof(tab));
+  tab.count = batch;
+  tab.splits = 1;
   int budget = m->n_sm / batch;
   if (budget < 1) budget = 1;
+  int n_max = 1;
   for (int b = 0; b < batch; ++b) {
     specasr_kv* u = kv[b];
     const int n_b = node_offsets[b + 1] - node_offsets[b];
@@ -605,36 +621,31 @@ extern "C" specasr_status specasr_verify_tree_batch(specasr_model* m, int32_t ba
       return SPECASR_ERR_UNSUPPORTED;
     }
     refresh_len(u, false);
-    int cap_b = u->max_pages * m->cfg.page_size;
-    if (cap < cap_b) cap_b = cap;
-    if (u->len_exact && u->len_host + n_b > cap_b) {
+    tab.seg[b] = seg_entry(u, node_offsets[b], n_b);
+    if (u->len_exact && u->len_host + n_b > tab.seg[b].capacity) {
       set_error("%s: utterance %d: %d committed + %d tree slots exceed the capacity of %d", who, b, u->len_host, n_b,
-                cap_b);
+                tab.seg[b].capacity);
       return SPECASR_ERR_KV_CAPACITY;
     }
     bool use_tc = false;
-    const int sp = attention_splits(u, n_b, u->len_upper, budget, &use_tc, &plan.chunk[b]);
+    const int sp = attention_splits(u, n_b, u->len_upper, budget, &use_tc, &tab.seg[b].chunk);
     if (!use_tc) {
       set_error("%s: utterance %d: cache of up to %d positions needs more key blocks than the workspace holds", who, b,
                 u->len_upper + n_b);
       return SPECASR_ERR_UNSUPPORTED;
     }
-    if (sp > plan.splits) plan.splits = sp;
+    if (sp > tab.splits) tab.splits = sp;
+    if (n_b > n_max) n_max = n_b;
   }
   cudaStream_t s = (cudaStream_t)stream;
   int32_t* ctl_shared = wk->ws.ctl + kCtlBatch;
   CUDA_TRY(cudaMemsetAsync(ctl_shared, 0, sizeof(int32_t) * 4, s));
-  Rows segs[SPECASR_MAX_BATCH];
-  for (int b = 0; b < batch; ++b) segs[b] = Rows{kv[b], node_offsets[b], node_offsets[b + 1] - node_offsets[b]};
-  for (int b = 0; b < batch; ++b) launch_tree_prep(wk, segs[b], tokens + segs[b].row0, parent_idx + segs[b].row0, s);
-  for (int b = 0; b < batch; ++b) launch_embed_tokens(wk, segs[b], tokens + segs[b].row0, s);
-  run_stack(m, wk, segs, batch, total, ctl_shared, plan, true, nullptr, s);
-  for (int b = 0; b < batch; ++b) {
-    const int o = segs[b].row0;
-    launch_accept(wk, segs[b], ctl_shared, tokens + o, parent_idx + o, lm_tiles_of(m), out_argmax + o,
-                  out_accept_len + b, out_path + o, out_bonus ? out_bonus + b : nullptr, s);
-    kv[b]->pending_n = segs[b].n;
-  }
+  launch_tree_prep(wk, tab, tokens, parent_idx, s);
+  launch_embed_tokens(wk, tab, total, tokens, s);
+  run_stack(m, wk, tab, total, n_max, true, ctl_shared, true, nullptr, s);
+  launch_accept(wk, tab, ctl_shared, tokens, parent_idx, lm_tiles_of(m), out_argmax, out_accept_len, out_path, out_bonus,
+                s);
+  for (int b = 0; b < batch; ++b) kv[b]->pending_n = tab.seg[b].n;
   CUDA_TRY(cudaGetLastError());
   return SPECASR_OK;
 }

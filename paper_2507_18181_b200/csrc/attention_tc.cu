@@ -56,8 +56,7 @@ struct AttnParams {
 
 template <int DH>
 __global__ void __launch_bounds__(64 + SOFTMAX_THREADS, 1) k_tree_attention_tc(const __grid_constant__ CUtensorMap tmQ,
-                                                              const __grid_constant__ CUtensorMap tmK,
-                                                              const __grid_constant__ CUtensorMap tmV, AttnParams p) {
+                                                              const __grid_constant__ SegTable tab, AttnParams p) {
   constexpr int H = DH / 64;                               // 64-wide halves of the head
   constexpr int A_BYTES = 4 * SUB;                         // Q planes (2 H sub-tiles), later two P planes of 128 keys
   constexpr int KV_BYTES = 2 * H * KVSUB;
@@ -65,8 +64,22 @@ __global__ void __launch_bounds__(64 + SOFTMAX_THREADS, 1) k_tree_attention_tc(c
   pdl_launch_dependents();
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int kvh = blockIdx.x, split = blockIdx.z;
+  // grid z = utterance * (key blocks per utterance) + key block; the utterance's own values complete the parameters
+  const int kvh = blockIdx.x, split = blockIdx.z % tab.splits;
+  const SegDev& sg = tab.seg[blockIdx.z / tab.splits];
   const int node0 = blockIdx.y * p.nodes_per_tile;
+  if (node0 >= sg.n) return;                               // this utterance has fewer row tiles than the largest one
+  p.ctl = sg.ctl;
+  p.page_table = sg.page_table;
+  p.n_pages = sg.n_pages;
+  p.n = sg.n;
+  p.chunk = sg.chunk;
+  p.row0 = sg.row0;
+  p.anc += (size_t)sg.row0 * 4;
+  p.attO += (size_t)sg.row0 * p.Hq * DH;
+  p.attML += (size_t)sg.row0 * p.Hq;
+  const CUtensorMap* tmK = sg.tmK;
+  const CUtensorMap* tmV = sg.tmV;
   const int rows_used = p.nodes_per_tile * p.group;
   const int k_begin = split * p.chunk;
 
@@ -85,8 +98,8 @@ __global__ void __launch_bounds__(64 + SOFTMAX_THREADS, 1) k_tree_attention_tc(c
     sc->abort = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tmQ);
-    tma_prefetch_desc(&tmK);
-    tma_prefetch_desc(&tmV);
+    tma_prefetch_desc(tmK);
+    tma_prefetch_desc(tmV);
   }
   if (rows_used < 128) {             // query rows the TMA box does not cover must not hold garbage
     const int chunks = (128 - rows_used) * 8;
@@ -144,14 +157,14 @@ __global__ void __launch_bounds__(64 + SOFTMAX_THREADS, 1) k_tree_attention_tc(c
       c4 = p.layer * p.n_pages + p.page_table[k_begin / p.page_size + lane];
       for (int plane = 0; plane < 2; ++plane)
         for (int h = 0; h < H; ++h)
-          tma_load_5d(KVs + (plane * H + h) * KVSUB + off, &tmK, h * 64, 0, plane, kvh, c4, &sc->bar_qk);
+          tma_load_5d(KVs + (plane * H + h) * KVSUB + off, tmK, h * 64, 0, plane, kvh, c4, &sc->bar_qk);
     }
     // V takes K's place once the S MMAs have read K
     const bool ok = mbar_wait(&sc->bar_s, 0u, abort, status);
     if (ok && lane < pages) {
       for (int plane = 0; plane < 2; ++plane)
         for (int h = 0; h < H; ++h)
-          tma_load_5d(KVs + (plane * H + h) * KVSUB + off, &tmV, h * 64, 0, plane, kvh, c4, &sc->bar_v);
+          tma_load_5d(KVs + (plane * H + h) * KVSUB + off, tmV, h * 64, 0, plane, kvh, c4, &sc->bar_v);
     }
   } else if (warp == 1 && lane == 0) {
     // ---------------- MMA issuer
@@ -341,10 +354,8 @@ __global__ void __launch_bounds__(64 + SOFTMAX_THREADS, 1) k_tree_attention_tc(c
 }
 
 template <int DH>
-void launch_dh(specasr_kv* wk, const Rows& r, int layer, int n_splits, int chunk, cudaStream_t s) {
+void launch_dh(specasr_kv* wk, const SegTable& t, int n_max, int layer, cudaStream_t s) {
   const specasr_model* m = wk->m;
-  specasr_kv* kv = r.kv;
-  const int n = r.n;
   const specasr_model_config& c = m->cfg;
   constexpr int H = DH / 64;
   const size_t smem = 4 * SUB + 2 * H * KVSUB + sizeof(AttnCtl) + 1024;
@@ -354,26 +365,21 @@ void launch_dh(specasr_kv* wk, const Rows& r, int layer, int n_splits, int chunk
     configured = true;
   }
   AttnParams p;
-  p.ctl = kv->ws.ctl;
-  p.page_table = kv->page_table;
-  p.anc = wk->ws.anc + (size_t)r.row0 * 4;
-  p.attO = wk->ws.attO + (size_t)r.row0 * c.n_heads * DH;
-  p.attML = wk->ws.attML + (size_t)r.row0 * c.n_heads;
+  memset(&p, 0, sizeof(p));          // ctl, page table, n, chunk, row0, n_pages come from the utterance's table entry
+  p.anc = wk->ws.anc;
+  p.attO = wk->ws.attO;
+  p.attML = wk->ws.attML;
   p.rows_alloc = (size_t)wk->n_alloc * c.n_heads;
-  p.row0 = r.row0;
-  p.n_pages = kv->n_pages;
   p.page_size = c.page_size;
   p.layer = layer;
   p.Hq = c.n_heads;
   p.Hkv = c.n_kv_heads;
   p.group = c.n_heads / c.n_kv_heads;
   p.nodes_per_tile = 128 / p.group;
-  p.n = n;
-  p.chunk = chunk;
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
-  dim3 grid(c.n_kv_heads, (n + p.nodes_per_tile - 1) / p.nodes_per_tile, n_splits);
+  dim3 grid(c.n_kv_heads, (n_max + p.nodes_per_tile - 1) / p.nodes_per_tile, t.count * t.splits);
   LaunchScope scope(wk, SPECASR_KIND_ATTN, s);
-  launch_pdl(k_tree_attention_tc<DH>, grid, dim3(64 + SOFTMAX_THREADS), smem, s, wk->tm_Q, kv->tm_K, kv->tm_V, p);
+  launch_pdl(k_tree_attention_tc<DH>, grid, dim3(64 + SOFTMAX_THREADS), smem, s, wk->tm_Q, t, p);
 }
 
 }  // namespace
@@ -426,11 +432,20 @@ bool attention_tc_make_maps(specasr_kv* kv) {
   uint64_t dims[5] = {dh, ps, 2, (uint64_t)c.n_kv_heads, (uint64_t)c.n_layers * kv->n_pages};
   uint64_t strides[4] = {dh * 2, ps * dh * 2, 2 * ps * dh * 2, (uint64_t)c.n_kv_heads * 2 * ps * dh * 2};
   uint32_t box[5] = {64, (uint32_t)ps, 1, 1, 1};
-  return make_tensor_map_nd(&kv->tm_K, kv->k_pool, 5, dims, strides, box) &&
-         make_tensor_map_nd(&kv->tm_V, kv->v_pool, 5, dims, strides, box);
+  if (!make_tensor_map_nd(&kv->tm_K, kv->k_pool, 5, dims, strides, box) ||
+      !make_tensor_map_nd(&kv->tm_V, kv->v_pool, 5, dims, strides, box))
+    return false;
+  // the kernel reads the pool descriptors through the utterance table, i.e. from global memory
+  cudaError_t e = cudaMemcpy(kv->ws.tmKV, &kv->tm_K, sizeof(CUtensorMap), cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaMemcpy(kv->ws.tmKV + 1, &kv->tm_V, sizeof(CUtensorMap), cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) {
+    set_error("attention descriptors: %s", cudaGetErrorString(e));
+    return false;
+  }
+  return true;
 }
 
-void launch_tree_attention_tc(specasr_kv* wk, const Rows& r, int layer, int n_splits, int chunk, cudaStream_t s) {
-  if (wk->m->cfg.head_dim == 64) launch_dh<64>(wk, r, layer, n_splits, chunk, s);
-  else launch_dh<128>(wk, r, layer, n_splits, chunk, s);
+void launch_tree_attention_tc(specasr_kv* wk, const SegTable& t, int n_max, int layer, cudaStream_t s) {
+  if (wk->m->cfg.head_dim == 64) launch_dh<64>(wk, t, n_max, layer, s);
+  else launch_dh<128>(wk, t, n_max, layer, s);
 }

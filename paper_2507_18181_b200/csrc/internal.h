@@ -60,6 +60,7 @@ struct Workspace {
   float* attO;              // [kMaxAttnSplits][n_alloc * Hq][dh] unnormalised partial outputs
   float2* attML;            // [kMaxAttnSplits][n_alloc * Hq]     (running max in log2 units, sum)
   unsigned long long* amax; // [lm_tiles][n_alloc] packed (ordered logit, ~token id) per vocab tile
+  CUtensorMap* tmKV;        // [2] device copies of the K and V pool descriptors (tensor-core attention)
   size_t bytes;
 };
 
@@ -161,13 +162,29 @@ inline void launch_pdl_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, 
   cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
-// The rows of one utterance in a (possibly batched) call: its handle (control words, pools, page table),
-// the first workspace row it occupies and its number of rows.  A plain call is one such segment at row 0
-// of its own workspace.
-struct Rows {
-  specasr_kv* kv;
-  int row0;
-  int n;
+// One utterance of a (possibly batched) call as the kernels see it: its control block, cache and the workspace
+// rows it occupies.  A plain call is one such entry at row 0 of its own workspace.  The table travels as a
+// kernel parameter, so the per-utterance kernels (tree prep, embedding, rotary + append, attention, accept) run
+// once per call over all utterances.
+struct SegDev {
+  int32_t* ctl;                 // the utterance's control block
+  const int32_t* page_table;
+  bf16* k_pool;
+  bf16* v_pool;
+  const CUtensorMap* tmK;       // device copies of the pool descriptors (tensor-core attention), else null
+  const CUtensorMap* tmV;
+  int n_pages;
+  int row0;                     // first workspace row
+  int n;                        // rows
+  int chunk;                    // keys per attention CTA
+  int capacity;                 // positions the cache can hold
+  int pad;
+};
+struct SegTable {
+  int count;
+  int splits;                   // grid depth of the attention launch per utterance (largest any of them needs)
+  int pad[2];
+  SegDev seg[SPECASR_MAX_BATCH];
 };
 
 void set_error(const char* fmt, ...);
@@ -175,17 +192,17 @@ Workspace carve_workspace(const specasr_model* m, int n_alloc, void* base);
 int lm_tiles_of(const specasr_model* m);
 
 // ---- kernels_small.cu
-void launch_tree_prep(specasr_kv* wk, const Rows& r, const int32_t* tokens, const int32_t* parent, cudaStream_t s);
+void launch_tree_prep(specasr_kv* wk, const SegTable& t, const int32_t* tokens, const int32_t* parent, cudaStream_t s);
 void launch_chain_prep(specasr_kv* kv, int n, cudaStream_t s);
-void launch_embed_tokens(specasr_kv* wk, const Rows& r, const int32_t* tokens, cudaStream_t s);
+void launch_embed_tokens(specasr_kv* wk, const SegTable& t, int n_total, const int32_t* tokens, cudaStream_t s);
 void launch_copy_embeds(specasr_kv* kv, const float* embeds, int n, cudaStream_t s);
 void launch_rmsnorm_split(specasr_kv* wk, const int32_t* ctl, const float* gain, int n, int n_pad, int n_partials,
                           cudaStream_t s);
-void launch_rope_append(specasr_kv* wk, const Rows& r, int layer, int n_partials, cudaStream_t s);
+void launch_rope_append(specasr_kv* wk, const SegTable& t, int n_total, int layer, int n_partials, cudaStream_t s);
 void launch_attn_merge(specasr_kv* wk, const int32_t* ctl, int n, int n_pad, int n_splits, cudaStream_t s);
-void launch_accept(specasr_kv* wk, const Rows& r, const int32_t* ctl_shared, const int32_t* tokens, const int32_t* parent, int n_tiles,
-                   int32_t* out_argmax, int32_t* out_accept_len, int32_t* out_path, int32_t* out_bonus,
-                   cudaStream_t s);
+void launch_accept(specasr_kv* wk, const SegTable& t, const int32_t* ctl_shared, const int32_t* tokens,
+                   const int32_t* parent, int n_tiles, int32_t* out_argmax, int32_t* out_accept_len, int32_t* out_path,
+                   int32_t* out_bonus, cudaStream_t s);
 void launch_advance_len(specasr_kv* kv, int n, cudaStream_t s);
 void launch_set_len(specasr_kv* kv, int len, cudaStream_t s);
 void launch_commit(specasr_kv* kv, const int32_t* path, const int32_t* accept_len, cudaStream_t s);
@@ -196,7 +213,7 @@ bool attention_tc_supported(const specasr_model* m);
 bool attention_tc_plan(const specasr_model* m, int n, int total_len, int sm_budget, int max_splits, int* n_splits,
                        int* chunk);
 bool attention_tc_make_maps(specasr_kv* kv);
-void launch_tree_attention_tc(specasr_kv* wk, const Rows& r, int layer, int n_splits, int chunk, cudaStream_t s);
+void launch_tree_attention_tc(specasr_kv* wk, const SegTable& t, int n_max, int layer, cudaStream_t s);
 
 // ---- gemm_fma.cu / gemm_tcgen05.cu
 enum GemmEpilogue {

@@ -9,12 +9,20 @@
 // Tree preparation: validates the parent array, derives depth, position and the ancestor-or-self
 // bitmask of every node (the rows of the 2-D tree attention mask), and sets the status word that
 // every later kernel of the call checks.
-__global__ void k_tree_prep(int32_t* __restrict__ ctl, const int32_t* __restrict__ tokens,
-                            const int32_t* __restrict__ parent, int n, int vocab, int capacity,
-                            int32_t* __restrict__ depth, int32_t* __restrict__ pos,
-                            unsigned long long* __restrict__ anc) {
+// One block per utterance of the call; tokens / parent / depth / pos / anc are indexed by workspace row.
+__global__ void k_tree_prep(const __grid_constant__ SegTable tab, const int32_t* __restrict__ tokens,
+                            const int32_t* __restrict__ parent, int vocab, int32_t* __restrict__ depth,
+                            int32_t* __restrict__ pos, unsigned long long* __restrict__ anc) {
   __shared__ int s_bad;
   const int i = threadIdx.x;
+  const SegDev& sg = tab.seg[blockIdx.x];
+  int32_t* ctl = sg.ctl;
+  const int n = sg.n, capacity = sg.capacity;
+  if (tokens) tokens += sg.row0;
+  parent += sg.row0;
+  depth += sg.row0;
+  pos += sg.row0;
+  anc += (size_t)sg.row0 * 4;
   grid_dep_launch();
   grid_dep_wait();
   if (i == 0) s_bad = 0;
@@ -82,13 +90,10 @@ __global__ void k_chain_prep(int32_t* __restrict__ ctl, int n, int capacity, int
   }
 }
 
-void launch_tree_prep(specasr_kv* wk, const Rows& r, const int32_t* tokens, const int32_t* parent, cudaStream_t s) {
-  const specasr_model* m = wk->m;
-  int cap = r.kv->max_pages * m->cfg.page_size;
-  if (m->cfg.max_positions < cap) cap = m->cfg.max_positions;
+void launch_tree_prep(specasr_kv* wk, const SegTable& t, const int32_t* tokens, const int32_t* parent, cudaStream_t s) {
   LaunchScope scope(wk, SPECASR_KIND_PREP, s);
-  launch_pdl(k_tree_prep, dim3(1), dim3(256), 0, s, r.kv->ws.ctl, tokens, parent, r.n, m->cfg.vocab, cap,
-             wk->ws.depth + r.row0, wk->ws.pos + r.row0, wk->ws.anc + (size_t)r.row0 * 4);
+  launch_pdl(k_tree_prep, dim3(t.count), dim3(256), 0, s, t, tokens, parent, wk->m->cfg.vocab, wk->ws.depth,
+             wk->ws.pos, wk->ws.anc);
 }
 
 void launch_chain_prep(specasr_kv* kv, int n, cudaStream_t s) {
@@ -101,12 +106,19 @@ void launch_chain_prep(specasr_kv* kv, int n, cudaStream_t s) {
 
 // ------------------------------------------------------------------------------------------------
 // Layer-0 inputs: embedding rows (bf16 -> fp32 residual stream), or caller-provided vectors.
-__global__ void k_embed_tokens(const int32_t* __restrict__ ctl, const int32_t* __restrict__ tokens,
+// The utterance that owns workspace row `row` (segments are laid out back to back in table order).
+__device__ __forceinline__ int segment_of_row(const SegTable& tab, int row) {
+  int b = 0;
+  while (b + 1 < tab.count && row >= tab.seg[b].row0 + tab.seg[b].n) ++b;
+  return b;
+}
+
+__global__ void k_embed_tokens(const __grid_constant__ SegTable tab, const int32_t* __restrict__ tokens,
                                const bf16* __restrict__ E, int d, float* __restrict__ X) {
   grid_dep_launch();
   grid_dep_wait();
-  if (ctl[CTL_STATUS] != 0) return;
   const int i = blockIdx.x;
+  if (tab.seg[segment_of_row(tab, i)].ctl[CTL_STATUS] != 0) return;
   const bf16* row = E + (size_t)tokens[i] * d;
   float* x = X + (size_t)i * d;
   for (int k = threadIdx.x * 8; k < d; k += blockDim.x * 8) {
@@ -132,11 +144,9 @@ __global__ void k_copy_embeds(const int32_t* __restrict__ ctl, const float* __re
     *reinterpret_cast<float4*>(X + (size_t)i * d + k) = *reinterpret_cast<const float4*>(src + (size_t)i * d + k);
 }
 
-void launch_embed_tokens(specasr_kv* wk, const Rows& r, const int32_t* tokens, cudaStream_t s) {
-  const int d = wk->m->cfg.d_model;
+void launch_embed_tokens(specasr_kv* wk, const SegTable& t, int n_total, const int32_t* tokens, cudaStream_t s) {
   LaunchScope scope(wk, SPECASR_KIND_PREP, s);
-  launch_pdl(k_embed_tokens, dim3(r.n), dim3(128), 0, s, r.kv->ws.ctl, tokens, wk->m->embed, d,
-             wk->ws.X + (size_t)r.row0 * d);
+  launch_pdl(k_embed_tokens, dim3(n_total), dim3(128), 0, s, t, tokens, wk->m->embed, wk->m->cfg.d_model, wk->ws.X);
 }
 
 void launch_copy_embeds(specasr_kv* kv, const float* embeds, int n, cudaStream_t s) {
@@ -260,15 +270,15 @@ void launch_rmsnorm_split(specasr_kv* kv, const int32_t* ctl, const float* gain,
 // rotates Q and K heads by the angle of
 // the node's position (rotate-half pairing, table built in fp64 on the host), writes Q as hi/lo planes
 // and K,V as hi/lo planes into cache slot L + node.
-__global__ void k_rope_append(const int32_t* __restrict__ ctl, const float* __restrict__ P, int n_partials,
+__global__ void k_rope_append(const __grid_constant__ SegTable tab, const float* __restrict__ P, int n_partials,
                               size_t partial_stride, int qkv_dim, int Hq, int Hkv, int dh, const int32_t* __restrict__ pos, const float2* __restrict__ rope,
-                              int layer, bf16* __restrict__ Q, size_t q_plane_stride, bf16* __restrict__ k_pool,
-                              bf16* __restrict__ v_pool, const int32_t* __restrict__ page_table, int n_pages,
-                              int page_size) {
+                              int layer, bf16* __restrict__ Q, size_t q_plane_stride, int page_size) {
   grid_dep_launch();
   grid_dep_wait();
+  const int i = blockIdx.x;                    // workspace row
+  const SegDev& sg = tab.seg[segment_of_row(tab, i)];
+  const int32_t* ctl = sg.ctl;
   if (ctl[CTL_STATUS] != 0) return;
-  const int i = blockIdx.x;
   const int half = dh >> 1;
   const int head = blockIdx.y * (blockDim.x / half) + threadIdx.x / half;     // several heads per block
   const int k = threadIdx.x % half;
@@ -306,11 +316,11 @@ __global__ void k_rope_append(const int32_t* __restrict__ ctl, const float* __re
     q[q_plane_stride + k + half] = l2;
   } else {
     const int kvh = is_v ? head - Hq - Hkv : head - Hq;
-    const int slot = ctl[CTL_LEN] + i;
-    const int page = page_table[slot / page_size];
+    const int slot = ctl[CTL_LEN] + (i - sg.row0);
+    const int page = sg.page_table[slot / page_size];
     const int off = slot % page_size;
-    bf16* pool = is_v ? v_pool : k_pool;
-    bf16* dst = pool + kv_plane_offset(layer, n_pages, Hkv, page_size, dh, page, kvh, 0) + (size_t)off * dh;
+    bf16* pool = is_v ? sg.v_pool : sg.k_pool;
+    bf16* dst = pool + kv_plane_offset(layer, sg.n_pages, Hkv, page_size, dh, page, kvh, 0) + (size_t)off * dh;
     const size_t plane = (size_t)page_size * dh;
     dst[k] = h1;
     dst[k + half] = h2;
@@ -319,16 +329,15 @@ __global__ void k_rope_append(const int32_t* __restrict__ ctl, const float* __re
   }
 }
 
-void launch_rope_append(specasr_kv* wk, const Rows& r, int layer, int n_partials, cudaStream_t s) {
+void launch_rope_append(specasr_kv* wk, const SegTable& t, int n_total, int layer, int n_partials, cudaStream_t s) {
   const specasr_model* m = wk->m;
   const specasr_model_config& c = m->cfg;
   const int heads_per_block = 256 / (c.head_dim / 2);
-  dim3 grid(r.n, (c.n_heads + 2 * c.n_kv_heads + heads_per_block - 1) / heads_per_block);
+  dim3 grid(n_total, (c.n_heads + 2 * c.n_kv_heads + heads_per_block - 1) / heads_per_block);
   LaunchScope scope(wk, SPECASR_KIND_ROPE, s);
-  launch_pdl(k_rope_append, grid, dim3(256), 0, s, r.kv->ws.ctl, wk->ws.P + (size_t)r.row0 * m->qkv_dim, n_partials,
-             (size_t)wk->n_alloc * m->qkv_dim, m->qkv_dim, c.n_heads, c.n_kv_heads, c.head_dim, wk->ws.pos + r.row0,
-             m->rope_table, layer, wk->ws.Q + (size_t)r.row0 * m->q_dim, (size_t)wk->n_alloc * m->q_dim, r.kv->k_pool,
-             r.kv->v_pool, r.kv->page_table, r.kv->n_pages, c.page_size);
+  launch_pdl(k_rope_append, grid, dim3(256), 0, s, t, wk->ws.P, n_partials, (size_t)wk->n_alloc * m->qkv_dim, m->qkv_dim,
+             c.n_heads, c.n_kv_heads, c.head_dim, wk->ws.pos, m->rope_table, layer, wk->ws.Q,
+             (size_t)wk->n_alloc * m->q_dim, c.page_size);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -405,16 +414,28 @@ void launch_attn_merge(specasr_kv* kv, const int32_t* ctl, int n, int n_pad, int
 // ------------------------------------------------------------------------------------------------
 // Accept: reduce the per-vocab-tile argmax candidates, then follow draft tokens while they equal the
 // target's greedy token at their parent; the deepest such node (lowest index among equals) wins.
-__global__ void __launch_bounds__(256) k_accept(int32_t* __restrict__ ctl, const int32_t* __restrict__ ctl_shared,
+// One block per utterance; arrays indexed by workspace row, out_accept_len / out_bonus by utterance.
+__global__ void __launch_bounds__(256) k_accept(const __grid_constant__ SegTable tab, const int32_t* __restrict__ ctl_shared,
                                                 const unsigned long long* __restrict__ amax, int n_tiles,
                                                 int n_alloc, const int32_t* __restrict__ tokens,
                                                 const int32_t* __restrict__ parent,
-                                                const int32_t* __restrict__ depth, int n,
+                                                const int32_t* __restrict__ depth,
                                                 int32_t* __restrict__ out_argmax, int32_t* __restrict__ out_accept_len,
                                                 int32_t* __restrict__ out_path, int32_t* __restrict__ out_bonus) {
   __shared__ int s_arg[SPECASR_MAX_NODES];
   __shared__ unsigned int s_best;
   const int i = threadIdx.x;
+  const SegDev& sg = tab.seg[blockIdx.x];
+  int32_t* ctl = sg.ctl;
+  const int n = sg.n;
+  amax += sg.row0;
+  tokens += sg.row0;
+  parent += sg.row0;
+  depth += sg.row0;
+  out_argmax += sg.row0;
+  out_path += sg.row0;
+  out_accept_len += blockIdx.x;
+  if (out_bonus) out_bonus += blockIdx.x;
   grid_dep_launch();
   grid_dep_wait();
   // a failure of the kernels shared by a whole batch (a bounded wait that ran out) fails every utterance
@@ -485,12 +506,12 @@ __global__ void __launch_bounds__(256) k_accept(int32_t* __restrict__ ctl, const
   }
 }
 
-void launch_accept(specasr_kv* wk, const Rows& r, const int32_t* ctl_shared, const int32_t* tokens, const int32_t* parent, int n_tiles,
-                   int32_t* out_argmax, int32_t* out_accept_len, int32_t* out_path, int32_t* out_bonus,
-                   cudaStream_t s) {
+void launch_accept(specasr_kv* wk, const SegTable& t, const int32_t* ctl_shared, const int32_t* tokens,
+                   const int32_t* parent, int n_tiles, int32_t* out_argmax, int32_t* out_accept_len, int32_t* out_path,
+                   int32_t* out_bonus, cudaStream_t s) {
   LaunchScope scope(wk, SPECASR_KIND_ACCEPT, s);
-  launch_pdl(k_accept, dim3(1), dim3(256), 0, s, r.kv->ws.ctl, ctl_shared, wk->ws.amax + r.row0, n_tiles, wk->n_alloc, tokens,
-             parent, wk->ws.depth + r.row0, r.n, out_argmax, out_accept_len, out_path, out_bonus);
+  launch_pdl(k_accept, dim3(t.count), dim3(256), 0, s, t, ctl_shared, wk->ws.amax, n_tiles, wk->n_alloc, tokens, parent,
+             wk->ws.depth, out_argmax, out_accept_len, out_path, out_bonus);
 }
 
 // ------------------------------------------------------------------------------------------------

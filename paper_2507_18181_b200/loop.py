@@ -29,8 +29,9 @@ class SpeculativeBatchLoop:
         if self.draft_kvs is not None:
             self.draft_len = [kv.length() for kv in self.draft_kvs]
             self._minus_one = torch.full((self.B,), -1, dtype=torch.int32, device=self.device)
-        self.rounds = 0
-        self.draft_steps = 0
+        self.rounds = 0               # batched verification calls
+        self.utterance_rounds = 0     # trees verified (rounds summed over utterances)
+        self.draft_steps = 0          # batched draft-model calls
 
     # ---- draft phase -----------------------------------------------------------------------------------------
     def _verifier(self, kvs, members):
@@ -96,6 +97,7 @@ class SpeculativeBatchLoop:
             self.target_len[b] += a + 1
             out[b] = (a, path[offsets[i]:offsets[i] + a + 1].copy(), int(bonus[i]))
         self.rounds += 1
+        self.utterance_rounds += len(members)
         return out
 
     # ---- the loop --------------------------------------------------------------------------------------------
