@@ -32,6 +32,8 @@ WORKLOADS = {
     "config1": dict(model="tiny", n_audio=64, n_text=8, n_nodes=15, levels=None, chain=False),
     # config3 cut to two layers: same kernels and launch shapes, small enough for a profiler capture
     "config3_2layers": dict(model="7b", n_layers=2, n_audio=1500, n_text=201, n_nodes=64, levels=12, chain=False),
+    # a 256-node point of the config 4 sweep cut to two layers, for a profiler capture of the large-tree regime
+    "config4_n256_2layers": dict(model="7b", n_layers=2, n_audio=1500, n_text=201, n_nodes=256, levels=None, chain=False),
 }
 METRIC = "tree_tokens_per_s"
 UNIT = "tree tokens/s"
@@ -60,6 +62,30 @@ def algorithmic_flops(cfg, L, n):
     params = cfg.n_layers * (cfg.d_model * (cfg.q_dim + 2 * cfg.kv_dim) + cfg.q_dim * cfg.d_model
                              + 3 * cfg.d_model * cfg.ffn) + cfg.d_model * cfg.vocab
     return 2 * n * params + 4 * n * cfg.q_dim * (L + n) * cfg.n_layers
+
+
+# DRAM traffic (read + write, MB per launch) of the projection kernel from the ncu capture summarised in
+# profiles/k_proj_config3_2layers.md: 7B shape, 64 tokens.  Valid only for the kernel source it was taken on.
+PROJ_TRAFFIC_MB = {"gemm_qkv": 51.46, "gemm_o": 34.65, "gemm_gu": 248.17, "gemm_down": 124.97, "gemm_lm": 276.25}
+PROJ_TRAFFIC_SOURCE_SHA256 = {
+    "gemm_tcgen05.cu": "327d2dd19f59270026f244e963c296d2727f02cc697402de3905cf5e1766e658",
+    "sm100_ptx.cuh": "3a0c294121fb64b742ab3700569cef82a1922484c98acd5238167235b990940f",
+}
+
+
+def proj_traffic_per_launch(wl, cfg):
+    """Average DRAM bytes per projection launch from the committed capture, or None when the capture does not
+    describe this run (another shape, or the kernel source changed since)."""
+    import hashlib
+    if wl.get("model") != "7b" or wl.get("n_nodes") != 64:
+        return None
+    for name, want in PROJ_TRAFFIC_SOURCE_SHA256.items():
+        path = os.path.join(ROOT, "paper_2507_18181_b200", "csrc", name)
+        if not os.path.exists(path) or hashlib.sha256(open(path, "rb").read()).hexdigest() != want:
+            return None
+    t = PROJ_TRAFFIC_MB
+    per_layer = t["gemm_qkv"] + t["gemm_o"] + t["gemm_gu"] + t["gemm_down"]
+    return (cfg.n_layers * per_layer + t["gemm_lm"]) * 1e6 / (4 * cfg.n_layers + 1)
 
 
 def measured_peaks():
@@ -365,7 +391,7 @@ def run_ours(args, wl):
                           "frac_of_nominal_8TBs": (ab["total"] / 8e12 * 1e3) / ms_per_step},
         "roofline": {"kernel": "k_gemm_tc (all projections)", "bound": "hbm", "achieved": achieved,
                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                     "peak_source": peaks["source"], "traffic": None,
+                     "peak_source": peaks["source"], "traffic": proj_traffic_per_launch(wl, cfg),
                      "algorithmic_bytes_per_launch": gemm_bytes_step / gemm_launches,
                      "avg_launch_ms": gemm_ms_step / gemm_launches},
         "kernels": kernels,

@@ -10,6 +10,9 @@
 // adds the two halves of the accumulator.
 // A pipeline stage holds one k-block of `tm` adjacent weight tiles and the matching activation block,
 // so with tm = 2 the activation bytes (which every CTA re-reads from L2) are half the weight bytes.
+// From 128 tokens on the two planes are "folded": one MMA per plane (N = tokens of the box), both accumulating
+// into the same TMEM columns, so a tile costs n instead of 2 n columns and two accumulator sets of 256 tokens
+// fit the 512 columns.
 //
 // Scheduling.  The kernel is persistent, at most one CTA per SM, over (tile group, k-block) units.
 //  - Linear outputs (QKV, O, down): the k-blocks of every tile group are cut into `splits` equal
@@ -60,6 +63,7 @@ struct alignas(16) SharedCtl {
 
 struct TcParams {
   int M, K, n, n_pad, n_alloc, box_rows, stages, ksub, tm, n_buf, tmem_cols, KB, tiles, groups, splits, epoch;
+  int fold;                 // launch the FOLD instantiation: hi and lo products share the TMEM columns
   int32_t* ctl;
   float* fixP;              // [grid][tm][n_pad][128] parked partial sums (hi + lo halves added) of split tile groups
   int32_t* fixFlag;         // [grid] launch number of the partial sums each CTA parked last
@@ -80,7 +84,7 @@ __device__ __forceinline__ void st_release(int32_t* p, int v) {
 constexpr int EPI_THREADS = 256;      // warps 2..9
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
-template <int EPI>
+template <int EPI, bool FOLD>
 __global__ void __launch_bounds__(64 + EPI_THREADS, 1) k_proj(const __grid_constant__ CUtensorMap tmW,
                                                  const __grid_constant__ CUtensorMap tmAct, TcParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -89,7 +93,7 @@ __global__ void __launch_bounds__(64 + EPI_THREADS, 1) k_proj(const __grid_const
   const int act_sub = p.n_pad * 2 * SUB_K * 2;         // both planes of one 64-wide k sub-block
   const int stage_bytes = w_bytes + p.ksub * act_sub;
   SharedCtl* sc = (SharedCtl*)(tiles + (size_t)p.stages * stage_bytes);
-  bf16* epi_stage = (bf16*)(sc + 1);                    // EPI_SWIGLU: [2 planes][n_pad][64] output tile
+  bf16* epi_stage = (bf16*)(sc + 1);                    // EPI_SWIGLU: [2 planes][<= 64 tokens][64] output tile
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = gridDim.x, cta = blockIdx.x;
@@ -105,7 +109,8 @@ __global__ void __launch_bounds__(64 + EPI_THREADS, 1) k_proj(const __grid_const
     u1 = (cta + 1) * U / G;
   }
   const int n_blocks = p.n_pad / p.box_rows;
-  const int acc_cols = p.tm * 2 * p.n_pad;              // TMEM columns of one accumulator set (hi | lo halves)
+  const int tile_cols = FOLD ? p.n_pad : 2 * p.n_pad;   // TMEM columns of one tile: hi | lo halves unless folded
+  const int acc_cols = p.tm * tile_cols;                // one accumulator set
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) {
@@ -174,7 +179,8 @@ __global__ void __launch_bounds__(64 + EPI_THREADS, 1) k_proj(const __grid_const
     // ---------------- MMA issuer
     pdl_wait();
     if (*(volatile int32_t*)status == 0) {
-      const uint32_t idesc = make_idesc_bf16(2 * p.box_rows);      // both planes of a token block in one MMA
+      // both planes of a token block in one MMA of N = 2 * box rows, or (folded) one MMA per plane into the same columns
+      const uint32_t idesc = make_idesc_bf16(FOLD ? p.box_rows : 2 * p.box_rows);
       int i = 0, seg = 0;
       bool ok = true;
       for (long long u = u0; u < u1 && ok; ++seg) {
@@ -199,12 +205,16 @@ __global__ void __launch_bounds__(64 + EPI_THREADS, 1) k_proj(const __grid_const
               const uint32_t a_addr = w_addr + (t * p.ksub + q) * W_SUB_BYTES;
               for (int jb = 0; jb < n_blocks; ++jb) {
                 const uint32_t b_addr = act_addr + q * act_sub + (uint32_t)(jb * 2 * p.box_rows * SUB_K * 2);
-                const uint32_t d_addr = d_base + (uint32_t)(t * 2 * p.n_pad + jb * 2 * p.box_rows);
+                const uint32_t d_addr = d_base + (uint32_t)(t * tile_cols + jb * (FOLD ? 1 : 2) * p.box_rows);
+                const uint32_t lo_addr = b_addr + (uint32_t)(p.box_rows * SUB_K * 2);   // lo rows follow the hi rows
 #pragma unroll
                 for (int k = 0; k < SUB_K / UMMA_K; ++k) {
                   const uint32_t acc = (kb > kb0 || q > 0 || k > 0) ? 1u : 0u;
                   umma_bf16(d_addr, make_smem_desc(a_addr + k * UMMA_K * 2), make_smem_desc(b_addr + k * UMMA_K * 2),
                             idesc, acc);
+                  if (FOLD)
+                    umma_bf16(d_addr, make_smem_desc(a_addr + k * UMMA_K * 2), make_smem_desc(lo_addr + k * UMMA_K * 2),
+                              idesc, 1u);
                 }
               }
             }
@@ -226,6 +236,10 @@ __global__ void __launch_bounds__(64 + EPI_THREADS, 1) k_proj(const __grid_const
     int seg = 0;
     // value of token block [c0, c0 + 16) of tile t2: hi half + lo half of the accumulator
     auto load16 = [&](uint32_t lane_addr, int t2, int c0, float* v) {
+      if (FOLD) {
+        tmem_ld16(lane_addr + (uint32_t)(t2 * p.n_pad + c0), v);
+        return;
+      }
       const uint32_t col = (uint32_t)(t2 * 2 * p.n_pad + (c0 / p.box_rows) * 2 * p.box_rows + c0 % p.box_rows);
       float lo[16];
       tmem_ld16x2(lane_addr + col, lane_addr + col + (uint32_t)p.box_rows, v, lo);
@@ -331,85 +345,92 @@ __global__ void __launch_bounds__(64 + EPI_THREADS, 1) k_proj(const __grid_const
           for (int t = etid; t < SPECASR_MAX_NODES; t += EPI_THREADS) sc->key[t] = 0ull;
           epi_bar();
         }
-        if (ok) {
-          // parked sums of this tile (requested a tile ahead); the next tile's are requested now
-          float cur0[16], cur1[16];
-          if (last > cta && quick) {
-#pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              cur0[j] = pk0[j];
-              cur1[j] = pk1[j];
-            }
-            if (t2 + 1 < p.tm) {
-              load_parked(t2 + 1, c_first, pk0);
-              load_parked(t2 + 1, c_first + 32, pk1);
-            }
-          }
-          for (int c0 = c_first; c0 < p.n_pad; c0 += 32) {
-            float v[16];
-            load16(lane_addr, t2, c0, v);
-            if (last > cta) {
-              if (quick) {
-                const bool first = c0 == c_first;
-#pragma unroll
-                for (int j = 0; j < 16; ++j) v[j] += first ? cur0[j] : cur1[j];
-              } else {
-                float f[16];
-                load_parked(t2, c0, f);
-#pragma unroll
-                for (int j = 0; j < 16; ++j) v[j] += f[j];
-              }
-            }
-            if (EPI == EPI_SWIGLU) {
-              // rows 2f / 2f + 1 of the tile are gate / up of feature f: the even lane keeps the hi plane of
-              // the product, the odd lane the lo plane, staged in shared memory for 16-byte global stores
-              float a[16];
-#pragma unroll
-              for (int j = 0; j < 16; ++j) {
-                const float other = __shfl_xor_sync(0xFFFFFFFFu, v[j], 1);
-                const float g = (lane & 1) ? other : v[j];
-                const float up = (lane & 1) ? v[j] : other;
-                a[j] = __fdividef(g, 1.f + __expf(-g)) * up;
-              }
-              bf16* st = epi_stage + (size_t)(lane & 1) * p.n_pad * 64 + (size_t)c0 * 64 + (row >> 1);
-#pragma unroll
-              for (int j = 0; j < 16; ++j) {
-                bf16 hi, lo;
-                split_bf16(a[j], hi, lo);
-                st[j * 64] = (lane & 1) ? lo : hi;
-              }
-            } else if (EPI == EPI_ARGMAX) {
-#pragma unroll
-              for (int j = 0; j < 16; ++j) {
-                const int t = c0 + j;
-                if (p.logits && t < p.n && row_ok) p.logits[(size_t)t * p.M + m] = v[j];
-                // warp arg-max: largest ordered key, then the lowest row among its holders
-                uint32_t key = __float_as_uint(v[j]);
-                key = (key & 0x80000000u) ? ~key : (key | 0x80000000u);
-                if (!row_ok) key = 0u;
-                const uint32_t best = __reduce_max_sync(0xFFFFFFFFu, key);
-                const uint32_t who = __reduce_min_sync(0xFFFFFFFFu, key == best ? (uint32_t)m : 0xFFFFFFFFu);
-                if (lane == 0 && t < p.n && best != 0u)
-                  atomicMax(&sc->key[t], ((unsigned long long)best << 32) | (unsigned long long)(0xFFFFFFFFu - who));
-              }
-            }
-          }
-        }
-        if (EPI == EPI_SWIGLU) {
-          epi_bar();
+        // the SwiGLU output of 128 tokens or more is staged in shared memory 64 tokens at a time
+        constexpr bool CHUNKED = FOLD && EPI == EPI_SWIGLU;      // folded launches have at least 128 tokens
+        const int tok_chunk = CHUNKED ? 64 : p.n_pad;
+        for (int tc0 = 0; tc0 < (CHUNKED ? p.n_pad : 1); tc0 += tok_chunk) {
           if (ok) {
-            const int F = p.M >> 1;
-            const int f0 = tile * 64;
-            const int chunks = 2 * p.n * 8;                 // 16-byte pieces of the [2][n][64] tile
-            for (int idx = etid; idx < chunks; idx += EPI_THREADS) {
-              const int plane = idx / (p.n * 8), rem = idx % (p.n * 8);
-              const int t = rem >> 3, ch = rem & 7;
-              if (f0 + ch * 8 < F)
-                *reinterpret_cast<uint4*>(p.A + (size_t)plane * p.n_alloc * F + (size_t)t * F + f0 + ch * 8) =
-                    *reinterpret_cast<const uint4*>(epi_stage + (size_t)plane * p.n_pad * 64 + t * 64 + ch * 8);
+            // parked sums of this tile (requested a tile ahead); the next tile's are requested now
+            float cur0[16], cur1[16];
+            if (last > cta && quick) {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                cur0[j] = pk0[j];
+                cur1[j] = pk1[j];
+              }
+              if (t2 + 1 < p.tm) {
+                load_parked(t2 + 1, c_first, pk0);
+                load_parked(t2 + 1, c_first + 32, pk1);
+              }
+            }
+            for (int c0 = tc0 + c_first; c0 < tc0 + tok_chunk; c0 += 32) {
+              float v[16];
+              load16(lane_addr, t2, c0, v);
+              if (last > cta) {
+                if (quick) {
+                  const bool first = c0 == c_first;
+#pragma unroll
+                  for (int j = 0; j < 16; ++j) v[j] += first ? cur0[j] : cur1[j];
+                } else {
+                  float f[16];
+                  load_parked(t2, c0, f);
+#pragma unroll
+                  for (int j = 0; j < 16; ++j) v[j] += f[j];
+                }
+              }
+              if (EPI == EPI_SWIGLU) {
+                // rows 2f / 2f + 1 of the tile are gate / up of feature f: the even lane keeps the hi plane of
+                // the product, the odd lane the lo plane, staged in shared memory for 16-byte global stores
+                float a[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                  const float other = __shfl_xor_sync(0xFFFFFFFFu, v[j], 1);
+                  const float g = (lane & 1) ? other : v[j];
+                  const float up = (lane & 1) ? v[j] : other;
+                  a[j] = __fdividef(g, 1.f + __expf(-g)) * up;
+                }
+                bf16* st = epi_stage + (size_t)(lane & 1) * tok_chunk * 64 + (size_t)(c0 - tc0) * 64 + (row >> 1);
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                  bf16 hi, lo;
+                  split_bf16(a[j], hi, lo);
+                  st[j * 64] = (lane & 1) ? lo : hi;
+                }
+              } else if (EPI == EPI_ARGMAX) {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                  const int t = c0 + j;
+                  if (p.logits && t < p.n && row_ok) p.logits[(size_t)t * p.M + m] = v[j];
+                  // warp arg-max: largest ordered key, then the lowest row among its holders
+                  uint32_t key = __float_as_uint(v[j]);
+                  key = (key & 0x80000000u) ? ~key : (key | 0x80000000u);
+                  if (!row_ok) key = 0u;
+                  const uint32_t best = __reduce_max_sync(0xFFFFFFFFu, key);
+                  const uint32_t who = __reduce_min_sync(0xFFFFFFFFu, key == best ? (uint32_t)m : 0xFFFFFFFFu);
+                  if (lane == 0 && t < p.n && best != 0u)
+                    atomicMax(&sc->key[t], ((unsigned long long)best << 32) | (unsigned long long)(0xFFFFFFFFu - who));
+                }
+              }
             }
           }
-          epi_bar();
+          if (EPI == EPI_SWIGLU) {
+            epi_bar();
+            if (ok) {
+              const int F = p.M >> 1;
+              const int f0 = tile * 64;
+              int nt = p.n - tc0;                             // tokens of this chunk that exist
+              nt = nt < 0 ? 0 : (nt > tok_chunk ? tok_chunk : nt);
+              const int chunks = 2 * nt * 8;                  // 16-byte pieces of the [2][nt][64] tile
+              for (int idx = etid; idx < chunks; idx += EPI_THREADS) {
+                const int plane = idx / (nt * 8), rem = idx % (nt * 8);
+                const int t = rem >> 3, ch = rem & 7;
+                if (f0 + ch * 8 < F)
+                  *reinterpret_cast<uint4*>(p.A + (size_t)plane * p.n_alloc * F + (size_t)(tc0 + t) * F + f0 + ch * 8) =
+                      *reinterpret_cast<const uint4*>(epi_stage + (size_t)plane * tok_chunk * 64 + t * 64 + ch * 8);
+              }
+            }
+            epi_bar();
+          }
         }
         if (EPI == EPI_ARGMAX) {
           epi_bar();
@@ -461,15 +482,15 @@ int pick_box_rows(int n_pad) {
   return b;
 }
 
-template <int EPI>
+template <int EPI, bool FOLD>
 void launch_epi(const CUtensorMap& tmW, const CUtensorMap& tmAct, const TcParams& p, int grid, size_t smem,
                 cudaStream_t s) {
   static bool configured = false;
   if (!configured) {
-    cudaFuncSetAttribute(k_proj<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);
+    cudaFuncSetAttribute(k_proj<EPI, FOLD>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);
     configured = true;
   }
-  launch_pdl(k_proj<EPI>, dim3(grid), dim3(64 + EPI_THREADS), smem, s, tmW, tmAct, p);
+  launch_pdl(k_proj<EPI, FOLD>, dim3(grid), dim3(64 + EPI_THREADS), smem, s, tmW, tmAct, p);
 }
 
 }  // namespace
@@ -549,6 +570,11 @@ static void tc_shape(int n_pad, int* tm, int* ksub) {
   // One weight tile per stage: with 64 tokens a stage is 64 KB and three stages fit, which measured faster
   // than two stages of a tile pair (tm = 2, activation block shared by both tiles) although the pair halves
   // the activation traffic; the kernel keeps tm as a parameter.
+  // From 128 tokens on the hi / lo products are folded into one accumulator, which keeps two accumulator sets
+  // within the 512 TMEM columns up to 256 tokens (the epilogue of one tile overlaps the next tile's main loop).
+  // A tile pair per stage (tm = 2) was measured there as well: it halves the activation bytes per weight byte
+  // but leaves only two 96 KB stages at 256 tokens, and the step is bound by the latency of a stage, not by
+  // bandwidth (256 tokens, gate/up: 175 us with pairs, 144 us without).
   *tm = 1;
   *ksub = n_pad <= 64 ? 2 : 1;                    // 256 contiguous bytes per weight row keep DRAM pages busy
 }
@@ -579,11 +605,12 @@ void launch_gemm_tc(specasr_kv* kv, const GemmArgs& a, int kind, cudaStream_t s)
   p.box_rows = pick_box_rows(a.n_pad);
   tc_shape(a.n_pad, &p.tm, &p.ksub);
   const int stage_bytes = p.ksub * (p.tm * W_SUB_BYTES + a.n_pad * 2 * SUB_K * 2);
-  const int epi_bytes = a.epilogue == EPI_SWIGLU ? 2 * a.n_pad * 64 * 2 : 0;     // staged output tile
+  p.fold = a.n_pad >= 128 ? 1 : 0;
+  const int epi_bytes = a.epilogue == EPI_SWIGLU ? 2 * (a.n_pad < 64 ? a.n_pad : 64) * 64 * 2 : 0;   // staged output tile
   int stages = (SMEM_LIMIT - (int)sizeof(SharedCtl) - epi_bytes - 1024) / stage_bytes;
   if (stages > MAX_STAGES) stages = MAX_STAGES;
   p.stages = stages;
-  const int acc_cols = p.tm * 2 * a.n_pad;
+  const int acc_cols = p.tm * (p.fold ? 1 : 2) * a.n_pad;
   p.n_buf = 2 * acc_cols <= 512 ? 2 : 1;
   int cols = 32;
   while (cols < p.n_buf * acc_cols) cols <<= 1;
@@ -604,9 +631,17 @@ void launch_gemm_tc(specasr_kv* kv, const GemmArgs& a, int kind, cudaStream_t s)
   for (int b = 16; b < p.box_rows; b <<= 1) ++idx;
   const CUtensorMap& act = a.tmAct[idx];
   LaunchScope scope(kv, kind, s);
-  switch (a.epilogue) {
-    case EPI_PARTIAL: launch_epi<EPI_PARTIAL>(*a.tmW, act, p, grid, smem, s); break;
-    case EPI_SWIGLU: launch_epi<EPI_SWIGLU>(*a.tmW, act, p, grid, smem, s); break;
-    default: launch_epi<EPI_ARGMAX>(*a.tmW, act, p, grid, smem, s); break;
+  if (p.fold) {
+    switch (a.epilogue) {
+      case EPI_PARTIAL: launch_epi<EPI_PARTIAL, true>(*a.tmW, act, p, grid, smem, s); break;
+      case EPI_SWIGLU: launch_epi<EPI_SWIGLU, true>(*a.tmW, act, p, grid, smem, s); break;
+      default: launch_epi<EPI_ARGMAX, true>(*a.tmW, act, p, grid, smem, s); break;
+    }
+  } else {
+    switch (a.epilogue) {
+      case EPI_PARTIAL: launch_epi<EPI_PARTIAL, false>(*a.tmW, act, p, grid, smem, s); break;
+      case EPI_SWIGLU: launch_epi<EPI_SWIGLU, false>(*a.tmW, act, p, grid, smem, s); break;
+      default: launch_epi<EPI_ARGMAX, false>(*a.tmW, act, p, grid, smem, s); break;
+    }
   }
 }
