@@ -37,7 +37,8 @@ Parity pins (tests/test_oracle_*.py): an independent library decoder
 pairing and GQA grouping; torch's scaled_dot_product_attention for the masked
 attention; closed forms for RMSNorm / softmax / SiLU / RoPE; brute force over
 root paths for the tree forward and for the accept rule; a plain prefill of the
-accepted path for the commit.  The paper prints no worked numbers for this step,
+accepted path for the commit; scipy's softmax, a hand-computed row and a brute-force sort for
+top2_probs.  The paper prints no worked numbers for this step,
 so parity with numbers *in the paper* is unpinned; only its lossless property
 binds, and the tests check it.
 """
@@ -248,6 +249,28 @@ def tree_prep(parent) -> tuple[np.ndarray, np.ndarray]:
 def top2_gap(logits: np.ndarray) -> np.ndarray:
     part = np.partition(logits, -2, axis=-1)
     return part[..., -1] - part[..., -2]
+
+
+def top2_probs(logits: np.ndarray) -> tuple[np.ndarray, np.ndarray]:
+    """The two most probable tokens of every row and their probabilities under the softmax over the whole
+    vocabulary ("normalized logits", Section IV-A: drafting stops where the top-1 value falls below a threshold;
+    Section IV-C: the second-ranked token seeds a side branch).  Ties go to the lower token id.
+    Returns (ids [n, 2] int32, probs [n, 2] fp64)."""
+    logits = np.asarray(logits, dtype=F64)
+    n, v = logits.shape
+    ids = np.zeros((n, 2), dtype=np.int32)
+    probs = np.zeros((n, 2), dtype=F64)
+    for i in range(n):
+        row = logits[i]
+        e = np.exp(row - row.max())
+        sm = e / e.sum()
+        first = int(np.argmax(row))                       # lowest id among equal maxima
+        rest = row.copy()
+        rest[first] = -np.inf
+        second = int(np.argmax(rest)) if v > 1 else first
+        ids[i] = (first, second)
+        probs[i] = (sm[first], sm[second])
+    return ids, probs
 
 
 def accept(tokens, parent, argmax) -> dict:

@@ -132,3 +132,27 @@ def test_causal_forward_matches_library_llama(name):
     with torch.no_grad():
         ref_t = model(input_ids=torch.from_numpy(toks.astype(np.int64))[None]).logits[0].numpy()
     assert np.abs(ours_t - ref_t).max() < 1e-6
+
+
+def test_top2_probs_against_library_softmax_hand_values_and_sorting():
+    from scipy.special import softmax
+    # a row worked by hand: logits (0, ln 2, ln 5) -> probabilities (1/8, 2/8, 5/8)
+    ids, probs = O.top2_probs(np.array([[0.0, np.log(2.0), np.log(5.0)]]))
+    assert ids.tolist() == [[2, 1]]
+    assert np.allclose(probs, [[5 / 8, 2 / 8]], rtol=0, atol=1e-15)
+    # ties: the lower id first, then the other holder of the maximum
+    ids, probs = O.top2_probs(np.array([[1.0, 3.0, 3.0, -1.0], [2.0, 2.0, 2.0, 2.0]]))
+    assert ids.tolist() == [[1, 2], [0, 1]]
+    assert np.allclose(probs[1], [0.25, 0.25])
+    # random rows: library softmax and a full stable sort
+    rng = np.random.default_rng(7)
+    logits = rng.standard_normal((9, 501)) * 4.0
+    ids, probs = O.top2_probs(logits)
+    sm = softmax(logits, axis=-1)
+    order = np.argsort(-logits, axis=-1, kind="stable")
+    assert np.array_equal(ids, order[:, :2].astype(np.int32))
+    assert np.allclose(probs, np.take_along_axis(sm, order[:, :2], axis=-1), rtol=1e-13, atol=0)
+    assert np.all(probs[:, 0] >= probs[:, 1]) and np.all(probs.sum(-1) <= 1.0 + 1e-15)
+    # shifting a row by a constant changes nothing; a huge offset must not overflow
+    ids2, probs2 = O.top2_probs(logits + 1000.0)
+    assert np.array_equal(ids2, ids) and np.allclose(probs2, probs, rtol=1e-10)
