@@ -174,6 +174,7 @@ specasr_status specasr_verify_tree_ex(specasr_model* m, specasr_kv* kv, const in
  *   out_argmax, out_path : [device] int32[node_offsets[batch]], per utterance as in specasr_verify_tree
  *                        (path entries are local node indices)
  *   out_accept_len     : [device] int32[batch]
+ *   out_logits         : [device] fp32 [node_offsets[batch], vocab] or NULL: the target logits after every node
  *   out_bonus          : [device] int32[batch] or NULL
  * Each handle becomes "pending" and is committed on its own:
  *   specasr_commit_kv(m, kv[b], out_path + node_offsets[b], out_accept_len + b, stream).
@@ -186,7 +187,7 @@ specasr_status specasr_verify_tree_ex(specasr_model* m, specasr_kv* kv, const in
 specasr_status specasr_verify_tree_batch(specasr_model* m, int32_t batch, specasr_kv* const* kv,
                                          const int32_t* tokens, const int32_t* parent_idx,
                                          const int32_t* node_offsets, int32_t* out_argmax, int32_t* out_accept_len,
-                                         int32_t* out_path, int32_t* out_bonus, void* stream);
+                                         int32_t* out_path, float* out_logits, int32_t* out_bonus, void* stream);
 
 /*
  * Keep the accepted path (the "revert to the draft model" step of Section II-B needs the cache to
@@ -268,6 +269,21 @@ specasr_status specasr_accept_logits_static(const float* logits, int32_t vocab, 
                                             const int32_t* parent_idx, int32_t n_nodes, int32_t* out_argmax,
                                             int32_t* out_accept_len, int32_t* out_path, int32_t* out_bonus,
                                             void* stream);
+
+/*
+ * Top-2 tokens and their probabilities for every row of a logits matrix (the draft side of the method:
+ * Section IV-A truncates a draft where the normalised value of its top-1 token falls below a threshold,
+ * Section IV-C branches on the second-ranked token there).
+ *   logits    : [device] fp32 [n_rows, vocab], row-major, finite values (e.g. out_logits of
+ *               specasr_verify_tree_ex run on the draft model)
+ *   out_ids   : [device] int32 [n_rows, 2]  most probable and second most probable token (ties: lower id first;
+ *               both entries equal when vocab == 1)
+ *   out_probs : [device] fp32 [n_rows, 2]   their probabilities under the softmax over the whole row
+ * No scratch memory; one kernel on `stream`.  Errors: null pointer, n_rows < 1, vocab < 1 ->
+ * SPECASR_ERR_INVALID_ARG with nothing enqueued.
+ */
+specasr_status specasr_top2_probs(const float* logits, int32_t n_rows, int32_t vocab, int32_t* out_ids,
+                                  float* out_probs, void* stream);
 
 const char* specasr_last_error(void);
 

@@ -21,7 +21,7 @@ EXPORTS = [
     "specasr_kv_create", "specasr_kv_destroy", "specasr_kv_length", "specasr_kv_truncate",
     "specasr_prefill_embeds", "specasr_prefill_tokens", "specasr_verify_tree", "specasr_verify_tree_ex",
     "specasr_verify_tree_batch", "specasr_commit_kv", "specasr_poll_status", "specasr_launch_count", "specasr_last_error",
-    "specasr_profile_enable", "specasr_profile_read", "specasr_accept_logits_static",
+    "specasr_profile_enable", "specasr_profile_read", "specasr_accept_logits_static", "specasr_top2_probs",
 ]
 KIND_NAMES = ["prep", "norm", "gemm_qkv", "rope", "attn", "attn_merge", "gemm_o", "gemm_gu", "gemm_down", "gemm_lm",
               "accept", "commit"]
@@ -75,7 +75,7 @@ def lib() -> C.CDLL:
         L.specasr_verify_tree.restype = st
         L.specasr_verify_tree_ex.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp]
         L.specasr_verify_tree_ex.restype = st
-        L.specasr_verify_tree_batch.argtypes = [vp, i32, C.POINTER(vp), vp, vp, C.POINTER(i32), vp, vp, vp, vp, vp]
+        L.specasr_verify_tree_batch.argtypes = [vp, i32, C.POINTER(vp), vp, vp, C.POINTER(i32), vp, vp, vp, vp, vp, vp]
         L.specasr_verify_tree_batch.restype = st
         L.specasr_commit_kv.argtypes = [vp, vp, vp, vp, vp]
         L.specasr_commit_kv.restype = st
@@ -89,6 +89,8 @@ def lib() -> C.CDLL:
         L.specasr_profile_read.restype = st
         L.specasr_accept_logits_static.argtypes = [vp, i32, vp, vp, i32, vp, vp, vp, vp, vp]
         L.specasr_accept_logits_static.restype = st
+        L.specasr_top2_probs.argtypes = [vp, i32, i32, vp, vp, vp]
+        L.specasr_top2_probs.restype = st
         L.specasr_last_error.argtypes = []
         L.specasr_last_error.restype = C.c_char_p
         _lib = L
@@ -172,7 +174,8 @@ def specasr_verify_tree_ex(model: int, kv: int, tokens: int, parent_idx: int, n_
 
 
 def specasr_verify_tree_batch(model: int, kv_handles, tokens: int, parent_idx: int, node_offsets, out_argmax: int,
-                              out_accept_len: int, out_path: int, out_bonus: int = 0, stream: int = 0) -> None:
+                              out_accept_len: int, out_path: int, out_logits: int = 0, out_bonus: int = 0,
+                              stream: int = 0) -> None:
     """kv_handles: sequence of handles; node_offsets: sequence of batch + 1 ints (both host side);
     the other arguments are device addresses covering all utterances back to back."""
     batch = len(kv_handles)
@@ -181,7 +184,7 @@ def specasr_verify_tree_batch(model: int, kv_handles, tokens: int, parent_idx: i
     if len(node_offsets) != batch + 1:
         raise ValueError("node_offsets needs batch + 1 entries")
     _check(lib().specasr_verify_tree_batch(model, batch, handles, tokens, parent_idx, offsets, out_argmax,
-                                           out_accept_len, out_path, out_bonus or None, stream))
+                                           out_accept_len, out_path, out_logits or None, out_bonus or None, stream))
 
 
 def specasr_commit_kv(model: int, kv: int, path: int, accept_len: int, stream: int = 0) -> None:
@@ -189,11 +192,16 @@ def specasr_commit_kv(model: int, kv: int, path: int, accept_len: int, stream: i
 
 
 def specasr_accept_logits_static(logits: int, vocab: int, tokens: int, parent_idx: int, n_nodes: int, out_argmax: int,
-                                 out_accept_len: int, out_path: int, out_bonus: int = 0, stream: int = 0) -> None:
+                                 out_accept_len: int, out_path: int, out_logits: int = 0, out_bonus: int = 0,
+                              stream: int = 0) -> None:
     """Accept step from a logits matrix for callers that cannot allocate device memory (see the header):
     all arguments are device addresses of caller-owned buffers; the library's built-in array is the only scratch."""
     _check(lib().specasr_accept_logits_static(logits, vocab, tokens, parent_idx, n_nodes, out_argmax, out_accept_len,
                                               out_path, out_bonus or None, stream))
+
+
+def specasr_top2_probs(logits: int, n_rows: int, vocab: int, out_ids: int, out_probs: int, stream: int = 0) -> None:
+    _check(lib().specasr_top2_probs(logits, n_rows, vocab, out_ids, out_probs, stream))
 
 
 def specasr_poll_status(kv: int, stream: int = 0) -> int:

@@ -570,8 +570,8 @@ extern "C" specasr_status specasr_verify_tree(specasr_model* m, specasr_kv* kv, 
 extern "C" specasr_status specasr_verify_tree_batch(specasr_model* m, int32_t batch, specasr_kv* const* kv,
                                                     const int32_t* tokens, const int32_t* parent_idx,
                                                     const int32_t* node_offsets, int32_t* out_argmax,
-                                                    int32_t* out_accept_len, int32_t* out_path, int32_t* out_bonus,
-                                                    void* stream) {
+                                                    int32_t* out_accept_len, int32_t* out_path, float* out_logits,
+                                                    int32_t* out_bonus, void* stream) {
   const char* who = "specasr_verify_tree_batch";
   if (!m || !kv || !tokens || !parent_idx || !node_offsets || !out_argmax || !out_accept_len || !out_path) {
     set_error("%s: null argument", who);
@@ -642,7 +642,7 @@ extern "C" specasr_status specasr_verify_tree_batch(specasr_model* m, int32_t ba
   CUDA_TRY(cudaMemsetAsync(ctl_shared, 0, sizeof(int32_t) * 4, s));
   launch_tree_prep(wk, tab, tokens, parent_idx, s);
   launch_embed_tokens(wk, tab, total, tokens, s);
-  run_stack(m, wk, tab, total, n_max, true, ctl_shared, true, nullptr, s);
+  run_stack(m, wk, tab, total, n_max, true, ctl_shared, true, out_logits, s);
   launch_accept(wk, tab, ctl_shared, tokens, parent_idx, lm_tiles_of(m), out_argmax, out_accept_len, out_path, out_bonus,
                 s);
   for (int b = 0; b < batch; ++b) kv[b]->pending_n = tab.seg[b].n;

@@ -12,7 +12,8 @@ Control flow only: every forward pass, the accept rule and the cache compaction 
 import numpy as np
 import torch
 
-from .runtime import BatchVerifier
+from . import binding as B
+from .runtime import BatchVerifier, DeviceKV
 
 
 class SpeculativeBatchLoop:
@@ -27,7 +28,8 @@ class SpeculativeBatchLoop:
         self._verifiers = {}
         self.target_len = [kv.length() for kv in self.target_kvs]
         if self.draft_kvs is not None:
-            self.draft_len = [kv.length() for kv in self.draft_kvs]
+            self.draft_len = [kv.length() for kv in self.draft_kvs]     # entries that match the committed text
+            self.draft_dev_len = list(self.draft_len)                   # entries the device cache holds
             self._minus_one = torch.full((self.B,), -1, dtype=torch.int32, device=self.device)
         self.rounds = 0               # batched verification calls
         self.utterance_rounds = 0     # trees verified (rounds summed over utterances)
@@ -57,6 +59,7 @@ class SpeculativeBatchLoop:
             bv.commit()
             for b in members:
                 self.draft_len[b] += 1
+                self.draft_dev_len[b] += 1
             self.draft_steps += 1
 
     def align_draft(self, b, committed_tokens):
@@ -67,12 +70,13 @@ class SpeculativeBatchLoop:
             return
         want = self.target_len[b]
         kv = self.draft_kvs[b]
-        if self.draft_len[b] > want:
-            kv.truncate(want)
-        elif self.draft_len[b] < want:
-            missing = committed_tokens[len(committed_tokens) - 1 - (want - self.draft_len[b]):len(committed_tokens) - 1]
+        have = min(self.draft_len[b], want)
+        if self.draft_dev_len[b] != have:
+            kv.truncate(have)
+        if have < want:
+            missing = committed_tokens[len(committed_tokens) - 1 - (want - have):len(committed_tokens) - 1]
             kv.prefill_tokens(torch.tensor([int(t) for t in missing], dtype=torch.int32, device=self.device))
-        self.draft_len[b] = want
+        self.draft_len[b] = self.draft_dev_len[b] = want
 
     # ---- verification ----------------------------------------------------------------------------------------
     def verify_round(self, trees):
@@ -125,4 +129,83 @@ class SpeculativeBatchLoop:
                 emitted[b] += accepted + [bonus]
                 history[b] += accepted + [bonus]
                 proposer.observe(b, a)
+        return [e[:n_tokens] for e in emitted]
+
+    # ---- drafts from the draft model itself ------------------------------------------------------------------
+    def draft_trees(self, members, roots, threshold, max_len):
+        """Greedy single-sequence drafting with the draft model for the utterances in `members` (all of them in
+        one batched single-node call per step).  After every step the top-2 tokens and their softmax
+        probabilities are read back: the top-1 token extends the trunk; where its probability is below
+        `threshold` the second-ranked token becomes a one-node side branch at that position and the utterance
+        stops drafting (adaptive truncation, Section IV-A, with the limited-width expansion of Section IV-C at
+        the point of uncertainty); nobody drafts more than `max_len` tokens.  Returns {b: (tokens, parent)}."""
+        vocab = self.draft_kvs[0].model.cfg.vocab
+        trunk = {b: [] for b in members}
+        branch = {b: None for b in members}            # (depth of the parent on the trunk, token)
+        cur = {b: int(roots[b]) for b in members}
+        live = list(members)
+        for _ in range(max_len):
+            if not live:
+                break
+            bv = self._verifier(self.draft_kvs, live)
+            nb = len(live)
+            if not hasattr(bv, "logits"):
+                bv.logits = torch.empty(nb, vocab, dtype=torch.float32, device=self.device)
+                bv.top_ids = torch.empty(nb, 2, dtype=torch.int32, device=self.device)
+                bv.top_probs = torch.empty(nb, 2, dtype=torch.float32, device=self.device)
+            toks = torch.tensor([cur[b] for b in live], dtype=torch.int32, device=self.device)
+            bv.verify(toks, self._minus_one[:nb], list(range(nb + 1)), bv.logits)
+            bv.commit()
+            B.specasr_top2_probs(bv.logits.data_ptr(), nb, vocab, bv.top_ids.data_ptr(), bv.top_probs.data_ptr(),
+                                 DeviceKV._stream())
+            ids = bv.top_ids.cpu().numpy()             # synchronises: the host decides who goes on
+            probs = bv.top_probs.cpu().numpy()
+            self.draft_steps += 1
+            still = []
+            for i, b in enumerate(live):
+                self.draft_len[b] += 1
+                self.draft_dev_len[b] += 1
+                trunk[b].append(int(ids[i, 0]))
+                cur[b] = int(ids[i, 0])
+                if probs[i, 0] < threshold:
+                    branch[b] = (len(trunk[b]) - 1, int(ids[i, 1]))
+                else:
+                    still.append(b)
+            live = still
+        trees = {}
+        for b in members:
+            k = len(trunk[b])
+            tokens = [int(roots[b])] + trunk[b]
+            parent = [-1] + list(range(k))
+            if branch[b] is not None and branch[b][1] != trunk[b][branch[b][0]]:
+                parent.append(branch[b][0])            # sibling of trunk node depth + 1
+                tokens.append(branch[b][1])
+            trees[b] = (np.asarray(tokens, np.int32), np.asarray(parent, np.int32))
+        return trees
+
+    def decode_with_draft_model(self, roots, n_tokens, threshold=0.4, max_len=24):
+        """The loop with the draft model's own proposals (no stand-in): rounds of draft_trees -> batched
+        verification -> commit until every utterance has emitted n_tokens tokens."""
+        if self.draft_kvs is None:
+            raise ValueError("no draft caches were given")
+        emitted = [[] for _ in range(self.B)]
+        history = [[int(r)] for r in roots]
+        while True:
+            active = [b for b in range(self.B) if len(emitted[b]) < n_tokens]
+            if not active:
+                break
+            for b in active:
+                self.align_draft(b, history[b])
+            start = {b: self.draft_len[b] for b in active}
+            trees = self.draft_trees(active, {b: history[b][-1] for b in active}, threshold, max_len)
+            for b, (a, path, bonus) in self.verify_round(trees).items():
+                tokens = trees[b][0]
+                accepted = [int(tokens[i]) for i in path[1:]]
+                emitted[b] += accepted + [bonus]
+                history[b] += accepted + [bonus]
+                # the draft cache holds the root and the trunk tokens it was stepped on: keep what the target kept
+                on_trunk = 0
+                while on_trunk < a and int(path[on_trunk + 1]) == on_trunk + 1:
+                    on_trunk += 1
+                self.draft_len[b] = min(self.draft_len[b], start[b] + on_trunk + 1)
         return [e[:n_tokens] for e in emitted]

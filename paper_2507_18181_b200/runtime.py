@@ -193,13 +193,14 @@ class BatchVerifier:
         self.out_bonus = torch.empty(len(self.kvs), dtype=torch.int32, device=dev)
         self.offsets = [0] * (len(self.kvs) + 1)
 
-    def verify(self, tokens: torch.Tensor, parent: torch.Tensor, node_offsets):
+    def verify(self, tokens: torch.Tensor, parent: torch.Tensor, node_offsets, logits: torch.Tensor | None = None):
         """tokens / parent: int32 device tensors over all utterances back to back (parents local to the
-        utterance); node_offsets: batch + 1 host ints."""
+        utterance); node_offsets: batch + 1 host ints; logits: optional fp32 [total nodes, vocab] output."""
         self.offsets = [int(o) for o in node_offsets]
         B.specasr_verify_tree_batch(self.model.handle, [kv.handle for kv in self.kvs], tokens.data_ptr(),
                                     parent.data_ptr(), self.offsets, self.out_argmax.data_ptr(),
-                                    self.out_accept.data_ptr(), self.out_path.data_ptr(), self.out_bonus.data_ptr(),
+                                    self.out_accept.data_ptr(), self.out_path.data_ptr(),
+                                    logits.data_ptr() if logits is not None else 0, self.out_bonus.data_ptr(),
                                     DeviceKV._stream())
 
     def commit(self):

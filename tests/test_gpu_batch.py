@@ -47,22 +47,27 @@ class _Utterance:
         return np.asarray(tokens, np.int32), np.asarray(parent, np.int32)
 
 
-def _run_batch(bv, trees):
+def _run_batch(bv, trees, vocab=None):
     offsets = np.concatenate([[0], np.cumsum([len(t) for t, _ in trees])]).astype(int)
     tokens = torch.from_numpy(np.concatenate([t for t, _ in trees])).cuda()
     parent = torch.from_numpy(np.concatenate([p for _, p in trees])).cuda()
-    bv.verify(tokens, parent, offsets)
+    logits = torch.empty(int(offsets[-1]), vocab, dtype=torch.float32, device="cuda") if vocab else None
+    bv.verify(tokens, parent, offsets, logits)
     torch.cuda.synchronize()
     out = []
     for b in range(len(trees)):
         lo, hi = offsets[b], offsets[b + 1]
         out.append({"argmax": bv.out_argmax[lo:hi].cpu().numpy(), "path": bv.out_path[lo:hi].cpu().numpy(),
                     "accept_len": int(bv.out_accept[b].item()), "bonus": int(bv.out_bonus[b].item())})
+        if vocab:
+            out[-1]["logits"] = logits[lo:hi].cpu().numpy().astype(np.float64)
     return out
 
 
 def _check_utterance(got, want, tokens, parent):
     n = len(tokens)
+    if "logits" in got:
+        assert np.abs(got["logits"] - want["logits"]).max() < LOGIT_TOL
     clear = want["gap"] > GAP
     assert np.array_equal(got["argmax"][clear], want["argmax"][clear])
     top = want["logits"].max(-1)
@@ -91,7 +96,7 @@ def test_batch_matches_oracle_per_utterance_over_two_rounds(cfg_name, shapes):
     for rnd in range(2):
         trees = [u.draft(kind, seed=rnd) for u, (_, _, kind) in zip(utts, shapes)]
         wants = [O.verify_tree(cfg, W, u.cache, t, p) for u, (t, p) in zip(utts, trees)]
-        gots = _run_batch(bv, trees)
+        gots = _run_batch(bv, trees, cfg.vocab if rnd == 0 else None)
         for u, got, want, (t, p) in zip(utts, gots, wants, trees):
             assert u.kv.status() == 0
             _check_utterance(got, want, t, p)
@@ -158,7 +163,7 @@ def test_batch_host_side_errors_enqueue_nothing():
 
     def call(handles, offsets):
         B.specasr_verify_tree_batch(model.handle, handles, buf.data_ptr(), buf.data_ptr(), offsets, buf.data_ptr(),
-                                    buf.data_ptr(), buf.data_ptr(), 0, 0)
+                                    buf.data_ptr(), buf.data_ptr(), 0, 0, 0)
 
     for handles, offsets in [
         ([kvs[0].handle, kvs[0].handle], [0, 4, 8]),      # the same handle twice

@@ -85,3 +85,59 @@ def test_draft_shape_matches_oracle():
         assert np.array_equal(kv.out_argmax[:n].cpu().numpy()[clear], want["argmax"][clear])
         if want["decisive"]:
             assert int(kv.out_accept.item()) == want["accept_len"]
+
+
+def test_top2_probs_matches_oracle():
+    from paper_2507_18181_b200 import binding as B
+    rng = np.random.default_rng(11)
+    for n, vocab, scale in ((1, 1, 1.0), (3, 2, 1.0), (5, 257, 3.0), (64, 32000, 1.5), (2, 4099, 30.0)):
+        logits = (rng.standard_normal((n, vocab)) * scale).astype(np.float32)
+        if vocab > 300:
+            logits[0, 17] = logits[0, 230] = logits[0].max() + 1.0      # a tie at the top: lower id first
+        d = torch.from_numpy(logits).cuda()
+        ids = torch.empty(n, 2, dtype=torch.int32, device="cuda")
+        probs = torch.empty(n, 2, dtype=torch.float32, device="cuda")
+        B.specasr_top2_probs(d.data_ptr(), n, vocab, ids.data_ptr(), probs.data_ptr())
+        torch.cuda.synchronize()
+        want_ids, want_probs = O.top2_probs(logits)
+        assert np.array_equal(ids.cpu().numpy(), want_ids)                       # decided on the same fp32 values
+        assert np.allclose(probs.cpu().numpy(), want_probs, rtol=2e-5, atol=1e-9)
+    with pytest.raises(B.SpecasrError):
+        B.specasr_top2_probs(0, 1, 8, ids.data_ptr(), probs.data_ptr())
+
+
+@pytest.mark.parametrize("same_model,threshold,max_len", [(True, 0.0, 6), (True, 2.0, 6), (False, 0.0, 4)])
+def test_loop_with_the_draft_models_own_proposals(same_model, threshold, max_len):
+    """Drafts come from the draft model (top-1 extends the trunk, a low-probability top-1 ends it and adds the
+    second-ranked token as a sibling).  With the target's own weights as the draft every trunk token is the
+    target's greedy token, so rounds accept whole trunks; with another model nearly nothing is accepted.  Either
+    way the transcript is the oracle's greedy one."""
+    from paper_2507_18181_b200.runtime import DeviceModel, DeviceKV
+    from paper_2507_18181_b200.loop import SpeculativeBatchLoop
+    cfg = gen.get_config("tiny")
+    store = gen.WeightStore(cfg, 0)
+    W = O.Weights(store, cache_layers=True)
+    target = DeviceModel(cfg, store, gemm_path=0)
+    draft = target if same_model else DeviceModel(cfg, gen.WeightStore(cfg, 5), gemm_path=0)
+    n_tokens = 18
+    prefixes = (33, 58)
+    kvs, dkvs, roots, truth = [], [], [], []
+    for b, n_audio in enumerate(prefixes):
+        prompt = gen.prompt_tokens(4, cfg.vocab, 0, utterance=b)
+        kv, cache = _fill(cfg, target, DeviceKV, b, n_audio, prompt, W)
+        kvs.append(kv)
+        dkvs.append(_fill(cfg, draft, DeviceKV, b, n_audio, prompt)[0])
+        roots.append(int(prompt[-1]))
+        truth.append(O.greedy_continuation(cfg, W, cache, roots[-1], n_tokens + max_len + 2))
+    loop = SpeculativeBatchLoop(kvs, dkvs)
+    out = loop.decode_with_draft_model(roots, n_tokens, threshold=threshold, max_len=max_len)
+    for b in range(len(prefixes)):
+        assert out[b] == truth[b][:n_tokens]
+        assert kvs[b].status() == 0 and dkvs[b].status() == 0
+        assert kvs[b].length() == loop.target_len[b]
+    if same_model and threshold == 0.0:
+        assert loop.rounds <= -(-n_tokens // (max_len + 1)) + 1       # whole trunks accepted
+    if same_model and threshold == 2.0:
+        assert loop.rounds <= n_tokens // 2 + 1                       # one draft token + the bonus per round
+    if not same_model:
+        assert loop.rounds >= n_tokens - 3
