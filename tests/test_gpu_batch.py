@@ -180,3 +180,35 @@ def test_batch_host_side_errors_enqueue_nothing():
     with pytest.raises(B.SpecasrError) as e:
         call([kvs[0].handle, kvs[1].handle], [0, 4, 16])
     assert e.value.status == B.SPECASR_ERR_KV_CAPACITY
+
+
+def test_largest_batch_of_single_node_trees_equals_plain_calls():
+    """32 utterances (the most one call takes) of one node each: every row is an ordinary decoding step."""
+    from paper_2507_18181_b200.runtime import DeviceModel, DeviceKV, BatchVerifier
+    from paper_2507_18181_b200 import binding as B
+    cfg = gen.get_config("tiny")
+    model = DeviceModel(cfg, gen.WeightStore(cfg, 0), gemm_path=0)
+    nb = B.SPECASR_MAX_BATCH
+    kvs, toks = [], []
+    for b in range(nb):
+        kv = DeviceKV(model, max_tokens=64, max_nodes=32)
+        kv.prefill_tokens(torch.from_numpy(gen.prompt_tokens(3 + b % 7, cfg.vocab, 0, utterance=b)).cuda())
+        kvs.append(kv)
+        toks.append(int(gen.prompt_tokens(1, cfg.vocab, 9, utterance=b)[0]))
+    bv = BatchVerifier(kvs)
+    d_toks = torch.tensor(toks, dtype=torch.int32, device="cuda")
+    minus = torch.full((nb,), -1, dtype=torch.int32, device="cuda")
+    bv.verify(d_toks, minus, list(range(nb + 1)))
+    torch.cuda.synchronize()
+    got = bv.out_argmax[:nb].cpu().numpy()
+    assert np.all(bv.out_accept.cpu().numpy() == 0) and np.all(bv.out_path[:nb].cpu().numpy() == 0)
+    assert np.array_equal(bv.out_bonus.cpu().numpy(), got)
+    for b in range(nb):
+        kvs[b].verify(d_toks[b:b + 1], minus[:1])
+        torch.cuda.synchronize()
+        assert int(kvs[b].out_argmax[0].item()) == int(got[b])
+    with pytest.raises(B.SpecasrError) as e:          # one utterance more than a call takes
+        B.specasr_verify_tree_batch(model.handle, [kv.handle for kv in kvs] + [kvs[0].handle], d_toks.data_ptr(),
+                                    minus.data_ptr(), list(range(nb + 2)), bv.out_argmax.data_ptr(),
+                                    bv.out_accept.data_ptr(), bv.out_path.data_ptr(), 0, 0, 0)
+    assert e.value.status == B.SPECASR_ERR_INVALID_ARG
