@@ -192,8 +192,7 @@ def specasr_commit_kv(model: int, kv: int, path: int, accept_len: int, stream: i
 
 
 def specasr_accept_logits_static(logits: int, vocab: int, tokens: int, parent_idx: int, n_nodes: int, out_argmax: int,
-                                 out_accept_len: int, out_path: int, out_logits: int = 0, out_bonus: int = 0,
-                              stream: int = 0) -> None:
+                                 out_accept_len: int, out_path: int, out_bonus: int = 0, stream: int = 0) -> None:
     """Accept step from a logits matrix for callers that cannot allocate device memory (see the header):
     all arguments are device addresses of caller-owned buffers; the library's built-in array is the only scratch."""
     _check(lib().specasr_accept_logits_static(logits, vocab, tokens, parent_idx, n_nodes, out_argmax, out_accept_len,
