@@ -51,6 +51,6 @@ class CorruptedGreedyProposer:
         return tokens, parent, feed
 
     def observe(self, b, accept_len):
-        """The round's verdict: proposals beyond the rejected one stay valid for the positions they were
+        """The outcome of the verification: proposals beyond the rejected one stay valid for the positions they were
         drafted for and head the next trunk."""
         self.tail[b] = self.trunk[b][accept_len + 1:]
