@@ -56,3 +56,49 @@ def test_tree_generators():
     assert all(0 <= p2[i] < i for i in range(1, 64)) and sorted(old) == list(range(64))
     for new in range(1, 64):
         assert old[p2[new]] == p[old[new]] and t2[new] == toks[old[new]]
+
+
+def test_trunk_tree_and_proposer_follow_their_contracts():
+    """trunk_tree: the trunk is the main path and parents precede children; the proposer replays a transcript with
+    seeded corruption, recycles the tail past a rejection and asks for one draft step per new trunk token."""
+    for n, k, seed in ((32, 4, 0), (32, 16, 1), (12, 11, 2), (2, 1, 3)):
+        parent = gen.trunk_tree(n, k, seed=seed)
+        assert len(parent) == n and parent[0] == -1 and all(0 <= parent[i] < i for i in range(1, n))
+        assert list(gen.main_path(parent)) == list(range(k + 1))
+        assert np.array_equal(parent, gen.trunk_tree(n, k, seed=seed))
+    rng = np.random.default_rng(3)
+    T = [list(rng.integers(0, 1000, 120)), list(rng.integers(0, 1000, 120))]
+    roots = [7, 9]
+    P = gen.CorruptedGreedyProposer(T, roots, 1000, seed=4, n_nodes=32, k_min=4, k_max=16, corrupt_p=0.2)
+    Q = gen.CorruptedGreedyProposer(T, roots, 1000, seed=4, n_nodes=32, k_min=4, k_max=16, corrupt_p=0.2)
+    for b in range(2):
+        emitted, steps, drafted = [], 0, 0
+        prev_trunk, prev_a = None, None
+        while len(emitted) < 80:
+            tokens, parent, feed = P.propose(b, emitted)
+            t2, p2, f2 = Q.propose(b, emitted)
+            assert np.array_equal(tokens, t2) and np.array_equal(parent, p2) and list(feed) == list(f2)   # seeded
+            k = len(gen.main_path(parent)) - 1
+            assert 1 <= k <= 16 and len(tokens) == 32 and tokens[0] == (emitted[-1] if emitted else roots[b])
+            trunk = [int(x) for x in tokens[1:k + 1]]
+            if prev_trunk is not None:
+                tail = prev_trunk[prev_a + 1:][:k]
+                assert trunk[:len(tail)] == tail                        # recycled proposals head the new trunk
+                assert len(feed) == k - len(tail)                       # one draft step per new token
+                assert list(feed) == ([int(tokens[0])] + trunk)[len(tail):k]
+            else:
+                assert len(feed) == k
+            # siblings carry different tokens
+            for i in range(1, 32):
+                assert all(tokens[i] != tokens[j] for j in range(1, 32) if j != i and parent[j] == parent[i])
+            a = 0
+            while a < k and trunk[a] == T[b][len(emitted) + a]:
+                a += 1
+            emitted += trunk[:a] + [T[b][len(emitted) + a]]
+            P.observe(b, a)
+            Q.observe(b, a)
+            prev_trunk, prev_a = trunk, a
+            steps += 1
+            drafted += len(feed)
+        assert emitted == T[b][:len(emitted)]
+        assert steps < 40 and drafted < sum(1 for _ in emitted) * 4
