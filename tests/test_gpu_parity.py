@@ -19,11 +19,11 @@ LOGIT_TOL = 2e-2
 GAP = 1e-2
 
 
-def _gpu_stack(cfg_name, seed, gemm_path, max_tokens=512, max_nodes=64, shuffle=None):
+def _gpu_stack(cfg_name, seed, gemm_path, max_tokens=512, max_nodes=64, shuffle=None, page_size=16):
     from paper_2507_18181_b200.runtime import DeviceModel, DeviceKV
     cfg = gen.get_config(cfg_name)
     store = gen.WeightStore(cfg, seed)
-    model = DeviceModel(cfg, store, gemm_path=gemm_path)
+    model = DeviceModel(cfg, store, gemm_path=gemm_path, page_size=page_size)
     kv = DeviceKV(model, max_tokens=max_tokens, max_nodes=max_nodes, shuffle_pages_seed=shuffle)
     return cfg, store, model, kv
 
@@ -138,6 +138,36 @@ def test_verify_matches_oracle(cfg_name, gemm_path, n_audio, n_prompt, tree):
         moves = O.commit(cache, want)
         assert moves == [(int(s), L + j) for j, s in enumerate(src)]
         assert np.abs(after_k - cache.K[-1]).max() < 2e-3 and np.abs(after_v - cache.V[-1]).max() < 2e-3
+
+
+@pytest.mark.parametrize("page_size", [8, 24, 32, 64, 208])
+def test_page_sizes_and_an_exactly_full_cache(page_size):
+    """Pages of 32 / 64 / 208 slots run the tensor-core attention (one TMA box per page), 8 and 24 the plain one;
+    the cache is sized so that the tree's last node lands in its last slot."""
+    n_audio, n_prompt, n = 150, 6, 40
+    L = n_audio + n_prompt - 1
+    cap = -(-(L + n) // page_size) * page_size
+    extra = cap - (L + n)                       # audio frames added so that L + n == capacity
+    cfg, store, model, kv = _gpu_stack("small", 4, 0, max_tokens=cap, max_nodes=64, shuffle=5, page_size=page_size)
+    W, cache, prompt = _fill_both(cfg, store, kv, n_audio + extra, n_prompt, 4)
+    assert kv.length() + n == kv.max_pages * page_size
+    parent = gen.sparse_tree(n, seed=4)
+    root = int(prompt[-1])
+    greedy = O.greedy_continuation(cfg, W, cache, root, len(gen.main_path(parent)) - 1)
+    tokens = gen.fill_tree_tokens(parent, cfg.vocab, seed=4, root_token=root, main_tokens=greedy, corrupt_p=0.2)
+    got = _verify_gpu(cfg, kv, tokens, parent)
+    _check_against_oracle(got, O.verify_tree(cfg, W, cache, tokens, parent), tokens, parent)
+    before = kv.length()
+    kv.commit()
+    assert kv.length() == before + got["accept_len"] + 1
+    # one node more than fits is refused on the host
+    from paper_2507_18181_b200 import binding as B
+    kv.truncate(before)
+    bigger = gen.chain_tree(n)                  # n + 1 nodes
+    t = torch.zeros(n + 1, dtype=torch.int32, device="cuda")
+    with pytest.raises(B.SpecasrError) as e:
+        kv.verify(t, torch.from_numpy(bigger).cuda())
+    assert e.value.status == B.SPECASR_ERR_KV_CAPACITY
 
 
 def test_tensor_core_and_fma_projections_agree():
