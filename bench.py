@@ -32,6 +32,8 @@ WORKLOADS = {
     "config1": dict(model="tiny", n_audio=64, n_text=8, n_nodes=15, levels=None, chain=False),
     # config3 cut to two layers: same kernels and launch shapes, small enough for a profiler capture
     "config3_2layers": dict(model="7b", n_layers=2, n_audio=1500, n_text=201, n_nodes=64, levels=12, chain=False),
+    # the 13B-class shape as a second target (same tree and context as config 3)
+    "config3_13b": dict(model="13b", n_audio=1500, n_text=201, n_nodes=64, levels=12, chain=False),
     # a 256-node point of the config 4 sweep cut to two layers, for a profiler capture of the large-tree regime
     "config4_n256_2layers": dict(model="7b", n_layers=2, n_audio=1500, n_text=201, n_nodes=256, levels=None, chain=False),
 }

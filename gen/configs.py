@@ -48,6 +48,8 @@ CONFIGS = {
     "1b": ModelConfig("1b", 16, 2048, 32, 8, 64, 8192, 32000),
     "7b": ModelConfig("7b", 32, 4096, 32, 8, 128, 14336, 32000),
     "0.5b": ModelConfig("0.5b", 24, 896, 14, 2, 64, 4864, 32000),
+    # 13B-class target (the largest target of Section V-A): multi-head attention, 40 layers.
+    "13b": ModelConfig("13b", 40, 5120, 40, 40, 128, 13824, 32000),
 }
 
 

@@ -294,6 +294,23 @@ def test_single_node_tree_and_max_nodes():
     _check_against_oracle(got, O.verify_tree(cfg, W, cache, tokens, parent), tokens, parent)
 
 
+def test_13b_shape_two_layers():
+    """13B-class head geometry: 40 query heads = 40 KV heads (a row tile holds 128 nodes of one head), d_model 5120,
+    120 weight tiles in the QKV projection (no k-split)."""
+    from paper_2507_18181_b200.runtime import DeviceModel, DeviceKV
+    cfg = gen.get_config("13b", n_layers=2)
+    store = gen.WeightStore(cfg, 6)
+    model = DeviceModel(cfg, store, gemm_path=0)
+    kv = DeviceKV(model, max_tokens=512, max_nodes=64, shuffle_pages_seed=2)
+    W2, cache, prompt = _fill_both(cfg, store, kv, 230, 5, 6)
+    root = int(prompt[-1])
+    parent = gen.sparse_tree(64, seed=6, levels=12)
+    greedy = O.greedy_continuation(cfg, W2, cache, root, len(gen.main_path(parent)) - 1)
+    tokens = gen.fill_tree_tokens(parent, cfg.vocab, seed=6, root_token=root, main_tokens=greedy, corrupt_p=0.2)
+    got = _verify_gpu(cfg, kv, tokens, parent)
+    _check_against_oracle(got, O.verify_tree(cfg, W2, cache, tokens, parent), tokens, parent)
+
+
 def _bench_shape_case(cfg, n_audio, n_text, parent, seed, max_nodes):
     """Same launch configuration as bench.py for that shape: prefill in chunks of max_nodes, page size 16,
     tensor-core path; the oracle runs the same seeded inputs in fp64."""
