@@ -162,7 +162,9 @@ void launch_copy_embeds(specasr_kv* kv, const float* embeds, int n, cudaStream_t
 // A cluster of four CTAs owns a row, one quarter each, so that the few megabytes of partial planes are
 // pulled through 4 x n SMs at once and every thread has all its loads (x and up to 12 planes) in flight
 // together: an in-order core would otherwise pay one L2 round trip per plane.  The four partial sums of
-// squares meet through distributed shared memory and are added in rank order.
+// squares meet through distributed shared memory (each CTA writes its own into all four) and are added in rank
+// order.  (Two CTAs per row, i.e. at most
+// one block per SM at 64 rows, measured the same.)
 constexpr int kNormCluster = 4;
 
 template <int ITER>
@@ -172,7 +174,7 @@ __global__ void __launch_bounds__(256) k_rmsnorm_split(const int32_t* __restrict
                                                        int d, int d_part, float eps, int n, size_t plane_stride,
                                                        bf16* __restrict__ H) {
   namespace cg = cooperative_groups;
-  __shared__ float s_ss;
+  __shared__ float s_ss[kNormCluster];
   grid_dep_launch();
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = (int)cluster.block_rank();
@@ -228,12 +230,13 @@ __global__ void __launch_bounds__(256) k_rmsnorm_split(const int32_t* __restrict
     ss += v[it].x * v[it].x + v[it].y * v[it].y + v[it].z * v[it].z + v[it].w * v[it].w;
   }
   ss = block_sum_256(ss);
-  if (tid == 0) s_ss = ss;
+  // every CTA hands its sum to all four (slot = its rank) before the one cluster barrier; afterwards each reads
+  // only its own shared memory, so nobody has to wait for a peer before leaving
+  if (tid < kNormCluster) *cluster.map_shared_rank(&s_ss[rank], tid) = ss;
   cluster.sync();
   float total = 0.f;
 #pragma unroll
-  for (int r = 0; r < kNormCluster; ++r) total += *cluster.map_shared_rank(&s_ss, r);
-  cluster.sync();                            // nobody leaves while a peer may still read its sum
+  for (int r = 0; r < kNormCluster; ++r) total += s_ss[r];
   const float inv = rsqrtf(total / (float)d + eps);
 #pragma unroll
   for (int it = 0; it < ITER; ++it) {
@@ -265,14 +268,19 @@ void launch_rmsnorm_split(specasr_kv* kv, const int32_t* ctl, const float* gain,
 }
 
 // ------------------------------------------------------------------------------------------------
-// Rotary embedding at tree positions + KV append.  One thread per (node, head of the fused QKV row, rotation pair).
-// Sums the QKV projection's partial planes (their columns follow the rotary-paired row order of Wqkv),
-// rotates Q and K heads by the angle of
-// the node's position (rotate-half pairing, table built in fp64 on the host), writes Q as hi/lo planes
+// Rotary embedding at tree positions + KV append.  One thread per (node, head of the fused QKV row, four
+// adjacent rotation pairs).  Sums the QKV projection's partial planes (their columns follow the rotary-paired
+// row order of Wqkv, in which four adjacent features are four adjacent columns), rotates Q and K heads by the
+// angle of the node's position (rotate-half pairing, table built in fp64 on the host), writes Q as hi/lo planes
 // and K,V as hi/lo planes into cache slot L + node.
-__global__ void k_rope_append(const __grid_constant__ SegTable tab, const float* __restrict__ P, int n_partials,
-                              size_t partial_stride, int qkv_dim, int Hq, int Hkv, int dh, const int32_t* __restrict__ pos, const float2* __restrict__ rope,
-                              int layer, bf16* __restrict__ Q, size_t q_plane_stride, int page_size) {
+// The grid is kept small (a few hundred blocks) on purpose: launched with programmatic stream serialization the
+// blocks become resident while the QKV projection still runs, and only a grid that fits beside it in one wave
+// starts working the moment the projection ends.
+__global__ void __launch_bounds__(128) k_rope_append(const __grid_constant__ SegTable tab, const float* __restrict__ P,
+                                                     int n_partials, size_t partial_stride, int qkv_dim, int Hq, int Hkv,
+                                                     int dh, const int32_t* __restrict__ pos,
+                                                     const float2* __restrict__ rope, int layer, bf16* __restrict__ Q,
+                                                     size_t q_plane_stride, int page_size) {
   grid_dep_launch();
   grid_dep_wait();
   const int i = blockIdx.x;                    // workspace row
@@ -280,62 +288,71 @@ __global__ void k_rope_append(const __grid_constant__ SegTable tab, const float*
   const int32_t* ctl = sg.ctl;
   if (ctl[CTL_STATUS] != 0) return;
   const int half = dh >> 1;
-  const int head = blockIdx.y * (blockDim.x / half) + threadIdx.x / half;     // several heads per block
-  const int k = threadIdx.x % half;
+  const int per_head = half >> 2;              // threads per head: four rotation pairs each
+  const int head = blockIdx.y * (blockDim.x / per_head) + threadIdx.x / per_head;
+  const int k = (threadIdx.x % per_head) * 4;
   if (head >= Hq + 2 * Hkv) return;
   const size_t col = (size_t)i * qkv_dim + (size_t)head * dh;
   const size_t c1 = col + qkv_row_of_feature(k, dh), c2 = col + qkv_row_of_feature(k + half, dh);
-  float a1[kMaxSplitK], a2[kMaxSplitK];      // all plane loads in flight together, summed in plane order
-#pragma unroll
-  for (int s = 0; s < kMaxSplitK; ++s) {
-    a1[s] = s < n_partials ? __ldcg(P + s * partial_stride + c1) : 0.f;
-    a2[s] = s < n_partials ? __ldcg(P + s * partial_stride + c2) : 0.f;
-  }
-  float x1 = 0.f, x2 = 0.f;
-#pragma unroll
-  for (int s = 0; s < kMaxSplitK; ++s) {
-    x1 += a1[s];
-    x2 += a2[s];
-  }
   const bool is_v = head >= Hq + Hkv;
+  float4 x1 = make_float4(0.f, 0.f, 0.f, 0.f), x2 = x1;
+  float4 cs01 = make_float4(1.f, 0.f, 1.f, 0.f), cs23 = cs01;      // (cos, sin) of pairs k, k+1 and k+2, k+3
   if (!is_v) {
-    const float2 cs = rope[(size_t)pos[i] * half + k];
-    const float r1 = x1 * cs.x - x2 * cs.y;
-    const float r2 = x2 * cs.x + x1 * cs.y;
-    x1 = r1;
-    x2 = r2;
+    const float4* t = reinterpret_cast<const float4*>(rope + (size_t)pos[i] * half + k);
+    cs01 = t[0];
+    cs23 = t[1];
   }
-  bf16 h1, l1, h2, l2;
-  split_bf16(x1, h1, l1);
-  split_bf16(x2, h2, l2);
+  for (int s0 = 0; s0 < n_partials; s0 += 4) {   // four planes in flight, summed in plane order
+    float4 a1[4], a2[4];
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+      const bool on = s0 + s < n_partials;
+      a1[s] = on ? __ldcg(reinterpret_cast<const float4*>(P + (s0 + s) * partial_stride + c1)) : make_float4(0.f, 0.f, 0.f, 0.f);
+      a2[s] = on ? __ldcg(reinterpret_cast<const float4*>(P + (s0 + s) * partial_stride + c2)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+      x1.x += a1[s].x; x1.y += a1[s].y; x1.z += a1[s].z; x1.w += a1[s].w;
+      x2.x += a2[s].x; x2.y += a2[s].y; x2.z += a2[s].z; x2.w += a2[s].w;
+    }
+  }
+  // r1 = x1 cos - x2 sin, r2 = x2 cos + x1 sin (identity for V: cos = 1, sin = 0)
+  const float4 r1 = make_float4(x1.x * cs01.x - x2.x * cs01.y, x1.y * cs01.z - x2.y * cs01.w,
+                                x1.z * cs23.x - x2.z * cs23.y, x1.w * cs23.z - x2.w * cs23.w);
+  const float4 r2 = make_float4(x2.x * cs01.x + x1.x * cs01.y, x2.y * cs01.z + x1.y * cs01.w,
+                                x2.z * cs23.x + x1.z * cs23.y, x2.w * cs23.z + x1.w * cs23.w);
+  uint32_t h1[2], l1[2], h2[2], l2[2];
+  split2_pack(r1.x, r1.y, h1[0], l1[0]);
+  split2_pack(r1.z, r1.w, h1[1], l1[1]);
+  split2_pack(r2.x, r2.y, h2[0], l2[0]);
+  split2_pack(r2.z, r2.w, h2[1], l2[1]);
+  bf16* dst;
+  size_t plane;
   if (head < Hq) {
-    bf16* q = Q + (size_t)i * Hq * dh + (size_t)head * dh;
-    q[k] = h1;
-    q[k + half] = h2;
-    q[q_plane_stride + k] = l1;
-    q[q_plane_stride + k + half] = l2;
+    dst = Q + (size_t)i * Hq * dh + (size_t)head * dh;
+    plane = q_plane_stride;
   } else {
     const int kvh = is_v ? head - Hq - Hkv : head - Hq;
     const int slot = ctl[CTL_LEN] + (i - sg.row0);
     const int page = sg.page_table[slot / page_size];
     const int off = slot % page_size;
-    bf16* pool = is_v ? sg.v_pool : sg.k_pool;
-    bf16* dst = pool + kv_plane_offset(layer, sg.n_pages, Hkv, page_size, dh, page, kvh, 0) + (size_t)off * dh;
-    const size_t plane = (size_t)page_size * dh;
-    dst[k] = h1;
-    dst[k + half] = h2;
-    dst[plane + k] = l1;
-    dst[plane + k + half] = l2;
+    dst = (is_v ? sg.v_pool : sg.k_pool) + kv_plane_offset(layer, sg.n_pages, Hkv, page_size, dh, page, kvh, 0) +
+          (size_t)off * dh;
+    plane = (size_t)page_size * dh;
   }
+  *reinterpret_cast<uint2*>(dst + k) = make_uint2(h1[0], h1[1]);
+  *reinterpret_cast<uint2*>(dst + k + half) = make_uint2(h2[0], h2[1]);
+  *reinterpret_cast<uint2*>(dst + plane + k) = make_uint2(l1[0], l1[1]);
+  *reinterpret_cast<uint2*>(dst + plane + k + half) = make_uint2(l2[0], l2[1]);
 }
 
 void launch_rope_append(specasr_kv* wk, const SegTable& t, int n_total, int layer, int n_partials, cudaStream_t s) {
   const specasr_model* m = wk->m;
   const specasr_model_config& c = m->cfg;
-  const int heads_per_block = 256 / (c.head_dim / 2);
+  const int heads_per_block = 128 / (c.head_dim / 8);
   dim3 grid(n_total, (c.n_heads + 2 * c.n_kv_heads + heads_per_block - 1) / heads_per_block);
   LaunchScope scope(wk, SPECASR_KIND_ROPE, s);
-  launch_pdl(k_rope_append, grid, dim3(256), 0, s, t, wk->ws.P, n_partials, (size_t)wk->n_alloc * m->qkv_dim, m->qkv_dim,
+  launch_pdl(k_rope_append, grid, dim3(128), 0, s, t, wk->ws.P, n_partials, (size_t)wk->n_alloc * m->qkv_dim, m->qkv_dim,
              c.n_heads, c.n_kv_heads, c.head_dim, wk->ws.pos, m->rope_table, layer, wk->ws.Q,
              (size_t)wk->n_alloc * m->q_dim, c.page_size);
 }
@@ -344,7 +361,8 @@ void launch_rope_append(specasr_kv* wk, const SegTable& t, int n_total, int laye
 // Merge of the attention kernel's KV splits (log-sum-exp combination in base 2), normalisation and
 // hi/lo split of the result for the O projection.  One warp per (node, head) row: lane s holds the
 // (max, sum) of splits s and s + 32, lane c the output columns 4c .. 4c + 3; the partial outputs of
-// eight splits are requested together.  Rows n..n_pad-1 are zeroed.
+// six splits are requested together (more would cost the registers that let the blocks wait beside the attention
+// kernel in one wave).  Rows n..n_pad-1 are zeroed.
 __global__ void __launch_bounds__(128) k_attn_merge(const int32_t* __restrict__ ctl, const float* __restrict__ attO,
                                                     const float2* __restrict__ attML, int n_splits, size_t rows_alloc,
                                                     int Hq, int dh, int n, int rows_total, bf16* __restrict__ AO,
@@ -376,11 +394,11 @@ __global__ void __launch_bounds__(128) k_attn_merge(const int32_t* __restrict__ 
   float den = 0.f;
   for (int s = 0; s < n_splits; ++s) den += __shfl_sync(0xFFFFFFFFu, s < 32 ? ml0.y * w0 : ml1.y * w1, s & 31);
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int s0 = 0; s0 < n_splits; s0 += 8) {
-    float4 o[8];
-    float w[8];
+  for (int s0 = 0; s0 < n_splits; s0 += 6) {
+    float4 o[6];
+    float w[6];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
+    for (int u = 0; u < 6; ++u) {
       const int s = s0 + u;
       w[u] = __shfl_sync(0xFFFFFFFFu, s < 32 ? w0 : w1, s & 31);
       if (s >= n_splits) w[u] = 0.f;
@@ -388,7 +406,7 @@ __global__ void __launch_bounds__(128) k_attn_merge(const int32_t* __restrict__ 
                                     : make_float4(0.f, 0.f, 0.f, 0.f);
     }
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
+    for (int u = 0; u < 6; ++u) {
       acc.x += o[u].x * w[u]; acc.y += o[u].y * w[u]; acc.z += o[u].z * w[u]; acc.w += o[u].w * w[u];
     }
   }
