@@ -418,3 +418,35 @@ def test_7b_full_size_properties():
     assert kv.length() == L + al + 1
     k_after, _ = kv.read_kv(31, L + al + 1)
     assert np.array_equal(k_after[L:], k_before[L + res["path"][:al + 1]])
+
+
+@pytest.mark.parametrize("cfg_name", ["tiny", "micro", "small"])
+def test_random_tree_shapes(cfg_name):
+    """Seeded random topologies (any parent[i] < i: bushy, stringy, stars) and sizes from 1 to 70 nodes, several
+    rounds on one cache with commits in between, so that ragged tile tails, odd page offsets and every padding
+    width (16 / 32 / 64 / 128) are hit."""
+    cfg, store, model, kv = _gpu_stack(cfg_name, 8, 0, max_tokens=640, max_nodes=128, shuffle=9)
+    W, cache, prompt = _fill_both(cfg, store, kv, 45, 4, 8)
+    rng = np.random.default_rng(1234)
+    root = int(prompt[-1])
+    for rnd, n in enumerate([1, 2, 3, 7, 15, 17, 31, 33, 48, 63, 65, 70]):
+        shape = rnd % 3
+        if shape == 0:
+            parent = np.array([-1] + [int(rng.integers(0, i)) for i in range(1, n)], np.int32)              # bushy
+        elif shape == 1:
+            parent = np.array([-1] + [max(0, i - 1 - int(rng.integers(0, 2))) for i in range(1, n)], np.int32)  # stringy
+        else:
+            parent = np.array([-1] + [0 if rng.random() < 0.5 else int(rng.integers(0, i)) for i in range(1, n)], np.int32)
+        depth_main = len(gen.main_path(parent)) - 1
+        greedy = O.greedy_continuation(cfg, W, cache, root, depth_main) if depth_main else []
+        tokens = gen.fill_tree_tokens(parent, cfg.vocab, seed=50 + rnd, root_token=root, main_tokens=greedy,
+                                      corrupt_p=0.15)
+        want = O.verify_tree(cfg, W, cache, tokens, parent)
+        got = _verify_gpu(cfg, kv, tokens, parent)
+        _check_against_oracle(got, want, tokens, parent)
+        if not want["decisive"]:
+            break                                   # a near-tie: the two sides may legitimately part ways from here
+        kv.commit()
+        O.commit(cache, want)
+        assert kv.length() == cache.length
+        root = got["bonus"]
