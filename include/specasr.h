@@ -129,7 +129,7 @@ specasr_status specasr_kv_length(specasr_kv* kv, int32_t* out_len, void* stream)
 /* Rewinds (or empties) the cache to `len` <= current length.  Drops any pending verify. */
 specasr_status specasr_kv_truncate(specasr_kv* kv, int32_t len, void* stream);
 
-/* Context fill (the prefill of Section II-A: audio vectors "alongside text prompts"), causal
+/* Context fill (the prefill of Section II-A: audio-embedding vectors followed by prompt text), causal
  * attention, no logits.  embeds [device] fp32 [n, d_model] enter layer 0 directly; tokens [device]
  * int32[n] go through the embedding table.  Any n >= 1 (processed in chunks); advances the length. */
 specasr_status specasr_prefill_embeds(specasr_model* m, specasr_kv* kv, const float* embeds, int32_t n, void* stream);
@@ -190,7 +190,7 @@ specasr_status specasr_verify_tree_batch(specasr_model* m, int32_t batch, specas
                                          int32_t* out_path, float* out_logits, int32_t* out_bonus, void* stream);
 
 /*
- * Keep the accepted path (the "revert to the draft model" step of Section II-B needs the cache to
+ * Keep the accepted path (after a round control goes back to the draft model, Section II-B, so the cache must
  * hold exactly prefix + accepted tokens): slot L+j <- slot L+path[j] for j = 0..accept_len, all
  * layers, K and V; then L <- L + accept_len + 1.  path / accept_len are the [device] arrays a
  * preceding verify wrote (or the caller's own choice of a root path of that tree).  Requires a
