@@ -219,6 +219,65 @@ def run_reference(args, wl):
 
 # ------------------------------------------------------------------------------------------------ CUDA leg
 
+def in_flow_times(kv, step, kind_names):
+    """Per-kernel contribution to one step from the library's device-side trace: block records are grouped into
+    launches (same kind, starts close together); a launch adds (its last block's end - the latest end of all
+    launches before it).  Returns {kind name: {"launches", "us_per_step"}} or None if nothing was recorded."""
+    rec = kv.trace(step, capacity=1 << 18)
+    if len(rec) == 0:
+        return None
+    launches = []                      # [kind, first start, last start, last end]
+    for kind, start, end, _ in rec:
+        if launches and launches[-1][0] == kind and start - launches[-1][2] < 20000:
+            launches[-1][2] = max(launches[-1][2], start)
+            launches[-1][3] = max(launches[-1][3], end)
+        else:
+            launches.append([int(kind), int(start), int(start), int(end)])
+    out = {}
+    latest = launches[0][1]
+    for kind, _, _, end in launches:
+        name = kind_names[kind]
+        d = out.setdefault(name, {"launches": 0, "us_per_step": 0.0})
+        d["launches"] += 1
+        d["us_per_step"] += max(0, end - latest) / 1e3
+        latest = max(latest, end)
+    return out
+
+
+def run_in_flow(args, wl):
+    """Child mode (--in-flow, with SPECASR_TRACE_LIB=1): one traced step of the workload, result as a JSON line."""
+    import torch
+    from paper_2507_18181_b200 import binding as B
+    device = "cuda:0"
+    torch.cuda.set_device(0)
+    cfg, model, kv, L, tokens, parent = build_workload(wl, device)
+    d_tokens, d_parent = torch.from_numpy(tokens).to(device), torch.from_numpy(parent).to(device)
+
+    def step():
+        kv.verify(d_tokens, d_parent)
+        kv.commit()
+        kv.truncate(L)
+
+    for _ in range(5):
+        step()
+    print(json.dumps({"in_flow": in_flow_times(kv, step, B.KIND_NAMES)}))
+
+
+def in_flow_from_child(args):
+    """The device-side trace lives in a build variant of the library (it costs ~2 % even when off), so the traced
+    step runs in a child process that loads that variant."""
+    env = dict(os.environ, SPECASR_TRACE_LIB="1")
+    for k in ("RANK", "LOCAL_RANK", "WORLD_SIZE"):
+        env.pop(k, None)
+    try:
+        res = subprocess.run([sys.executable, os.path.abspath(__file__), "--workload", args.workload, "--in-flow"],
+                             env=env, capture_output=True, text=True, timeout=600)
+        lines = [l for l in res.stdout.splitlines() if l.startswith("{")]
+        return json.loads(lines[-1])["in_flow"] if res.returncode == 0 and lines else None
+    except Exception:
+        return None
+
+
 def slowest_rank(elapsed, world, device):
     """Replicas do not exchange data: the job's time is the slowest rank's (max over ranks)."""
     if world <= 1:
@@ -239,7 +298,8 @@ def build_workload(wl, device, seed=1):
     import torch
     from paper_2507_18181_b200 import build as _build
     from paper_2507_18181_b200.runtime import DeviceModel, DeviceKV
-    _build.build()
+    from paper_2507_18181_b200 import binding as _binding
+    _build.build(trace=_binding.TRACE_LIB)
     cfg = model_config(wl)
     store = gen.WeightStore(cfg, seed)
     model = DeviceModel(cfg, store, device=device)
@@ -364,6 +424,7 @@ def run_ours(args, wl):
     ms, cnt = B.specasr_profile_read(kv.handle, stream.cuda_stream)
     B.specasr_profile_enable(kv.handle, 0)
     kernels = {k: {"launches_per_step": cnt[k] / prof_steps, "ms_per_step": ms[k] / prof_steps} for k in ms if cnt[k]}
+    in_flow = in_flow_from_child(args) if world == 1 else None
     gb = gemm_weight_bytes(cfg)
     gemm_bytes_step = cfg.n_layers * (gb["gemm_qkv"] + gb["gemm_o"] + gb["gemm_gu"] + gb["gemm_down"]) + gb["gemm_lm"]
     gemm_ms_step = sum(ms[k] for k in gb) / prof_steps
@@ -397,11 +458,22 @@ def run_ours(args, wl):
                      "algorithmic_bytes_per_launch": gemm_bytes_step / gemm_launches,
                      "avg_launch_ms": gemm_ms_step / gemm_launches},
         "kernels": kernels,
+        "in_flow": None,
         "gpu_launches": int(launches),
         "clocks": clocks,
         "e2e": {"value": world * n * args.steps / e2e_s, "unit": UNIT, "ms_per_step": e2e_s / args.steps * 1e3,
                 "h2d_bytes_per_step": int(2 * n * 4), "d2h_bytes_per_step": int((2 * n + 2) * 4)},
     }
+    if in_flow:
+        gemm_us = sum(in_flow[k]["us_per_step"] for k in gb if k in in_flow)
+        line["in_flow"] = {
+            "how": "one extra step with the device-side trace on: time from the previous kernel's last block end to "
+                   "this kernel's last block end (%globaltimer), i.e. what the kernel adds to the step with the "
+                   "overlap of consecutive kernels intact",
+            "us_per_launch": {k: round(v["us_per_step"] / v["launches"], 2) for k, v in in_flow.items()},
+            "projections": {"us_per_step": gemm_us, "achieved_gbs": gemm_bytes_step / (gemm_us * 1e-6) / 1e9,
+                            "frac_of_" + peaks["source"]: gemm_bytes_step / (gemm_us * 1e-6) / 1e9 / peaks["hbm_gbs"]},
+        }
     if world == 1 and not args.no_cpu_baseline:
         run_once, desc = oracle_sample(wl)
         run_once()
@@ -624,6 +696,7 @@ def main():
     ap.add_argument("--workload", default="config3", choices=sorted(WORKLOADS) + ["config5", "config5_small"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="config 4: one JSON line per (draft shape, KV length) point")
+    ap.add_argument("--in-flow", action="store_true", help=argparse.SUPPRESS)
     args = ap.parse_args()
     if args.sweep:
         run_sweep(args)
@@ -634,6 +707,9 @@ def main():
         run_loop(args)
         return
     wl = WORKLOADS[args.workload]
+    if args.in_flow:
+        run_in_flow(args, wl)
+        return
     if args.impl == "reference":
         run_reference(args, wl)
     else:

@@ -230,6 +230,19 @@ enum {
   SPECASR_KIND_COUNT = 12
 };
 specasr_status specasr_profile_enable(specasr_kv* kv, int32_t enable);
+/*
+ * Device-side trace.  The event pairs of specasr_profile_* sit between launches and thereby switch off the
+ * overlap of consecutive kernels (programmatic dependent launch); with a trace buffer set, every thread block of
+ * the tree-prep, embedding, norm, projection, rotary, attention, merge and accept kernels instead appends one
+ * record of four uint64 words {SPECASR_KIND_*, start, end, wait_end} in %globaltimer nanoseconds (wait_end = when
+ * the block's wait for the previous kernel of the stream returned; 0 if it never got there).
+ *   buffer : [device] uint64 words, 8-byte aligned: word 0 = number of records appended so far (the caller zeroes it
+ *            before a traced call; counting continues past the capacity), word 1 unused, records from word 2 on;
+ *            at least 2 + 4 * capacity_records words.  NULL switches tracing off (the default).
+ * For a batched call the buffer of the first handle is used.  The buffer is borrowed until it is replaced or the
+ * handle is destroyed.  (No counterpart in the paper: instrumentation of this implementation.)
+ */
+specasr_status specasr_trace_set(specasr_kv* kv, void* buffer, int64_t capacity_records);
 specasr_status specasr_profile_read(specasr_kv* kv, double* out_ms, int64_t* out_launches, void* stream);
 
 /*

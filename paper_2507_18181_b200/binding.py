@@ -8,7 +8,9 @@ import ctypes as C
 import os
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libspecasr.so")
+# SPECASR_TRACE_LIB=1 selects the variant built with -DSPECASR_TRACE (specasr_trace_set records; ~2 % slower)
+TRACE_LIB = os.environ.get("SPECASR_TRACE_LIB") == "1"
+LIB_PATH = os.path.join(_HERE, "libspecasr_trace.so" if TRACE_LIB else "libspecasr.so")
 
 SPECASR_MAX_NODES = 256
 SPECASR_MAX_BATCH = 32
@@ -21,7 +23,7 @@ EXPORTS = [
     "specasr_kv_create", "specasr_kv_destroy", "specasr_kv_length", "specasr_kv_truncate",
     "specasr_prefill_embeds", "specasr_prefill_tokens", "specasr_verify_tree", "specasr_verify_tree_ex",
     "specasr_verify_tree_batch", "specasr_commit_kv", "specasr_poll_status", "specasr_launch_count", "specasr_last_error",
-    "specasr_profile_enable", "specasr_profile_read", "specasr_accept_logits_static", "specasr_top2_probs",
+    "specasr_profile_enable", "specasr_profile_read", "specasr_trace_set", "specasr_accept_logits_static", "specasr_top2_probs",
 ]
 KIND_NAMES = ["prep", "norm", "gemm_qkv", "rope", "attn", "attn_merge", "gemm_o", "gemm_gu", "gemm_down", "gemm_lm",
               "accept", "commit"]
@@ -87,6 +89,8 @@ def lib() -> C.CDLL:
         L.specasr_profile_enable.restype = st
         L.specasr_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64), vp]
         L.specasr_profile_read.restype = st
+        L.specasr_trace_set.argtypes = [vp, vp, C.c_int64]
+        L.specasr_trace_set.restype = st
         L.specasr_accept_logits_static.argtypes = [vp, i32, vp, vp, i32, vp, vp, vp, vp, vp]
         L.specasr_accept_logits_static.restype = st
         L.specasr_top2_probs.argtypes = [vp, i32, i32, vp, vp, vp]
@@ -215,6 +219,10 @@ def specasr_launch_count(kv: int) -> int:
 
 def specasr_profile_enable(kv: int, enable: int) -> None:
     _check(lib().specasr_profile_enable(kv, enable))
+
+
+def specasr_trace_set(kv: int, buffer: int, capacity_records: int) -> None:
+    _check(lib().specasr_trace_set(kv, buffer or None, capacity_records))
 
 
 def specasr_profile_read(kv: int, stream: int = 0):

@@ -235,6 +235,8 @@ extern "C" specasr_status specasr_kv_create(const specasr_model* m, void* k_pool
   kv->prof_on = false;
   kv->prof_used = 0;
   kv->attn_tc = false;
+  kv->trace.buf = nullptr;
+  kv->trace.cap = 0;
   cudaError_t e = cudaHostAlloc(&kv->pinned, 4 * sizeof(int32_t), cudaHostAllocDefault);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&kv->len_event, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaMemset(kv->ws.ctl, 0, sizeof(int32_t) * kCtlWords);
@@ -277,6 +279,22 @@ extern "C" void specasr_kv_destroy(specasr_kv* kv) {
 }
 
 extern "C" int64_t specasr_launch_count(const specasr_kv* kv) { return kv ? kv->launches : 0; }
+
+extern "C" specasr_status specasr_trace_set(specasr_kv* kv, void* buffer, int64_t capacity_records) {
+  if (!kv || capacity_records < 0 || (buffer && ((uintptr_t)buffer & 7))) {
+    set_error("specasr_trace_set: null handle, negative capacity or misaligned buffer");
+    return SPECASR_ERR_INVALID_ARG;
+  }
+#ifndef SPECASR_TRACE
+  if (buffer) {
+    set_error("specasr_trace_set: this library was built without -DSPECASR_TRACE (use libspecasr_trace.so)");
+    return SPECASR_ERR_UNSUPPORTED;
+  }
+#endif
+  kv->trace.buf = (unsigned long long*)buffer;
+  kv->trace.cap = buffer ? (unsigned long long)capacity_records : 0ull;
+  return SPECASR_OK;
+}
 
 extern "C" specasr_status specasr_profile_enable(specasr_kv* kv, int32_t enable) {
   if (!kv) {

@@ -52,6 +52,9 @@ struct AttnParams {
   size_t rows_alloc;      // n_alloc * Hq
   int n_pages, page_size, layer, Hq, Hkv, group, nodes_per_tile, n, chunk, row0;
   float scale_log2;
+#ifdef SPECASR_TRACE
+  TraceBuf tr;
+#endif
 };
 
 template <int DH>
@@ -113,7 +116,9 @@ __global__ void __launch_bounds__(64 + SOFTMAX_THREADS, 1) k_tree_attention_tc(c
   __syncthreads();
   tc_fence_after();
   // everything above is independent of the previous kernel; its results are read from here on
+  SPECASR_TRACE_SCOPE(p.tr, SPECASR_KIND_ATTN);
   pdl_wait();
+  SPECASR_TRACE_MARK();
   const bool live = p.ctl[CTL_STATUS] == 0;
   const int L = p.ctl[CTL_LEN];
   const int Ltot = L + p.n;
@@ -377,6 +382,9 @@ void launch_dh(specasr_kv* wk, const SegTable& t, int n_max, int layer, cudaStre
   p.group = c.n_heads / c.n_kv_heads;
   p.nodes_per_tile = 128 / p.group;
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
+#ifdef SPECASR_TRACE
+  p.tr = wk->trace;
+#endif
   dim3 grid(c.n_kv_heads, (n_max + p.nodes_per_tile - 1) / p.nodes_per_tile, t.count * t.splits);
   LaunchScope scope(wk, SPECASR_KIND_ATTN, s);
   launch_pdl(k_tree_attention_tc<DH>, grid, dim3(64 + SOFTMAX_THREADS), smem, s, wk->tm_Q, t, p);

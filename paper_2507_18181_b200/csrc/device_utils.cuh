@@ -58,6 +58,39 @@ __device__ __forceinline__ unsigned long long pack_max_key(float v, uint32_t idx
   return ((unsigned long long)u << 32) | (unsigned long long)(0xFFFFFFFFu - idx);
 }
 
+// One trace record per thread block (see TraceBuf): construct at kernel entry, mark() after the wait for the
+// previous kernel, the destructor stamps the end.  Only the library variant built with -DSPECASR_TRACE carries
+// it (through the SPECASR_TRACE_* macros): even switched off, the extra parameter and live value changed the
+// register allocation of several kernels and cost the step about 2 %.
+#ifdef SPECASR_TRACE
+struct TraceScope {
+  unsigned long long* e;
+  __device__ __forceinline__ static unsigned long long now() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+  }
+  __device__ __forceinline__ TraceScope(const TraceBuf& tr, int kind) : e(nullptr) {
+    if (tr.buf != nullptr && threadIdx.x == 0 && threadIdx.y == 0 && threadIdx.z == 0) {
+      const unsigned long long slot = atomicAdd(tr.buf, 1ull);
+      if (slot < tr.cap) {
+        e = tr.buf + 2 + slot * 4;
+        e[0] = (unsigned long long)kind;
+        e[1] = now();
+        e[2] = 0;
+        e[3] = 0;
+      }
+    }
+  }
+  __device__ __forceinline__ void mark() {
+    if (e) e[3] = now();
+  }
+  __device__ __forceinline__ ~TraceScope() {
+    if (e) e[2] = now();
+  }
+};
+#endif
+
 // Programmatic dependent launch (see launch_pdl): wait for the previous kernel of the stream, and let
 // the next one begin its prologue.
 __device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }

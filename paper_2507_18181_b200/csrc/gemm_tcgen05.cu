@@ -71,6 +71,10 @@ struct TcParams {
   bf16* A;                  // EPI_SWIGLU: [2][n_alloc][M/2]
   unsigned long long* amax; // EPI_ARGMAX: [tiles][n_alloc]
   float* logits;            // EPI_ARGMAX: optional [n][M]
+#ifdef SPECASR_TRACE
+  TraceBuf tr;
+  int kind;                 // SPECASR_KIND_* of this launch
+#endif
 };
 
 __device__ __forceinline__ int ld_acquire(const int32_t* p) {
@@ -88,6 +92,7 @@ template <int EPI, bool FOLD>
 __global__ void __launch_bounds__(64 + EPI_THREADS, 1) k_proj(const __grid_constant__ CUtensorMap tmW,
                                                  const __grid_constant__ CUtensorMap tmAct, TcParams p) {
   extern __shared__ uint8_t smem_raw[];
+  SPECASR_TRACE_SCOPE(p.tr, p.kind);
   uint8_t* tiles = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const int w_bytes = p.tm * p.ksub * W_SUB_BYTES;
   const int act_sub = p.n_pad * 2 * SUB_K * 2;         // both planes of one 64-wide k sub-block
@@ -162,6 +167,7 @@ __global__ void __launch_bounds__(64 + EPI_THREADS, 1) k_proj(const __grid_const
       load_w(i);
     }
     pdl_wait();
+    SPECASR_TRACE_MARK();
     if (*(volatile int32_t*)status != 0) {
       if (pre > 0) *abort = 1;       // weight tiles are in flight: hold the shared memory until they land
     } else {
@@ -624,6 +630,10 @@ void launch_gemm_tc(specasr_kv* kv, const GemmArgs& a, int kind, cudaStream_t s)
   p.fixP = kv->ws.fixP;
   p.fixFlag = kv->ws.fixFlag;
   p.P = a.P; p.A = a.A; p.amax = a.amax; p.logits = a.logits;
+#ifdef SPECASR_TRACE
+  p.tr = kv->trace;
+  p.kind = kind;
+#endif
   const long long units = (long long)p.groups * p.KB;
   const int grid = a.epilogue == EPI_PARTIAL ? p.groups * p.splits : (int)(units < m->n_sm ? units : m->n_sm);
   const size_t smem = (size_t)stages * stage_bytes + sizeof(SharedCtl) + epi_bytes + 1024;

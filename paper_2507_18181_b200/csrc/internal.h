@@ -23,6 +23,28 @@ enum { CTL_LEN = 0, CTL_STATUS = 1, CTL_N = 2 };
 // over all utterances: its status word only ever records a bounded wait that ran out.
 constexpr int kCtlBatch = 16;
 
+// Optional device-side trace (specasr_trace_set): every thread block of the traced kernels appends one record
+// {kind, start, end, time its wait for the previous kernel ended} of %globaltimer nanoseconds.  Event pairs around
+// a launch switch the overlap of consecutive kernels off; these stamps do not.
+struct TraceBuf {
+  unsigned long long* buf;  // [0] = records written so far, [1] unused, records of 4 words from [2]; null = off
+  unsigned long long cap;   // records the buffer holds
+};
+
+// The trace exists only in the library variant built with -DSPECASR_TRACE; in the product build these expand to
+// nothing, so that kernel signatures, parameter structs and register allocation are exactly those without it.
+#ifdef SPECASR_TRACE
+#define SPECASR_TRACE_PARAM , TraceBuf tr
+#define SPECASR_TRACE_ARG(kv) , (kv)->trace
+#define SPECASR_TRACE_SCOPE(tr, kind) TraceScope trace_(tr, kind)
+#define SPECASR_TRACE_MARK() trace_.mark()
+#else
+#define SPECASR_TRACE_PARAM
+#define SPECASR_TRACE_ARG(kv)
+#define SPECASR_TRACE_SCOPE(tr, kind)
+#define SPECASR_TRACE_MARK()
+#endif
+
 struct GemmMaps {           // TMA descriptors of one weight matrix (tcgen05 path)
   CUtensorMap w;
 };
@@ -89,6 +111,7 @@ struct specasr_kv {
   std::vector<cudaEvent_t> prof_events;   // 2 per recorded launch
   std::vector<int> prof_kinds;
   size_t prof_used;                       // launches recorded since the last read
+  TraceBuf trace;                         // device-side trace, off unless specasr_trace_set was called
   // activation TMA descriptors (tcgen05 path), one per box height 16 << i
   CUtensorMap tm_H[5], tm_AO[5], tm_A[5];
   // tensor-core attention: rotated queries and the two pools

@@ -12,8 +12,9 @@
 // One block per utterance of the call; tokens / parent / depth / pos / anc are indexed by workspace row.
 __global__ void k_tree_prep(const __grid_constant__ SegTable tab, const int32_t* __restrict__ tokens,
                             const int32_t* __restrict__ parent, int vocab, int32_t* __restrict__ depth,
-                            int32_t* __restrict__ pos, unsigned long long* __restrict__ anc) {
+                            int32_t* __restrict__ pos, unsigned long long* __restrict__ anc SPECASR_TRACE_PARAM) {
   __shared__ int s_bad;
+  SPECASR_TRACE_SCOPE(tr, SPECASR_KIND_PREP);
   const int i = threadIdx.x;
   const SegDev& sg = tab.seg[blockIdx.x];
   int32_t* ctl = sg.ctl;
@@ -25,6 +26,7 @@ __global__ void k_tree_prep(const __grid_constant__ SegTable tab, const int32_t*
   anc += (size_t)sg.row0 * 4;
   grid_dep_launch();
   grid_dep_wait();
+  SPECASR_TRACE_MARK();
   if (i == 0) s_bad = 0;
   __syncthreads();
   const int L = ctl[CTL_LEN];
@@ -93,7 +95,7 @@ __global__ void k_chain_prep(int32_t* __restrict__ ctl, int n, int capacity, int
 void launch_tree_prep(specasr_kv* wk, const SegTable& t, const int32_t* tokens, const int32_t* parent, cudaStream_t s) {
   LaunchScope scope(wk, SPECASR_KIND_PREP, s);
   launch_pdl(k_tree_prep, dim3(t.count), dim3(256), 0, s, t, tokens, parent, wk->m->cfg.vocab, wk->ws.depth,
-             wk->ws.pos, wk->ws.anc);
+             wk->ws.pos, wk->ws.anc SPECASR_TRACE_ARG(wk));
 }
 
 void launch_chain_prep(specasr_kv* kv, int n, cudaStream_t s) {
@@ -114,9 +116,11 @@ __device__ __forceinline__ int segment_of_row(const SegTable& tab, int row) {
 }
 
 __global__ void k_embed_tokens(const __grid_constant__ SegTable tab, const int32_t* __restrict__ tokens,
-                               const bf16* __restrict__ E, int d, float* __restrict__ X) {
+                               const bf16* __restrict__ E, int d, float* __restrict__ X SPECASR_TRACE_PARAM) {
   grid_dep_launch();
+  SPECASR_TRACE_SCOPE(tr, SPECASR_KIND_PREP);
   grid_dep_wait();
+  SPECASR_TRACE_MARK();
   const int i = blockIdx.x;
   if (tab.seg[segment_of_row(tab, i)].ctl[CTL_STATUS] != 0) return;
   const bf16* row = E + (size_t)tokens[i] * d;
@@ -146,7 +150,8 @@ __global__ void k_copy_embeds(const int32_t* __restrict__ ctl, const float* __re
 
 void launch_embed_tokens(specasr_kv* wk, const SegTable& t, int n_total, const int32_t* tokens, cudaStream_t s) {
   LaunchScope scope(wk, SPECASR_KIND_PREP, s);
-  launch_pdl(k_embed_tokens, dim3(n_total), dim3(128), 0, s, t, tokens, wk->m->embed, wk->m->cfg.d_model, wk->ws.X);
+  launch_pdl(k_embed_tokens, dim3(n_total), dim3(128), 0, s, t, tokens, wk->m->embed, wk->m->cfg.d_model, wk->ws.X
+             SPECASR_TRACE_ARG(wk));
 }
 
 void launch_copy_embeds(specasr_kv* kv, const float* embeds, int n, cudaStream_t s) {
@@ -172,10 +177,11 @@ __global__ void __launch_bounds__(256) k_rmsnorm_split(const int32_t* __restrict
                                                        const float* __restrict__ P, int n_partials,
                                                        size_t partial_stride, const float* __restrict__ gain,
                                                        int d, int d_part, float eps, int n, size_t plane_stride,
-                                                       bf16* __restrict__ H) {
+                                                       bf16* __restrict__ H SPECASR_TRACE_PARAM) {
   namespace cg = cooperative_groups;
   __shared__ float s_ss[kNormCluster];
   grid_dep_launch();
+  SPECASR_TRACE_SCOPE(tr, SPECASR_KIND_NORM);
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = (int)cluster.block_rank();
   const int row = blockIdx.x / kNormCluster;
@@ -189,6 +195,7 @@ __global__ void __launch_bounds__(256) k_rmsnorm_split(const int32_t* __restrict
     g[it] = kk[it] < k_end ? *reinterpret_cast<const float4*>(gain + kk[it]) : make_float4(0.f, 0.f, 0.f, 0.f);
   }
   grid_dep_wait();
+  SPECASR_TRACE_MARK();
   if (ctl[CTL_STATUS] != 0) return;          // same for the whole cluster
   bf16* hi = H + (size_t)row * d;
   bf16* lo = hi + plane_stride;
@@ -259,7 +266,8 @@ void launch_rmsnorm_split(specasr_kv* kv, const int32_t* ctl, const float* gain,
   LaunchScope scope(kv, SPECASR_KIND_NORM, s);
 #define NORM_LAUNCH(I)                                                                                           \
   launch_pdl_cluster(k_rmsnorm_split<I>, dim3(kNormCluster * n_pad), dim3(256), kNormCluster, s, ctl,          \
-                     kv->ws.X, kv->ws.P, n_partials, stride, gain, d, d_part, m->cfg.rms_eps, n, stride, kv->ws.H)
+                     kv->ws.X, kv->ws.P, n_partials, stride, gain, d, d_part, m->cfg.rms_eps, n, stride, kv->ws.H \
+                     SPECASR_TRACE_ARG(kv))
   if (d_part <= 1024) NORM_LAUNCH(1);
   else if (d_part <= 2048) NORM_LAUNCH(2);
   else if (d_part <= 4096) NORM_LAUNCH(4);
@@ -280,9 +288,11 @@ __global__ void __launch_bounds__(128) k_rope_append(const __grid_constant__ Seg
                                                      int n_partials, size_t partial_stride, int qkv_dim, int Hq, int Hkv,
                                                      int dh, const int32_t* __restrict__ pos,
                                                      const float2* __restrict__ rope, int layer, bf16* __restrict__ Q,
-                                                     size_t q_plane_stride, int page_size) {
+                                                     size_t q_plane_stride, int page_size SPECASR_TRACE_PARAM) {
   grid_dep_launch();
+  SPECASR_TRACE_SCOPE(tr, SPECASR_KIND_ROPE);
   grid_dep_wait();
+  SPECASR_TRACE_MARK();
   const int i = blockIdx.x;                    // workspace row
   const SegDev& sg = tab.seg[segment_of_row(tab, i)];
   const int32_t* ctl = sg.ctl;
@@ -354,7 +364,7 @@ void launch_rope_append(specasr_kv* wk, const SegTable& t, int n_total, int laye
   LaunchScope scope(wk, SPECASR_KIND_ROPE, s);
   launch_pdl(k_rope_append, grid, dim3(128), 0, s, t, wk->ws.P, n_partials, (size_t)wk->n_alloc * m->qkv_dim, m->qkv_dim,
              c.n_heads, c.n_kv_heads, c.head_dim, wk->ws.pos, m->rope_table, layer, wk->ws.Q,
-             (size_t)wk->n_alloc * m->q_dim, c.page_size);
+             (size_t)wk->n_alloc * m->q_dim, c.page_size SPECASR_TRACE_ARG(wk));
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -366,9 +376,11 @@ void launch_rope_append(specasr_kv* wk, const SegTable& t, int n_total, int laye
 __global__ void __launch_bounds__(128) k_attn_merge(const int32_t* __restrict__ ctl, const float* __restrict__ attO,
                                                     const float2* __restrict__ attML, int n_splits, size_t rows_alloc,
                                                     int Hq, int dh, int n, int rows_total, bf16* __restrict__ AO,
-                                                    size_t plane_stride) {
+                                                    size_t plane_stride SPECASR_TRACE_PARAM) {
   grid_dep_launch();
+  SPECASR_TRACE_SCOPE(tr, SPECASR_KIND_ATTN_MERGE);
   grid_dep_wait();
+  SPECASR_TRACE_MARK();
   if (ctl[CTL_STATUS] != 0) return;
   const int lane = threadIdx.x & 31;
   const int row = blockIdx.x * 4 + (threadIdx.x >> 5);       // = node * Hq + head
@@ -426,7 +438,7 @@ void launch_attn_merge(specasr_kv* kv, const int32_t* ctl, int n, int n_pad, int
   LaunchScope scope(kv, SPECASR_KIND_ATTN_MERGE, s);
   launch_pdl(k_attn_merge, dim3((rows_total + 3) / 4), dim3(128), 0, s, ctl, kv->ws.attO, kv->ws.attML, n_splits,
              (size_t)kv->n_alloc * c.n_heads, c.n_heads, c.head_dim, n, rows_total, kv->ws.AO,
-             (size_t)kv->n_alloc * kv->m->q_dim);
+             (size_t)kv->n_alloc * kv->m->q_dim SPECASR_TRACE_ARG(kv));
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -439,9 +451,11 @@ __global__ void __launch_bounds__(256) k_accept(const __grid_constant__ SegTable
                                                 const int32_t* __restrict__ parent,
                                                 const int32_t* __restrict__ depth,
                                                 int32_t* __restrict__ out_argmax, int32_t* __restrict__ out_accept_len,
-                                                int32_t* __restrict__ out_path, int32_t* __restrict__ out_bonus) {
+                                                int32_t* __restrict__ out_path, int32_t* __restrict__ out_bonus
+                                                SPECASR_TRACE_PARAM) {
   __shared__ int s_arg[SPECASR_MAX_NODES];
   __shared__ unsigned int s_best;
+  SPECASR_TRACE_SCOPE(tr, SPECASR_KIND_ACCEPT);
   const int i = threadIdx.x;
   const SegDev& sg = tab.seg[blockIdx.x];
   int32_t* ctl = sg.ctl;
@@ -456,6 +470,7 @@ __global__ void __launch_bounds__(256) k_accept(const __grid_constant__ SegTable
   if (out_bonus) out_bonus += blockIdx.x;
   grid_dep_launch();
   grid_dep_wait();
+  SPECASR_TRACE_MARK();
   // a failure of the kernels shared by a whole batch (a bounded wait that ran out) fails every utterance
   const int shared_status = ctl_shared ? ctl_shared[CTL_STATUS] : 0;
   if (ctl[CTL_STATUS] != 0 || shared_status != 0) {
@@ -529,7 +544,7 @@ void launch_accept(specasr_kv* wk, const SegTable& t, const int32_t* ctl_shared,
                    int32_t* out_bonus, cudaStream_t s) {
   LaunchScope scope(wk, SPECASR_KIND_ACCEPT, s);
   launch_pdl(k_accept, dim3(t.count), dim3(256), 0, s, t, ctl_shared, wk->ws.amax, n_tiles, wk->n_alloc, tokens, parent,
-             wk->ws.depth, out_argmax, out_accept_len, out_path, out_bonus);
+             wk->ws.depth, out_argmax, out_accept_len, out_path, out_bonus SPECASR_TRACE_ARG(wk));
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -152,6 +152,22 @@ class DeviceKV:
     def launches(self) -> int:
         return B.specasr_launch_count(self.handle)
 
+    def trace(self, fn, capacity: int = 1 << 16):
+        """Runs fn() with the device-side trace on and returns the records as an int64 array [records, 4]
+        (kind, start ns, end ns, wait-end ns), sorted by start time."""
+        buf = torch.zeros(2 + 4 * capacity, dtype=torch.int64, device=self.model.device)
+        torch.cuda.synchronize()
+        B.specasr_trace_set(self.handle, buf.data_ptr(), capacity)
+        try:
+            fn()
+            torch.cuda.synchronize()
+        finally:
+            B.specasr_trace_set(self.handle, 0, 0)
+        host = buf.cpu().numpy()
+        n = min(int(host[0]), capacity)
+        rec = host[2:2 + 4 * n].reshape(n, 4)
+        return rec[np.argsort(rec[:, 1], kind="stable")]
+
     def read_kv(self, layer: int, n_slots: int):
         """Host copy of K and V of slots [0, n_slots) of one layer as fp64 [n, Hkv, dh] (hi + lo)."""
         cfg = self.model.cfg

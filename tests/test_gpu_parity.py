@@ -450,3 +450,64 @@ def test_random_tree_shapes(cfg_name):
         O.commit(cache, want)
         assert kv.length() == cache.length
         root = got["bonus"]
+
+
+_TRACE_SCRIPT = r"""
+import numpy as np, torch, gen
+from paper_2507_18181_b200 import binding as B, build
+from paper_2507_18181_b200.runtime import DeviceModel, DeviceKV
+assert B.TRACE_LIB
+build.build(trace=True)
+cfg = gen.get_config("tiny")
+model = DeviceModel(cfg, gen.WeightStore(cfg, 0))
+kv = DeviceKV(model, max_tokens=256, max_nodes=64)
+kv.prefill_embeds(torch.from_numpy(gen.audio_prefix(40, cfg.d_model, 0)).cuda())
+parent = gen.complete_binary_tree(15)
+tokens = gen.fill_tree_tokens(parent, cfg.vocab, seed=0, root_token=7)
+d_t, d_p = torch.from_numpy(tokens).cuda(), torch.from_numpy(parent).cuda()
+kv.verify(d_t, d_p)
+torch.cuda.synchronize()
+plain = kv.out_argmax[:15].clone()
+rec = kv.trace(lambda: kv.verify(d_t, d_p))
+kinds = [B.KIND_NAMES[int(k)] for k in rec[:, 0]]
+# one launch each of prep, embedding, LM head and accept; per layer 2 norms, 4 projections, rotary, attention, merge
+assert kinds.count("accept") == 1 and "gemm_lm" in kinds
+for name in ("norm", "gemm_qkv", "rope", "attn", "attn_merge", "gemm_o", "gemm_gu", "gemm_down"):
+    assert name in kinds, name
+assert np.all(rec[:, 2] >= rec[:, 1])                              # every block ended after it started
+assert np.all((rec[:, 3] == 0) | ((rec[:, 3] >= rec[:, 1]) & (rec[:, 3] <= rec[:, 2])))
+assert kinds[0] == "prep" and int(np.argmax(rec[:, 2])) == kinds.index("accept")
+assert torch.equal(kv.out_argmax[:15], plain)                      # tracing does not change results
+# a buffer that is too small keeps counting but writes only what fits
+small = torch.zeros(2 + 4 * 8 + 4, dtype=torch.int64, device="cuda")
+B.specasr_trace_set(kv.handle, small.data_ptr(), 8)
+kv.verify(d_t, d_p)
+torch.cuda.synchronize()
+B.specasr_trace_set(kv.handle, 0, 0)
+assert int(small[0].item()) == len(rec) and int(small[2 + 4 * 8:].abs().sum().item()) == 0
+small.zero_()                                                      # off again: nothing is written
+kv.verify(d_t, d_p)
+torch.cuda.synchronize()
+assert int(small.abs().sum().item()) == 0
+print("trace ok", len(rec))
+"""
+
+
+def test_device_trace_variant_records_every_block_and_product_library_refuses():
+    """The device-side trace is a build variant (libspecasr_trace.so, selected by SPECASR_TRACE_LIB=1), exercised
+    in a child process; the product library accepts only 'off'."""
+    import os
+    import subprocess
+    import sys
+    from paper_2507_18181_b200 import binding as B
+    cfg, store, model, kv = _gpu_stack("tiny", 0, 0)
+    buf = torch.zeros(64, dtype=torch.int64, device="cuda")
+    B.specasr_trace_set(kv.handle, 0, 0)
+    with pytest.raises(B.SpecasrError) as e:
+        B.specasr_trace_set(kv.handle, buf.data_ptr(), 8)
+    assert e.value.status == B.SPECASR_ERR_UNSUPPORTED
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, SPECASR_TRACE_LIB="1", PYTHONPATH=root + os.pathsep + os.environ.get("PYTHONPATH", ""))
+    res = subprocess.run([sys.executable, "-c", _TRACE_SCRIPT], env=env, cwd=root, capture_output=True, text=True,
+                         timeout=600)
+    assert res.returncode == 0 and "trace ok" in res.stdout, res.stdout + res.stderr
