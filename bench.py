@@ -68,9 +68,9 @@ def algorithmic_flops(cfg, L, n):
 
 # DRAM traffic (read + write, MB per launch) of the projection kernel from the ncu capture summarised in
 # profiles/k_proj_config3_2layers.md: 7B shape, 64 tokens.  Valid only for the kernel source it was taken on.
-PROJ_TRAFFIC_MB = {"gemm_qkv": 51.46, "gemm_o": 34.65, "gemm_gu": 248.17, "gemm_down": 124.97, "gemm_lm": 276.25}
+PROJ_TRAFFIC_MB = {"gemm_qkv": 51.45, "gemm_o": 34.65, "gemm_gu": 247.58, "gemm_down": 125.01, "gemm_lm": 275.95}
 PROJ_TRAFFIC_SOURCE_SHA256 = {
-    "gemm_tcgen05.cu": "327d2dd19f59270026f244e963c296d2727f02cc697402de3905cf5e1766e658",
+    "gemm_tcgen05.cu": "821a4515b0ec6dcf6681b35259d549dae46c591a5b3d678ab23b82df97d84f86",
     "sm100_ptx.cuh": "3a0c294121fb64b742ab3700569cef82a1922484c98acd5238167235b990940f",
 }
 
@@ -424,7 +424,7 @@ def run_ours(args, wl):
     ms, cnt = B.specasr_profile_read(kv.handle, stream.cuda_stream)
     B.specasr_profile_enable(kv.handle, 0)
     kernels = {k: {"launches_per_step": cnt[k] / prof_steps, "ms_per_step": ms[k] / prof_steps} for k in ms if cnt[k]}
-    in_flow = in_flow_from_child(args) if world == 1 else None
+    in_flow = in_flow_from_child(args) if world == 1 and not args.no_in_flow else None
     gb = gemm_weight_bytes(cfg)
     gemm_bytes_step = cfg.n_layers * (gb["gemm_qkv"] + gb["gemm_o"] + gb["gemm_gu"] + gb["gemm_down"]) + gb["gemm_lm"]
     gemm_ms_step = sum(ms[k] for k in gb) / prof_steps
@@ -697,6 +697,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="config 4: one JSON line per (draft shape, KV length) point")
     ap.add_argument("--in-flow", action="store_true", help=argparse.SUPPRESS)
+    ap.add_argument("--no-in-flow", action="store_true", help="skip the traced step (it runs in a child process)")
     args = ap.parse_args()
     if args.sweep:
         run_sweep(args)
