@@ -511,3 +511,23 @@ def test_device_trace_variant_records_every_block_and_product_library_refuses():
     res = subprocess.run([sys.executable, "-c", _TRACE_SCRIPT], env=env, cwd=root, capture_output=True, text=True,
                          timeout=600)
     assert res.returncode == 0 and "trace ok" in res.stdout, res.stdout + res.stderr
+
+
+def test_config1_matches_the_stored_oracle_values():
+    """Config 1 against tests/golden/config1_tiny_verify.json (written from the oracle alone by make_golden.py)."""
+    import json
+    import os
+    stored = json.load(open(os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden",
+                                         "config1_tiny_verify.json")))
+    cfg, store, model, kv = _gpu_stack("tiny", 0, 0)
+    kv.prefill_embeds(torch.from_numpy(gen.audio_prefix(64, cfg.d_model, 0)).cuda())
+    prompt = gen.prompt_tokens(8, cfg.vocab, 0)
+    kv.prefill_tokens(torch.from_numpy(prompt[:-1].copy()).cuda())
+    tokens, parent = np.asarray(stored["tokens"], np.int32), np.asarray(stored["parent"], np.int32)
+    got = _verify_gpu(cfg, kv, tokens, parent)
+    assert stored["min_top2_gap"] > GAP                     # every arg-max of this workload is decided clearly
+    assert list(got["argmax"]) == stored["argmax"]
+    assert got["accept_len"] == stored["accept_len"] == 3
+    assert list(got["path"][:4]) == stored["path"] and got["bonus"] == stored["bonus"]
+    assert np.allclose(got["logits"][0, :8], stored["logits_row0_first8"], rtol=0, atol=LOGIT_TOL)
+    assert abs(np.abs(got["logits"]).sum() - stored["logits_abs_sum"]) < 1e-4 * stored["logits_abs_sum"]

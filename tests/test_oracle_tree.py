@@ -226,3 +226,24 @@ def test_planted_mistakes_are_caught():
     assert np.abs(res["logits"][2] - ref).max() < 1e-10
     leaky = O.causal_forward(cfg, W, np.concatenate([x, O.embed(W, [5, 9])]))[-1]
     assert np.abs(leaky - ref).max() > 1e-6
+
+
+def test_oracle_reproduces_the_stored_config1_values():
+    """tests/golden/config1_tiny_verify.json was written by tests/golden/make_golden.py from the oracle alone; a
+    change to the oracle's arithmetic (or to the seeded generators) shows up here."""
+    import importlib.util
+    import json
+    import os
+    here = os.path.dirname(os.path.abspath(__file__))
+    spec = importlib.util.spec_from_file_location("make_golden", os.path.join(here, "golden", "make_golden.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    now = mod.compute()
+    stored = json.load(open(os.path.join(here, "golden", "config1_tiny_verify.json")))
+    assert stored["accept_len"] == 3 and stored["path"] == [0, 1, 3, 7]      # the workload's stated outcome
+    for key in ("tokens", "parent", "greedy_continuation", "argmax", "accept_len", "path", "bonus", "top2_ids_row0"):
+        assert now[key] == stored[key], key
+    for key in ("logits_row0_first8", "top2_probs_row0"):
+        assert np.allclose(now[key], stored[key], rtol=1e-9, atol=1e-12), key
+    assert abs(now["logits_abs_sum"] - stored["logits_abs_sum"]) <= 1e-7 * stored["logits_abs_sum"]
+    assert abs(now["min_top2_gap"] - stored["min_top2_gap"]) < 1e-9
