@@ -445,7 +445,7 @@ void launch_attn_merge(specasr_kv* kv, const int32_t* ctl, int n, int n_pad, int
 // Accept: reduce the per-vocab-tile argmax candidates, then follow draft tokens while they equal the
 // target's greedy token at their parent; the deepest such node (lowest index among equals) wins.
 // One block per utterance; arrays indexed by workspace row, out_accept_len / out_bonus by utterance.
-__global__ void __launch_bounds__(256) k_accept(const __grid_constant__ SegTable tab, const int32_t* __restrict__ ctl_shared,
+__global__ void __launch_bounds__(1024) k_accept(const __grid_constant__ SegTable tab, const int32_t* __restrict__ ctl_shared,
                                                 const unsigned long long* __restrict__ amax, int n_tiles,
                                                 int n_alloc, const int32_t* __restrict__ tokens,
                                                 const int32_t* __restrict__ parent,
@@ -454,7 +454,9 @@ __global__ void __launch_bounds__(256) k_accept(const __grid_constant__ SegTable
                                                 int32_t* __restrict__ out_path, int32_t* __restrict__ out_bonus
                                                 SPECASR_TRACE_PARAM) {
   __shared__ int s_arg[SPECASR_MAX_NODES];
-  __shared__ unsigned int s_best;
+  __shared__ int s_parent[SPECASR_MAX_NODES], s_token[SPECASR_MAX_NODES];   // the walks below would otherwise be
+  __shared__ unsigned int s_best;                                           // chains of dependent global loads
+  __shared__ unsigned long long s_red[16][64];
   SPECASR_TRACE_SCOPE(tr, SPECASR_KIND_ACCEPT);
   const int i = threadIdx.x;
   const SegDev& sg = tab.seg[blockIdx.x];
@@ -486,31 +488,40 @@ __global__ void __launch_bounds__(256) k_accept(const __grid_constant__ SegTable
     return;
   }
   if (i == 0) s_best = 0u;
-  // arg-max over the vocabulary tiles: one warp per node, lanes stride over the tiles, eight loads in flight
-  for (int node = i >> 5; node < n; node += 8) {
-    const int lane = i & 31;
+  if (i < n) {
+    s_parent[i] = parent[i];
+    s_token[i] = tokens[i];
+  }
+  // arg-max over the vocabulary tiles, 64 nodes at a time: thread (node, g) scans tiles g, g + 16, ... so that a warp
+  // reads 32 adjacent nodes of one tile (the candidates are [tile][node]); the 16 partial results meet in shared
+  // memory.  (One warp per node with the lanes striding over the tiles touched every 32-byte sector four times and
+  // took 12 us on the single SM this kernel runs on.)
+  for (int node0 = 0; node0 < n; node0 += 64) {
+    const int node = node0 + (i & 63), g = i >> 6;
     unsigned long long best = 0ull;
-    for (int t0 = 0; t0 < n_tiles; t0 += 256) {
-      unsigned long long v[8];
+    if (node < n) {
+      for (int t0 = g; t0 < n_tiles; t0 += 16 * 8) {
+        unsigned long long v[8];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int t = t0 + u * 32 + lane;
-        v[u] = t < n_tiles ? __ldcg(amax + (size_t)t * n_alloc + node) : 0ull;
+        for (int u = 0; u < 8; ++u) {
+          const int t = t0 + u * 16;
+          v[u] = t < n_tiles ? __ldcg(amax + (size_t)t * n_alloc + node) : 0ull;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) best = v[u] > best ? v[u] : best;
       }
-#pragma unroll
-      for (int u = 0; u < 8; ++u) best = v[u] > best ? v[u] : best;
     }
+    s_red[g][i & 63] = best;
+    __syncthreads();
+    if (i < 64 && node < n) {
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const unsigned long long other = __shfl_xor_sync(0xFFFFFFFFu, best, o);
-      best = other > best ? other : best;
-    }
-    if (lane == 0) {
+      for (int q = 0; q < 16; ++q) best = s_red[q][i] > best ? s_red[q][i] : best;
       const int tok = (int)(0xFFFFFFFFu - (unsigned int)(best & 0xFFFFFFFFull));
       s_arg[node] = tok;
       out_argmax[node] = tok;
       out_path[node] = -1;
     }
+    __syncthreads();
   }
   __syncthreads();
   if (i < n) {
@@ -518,8 +529,8 @@ __global__ void __launch_bounds__(256) k_accept(const __grid_constant__ SegTable
     int j = i;
     int steps = 0;
     while (j > 0 && steps <= n) {
-      const int p = parent[j];
-      ok = ok && (tokens[j] == s_arg[p]);
+      const int p = s_parent[j];
+      ok = ok && (s_token[j] == s_arg[p]);
       j = p;
       ++steps;
     }
@@ -534,7 +545,7 @@ __global__ void __launch_bounds__(256) k_accept(const __grid_constant__ SegTable
     int j = best;
     for (int k = a; k >= 0 && j >= 0; --k) {
       out_path[k] = j;
-      j = parent[j];
+      j = s_parent[j];
     }
   }
 }
@@ -543,7 +554,7 @@ void launch_accept(specasr_kv* wk, const SegTable& t, const int32_t* ctl_shared,
                    const int32_t* parent, int n_tiles, int32_t* out_argmax, int32_t* out_accept_len, int32_t* out_path,
                    int32_t* out_bonus, cudaStream_t s) {
   LaunchScope scope(wk, SPECASR_KIND_ACCEPT, s);
-  launch_pdl(k_accept, dim3(t.count), dim3(256), 0, s, t, ctl_shared, wk->ws.amax, n_tiles, wk->n_alloc, tokens, parent,
+  launch_pdl(k_accept, dim3(t.count), dim3(1024), 0, s, t, ctl_shared, wk->ws.amax, n_tiles, wk->n_alloc, tokens, parent,
              wk->ws.depth, out_argmax, out_accept_len, out_path, out_bonus SPECASR_TRACE_ARG(wk));
 }
 
