@@ -14,6 +14,7 @@ __global__ void k_tree_prep(const __grid_constant__ SegTable tab, const int32_t*
                             const int32_t* __restrict__ parent, int vocab, int32_t* __restrict__ depth,
                             int32_t* __restrict__ pos, unsigned long long* __restrict__ anc SPECASR_TRACE_PARAM) {
   __shared__ int s_bad;
+  __shared__ int s_parent[SPECASR_MAX_NODES];     // the ancestor walk would otherwise be a chain of global loads
   SPECASR_TRACE_SCOPE(tr, SPECASR_KIND_PREP);
   const int i = threadIdx.x;
   const SegDev& sg = tab.seg[blockIdx.x];
@@ -32,6 +33,7 @@ __global__ void k_tree_prep(const __grid_constant__ SegTable tab, const int32_t*
   const int L = ctl[CTL_LEN];
   if (i < n) {
     const int p = parent[i];
+    s_parent[i] = p;
     const int t = tokens ? tokens[i] : 0;
     const bool bad = (i == 0 ? p != -1 : (p < 0 || p >= i)) || t < 0 || t >= vocab;
     if (bad) atomicOr(&s_bad, 1);
@@ -49,7 +51,7 @@ __global__ void k_tree_prep(const __grid_constant__ SegTable tab, const int32_t*
     // parent[j] < j was checked above, so the walk ends after at most i + 1 steps
     while (j >= 0 && d <= n) {
       m[j >> 6] |= 1ull << (j & 63);
-      j = parent[j];
+      j = s_parent[j];
       ++d;
     }
     depth[i] = d - 1;
@@ -592,9 +594,12 @@ __global__ void __launch_bounds__(256) k_commit(const int32_t* __restrict__ ctl,
                                                 int n_pages, int Hkv, int page_size, int dh) {
   grid_dep_launch();
   grid_dep_wait();
+  __shared__ int s_path[SPECASR_MAX_NODES];      // read once, side by side, instead of one dependent load per step
   const int a = accept_len[0];
   const int n = ctl[CTL_N];
   if (ctl[CTL_STATUS] != 0 || a < 0 || a >= n) return;
+  for (int j = threadIdx.x; j <= a; j += blockDim.x) s_path[j] = path[j];
+  __syncthreads();
   const int L = ctl[CTL_LEN];
   const int layer = blockIdx.x;
   bf16* pool = blockIdx.y == 0 ? k_pool : v_pool;
@@ -606,7 +611,7 @@ __global__ void __launch_bounds__(256) k_commit(const int32_t* __restrict__ ctl,
     const int ch = c % chunks_per_row;
     int prev = 0;
     for (int j = 1; j <= a; ++j) {
-      const int pj = path[j];
+      const int pj = s_path[j];
       if (pj <= prev || pj >= n) break;   // not a root path of the pending tree: stop copying
       prev = pj;
       if (pj == j) continue;
