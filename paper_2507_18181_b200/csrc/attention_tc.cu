@@ -115,6 +115,13 @@ __global__ void __launch_bounds__(64 + SOFTMAX_THREADS, 1) k_tree_attention_tc(c
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  // The page table does not change during a call: lane j of the producer warp looks up the page of its key block
+  // now, so that after the wait only the length stands between it and the first K load.
+  int my_page = 0;
+  if (warp == 0) {
+    const int idx = split * (p.chunk / p.page_size) + lane;
+    if (lane < p.chunk / p.page_size && idx * p.page_size < sg.capacity) my_page = p.page_table[idx];
+  }
   // everything above is independent of the previous kernel; its results are read from here on
   SPECASR_TRACE_SCOPE(p.tr, SPECASR_KIND_ATTN);
   pdl_wait();
@@ -159,7 +166,7 @@ __global__ void __launch_bounds__(64 + SOFTMAX_THREADS, 1) k_tree_attention_tc(c
     int c4 = 0;
     const int off = lane * p.page_size * 128;
     if (lane < pages) {
-      c4 = p.layer * p.n_pages + p.page_table[k_begin / p.page_size + lane];
+      c4 = p.layer * p.n_pages + my_page;
       for (int plane = 0; plane < 2; ++plane)
         for (int h = 0; h < H; ++h)
           tma_load_5d(KVs + (plane * H + h) * KVSUB + off, tmK, h * 64, 0, plane, kvh, c4, &sc->bar_qk);

@@ -198,7 +198,8 @@ __global__ void __launch_bounds__(256) k_rmsnorm_split(const int32_t* __restrict
   }
   grid_dep_wait();
   SPECASR_TRACE_MARK();
-  if (ctl[CTL_STATUS] != 0) return;          // same for the whole cluster
+  const int status = row < n ? 0 : ctl[CTL_STATUS];   // rows that exist read it behind their data loads (below)
+  if (status != 0) return;                   // same for the whole cluster
   bf16* hi = H + (size_t)row * d;
   bf16* lo = hi + plane_stride;
   if (row >= n) {                            // same for the whole cluster
@@ -215,6 +216,7 @@ __global__ void __launch_bounds__(256) k_rmsnorm_split(const int32_t* __restrict
 #pragma unroll
   for (int it = 0; it < ITER; ++it)
     v[it] = kk[it] < k_end ? *reinterpret_cast<const float4*>(x + kk[it]) : make_float4(0.f, 0.f, 0.f, 0.f);
+  const int late_status = ctl[CTL_STATUS];   // requested behind the row's data instead of in front of it
   constexpr int BATCH = ITER == 1 ? kMaxSplitK : (ITER == 2 ? 6 : 3);
   for (int s0 = 0; s0 < n_partials; s0 += BATCH) {
     float4 q[BATCH][ITER];
@@ -232,6 +234,7 @@ __global__ void __launch_bounds__(256) k_rmsnorm_split(const int32_t* __restrict
         v[it].x += q[u][it].x; v[it].y += q[u][it].y; v[it].z += q[u][it].z; v[it].w += q[u][it].w;
       }
   }
+  if (late_status != 0) return;              // same for the whole cluster; nothing has been written yet
   float ss = 0.f;
 #pragma unroll
   for (int it = 0; it < ITER; ++it) {
@@ -298,7 +301,6 @@ __global__ void __launch_bounds__(128) k_rope_append(const __grid_constant__ Seg
   const int i = blockIdx.x;                    // workspace row
   const SegDev& sg = tab.seg[segment_of_row(tab, i)];
   const int32_t* ctl = sg.ctl;
-  if (ctl[CTL_STATUS] != 0) return;
   const int half = dh >> 1;
   const int per_head = half >> 2;              // threads per head: four rotation pairs each
   const int head = blockIdx.y * (blockDim.x / per_head) + threadIdx.x / per_head;
@@ -309,11 +311,7 @@ __global__ void __launch_bounds__(128) k_rope_append(const __grid_constant__ Seg
   const bool is_v = head >= Hq + Hkv;
   float4 x1 = make_float4(0.f, 0.f, 0.f, 0.f), x2 = x1;
   float4 cs01 = make_float4(1.f, 0.f, 1.f, 0.f), cs23 = cs01;      // (cos, sin) of pairs k, k+1 and k+2, k+3
-  if (!is_v) {
-    const float4* t = reinterpret_cast<const float4*>(rope + (size_t)pos[i] * half + k);
-    cs01 = t[0];
-    cs23 = t[1];
-  }
+  int status = 0, len = 0;
   for (int s0 = 0; s0 < n_partials; s0 += 4) {   // four planes in flight, summed in plane order
     float4 a1[4], a2[4];
 #pragma unroll
@@ -322,12 +320,28 @@ __global__ void __launch_bounds__(128) k_rope_append(const __grid_constant__ Seg
       a1[s] = on ? __ldcg(reinterpret_cast<const float4*>(P + (s0 + s) * partial_stride + c1)) : make_float4(0.f, 0.f, 0.f, 0.f);
       a2[s] = on ? __ldcg(reinterpret_cast<const float4*>(P + (s0 + s) * partial_stride + c2)) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
+    if (s0 == 0) {
+      // the small loads that depend on one another (status, position -> table row, length) go out behind the
+      // plane loads instead of in front of them: an in-order core would otherwise wait for each before the next
+      status = ctl[CTL_STATUS];
+      len = ctl[CTL_LEN];
+      if (!is_v) {
+        const float4* t = reinterpret_cast<const float4*>(rope + (size_t)pos[i] * half + k);
+        cs01 = t[0];
+        cs23 = t[1];
+      }
+    }
 #pragma unroll
     for (int s = 0; s < 4; ++s) {
       x1.x += a1[s].x; x1.y += a1[s].y; x1.z += a1[s].z; x1.w += a1[s].w;
       x2.x += a2[s].x; x2.y += a2[s].y; x2.z += a2[s].z; x2.w += a2[s].w;
     }
   }
+  if (n_partials <= 0) {
+    status = ctl[CTL_STATUS];
+    len = ctl[CTL_LEN];
+  }
+  if (status != 0) return;                       // nothing is written for an utterance whose tree was refused
   // r1 = x1 cos - x2 sin, r2 = x2 cos + x1 sin (identity for V: cos = 1, sin = 0)
   const float4 r1 = make_float4(x1.x * cs01.x - x2.x * cs01.y, x1.y * cs01.z - x2.y * cs01.w,
                                 x1.z * cs23.x - x2.z * cs23.y, x1.w * cs23.z - x2.w * cs23.w);
@@ -345,7 +359,7 @@ __global__ void __launch_bounds__(128) k_rope_append(const __grid_constant__ Seg
     plane = q_plane_stride;
   } else {
     const int kvh = is_v ? head - Hq - Hkv : head - Hq;
-    const int slot = ctl[CTL_LEN] + (i - sg.row0);
+    const int slot = len + (i - sg.row0);
     const int page = sg.page_table[slot / page_size];
     const int off = slot % page_size;
     dst = (is_v ? sg.v_pool : sg.k_pool) + kv_plane_offset(layer, sg.n_pages, Hkv, page_size, dh, page, kvh, 0) +
@@ -399,29 +413,42 @@ __global__ void __launch_bounds__(128) k_attn_merge(const int32_t* __restrict__ 
   const float2 none = make_float2(-INFINITY, 0.f);
   const float2 ml0 = lane < n_splits ? __ldcg(attML + (size_t)lane * rows_alloc + row) : none;
   const float2 ml1 = lane + 32 < n_splits ? __ldcg(attML + (size_t)(lane + 32) * rows_alloc + row) : none;
+  // The partial outputs are requested whatever their weights turn out to be, the first six right behind the
+  // (max, sum) pairs, so that no load waits for another; an empty key block's output was never written and is
+  // dropped below.
+  constexpr int B6 = 6;
+  float4 o[B6];
+#pragma unroll
+  for (int u = 0; u < B6; ++u)
+    o[u] = (u < n_splits && c < dh) ? __ldcg(reinterpret_cast<const float4*>(attO + ((size_t)u * rows_alloc + row) * dh + c))
+                                    : make_float4(0.f, 0.f, 0.f, 0.f);
   float mx = fmaxf(ml0.y > 0.f ? ml0.x : -INFINITY, ml1.y > 0.f ? ml1.x : -INFINITY);
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+  for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
   const float w0 = ml0.y > 0.f ? exp2f(ml0.x - mx) : 0.f;
   const float w1 = ml1.y > 0.f ? exp2f(ml1.x - mx) : 0.f;
   // denominator: the terms are added one by one in split order, so the result does not depend on timing
   float den = 0.f;
   for (int s = 0; s < n_splits; ++s) den += __shfl_sync(0xFFFFFFFFu, s < 32 ? ml0.y * w0 : ml1.y * w1, s & 31);
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int s0 = 0; s0 < n_splits; s0 += 6) {
-    float4 o[6];
-    float w[6];
+  for (int s0 = 0; s0 < n_splits; s0 += B6) {
+    if (s0 > 0) {
 #pragma unroll
-    for (int u = 0; u < 6; ++u) {
-      const int s = s0 + u;
-      w[u] = __shfl_sync(0xFFFFFFFFu, s < 32 ? w0 : w1, s & 31);
-      if (s >= n_splits) w[u] = 0.f;
-      o[u] = (w[u] > 0.f && c < dh) ? __ldcg(reinterpret_cast<const float4*>(attO + ((size_t)s * rows_alloc + row) * dh + c))
-                                    : make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int u = 0; u < B6; ++u) {
+        const int s = s0 + u;
+        o[u] = (s < n_splits && c < dh) ? __ldcg(reinterpret_cast<const float4*>(attO + ((size_t)s * rows_alloc + row) * dh + c))
+                                        : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
     }
 #pragma unroll
-    for (int u = 0; u < 6; ++u) {
-      acc.x += o[u].x * w[u]; acc.y += o[u].y * w[u]; acc.z += o[u].z * w[u]; acc.w += o[u].w * w[u];
+    for (int u = 0; u < B6; ++u) {
+      const int s = s0 + u;
+      float w = __shfl_sync(0xFFFFFFFFu, s < 32 ? w0 : w1, s & 31);
+      if (s >= n_splits || !(w > 0.f)) {
+        w = 0.f;
+        o[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+      acc.x += o[u].x * w; acc.y += o[u].y * w; acc.z += o[u].z * w; acc.w += o[u].w * w;
     }
   }
   if (c < dh) {
