@@ -226,16 +226,24 @@ def in_flow_times(kv, step, kind_names):
     rec = kv.trace(step, capacity=1 << 18)
     if len(rec) == 0:
         return None
-    launches = []                      # [kind, first start, last start, last end]
-    for kind, start, end, _ in rec:
-        if launches and launches[-1][0] == kind and start - launches[-1][2] < 20000:
-            launches[-1][2] = max(launches[-1][2], start)
-            launches[-1][3] = max(launches[-1][3], end)
-        else:
-            launches.append([int(kind), int(start), int(start), int(end)])
+    # launches of one kind lie a whole layer (or half of one) apart, blocks of one launch start within a few us of
+    # one another: cut each kind's records where consecutive starts are more than 30 us apart
+    launches = []                      # [kind, first start, last end]
+    for kind in sorted(set(int(k) for k in rec[:, 0])):
+        r = rec[rec[:, 0] == kind]
+        r = r[np.argsort(r[:, 1], kind="stable")]
+        first, last_start, end = int(r[0, 1]), int(r[0, 1]), int(r[0, 2])
+        for _, start, e, _w in r[1:]:
+            if start - last_start > 30000:
+                launches.append([kind, first, end])
+                first, end = int(start), int(e)
+            last_start = int(start)
+            end = max(end, int(e))
+        launches.append([kind, first, end])
+    launches.sort(key=lambda l: l[1])
     out = {}
     latest = launches[0][1]
-    for kind, _, _, end in launches:
+    for kind, _, end in launches:
         name = kind_names[kind]
         d = out.setdefault(name, {"launches": 0, "us_per_step": 0.0})
         d["launches"] += 1
