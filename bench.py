@@ -41,6 +41,11 @@ METRIC = "tree_tokens_per_s"
 UNIT = "tree tokens/s"
 
 
+def workload_keys(wl):
+    """The workload's parameters for the JSON line (the decoder shape is named `decoder_shape`)."""
+    return {("decoder_shape" if k == "model" else k): v for k, v in wl.items()}
+
+
 def model_config(wl):
     over = {"n_layers": wl["n_layers"]} if "n_layers" in wl else {}
     return gen.get_config(wl["model"], **over)
@@ -210,7 +215,7 @@ def run_reference(args, wl):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_call * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": args.workload, **{k: v for k, v in wl.items()}},
+        "config": {"workload": args.workload, **workload_keys(wl)},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
@@ -452,7 +457,7 @@ def run_ours(args, wl):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": args.workload, **wl, "kv_len": L, "page_size": model.page_size,
+        "config": {"workload": args.workload, **workload_keys(wl), "kv_len": L, "page_size": model.page_size,
                    "kv_storage": "bf16 hi+lo planes (4 bytes/element)", "l2": "inputs larger than L2 (weights "
                    f"{ab['weights'] / 1e9:.2f} GB per step)", "parallelism": "replicas" if world > 1 else "single"},
         "latency_ms": {"mean": ms_per_step, "median": per_step[len(per_step) // 2], "min": per_step[0]},
