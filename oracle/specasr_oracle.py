@@ -38,7 +38,8 @@ pairing and GQA grouping; torch's scaled_dot_product_attention for the masked
 attention; closed forms for RMSNorm / softmax / SiLU / RoPE; brute force over
 root paths for the tree forward and for the accept rule; a plain prefill of the
 accepted path for the commit; scipy's softmax, a hand-computed row and a brute-force sort for
-top2_probs.  The paper prints no worked numbers for this step,
+top2_probs; a full sort, hand rows and a tie for top2_gap; hand-built trees with supplied logits for
+the `decisive` flag of `decide`.  The paper prints no worked numbers for this step,
 so parity with numbers *in the paper* is unpinned; only its lossless property
 binds, and the tests check it.
 """
@@ -247,6 +248,11 @@ def tree_prep(parent) -> tuple[np.ndarray, np.ndarray]:
 
 
 def top2_gap(logits: np.ndarray) -> np.ndarray:
+    """Largest entry minus second largest entry along the last axis (0 where the maximum is attained twice;
+    +inf for a single column, where nothing can overtake the only candidate)."""
+    logits = np.asarray(logits, dtype=F64)
+    if logits.shape[-1] < 2:
+        return np.full(logits.shape[:-1], np.inf)
     part = np.partition(logits, -2, axis=-1)
     return part[..., -1] - part[..., -2]
 
@@ -312,17 +318,52 @@ def verify_tree(cfg, weights: Weights, cache: KVCache, tokens, parent, decisive_
     pos = cache.length + depth
     hidden, tk, tv = decoder_stack(cfg, weights, embed(weights, tokens), pos, anc, cache)
     logits = lm_logits(cfg, weights, hidden)
+    res = decide(tokens, parent, logits, decisive_gap)
+    res.update({"depth": depth, "pos": pos, "tree_K": tk, "tree_V": tv})
+    return res
+
+
+def verify_tree_uncached(cfg, weights: Weights, prefix_inputs: np.ndarray, tokens, parent,
+                         decisive_gap: float = 1e-2) -> dict:
+    """The same round without a cache object: the context rows and the tree rows go through the layer
+    stack together, the context under causal attention, every tree node seeing the whole context and
+    its own root path (Section II-B: the tree is verified in one pass on top of the decoded text).
+    One pass over the weights instead of two, which is what makes the 7B shape affordable when the
+    layers are regenerated one at a time.  Equal to prefill + verify_tree (tested)."""
+    tokens = np.asarray(tokens, dtype=np.int64)
+    depth, anc = tree_prep(parent)
+    if np.any(tokens < 0) or np.any(tokens >= cfg.vocab):
+        raise TreeError("token id out of range")
+    L, n = prefix_inputs.shape[0], len(tokens)
+    x = np.concatenate([np.asarray(prefix_inputs, dtype=F64), embed(weights, tokens)], axis=0)
+    pos = np.concatenate([np.arange(L), L + depth])
+    mask = np.zeros((L + n, L + n), dtype=bool)
+    mask[:L, :L] = np.tril(np.ones((L, L), dtype=bool))
+    mask[L:, :L] = True
+    mask[L:, L:] = anc
+    hidden, nk, nv = decoder_stack(cfg, weights, x, pos, mask, None)
+    res = decide(tokens, parent, lm_logits(cfg, weights, hidden[L:]), decisive_gap)
+    res.update({"depth": depth, "pos": pos[L:], "tree_K": [k[L:] for k in nk], "tree_V": [v[L:] for v in nv],
+                "prefix_K": [k[:L] for k in nk], "prefix_V": [v[:L] for v in nv]})
+    return res
+
+
+def decide(tokens, parent, logits: np.ndarray, decisive_gap: float = 1e-2) -> dict:
+    """From the logits of every node to the round's outcome: greedy tokens, their margins, the accept
+    result, and whether that result is unambiguous.  The accept rule reads the arg-max of every node
+    that has a child (to test the child's token) and of the winning node (the bonus token); the result
+    is `decisive` when each of those was decided by more than `decisive_gap`.  A narrow margin at a
+    childless node that does not win changes nothing that is reported."""
+    logits = np.asarray(logits, dtype=F64)
+    n = len(tokens)
     argmax = np.argmax(logits, axis=-1).astype(np.int32)
     gap = top2_gap(logits)
     res = accept(tokens, parent, argmax)
-    is_parent = np.zeros(len(tokens), dtype=bool)
-    is_parent[np.asarray(parent)[1:]] = True
-    consulted = is_parent.copy()
+    consulted = np.zeros(n, dtype=bool)
+    consulted[np.asarray(parent, dtype=np.int64)[1:]] = True
     consulted[res["best"]] = True
     res.update({
-        "logits": logits, "argmax": argmax, "gap": gap, "depth": depth, "pos": pos,
-        "tree_K": tk, "tree_V": tv,
-        # the accept result is unambiguous when every argmax it reads is decided by a clear margin
+        "logits": logits, "argmax": argmax, "gap": gap, "consulted": consulted,
         "decisive": bool(np.all(gap[consulted] > decisive_gap)),
     })
     return res

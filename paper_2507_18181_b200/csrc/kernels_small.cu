@@ -117,15 +117,24 @@ __device__ __forceinline__ int segment_of_row(const SegTable& tab, int row) {
   return b;
 }
 
+// A token id outside [0, vocab) is never turned into an address: the row is skipped and the utterance's status
+// word is set, which turns the rest of the call into no-ops (tree verification has checked the ids before; a
+// context fill has not).
 __global__ void k_embed_tokens(const __grid_constant__ SegTable tab, const int32_t* __restrict__ tokens,
-                               const bf16* __restrict__ E, int d, float* __restrict__ X SPECASR_TRACE_PARAM) {
+                               const bf16* __restrict__ E, int d, int vocab, float* __restrict__ X SPECASR_TRACE_PARAM) {
   grid_dep_launch();
   SPECASR_TRACE_SCOPE(tr, SPECASR_KIND_PREP);
   grid_dep_wait();
   SPECASR_TRACE_MARK();
   const int i = blockIdx.x;
-  if (tab.seg[segment_of_row(tab, i)].ctl[CTL_STATUS] != 0) return;
-  const bf16* row = E + (size_t)tokens[i] * d;
+  int32_t* ctl = tab.seg[segment_of_row(tab, i)].ctl;
+  if (ctl[CTL_STATUS] != 0) return;
+  const int tok = tokens[i];
+  if (tok < 0 || tok >= vocab) {
+    if (threadIdx.x == 0) ctl[CTL_STATUS] = SPECASR_ERR_INVALID_TREE;
+    return;
+  }
+  const bf16* row = E + (size_t)tok * d;
   float* x = X + (size_t)i * d;
   for (int k = threadIdx.x * 8; k < d; k += blockDim.x * 8) {
     const uint4 v = *reinterpret_cast<const uint4*>(row + k);
@@ -152,8 +161,8 @@ __global__ void k_copy_embeds(const int32_t* __restrict__ ctl, const float* __re
 
 void launch_embed_tokens(specasr_kv* wk, const SegTable& t, int n_total, const int32_t* tokens, cudaStream_t s) {
   LaunchScope scope(wk, SPECASR_KIND_PREP, s);
-  launch_pdl(k_embed_tokens, dim3(n_total), dim3(128), 0, s, t, tokens, wk->m->embed, wk->m->cfg.d_model, wk->ws.X
-             SPECASR_TRACE_ARG(wk));
+  launch_pdl(k_embed_tokens, dim3(n_total), dim3(128), 0, s, t, tokens, wk->m->embed, wk->m->cfg.d_model,
+             wk->m->cfg.vocab, wk->ws.X SPECASR_TRACE_ARG(wk));
 }
 
 void launch_copy_embeds(specasr_kv* kv, const float* embeds, int n, cudaStream_t s) {
@@ -293,7 +302,8 @@ __global__ void __launch_bounds__(128) k_rope_append(const __grid_constant__ Seg
                                                      int n_partials, size_t partial_stride, int qkv_dim, int Hq, int Hkv,
                                                      int dh, const int32_t* __restrict__ pos,
                                                      const float2* __restrict__ rope, int layer, bf16* __restrict__ Q,
-                                                     size_t q_plane_stride, int page_size SPECASR_TRACE_PARAM) {
+                                                     size_t q_plane_stride, int page_size, int max_positions
+                                                     SPECASR_TRACE_PARAM) {
   grid_dep_launch();
   SPECASR_TRACE_SCOPE(tr, SPECASR_KIND_ROPE);
   grid_dep_wait();
@@ -326,7 +336,9 @@ __global__ void __launch_bounds__(128) k_rope_append(const __grid_constant__ Seg
       status = ctl[CTL_STATUS];
       len = ctl[CTL_LEN];
       if (!is_v) {
-        const float4* t = reinterpret_cast<const float4*>(rope + (size_t)pos[i] * half + k);
+        // the position is read before the status is known (a refused call never wrote it): keep the row inside the table
+        const int pp = min(max(pos[i], 0), max_positions - 1);
+        const float4* t = reinterpret_cast<const float4*>(rope + (size_t)pp * half + k);
         cs01 = t[0];
         cs23 = t[1];
       }
@@ -380,7 +392,7 @@ void launch_rope_append(specasr_kv* wk, const SegTable& t, int n_total, int laye
   LaunchScope scope(wk, SPECASR_KIND_ROPE, s);
   launch_pdl(k_rope_append, grid, dim3(128), 0, s, t, wk->ws.P, n_partials, (size_t)wk->n_alloc * m->qkv_dim, m->qkv_dim,
              c.n_heads, c.n_kv_heads, c.head_dim, wk->ws.pos, m->rope_table, layer, wk->ws.Q,
-             (size_t)wk->n_alloc * m->q_dim, c.page_size SPECASR_TRACE_ARG(wk));
+             (size_t)wk->n_alloc * m->q_dim, c.page_size, c.max_positions SPECASR_TRACE_ARG(wk));
 }
 
 // ------------------------------------------------------------------------------------------------

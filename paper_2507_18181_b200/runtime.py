@@ -89,7 +89,11 @@ class DeviceModel:
 class DeviceKV:
     """Paged KV cache + workspace for one utterance."""
 
-    def __init__(self, model: DeviceModel, max_tokens: int, max_nodes: int = 256, shuffle_pages_seed=None):
+    def __init__(self, model: DeviceModel, max_tokens: int, max_nodes: int = 256, shuffle_pages_seed=None,
+                 poison: bool = False):
+        """`poison` fills both pools and the workspace with 0xFF bytes (NaN as bf16 and fp32, -1 as int32)
+        instead of zeros before the handle is created: a kernel that reads something no kernel wrote then
+        produces NaN or an error instead of a silently plausible result."""
         self.model = model
         cfg = model.cfg
         dev = model.device
@@ -100,6 +104,9 @@ class DeviceKV:
         pool_bytes = B.specasr_kv_pool_bytes(model.handle, self.n_pages)
         self.k_pool = torch.zeros(pool_bytes // 2, dtype=torch.bfloat16, device=dev)
         self.v_pool = torch.zeros(pool_bytes // 2, dtype=torch.bfloat16, device=dev)
+        if poison:
+            self.k_pool.view(torch.uint8).fill_(0xFF)
+            self.v_pool.view(torch.uint8).fill_(0xFF)
         if shuffle_pages_seed is None:
             table = np.arange(self.max_pages, dtype=np.int32)
         else:
@@ -107,7 +114,7 @@ class DeviceKV:
         self.page_table_host = table
         self.page_table = torch.from_numpy(table).to(dev)
         ws_bytes = B.specasr_workspace_bytes(model.handle, max_nodes)
-        self.workspace = torch.zeros(ws_bytes + 256, dtype=torch.uint8, device=dev)
+        self.workspace = torch.full((ws_bytes + 256,), 0xFF if poison else 0, dtype=torch.uint8, device=dev)
         ws_ptr = (self.workspace.data_ptr() + 255) // 256 * 256
         self.handle = B.specasr_kv_create(model.handle, self.k_pool.data_ptr(), self.v_pool.data_ptr(), self.n_pages,
                                           self.page_table.data_ptr(), self.max_pages, ws_ptr, max_nodes)

@@ -156,3 +156,81 @@ def test_top2_probs_against_library_softmax_hand_values_and_sorting():
     # shifting a row by a constant changes nothing; a huge offset must not overflow
     ids2, probs2 = O.top2_probs(logits + 1000.0)
     assert np.array_equal(ids2, ids) and np.allclose(probs2, probs, rtol=1e-10)
+
+
+def test_top2_gap_against_a_full_sort_hand_rows_and_a_tie():
+    """The margin that decides which arg-max entries are compared bit-exactly: pinned to a full sort, to rows
+    worked by hand, to a tie (margin 0) and to the one-column case."""
+    rng = np.random.default_rng(3)
+    x = rng.standard_normal((7, 50))
+    s = np.sort(x, axis=-1)
+    assert np.array_equal(O.top2_gap(x), s[:, -1] - s[:, -2])
+    assert np.all(O.top2_gap(x) > 0)
+    # hand rows: 1-D input, 2-D input, negative values, the maximum in first / last place
+    assert O.top2_gap(np.array([0.25, -1.0, 0.75])) == 0.5
+    assert list(O.top2_gap(np.array([[3.0, 1.0, 2.0], [-5.0, -7.0, -4.0], [0.0, 0.0, 9.0]]))) == [1.0, 1.0, 9.0]
+    # a tie for the maximum has margin exactly 0, wherever the two entries sit
+    assert O.top2_gap(np.array([1.0, 5.0, 3.0, 5.0])) == 0.0
+    assert O.top2_gap(np.array([[2.0, 2.0]]))[0] == 0.0
+    # 3-D input keeps the leading axes
+    y = rng.standard_normal((2, 3, 9))
+    sy = np.sort(y, axis=-1)
+    assert np.array_equal(O.top2_gap(y), sy[..., -1] - sy[..., -2])
+    # a single column: nothing can overtake
+    assert np.all(np.isinf(O.top2_gap(np.array([[1.5], [2.5]]))))
+    # the margin is what separates a perturbed arg-max from the original: shifting the runner-up by more than
+    # the margin changes the arg-max, by less does not
+    row = x[0].copy()
+    first, second = np.argsort(row)[-1], np.argsort(row)[-2]
+    g = O.top2_gap(row)
+    bumped = row.copy(); bumped[second] += 0.99 * g
+    assert np.argmax(bumped) == first
+    bumped[second] = row[second] + 1.01 * g
+    assert np.argmax(bumped) == second
+
+
+def _hand_logits(n, vocab, winners, margins):
+    """Rows whose largest entry is winners[i] and whose runner-up sits margins[i] below it."""
+    lg = np.full((n, vocab), -3.0)
+    for i, (w, m) in enumerate(zip(winners, margins)):
+        lg[i, w] = 1.0
+        lg[i, (w + 1) % vocab] = 1.0 - m
+    return lg
+
+
+def test_decisive_flag_on_hand_built_trees():
+    """Tree 0 -> 1 -> 2 with a side leaf 3 below the root.  Node 1 carries the target's token after the root,
+    node 2 the target's token after node 1, so the path 0, 1, 2 is accepted and node 2 wins; node 3 carries
+    another token and is rejected.  The result reads the arg-max of nodes 0 and 1 (they have children) and of
+    node 2 (the bonus token); node 3's arg-max is read by nothing."""
+    parent = np.array([-1, 0, 1, 0])
+    vocab = 8
+    winners = [4, 6, 2, 5]                  # the target's greedy token after each node
+    tokens = np.array([7, 4, 6, 1])         # node 1 = winners[0], node 2 = winners[1], node 3 != winners[0]
+    wide = [1.0, 1.0, 1.0, 1.0]
+    r = O.decide(tokens, parent, _hand_logits(4, vocab, winners, wide))
+    assert r["accept_len"] == 2 and list(r["path"]) == [0, 1, 2] and r["bonus"] == 2 and r["decisive"]
+    assert list(r["consulted"]) == [True, True, True, False]
+    assert np.allclose(r["gap"], wide)
+    # a narrow margin at the rejected leaf changes nothing that is reported
+    r = O.decide(tokens, parent, _hand_logits(4, vocab, winners, [1.0, 1.0, 1.0, 1e-3]))
+    assert r["decisive"] and abs(r["gap"][3] - 1e-3) < 1e-12
+    # the same narrow margin at a node with a child, or at the winner, makes the round ambiguous
+    for node in (0, 1, 2):
+        m = list(wide)
+        m[node] = 1e-3
+        r = O.decide(tokens, parent, _hand_logits(4, vocab, winners, m))
+        assert not r["decisive"], node
+        assert r["accept_len"] == 2                      # the oracle's own outcome is unchanged
+    # the threshold is exclusive and adjustable: a margin equal to it is not clear
+    r = O.decide(tokens, parent, _hand_logits(4, vocab, winners, [0.5, 1.0, 1.0, 1.0]), decisive_gap=0.5)
+    assert not r["decisive"]
+    assert O.decide(tokens, parent, _hand_logits(4, vocab, winners, [0.5, 1.0, 1.0, 1.0]), decisive_gap=0.49)["decisive"]
+    # when the draft fails at the first step the winner is the root: only node 0 and the parents are read
+    tokens2 = np.array([7, 3, 6, 1])
+    r = O.decide(tokens2, parent, _hand_logits(4, vocab, winners, [1.0, 1.0, 1e-3, 1e-3]))
+    assert r["accept_len"] == 0 and r["best"] == 0 and r["decisive"]
+    assert list(r["consulted"]) == [True, True, False, False]
+    # a gap of zero everywhere (what a broken margin would report) must make every round ambiguous
+    flat = np.zeros((4, vocab))
+    assert not O.decide(tokens, parent, flat)["decisive"]

@@ -247,3 +247,30 @@ def test_oracle_reproduces_the_stored_config1_values():
         assert np.allclose(now[key], stored[key], rtol=1e-9, atol=1e-12), key
     assert abs(now["logits_abs_sum"] - stored["logits_abs_sum"]) <= 1e-7 * stored["logits_abs_sum"]
     assert abs(now["min_top2_gap"] - stored["min_top2_gap"]) < 1e-9
+
+
+def test_uncached_round_equals_prefill_then_verify():
+    """verify_tree_uncached (context and tree in one pass) against prefill + verify_tree, and through that against
+    the per-node brute force that pins verify_tree."""
+    cfg = gen.get_config("micro")
+    W = oracle_weights(cfg, 3)
+    cache, x, audio, prompt = filled_cache(cfg, W, 11, 4, seed=3)
+    parent = gen.sparse_tree(17, seed=3)
+    tokens = gen.fill_tree_tokens(parent, cfg.vocab, seed=3, root_token=int(prompt[-1]))
+    a = O.verify_tree(cfg, W, cache, tokens, parent)
+    b = O.verify_tree_uncached(cfg, W, x, tokens, parent)
+    assert np.abs(a["logits"] - b["logits"]).max() < 1e-10
+    assert a["accept_len"] == b["accept_len"] and list(a["path"]) == list(b["path"]) and a["bonus"] == b["bonus"]
+    for l in range(cfg.n_layers):
+        assert np.abs(a["tree_K"][l] - b["tree_K"][l]).max() < 1e-12
+        assert np.abs(a["tree_V"][l] - b["tree_V"][l]).max() < 1e-12
+        assert np.abs(cache.K[l] - b["prefix_K"][l]).max() < 1e-12
+    # one node against the plain definition: causal forward over context + its root path
+    i = int(np.argmax(a["depth"]))
+    path = []
+    j = i
+    while j >= 0:
+        path.append(j)
+        j = int(parent[j])
+    seq = np.concatenate([x, O.embed(W, tokens[path[::-1]])], 0)
+    assert np.abs(O.causal_forward(cfg, W, seq)[-1] - b["logits"][i]).max() < 1e-10
