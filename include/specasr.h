@@ -227,7 +227,9 @@ enum {
   SPECASR_KIND_GEMM_LM = 9,     /* vocabulary projection + argmax */
   SPECASR_KIND_ACCEPT = 10,
   SPECASR_KIND_COMMIT = 11,     /* KV compaction and length bookkeeping */
-  SPECASR_KIND_COUNT = 12
+  SPECASR_KIND_STACK = 12,      /* the whole layer stack (norms, projections, rotary, attention, arg-max) as one
+                                   persistent kernel; kinds 1..9 then name its steps in the device-side trace */
+  SPECASR_KIND_COUNT = 13
 };
 specasr_status specasr_profile_enable(specasr_kv* kv, int32_t enable);
 /*

@@ -26,7 +26,7 @@ EXPORTS = [
     "specasr_profile_enable", "specasr_profile_read", "specasr_trace_set", "specasr_accept_logits_static", "specasr_top2_probs",
 ]
 KIND_NAMES = ["prep", "norm", "gemm_qkv", "rope", "attn", "attn_merge", "gemm_o", "gemm_gu", "gemm_down", "gemm_lm",
-              "accept", "commit"]
+              "accept", "commit", "stack"]
 
 
 class ModelConfig(C.Structure):

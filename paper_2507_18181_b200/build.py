@@ -5,7 +5,7 @@ import sys
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
-SOURCES = ["api.cu", "kernels_small.cu", "attention.cu", "attention_tc.cu", "gemm_fma.cu", "gemm_tcgen05.cu", "accept_static.cu", "top2.cu"]
+SOURCES = ["api.cu", "kernels_small.cu", "attention.cu", "attention_tc.cu", "gemm_fma.cu", "gemm_tcgen05.cu", "fused_stack.cu", "accept_static.cu", "top2.cu"]
 LIB = os.path.join(HERE, "libspecasr.so")
 LIB_TRACE = os.path.join(HERE, "libspecasr_trace.so")      # same sources with -DSPECASR_TRACE (device-side trace)
 

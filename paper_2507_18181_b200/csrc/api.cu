@@ -69,13 +69,18 @@ Workspace carve_workspace(const specasr_model* m, int n_alloc, void* base) {
   w.attML = (float2*)take(sizeof(float2) * kMaxAttnSplits * n_alloc * c.n_heads);
   w.amax = (unsigned long long*)take(sizeof(unsigned long long) * lm_tiles_of(m) * n_alloc);
   w.tmKV = (CUtensorMap*)take(sizeof(CUtensorMap) * 2);
+  w.ssq = (float*)take(sizeof(float) * 2 * n_alloc);
+  w.sync = (int32_t*)take(fused_stack_sync_bytes(m));
   w.bytes = off;
   return w;
 }
 
 // ------------------------------------------------------------------------------------------------
-extern "C" specasr_status specasr_model_create(const specasr_model_config* cfg, const specasr_weight_ptrs* w,
-                                               specasr_model** out) {
+extern "C" void specasr_model_destroy(specasr_model* m);
+static thread_local specasr_model* g_creating = nullptr;   // handle under construction, for the catch block below
+
+static specasr_status model_create_impl(const specasr_model_config* cfg, const specasr_weight_ptrs* w,
+                                        specasr_model** out) {
   if (!cfg || !w || !out) {
     set_error("specasr_model_create: null argument");
     return SPECASR_ERR_INVALID_ARG;
@@ -101,6 +106,7 @@ extern "C" specasr_status specasr_model_create(const specasr_model_config* cfg, 
     set_error("out of host memory");
     return SPECASR_ERR_INVALID_ARG;
   }
+  g_creating = m;
   m->cfg = c;
   m->q_dim = c.n_heads * c.head_dim;
   m->kv_dim = c.n_kv_heads * c.head_dim;
@@ -109,6 +115,8 @@ extern "C" specasr_status specasr_model_create(const specasr_model_config* cfg, 
   m->lm_head = (const bf16*)w->lm_head;
   m->g_final = w->g_final;
   m->rope_table = nullptr;
+  m->w_maps_dev = nullptr;
+  m->gains_dev = nullptr;
   for (int l = 0; l < c.n_layers; ++l) {
     if (!w->wqkv[l] || !w->wo[l] || !w->wgu[l] || !w->wd[l] || !w->g_attn[l] || !w->g_ffn[l]) {
       delete m;
@@ -172,14 +180,60 @@ extern "C" specasr_status specasr_model_create(const specasr_model_config* cfg, 
       delete m;
       return SPECASR_ERR_CUDA;   // message set by make_tensor_map_2d
     }
+    // device copies of the weight descriptors and gain pointers, in the order the fused stack kernel walks them
+    std::vector<CUtensorMap> maps;
+    std::vector<const float*> gains;
+    for (int l = 0; l < c.n_layers; ++l) {
+      maps.push_back(m->tm_wqkv[l]);
+      maps.push_back(m->tm_wo[l]);
+      maps.push_back(m->tm_wgu[l]);
+      maps.push_back(m->tm_wd[l]);
+      gains.push_back(m->g_attn[l]);
+      gains.push_back(m->g_ffn[l]);
+    }
+    maps.push_back(m->tm_lm);
+    gains.push_back(m->g_final);
+    e = cudaMalloc(&m->w_maps_dev, maps.size() * sizeof(CUtensorMap));
+    if (e == cudaSuccess) e = cudaMalloc(&m->gains_dev, gains.size() * sizeof(const float*));
+    if (e == cudaSuccess)
+      e = cudaMemcpy(m->w_maps_dev, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess)
+      e = cudaMemcpy(m->gains_dev, gains.data(), gains.size() * sizeof(const float*), cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) {
+      if (m->w_maps_dev) cudaFree(m->w_maps_dev);
+      if (m->gains_dev) cudaFree(m->gains_dev);
+      cudaFree(m->rope_table);
+      delete m;
+      set_error("descriptor upload failed: %s", cudaGetErrorString(e));
+      return SPECASR_ERR_CUDA;
+    }
   }
   *out = m;
   return SPECASR_OK;
 }
 
+// No C++ exception crosses the boundary: the handle's vectors can throw std::bad_alloc.
+extern "C" specasr_status specasr_model_create(const specasr_model_config* cfg, const specasr_weight_ptrs* w,
+                                               specasr_model** out) {
+  g_creating = nullptr;
+  try {
+    const specasr_status st = model_create_impl(cfg, w, out);
+    g_creating = nullptr;
+    return st;
+  } catch (...) {
+    if (out) *out = nullptr;
+    if (g_creating) specasr_model_destroy(g_creating);
+    g_creating = nullptr;
+    set_error("specasr_model_create: out of host memory");
+    return SPECASR_ERR_INVALID_ARG;
+  }
+}
+
 extern "C" void specasr_model_destroy(specasr_model* m) {
   if (!m) return;
   if (m->rope_table) cudaFree(m->rope_table);
+  if (m->w_maps_dev) cudaFree(m->w_maps_dev);
+  if (m->gains_dev) cudaFree(m->gains_dev);
   delete m;
 }
 
@@ -444,6 +498,10 @@ static void run_stack(specasr_model* m, specasr_kv* wk, const SegTable& tab, int
                       const int32_t* ctl_shared, bool want_head, float* out_logits, cudaStream_t s) {
   const specasr_model_config& c = m->cfg;
   const int n = n_total;
+  if (fused_stack_supported(wk, n_total, att_tc, tab.splits)) {
+    launch_fused_stack(m, wk, tab, n_total, n_max, ctl_shared, want_head, out_logits, s);
+    return;
+  }
   const int n_pad = pad_tokens(n);
   const bool tc = c.gemm_path == 0;
   int pending = 0;               // partial planes of the last down projection still to be added to X

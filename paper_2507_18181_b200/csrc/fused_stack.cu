@@ -1,0 +1,1284 @@
+// The whole layer stack of one verification round as ONE persistent kernel (sm_100a), one CTA per SM.
+//
+// A round is a chain of dependent steps per layer (RMSNorm -> QKV projection -> rotary + cache append -> tree
+// attention -> merge of the key blocks -> O projection -> RMSNorm -> gate/up projection with SiLU * up -> down
+// projection) followed by the final norm and the vocabulary projection with arg-max.  Run as separate kernels,
+// every step pays a drain of the GPU, a launch, and a refill of the weight pipeline, and HBM idles meanwhile;
+// at 64 tree tokens that was more than half of the time of a layer.  Here the CTAs stay resident for the whole
+// stack:
+//   * warp 0 streams weight tiles (TMA, 128-byte swizzle) into a shared-memory ring and never waits for
+//     anything but a free ring slot, so the next projection's first tiles arrive while the small steps run;
+//   * warp 10 fetches the matching activation blocks (hi / lo bf16 planes) once the step that produces them
+//     has finished on every CTA, and is the TMA producer of the attention step;
+//   * one thread of warp 1 issues every tcgen05.mma (projections: weights as the A operand, tokens as N, both
+//     planes in one MMA of N = 2 x tokens; attention: S = Q K^T and O = P V as three hi/lo terms each);
+//   * warps 2..9 drain TMEM (projection epilogues, softmax) and run the element-wise steps.
+// Steps are separated by a grid-wide arrival counter in global memory instead of kernel boundaries: a CTA
+// adds one when its part of a step is written, and whoever needs the step's output polls the counter (the
+// activation producer for the projections' inputs, the worker warps for the element-wise steps).  The launch is
+// cooperative, so all CTAs are co-resident; every wait is bounded by wall-clock time and ends the call with
+// SPECASR_ERR_TIMEOUT in the status word instead of hanging.
+//
+// Work split.  Linear projections (QKV, O, down): weight tiles x k-parts, one CTA each; fp32 partial planes
+// that the consuming step adds in plane order.  Non-linear epilogues (SiLU * up, arg-max): the (tile, k-block)
+// list is cut into equal contiguous ranges, a tile that straddles two ranges is completed through a parked
+// partial and a flag, in CTA order.  All of this is independent of timing, so results are deterministic.
+//
+// RMSNorm is split in two: the norm step adds the previous projection's planes to the residual stream,
+// writes x * gain as hi / lo planes and leaves the row's sums of squares (two fixed halves per row); the
+// consumer of the projection multiplies by rsqrt(mean(x^2) + eps), which commutes with the projection.  That
+// removes the row-wide reduction from the path between two projections.
+//
+// The attention step borrows the ring's shared memory (Q / P tiles and K / V pages of one key block), so the
+// weight producer resumes when the CTA's attention units are done.
+#include "internal.h"
+#include "device_utils.cuh"
+#include "sm100_ptx.cuh"
+
+using namespace sm100;
+
+namespace {
+
+constexpr int TILE_M = 128;
+constexpr int SUB_K = 64;               // bf16 elements = 128 bytes = one swizzle row
+constexpr int UMMA_K = 16;
+constexpr int KSUB = 2;                 // 64-wide k sub-blocks per ring stage (256 contiguous bytes per weight row)
+constexpr int W_SUB_BYTES = TILE_M * SUB_K * 2;
+constexpr int W_STAGE_BYTES = KSUB * W_SUB_BYTES;
+constexpr int MAX_STAGES = 6;
+constexpr int SMEM_LIMIT = 227 * 1024;
+constexpr int WORKERS = 256;            // warps 2..9
+constexpr int NUM_THREADS = 352;        // + TMA weights, MMA, TMA activations
+constexpr int NORM_PARTS = 2;           // fixed halves of a row whose sums of squares are kept apart
+
+constexpr int KEYS_MAX = 208;           // cache positions per attention unit (13 pages of 16)
+constexpr int ROUND = 128;              // keys whose probabilities fit the P tile at once
+constexpr int SUB = 128 * 64 * 2;       // [128 rows][64 bf16] swizzled sub-tile (Q, P)
+constexpr int KVSUB = KEYS_MAX * 64 * 2;
+
+// steps of a layer, in order; step k of the call has its own arrival counter, complete when it equals the CTA count
+// (one shared counter would not do: a CTA without work in a step runs ahead and would be counted for a later one)
+enum { ST_NORM1 = 0, ST_QKV, ST_ROPE, ST_ATTN, ST_MERGE, ST_O, ST_NORM2, ST_GU, ST_DOWN, ST_PER_LAYER };
+
+struct alignas(16) StackCtl {
+  unsigned long long full[MAX_STAGES];
+  unsigned long long empty[MAX_STAGES];
+  unsigned long long acc_full[2];
+  unsigned long long acc_empty[2];
+  unsigned long long bar_qk, bar_v, bar_s, bar_p[2], bar_o[2];
+  unsigned long long key[64];
+  float red_max[2][128];
+  float red_sum[2][128];
+  float inv[64];                        // 1 / rms of every token row, for the epilogue in progress
+  float red[8];
+  uint32_t tmem_base;
+  int abort;
+  int attn_done;                        // attention steps this CTA has finished (its ring memory is free again)
+  int step_ok;                          // verdict of a wait that one worker made for all of them
+};
+
+struct StackParams {
+  int n_layers, d, qkv_dim, q_dim, Hq, Hkv, ffn, vocab, page_size, max_positions;
+  float eps, scale_log2;
+  const CUtensorMap* w_maps;            // [4 * n_layers + 1]: QKV, O, gate/up, down per layer, then the vocabulary
+  const float* const* gains;            // [2 * n_layers + 1]: attention / FFN norm per layer, then the final norm
+  const float2* rope;
+  int n, n_pad, n_alloc, stages, stage_bytes, ring_bytes;
+  int splits_qkv, splits_o, splits_down, epoch0, want_head, group, nodes_per_tile, row_tiles, attn_units;
+  int32_t* ctl;                         // control block whose status word ends the call
+  int32_t* sync;                        // [steps of the call] arrival counters, zeroed before the launch
+  float* X;
+  float* P;
+  float* fixP;
+  int32_t* fixFlag;
+  bf16* H;
+  bf16* Q;
+  bf16* AO;
+  bf16* A;
+  float* attO;
+  float2* attML;
+  float* ssq;                           // [NORM_PARTS][n_alloc]
+  unsigned long long* amax;
+  float* logits;
+  const int32_t* pos;
+  const unsigned long long* anc;
+#ifdef SPECASR_TRACE
+  TraceBuf tr;
+#endif
+};
+
+__device__ __forceinline__ int ld_acquire(const int32_t* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release(int32_t* p, int v) {
+  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void red_release_add(int32_t* p, int v) {
+  asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+// generic-proxy accesses (ordinary loads / stores) <-> async-proxy accesses (TMA) of the same memory
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ void worker_bar() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+// One projection as this CTA sees it.
+struct Gemm {
+  const CUtensorMap* tmW;
+  int M, K, KB, tiles, splits;          // splits > 0: linear output in `splits` k-parts per tile
+  int g_eff;                            // CTAs that take part
+  long long U, u0, u1;                  // all (tile, k-block) units; this CTA's range
+};
+
+__device__ __forceinline__ Gemm gemm_of(const StackParams& p, int layer, int which, int cta, int G) {
+  Gemm g;
+  switch (which) {
+    case ST_QKV: g.M = p.qkv_dim; g.K = p.d; g.splits = p.splits_qkv; g.tmW = p.w_maps + 4 * layer; break;
+    case ST_O: g.M = p.d; g.K = p.q_dim; g.splits = p.splits_o; g.tmW = p.w_maps + 4 * layer + 1; break;
+    case ST_GU: g.M = 2 * p.ffn; g.K = p.d; g.splits = 0; g.tmW = p.w_maps + 4 * layer + 2; break;
+    case ST_DOWN: g.M = p.d; g.K = p.ffn; g.splits = p.splits_down; g.tmW = p.w_maps + 4 * layer + 3; break;
+    default: g.M = p.vocab; g.K = p.d; g.splits = 0; g.tmW = p.w_maps + 4 * p.n_layers; break;      // vocabulary
+  }
+  g.KB = (g.K + KSUB * SUB_K - 1) / (KSUB * SUB_K);
+  g.tiles = (g.M + TILE_M - 1) / TILE_M;
+  g.U = (long long)g.tiles * g.KB;
+  if (g.splits > 0) {
+    g.g_eff = g.tiles * g.splits;
+    if (cta < g.g_eff) {
+      const int tile = cta / g.splits, split = cta % g.splits;
+      g.u0 = (long long)tile * g.KB + (long long)split * g.KB / g.splits;
+      g.u1 = (long long)tile * g.KB + (long long)(split + 1) * g.KB / g.splits;
+    } else {
+      g.u0 = g.u1 = 0;
+    }
+  } else {
+    g.g_eff = g.U < G ? (int)g.U : G;
+    if (cta < g.g_eff) {
+      g.u0 = cta * g.U / g.g_eff;
+      g.u1 = (cta + 1) * g.U / g.g_eff;
+    } else {
+      g.u0 = g.u1 = 0;
+    }
+  }
+  return g;
+}
+
+// Bounded poll of a word that only grows.  Returns false when the limit ran out or the call was aborted.
+__device__ __forceinline__ bool wait_word_ge(const int32_t* word, int target, volatile int* abort, int32_t* status) {
+  if (ld_acquire(word) >= target) return true;
+  const unsigned long long t0 = global_ns();
+  for (uint32_t it = 1;; ++it) {
+    __nanosleep(40);
+    if (ld_acquire(word) >= target) return true;
+    if ((it & 15u) == 0u) {
+      if (*abort) return false;
+      if (*(volatile int32_t*)status != 0) {
+        *abort = 1;
+        return false;
+      }
+      if (global_ns() - t0 > WAIT_LIMIT_NS) {
+        *abort = 1;
+        atomicExch(status, (int32_t)SPECASR_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ bool wait_smem_ge(volatile int* word, int target, volatile int* abort, int32_t* status) {
+  if (*word >= target) return true;
+  const unsigned long long t0 = global_ns();
+  for (uint32_t it = 1;; ++it) {
+    __nanosleep(40);
+    if (*word >= target) return true;
+    if ((it & 15u) == 0u) {
+      if (*abort) return false;
+      if (global_ns() - t0 > WAIT_LIMIT_NS) {
+        *abort = 1;
+        atomicExch(status, (int32_t)SPECASR_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+
+// The utterance that owns workspace row `row` (segments are laid out back to back in table order).
+__device__ __forceinline__ int seg_of_row(const SegTable& tab, int row) {
+  int b = 0;
+  while (b + 1 < tab.count && row >= tab.seg[b].row0 + tab.seg[b].n) ++b;
+  return b;
+}
+
+#ifdef SPECASR_TRACE
+#define STACK_TRACE_BEGIN() const unsigned long long tr_t0_ = wtid == 0 ? global_ns() : 0ull
+#define STACK_TRACE_END(kind, layer)                                                     \
+  do {                                                                                   \
+    if (wtid == 0 && p.tr.buf != nullptr) {                                              \
+      const unsigned long long slot_ = atomicAdd(p.tr.buf, 1ull);                        \
+      if (slot_ < p.tr.cap) {                                                            \
+        unsigned long long* e_ = p.tr.buf + 2 + slot_ * 4;                               \
+        e_[0] = (unsigned long long)(kind) | ((unsigned long long)((layer) + 1) << 8);   \
+        e_[1] = tr_t0_;                                                                  \
+        e_[2] = global_ns();                                                             \
+        e_[3] = tr_t0_;                                                                  \
+      }                                                                                  \
+    }                                                                                    \
+  } while (0)
+#else
+#define STACK_TRACE_BEGIN()
+#define STACK_TRACE_END(kind, layer)
+#endif
+
+template <int DH>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmAO,
+        const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmQ,
+        const __grid_constant__ SegTable tab, const StackParams p) {
+  constexpr int H2 = DH / 64;                           // 64-wide halves of a head
+  constexpr int A_BYTES = 4 * SUB;                      // Q planes, later two P planes of 128 keys
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* ring = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  StackCtl* sc = (StackCtl*)(ring + p.ring_bytes);
+  bf16* epi_stage = (bf16*)(sc + 1);                    // SiLU * up output tile [2 planes][tokens][64]
+  uint8_t* As = ring;                                   // attention: overlays the ring
+  uint8_t* KVs = ring + A_BYTES;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int G = gridDim.x, cta = blockIdx.x;
+  const int n_pad = p.n_pad;
+  const int act_sub = n_pad * 2 * SUB_K * 2;            // both planes of one 64-wide k sub-block
+  const int act_stage = KSUB * act_sub;
+  const int acc_cols = 2 * n_pad;                       // hi | lo halves of one accumulator set
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < MAX_STAGES; ++s) {
+      mbar_init(&sc->full[s], 2);                       // weight producer + activation producer
+      mbar_init(&sc->empty[s], 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&sc->acc_full[b], 1);
+      mbar_init(&sc->acc_empty[b], WORKERS);
+      mbar_init(&sc->bar_p[b], WORKERS);
+      mbar_init(&sc->bar_o[b], 1);
+    }
+    mbar_init(&sc->bar_qk, 1);
+    mbar_init(&sc->bar_v, 1);
+    mbar_init(&sc->bar_s, 1);
+    sc->abort = 0;
+    sc->attn_done = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&tmH);
+    tma_prefetch_desc(&tmAO);
+    tma_prefetch_desc(&tmA);
+    tma_prefetch_desc(&tmQ);
+  }
+  if (warp == 1) tmem_alloc(&sc->tmem_base, 512);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = sc->tmem_base;
+  volatile int* abort = &sc->abort;
+  int32_t* status = p.ctl + CTL_STATUS;
+  const bool live = *(volatile int32_t*)status == 0;
+  const int steps_total = p.n_layers * ST_PER_LAYER;    // index of the final norm; the vocabulary projection follows
+
+  // attention geometry shared by all roles
+  const int rows_used = p.nodes_per_tile * p.group;
+
+  if (!live) {
+    // the call was refused before it started (shared status): nothing to do
+  } else if (warp == 0 && lane == 0) {
+    // =========================================================== weight producer
+    int it = 0;                                          // ring slots used so far
+    bool ok = true;
+    auto stream_weights = [&](const Gemm& g) {
+      for (long long u = g.u0; u < g.u1 && ok; ++u, ++it) {
+        const int tile = (int)(u / g.KB), kb = (int)(u % g.KB), s = it % p.stages;
+        if (!mbar_wait(&sc->empty[s], (uint32_t)((it / p.stages) & 1) ^ 1u, abort, status)) {
+          ok = false;
+          break;
+        }
+        uint8_t* st = ring + (size_t)s * p.stage_bytes;
+        mbar_expect_tx(&sc->full[s], (uint32_t)W_STAGE_BYTES);
+        for (int q = 0; q < KSUB; ++q)                   // rows past M and columns past K read as zeros
+          tma_load_2d(st + q * W_SUB_BYTES, g.tmW, (kb * KSUB + q) * SUB_K, tile * TILE_M, &sc->full[s]);
+      }
+    };
+    for (int l = 0; l < p.n_layers && ok; ++l) {
+      stream_weights(gemm_of(p, l, ST_QKV, cta, G));
+      if (ok) ok = wait_smem_ge(&sc->attn_done, l + 1, abort, status);   // the attention step owns the ring meanwhile
+      if (ok) stream_weights(gemm_of(p, l, ST_O, cta, G));
+      if (ok) stream_weights(gemm_of(p, l, ST_GU, cta, G));
+      if (ok) stream_weights(gemm_of(p, l, ST_DOWN, cta, G));
+    }
+    if (ok && p.want_head) stream_weights(gemm_of(p, 0, -1, cta, G));
+  } else if (warp == 10) {
+    // =========================================================== activation producer / attention producer
+    int it = 0;
+    bool ok = true;
+    int au = 0;                                          // attention units this CTA has run
+    auto stream_acts = [&](const Gemm& g, const CUtensorMap* tmAct, int ready_step) {
+      if (g.u1 <= g.u0) return;
+      if (lane == 0) {
+        ok = wait_word_ge(p.sync + ready_step, G, abort, status);
+        fence_proxy_async_all();
+        for (long long u = g.u0; u < g.u1 && ok; ++u, ++it) {
+          const int kb = (int)(u % g.KB), s = it % p.stages;
+          if (!mbar_wait(&sc->empty[s], (uint32_t)((it / p.stages) & 1) ^ 1u, abort, status)) {
+            ok = false;
+            break;
+          }
+          uint8_t* st = ring + (size_t)s * p.stage_bytes + W_STAGE_BYTES;
+          mbar_expect_tx(&sc->full[s], (uint32_t)act_stage);
+          for (int q = 0; q < KSUB; ++q)
+            tma_load_3d(st + q * act_sub, tmAct, (kb * KSUB + q) * SUB_K, 0, 0, &sc->full[s]);
+        }
+      }
+      ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+      it = __shfl_sync(0xFFFFFFFFu, it, 0);
+    };
+    for (int l = 0; l < p.n_layers && ok; ++l) {
+      const int base = l * ST_PER_LAYER;
+      stream_acts(gemm_of(p, l, ST_QKV, cta, G), &tmH, base + ST_NORM1);
+      // ---- attention units of this CTA: lane 0 fetches Q, lane j page j of K and later of V
+      if (ok && cta < p.attn_units) {
+        if (lane == 0) {
+          ok = wait_word_ge(p.sync + base + ST_ROPE, G, abort, status);
+          fence_proxy_async_all();
+        }
+        ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+      }
+      for (int u = cta; u < p.attn_units && ok; u += G) {
+        const int kvh = u % p.Hkv, tile_y = (u / p.Hkv) % p.row_tiles, z = u / (p.Hkv * p.row_tiles);
+        const int split = z % tab.splits;
+        const SegDev& sg = tab.seg[z / tab.splits];
+        const int node0 = tile_y * p.nodes_per_tile;
+        if (node0 >= sg.n || sg.ctl[CTL_STATUS] != 0) continue;
+        const int L = sg.ctl[CTL_LEN];
+        const int Ltot = L + sg.n;
+        const int k_begin = split * sg.chunk;
+        if (k_begin >= Ltot) continue;
+        const int kc = min(sg.chunk, Ltot - k_begin);
+        const int pages = (kc + p.page_size - 1) / p.page_size;
+        const uint32_t par = (uint32_t)(au & 1);
+        ++au;
+        int my_page = 0;
+        if (lane < pages) my_page = sg.page_table[split * (sg.chunk / p.page_size) + lane];
+        const uint32_t q_bytes = 2 * H2 * rows_used * 128;
+        const uint32_t kv_bytes = 2 * H2 * pages * p.page_size * 128;
+        if (lane == 0) {
+          mbar_expect_tx(&sc->bar_qk, q_bytes + kv_bytes);
+          mbar_expect_tx(&sc->bar_v, kv_bytes);
+        }
+        __syncwarp();
+        if (lane == 0) {
+          for (int plane = 0; plane < 2; ++plane)
+            for (int h = 0; h < H2; ++h)
+              tma_load_4d(As + (plane * H2 + h) * SUB, &tmQ, h * 64, kvh * p.group, sg.row0 + node0, plane, &sc->bar_qk);
+        }
+        const int c4 = l * sg.n_pages + my_page;
+        const int off = lane * p.page_size * 128;
+        if (lane < pages) {
+          for (int plane = 0; plane < 2; ++plane)
+            for (int h = 0; h < H2; ++h)
+              tma_load_5d(KVs + (plane * H2 + h) * KVSUB + off, sg.tmK, h * 64, 0, plane, kvh, c4, &sc->bar_qk);
+        }
+        // V takes K's place once the S MMAs have read K
+        ok = mbar_wait(&sc->bar_s, par, abort, status);
+        if (ok && lane < pages) {
+          for (int plane = 0; plane < 2; ++plane)
+            for (int h = 0; h < H2; ++h)
+              tma_load_5d(KVs + (plane * H2 + h) * KVSUB + off, sg.tmV, h * 64, 0, plane, kvh, c4, &sc->bar_v);
+        }
+        ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+      }
+      if (ok) stream_acts(gemm_of(p, l, ST_O, cta, G), &tmAO, base + ST_MERGE);
+      if (ok) stream_acts(gemm_of(p, l, ST_GU, cta, G), &tmH, base + ST_NORM2);
+      if (ok) stream_acts(gemm_of(p, l, ST_DOWN, cta, G), &tmA, base + ST_GU);
+    }
+    if (ok && p.want_head) stream_acts(gemm_of(p, 0, -1, cta, G), &tmH, steps_total);
+  } else if (warp == 1 && lane == 0) {
+    // =========================================================== MMA issuer
+    int it = 0, seg = 0, au = 0, au2 = 0;
+    bool ok = true;
+    const uint32_t idesc = make_idesc_bf16(2 * n_pad);
+    auto run_gemm = [&](const Gemm& g) {
+      for (long long u = g.u0; u < g.u1 && ok; ++seg) {
+        const int kb0 = (int)(u % g.KB);
+        const int kb1 = (int)((g.u1 - u) < (long long)(g.KB - kb0) ? kb0 + (g.u1 - u) : g.KB);
+        const int b = seg & 1;
+        if (!mbar_wait(&sc->acc_empty[b], (uint32_t)((seg >> 1) & 1) ^ 1u, abort, status)) {
+          ok = false;
+          break;
+        }
+        tc_fence_after();
+        const uint32_t d_addr = tmem_base + (uint32_t)(b * acc_cols);
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
+          const int s = it % p.stages;
+          if (!mbar_wait(&sc->full[s], (uint32_t)((it / p.stages) & 1), abort, status)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t w_addr = smem_u32(ring + (size_t)s * p.stage_bytes);
+          const uint32_t act_addr = w_addr + W_STAGE_BYTES;
+#pragma unroll
+          for (int q = 0; q < KSUB; ++q) {
+#pragma unroll
+            for (int k = 0; k < SUB_K / UMMA_K; ++k) {
+              const uint32_t acc = (kb > kb0 || q > 0 || k > 0) ? 1u : 0u;
+              umma_bf16(d_addr, make_smem_desc(w_addr + q * W_SUB_BYTES + k * UMMA_K * 2),
+                        make_smem_desc(act_addr + q * act_sub + k * UMMA_K * 2), idesc, acc);
+            }
+          }
+          umma_commit(&sc->empty[s]);                    // arrives once these MMAs have read the stage
+        }
+        if (ok) umma_commit(&sc->acc_full[b]);
+        u += kb1 - kb0;
+      }
+    };
+    for (int l = 0; l < p.n_layers && ok; ++l) {
+      run_gemm(gemm_of(p, l, ST_QKV, cta, G));
+      // ---- attention units
+      for (int u = cta; u < p.attn_units && ok; u += G) {
+        const int tile_y = (u / p.Hkv) % p.row_tiles, z = u / (p.Hkv * p.row_tiles);
+        const int split = z % tab.splits;
+        const SegDev& sg = tab.seg[z / tab.splits];
+        if (tile_y * p.nodes_per_tile >= sg.n || sg.ctl[CTL_STATUS] != 0) continue;
+        const int Ltot = sg.ctl[CTL_LEN] + sg.n;
+        const int k_begin = split * sg.chunk;
+        if (k_begin >= Ltot) continue;
+        const int kc = min(sg.chunk, Ltot - k_begin);
+        const int kc_pad = (kc + 15) & ~15;
+        const int rounds = (kc_pad + ROUND - 1) / ROUND;
+        const uint32_t par = (uint32_t)(au & 1);
+        ++au;
+        const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 256;
+        ok = mbar_wait(&sc->bar_qk, par, abort, status);
+        if (!ok) break;
+        tc_fence_after();
+        {
+          const uint32_t idesc_s = make_idesc_bf16(kc_pad);
+          const uint32_t a0 = smem_u32(As), b0 = smem_u32(KVs);
+          uint32_t acc = 0u;
+#pragma unroll
+          for (int term = 0; term < 3; ++term) {
+            const int qp = term == 2 ? 1 : 0, kp = term == 1 ? 1 : 0;     // hi*hi, hi*lo, lo*hi
+            for (int h = 0; h < H2; ++h) {
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                umma_bf16(tmem_s, make_smem_desc(a0 + (qp * H2 + h) * SUB + k * 32),
+                          make_smem_desc(b0 + (kp * H2 + h) * KVSUB + k * 32), idesc_s, acc);
+                acc = 1u;
+              }
+            }
+          }
+          umma_commit(&sc->bar_s);
+        }
+        ok = mbar_wait(&sc->bar_v, par, abort, status);
+        const uint32_t idesc2 = make_idesc_bf16(DH, true);
+        uint32_t acc = 0u;
+        for (int rd = 0; rd < rounds && ok; ++rd) {
+          const uint32_t par_r = rd == 0 ? par : (uint32_t)(au2 & 1);
+          ok = mbar_wait(&sc->bar_p[rd], par_r, abort, status);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t a0 = smem_u32(As), b0 = smem_u32(KVs);
+          const int j_end = min(kc_pad - rd * ROUND, ROUND) / 16;
+#pragma unroll
+          for (int term = 0; term < 3; ++term) {
+            const int pp = term == 2 ? 1 : 0, vp = term == 1 ? 1 : 0;
+            for (int j = 0; j < j_end; ++j) {
+              umma_bf16(tmem_o, make_smem_desc(a0 + (pp * 2 + (j >> 2)) * SUB + (j & 3) * 32),
+                        make_smem_desc(b0 + vp * H2 * KVSUB + (rd * (ROUND / 16) + j) * 2048, KVSUB), idesc2, acc);
+              acc = 1u;
+            }
+          }
+          umma_commit(&sc->bar_o[rd]);
+        }
+        if (rounds == 2) ++au2;
+      }
+      if (ok) run_gemm(gemm_of(p, l, ST_O, cta, G));
+      if (ok) run_gemm(gemm_of(p, l, ST_GU, cta, G));
+      if (ok) run_gemm(gemm_of(p, l, ST_DOWN, cta, G));
+    }
+    if (ok && p.want_head) run_gemm(gemm_of(p, 0, -1, cta, G));
+  } else if (warp >= 2 && warp < 10) {
+    // =========================================================== workers
+    const int wtid = threadIdx.x - 64;
+    const int wwarp = warp - 2;
+    const int quad = warp & 3;
+    const int row = quad * 32 + lane;                   // TMEM lane = output row of a weight tile / query row
+    const int c_first = (wwarp >> 2) * 16;              // projections: this warp's first 16-token block, stride 32
+    const int eg = wwarp >> 2;                          // attention: which 32-key chunks this thread takes
+    const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
+    bool ok = true;
+    int seg = 0, au = 0, au2 = 0;
+    int arrived = 0;                                     // steps this CTA has signed off
+
+    // Barriers among the workers (worker_bar) are never placed under a condition that a failed wait could make
+    // differ between threads; `ok` only guards waits and memory traffic.  A wait's verdict is made uniform
+    // across the warp because the TMEM loads that follow are warp-wide instructions.
+    auto wwait = [&](void* bar, uint32_t parity) -> bool {
+      return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, abort, status) ? 1 : 0) != 0;
+    };
+    auto wwait_relaxed = [&](void* bar, uint32_t parity) -> bool {
+      return __all_sync(0xFFFFFFFFu, mbar_wait_relaxed(bar, parity, abort, status) ? 1 : 0) != 0;
+    };
+    // every worker's global writes of the step are done and visible -> one arrival for the CTA
+    auto arrive_step = [&]() {
+      __threadfence();
+      fence_proxy_async_all();
+      worker_bar();
+      if (wtid == 0) red_release_add(p.sync + arrived, 1);
+      ++arrived;
+    };
+    // all CTAs have signed off step `step`
+    auto wait_step = [&](int step) {
+      if (wtid == 0) sc->step_ok = (ok && wait_word_ge(p.sync + step, G, abort, status)) ? 1 : 0;
+      worker_bar();
+      ok = ok && sc->step_ok != 0;                       // the same verdict for every worker
+    };
+    auto worker_sum = [&](float v) -> float {            // fixed order: deterministic
+      v = warp_sum(v);
+      if (lane == 0) sc->red[wwarp] = v;
+      worker_bar();
+      float t = 0.f;
+#pragma unroll
+      for (int w = 0; w < 8; ++w) t += sc->red[w];
+      worker_bar();
+      return t;
+    };
+    // 1 / rms of every row from the sums of squares the last norm step left
+    auto load_inv = [&]() {
+      if (wtid < n_pad) {
+        float ss = 0.f;
+        if (wtid < p.n) {
+#pragma unroll
+          for (int q = 0; q < NORM_PARTS; ++q) ss += __ldcg(p.ssq + q * p.n_alloc + wtid);
+        }
+        sc->inv[wtid] = rsqrtf(ss / (float)p.d + p.eps);
+      }
+      worker_bar();
+    };
+
+    // ---------------- norm step: x += planes, h = x * g as hi / lo planes, sums of squares per half row
+    auto norm_step = [&](const float* __restrict__ gain, int n_planes, size_t plane_stride) {
+      const int d = p.d;
+      const int d_part = ((d + NORM_PARTS - 1) / NORM_PARTS + 3) & ~3;
+      const int items = p.n * NORM_PARTS;
+      const size_t h_plane = (size_t)p.n_alloc * d;
+      for (int item = cta; item < items; item += G) {
+        const int r = item / NORM_PARTS, part = item % NORM_PARTS;
+        const int k_end = min(d, (part + 1) * d_part);
+        float* x = p.X + (size_t)r * d;
+        float ss = 0.f;
+        for (int k0 = part * d_part + wtid * 4; k0 < k_end; k0 += 2 * WORKERS * 4) {
+          const int k1 = k0 + WORKERS * 4;
+          const bool on1 = k1 < k_end;
+          float4 v0 = *reinterpret_cast<const float4*>(x + k0);
+          float4 v1 = on1 ? *reinterpret_cast<const float4*>(x + k1) : make_float4(0.f, 0.f, 0.f, 0.f);
+          const float4 g0 = *reinterpret_cast<const float4*>(gain + k0);
+          const float4 g1 = on1 ? *reinterpret_cast<const float4*>(gain + k1) : make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int s0 = 0; s0 < n_planes; s0 += 4) {
+            float4 q0[4], q1[4];
+#pragma unroll
+            for (int s = 0; s < 4; ++s) {
+              const bool on = s0 + s < n_planes;
+              const float* src = p.P + (size_t)(s0 + s) * plane_stride + (size_t)r * d;
+              q0[s] = on ? __ldcg(reinterpret_cast<const float4*>(src + k0)) : make_float4(0.f, 0.f, 0.f, 0.f);
+              q1[s] = (on && on1) ? __ldcg(reinterpret_cast<const float4*>(src + k1)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int s = 0; s < 4; ++s) {
+              v0.x += q0[s].x; v0.y += q0[s].y; v0.z += q0[s].z; v0.w += q0[s].w;
+              v1.x += q1[s].x; v1.y += q1[s].y; v1.z += q1[s].z; v1.w += q1[s].w;
+            }
+          }
+          if (n_planes > 0) {
+            *reinterpret_cast<float4*>(x + k0) = v0;
+            if (on1) *reinterpret_cast<float4*>(x + k1) = v1;
+          }
+          ss += v0.x * v0.x + v0.y * v0.y + v0.z * v0.z + v0.w * v0.w;
+          ss += v1.x * v1.x + v1.y * v1.y + v1.z * v1.z + v1.w * v1.w;
+          bf16* hi = p.H + (size_t)r * d;
+          uint32_t ph[2], pl[2];
+          split2_pack(v0.x * g0.x, v0.y * g0.y, ph[0], pl[0]);
+          split2_pack(v0.z * g0.z, v0.w * g0.w, ph[1], pl[1]);
+          *reinterpret_cast<uint2*>(hi + k0) = make_uint2(ph[0], ph[1]);
+          *reinterpret_cast<uint2*>(hi + h_plane + k0) = make_uint2(pl[0], pl[1]);
+          if (on1) {
+            split2_pack(v1.x * g1.x, v1.y * g1.y, ph[0], pl[0]);
+            split2_pack(v1.z * g1.z, v1.w * g1.w, ph[1], pl[1]);
+            *reinterpret_cast<uint2*>(hi + k1) = make_uint2(ph[0], ph[1]);
+            *reinterpret_cast<uint2*>(hi + h_plane + k1) = make_uint2(pl[0], pl[1]);
+          }
+        }
+        ss = worker_sum(ss);
+        if (wtid == 0) p.ssq[part * p.n_alloc + r] = ss;
+      }
+    };
+
+    // ---------------- projection epilogues
+    auto load16 = [&](uint32_t lane_addr, int c0, float* v) {     // hi half + lo half of the accumulator
+      float lo[16];
+      tmem_ld16x2(lane_addr + (uint32_t)c0, lane_addr + (uint32_t)(c0 + n_pad), v, lo);
+#pragma unroll
+      for (int j = 0; j < 16; ++j) v[j] += lo[j];
+    };
+    // linear output: fp32 partial plane `split`
+    auto epi_partial = [&](const Gemm& g, size_t plane_stride) {
+      for (long long u = g.u0; u < g.u1; ++seg) {
+        const int tile = (int)(u / g.KB);
+        const int kb0 = (int)(u % g.KB);
+        const int kb1 = (int)((g.u1 - u) < (long long)(g.KB - kb0) ? kb0 + (g.u1 - u) : g.KB);
+        u += kb1 - kb0;
+        const int b = seg & 1;
+        if (ok) ok = wwait_relaxed(&sc->acc_full[b], (uint32_t)((seg >> 1) & 1));
+        tc_fence_after();
+        if (!ok) continue;
+        const uint32_t lane_addr = tmem_base + lane_off + (uint32_t)(b * acc_cols);
+        float* out = p.P + (size_t)(cta % g.splits) * plane_stride;
+        const int m = tile * TILE_M + row;
+        for (int c0 = c_first; c0 < n_pad; c0 += 32) {
+          float v[16];
+          load16(lane_addr, c0, v);
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            if (c0 + j < p.n && m < g.M) out[(size_t)(c0 + j) * g.M + m] = v[j];
+        }
+        tc_fence_before();
+        mbar_arrive(&sc->acc_empty[b]);
+      }
+    };
+    // SiLU(gate) * up (swiglu = true) or arg-max over the vocabulary (swiglu = false), equal unit ranges
+    auto epi_streamk = [&](const Gemm& g, bool swiglu, int epoch) {
+      for (long long u = g.u0; u < g.u1; ++seg) {
+        const int tile = (int)(u / g.KB);
+        const int kb0 = (int)(u % g.KB);
+        const int kb1 = (int)((g.u1 - u) < (long long)(g.KB - kb0) ? kb0 + (g.u1 - u) : g.KB);
+        u += kb1 - kb0;
+        const int b = seg & 1;
+        // the CTA that holds the first k-blocks of a split tile adds what the CTAs holding the rest have parked
+        int last = cta;
+        if (kb0 == 0 && kb1 != g.KB)
+          while (last + 1 < g.g_eff && (last + 1) * g.U / g.g_eff < (long long)(tile + 1) * g.KB) ++last;
+        float pk0[16], pk1[16];
+        auto load_parked = [&](int c0, float* f) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) f[j] = 0.f;
+          if (c0 < n_pad)
+            for (int cc = cta + 1; cc <= last; ++cc) {
+              const float* src = p.fixP + ((size_t)cc * n_pad + c0) * TILE_M + row;
+#pragma unroll
+              for (int j = 0; j < 16; ++j) f[j] += __ldcg(src + j * TILE_M);
+            }
+        };
+        if (last > cta) {
+          if (wtid == 0) {
+            bool got = ok;
+            for (int cc = cta + 1; cc <= last && got; ++cc)
+              got = wait_word_ge(p.fixFlag + cc, epoch, abort, status);            // flags carry the launch's epoch
+            sc->step_ok = got ? 1 : 0;
+          }
+          worker_bar();
+          ok = ok && sc->step_ok != 0;
+          if (ok) {
+            load_parked(c_first, pk0);
+            load_parked(c_first + 32, pk1);
+          }
+        }
+        if (ok) ok = wwait_relaxed(&sc->acc_full[b], (uint32_t)((seg >> 1) & 1));
+        tc_fence_after();
+        const uint32_t lane_addr = tmem_base + lane_off + (uint32_t)(b * acc_cols);
+
+        if (kb0 != 0) {
+          // later k-blocks of a tile whose first k-blocks belong to an earlier CTA: park the partial sums
+          float* dst = p.fixP + (size_t)cta * n_pad * TILE_M;
+          if (ok) {
+            for (int c0 = c_first; c0 < n_pad; c0 += 32) {
+              float v[16];
+              load16(lane_addr, c0, v);
+#pragma unroll
+              for (int j = 0; j < 16; ++j) dst[(size_t)(c0 + j) * TILE_M + row] = v[j];
+            }
+            tc_fence_before();
+            mbar_arrive(&sc->acc_empty[b]);
+            __threadfence();
+          }
+          worker_bar();
+          if (ok && wtid == 0) st_release(p.fixFlag + cta, epoch);
+          continue;
+        }
+
+        const int m = tile * TILE_M + row;
+        const bool row_ok = m < g.M;
+        if (!swiglu) {
+          if (wtid < 64) sc->key[wtid] = 0ull;
+          worker_bar();
+        }
+        if (ok) {
+          for (int c0 = c_first; c0 < n_pad; c0 += 32) {
+            float v[16];
+            load16(lane_addr, c0, v);
+            if (last > cta) {
+              const bool first = c0 == c_first;
+#pragma unroll
+              for (int j = 0; j < 16; ++j) v[j] += first ? pk0[j] : pk1[j];
+            }
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[j] *= sc->inv[c0 + j];
+            if (swiglu) {
+              // rows 2f / 2f + 1 of the tile are gate / up of feature f: the even lane keeps the hi plane of the
+              // product, the odd lane the lo plane, staged in shared memory for 16-byte global stores
+              float a[16];
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                const float other = __shfl_xor_sync(0xFFFFFFFFu, v[j], 1);
+                const float gt = (lane & 1) ? other : v[j];
+                const float up = (lane & 1) ? v[j] : other;
+                a[j] = __fdividef(gt, 1.f + __expf(-gt)) * up;
+              }
+              bf16* st = epi_stage + (size_t)(lane & 1) * n_pad * 64 + (size_t)c0 * 64 + (row >> 1);
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                bf16 hi, lo;
+                split_bf16(a[j], hi, lo);
+                st[j * 64] = (lane & 1) ? lo : hi;
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                const int t = c0 + j;
+                if (p.logits && t < p.n && row_ok) p.logits[(size_t)t * g.M + m] = v[j];
+                uint32_t key = __float_as_uint(v[j]);
+                key = (key & 0x80000000u) ? ~key : (key | 0x80000000u);
+                if (!row_ok) key = 0u;
+                const uint32_t best = __reduce_max_sync(0xFFFFFFFFu, key);
+                const uint32_t who = __reduce_min_sync(0xFFFFFFFFu, key == best ? (uint32_t)m : 0xFFFFFFFFu);
+                if (lane == 0 && t < p.n && best != 0u)
+                  atomicMax(&sc->key[t], ((unsigned long long)best << 32) | (unsigned long long)(0xFFFFFFFFu - who));
+              }
+            }
+          }
+        }
+        worker_bar();
+        if (ok) {
+          if (swiglu) {
+            const int F = g.M >> 1;
+            const int f0 = tile * 64;
+            const int nt = p.n;
+            const int chunks = 2 * nt * 8;                    // 16-byte pieces of the [2][nt][64] tile
+            for (int idx = wtid; idx < chunks; idx += WORKERS) {
+              const int plane = idx / (nt * 8), rem = idx % (nt * 8);
+              const int t = rem >> 3, ch = rem & 7;
+              if (f0 + ch * 8 < F)
+                *reinterpret_cast<uint4*>(p.A + (size_t)plane * p.n_alloc * F + (size_t)t * F + f0 + ch * 8) =
+                    *reinterpret_cast<const uint4*>(epi_stage + (size_t)plane * n_pad * 64 + t * 64 + ch * 8);
+            }
+          } else {
+            for (int t = wtid; t < p.n; t += WORKERS) p.amax[(size_t)tile * p.n_alloc + t] = sc->key[t];
+          }
+          tc_fence_before();
+          mbar_arrive(&sc->acc_empty[b]);
+        }
+        worker_bar();
+      }
+    };
+
+    // ---------------- rotary embedding at tree positions + cache append (from the QKV partial planes)
+    auto rope_step = [&](int layer) {
+      const int half = DH >> 1;
+      const int per_head = half >> 2;                    // threads per head: four rotation pairs each
+      const int heads_all = p.Hq + 2 * p.Hkv;
+      const long long total = (long long)p.n * heads_all * per_head;
+      const size_t pstride = (size_t)p.n_alloc * p.qkv_dim;
+      const size_t q_plane = (size_t)p.n_alloc * p.q_dim;
+      for (long long idx = (long long)cta * WORKERS + wtid; idx < total; idx += (long long)G * WORKERS) {
+        const int i = (int)(idx / (heads_all * per_head));
+        const int rem = (int)(idx % (heads_all * per_head));
+        const int head = rem / per_head, k = (rem % per_head) * 4;
+        const SegDev& sg = tab.seg[seg_of_row(tab, i)];
+        const size_t col = (size_t)i * p.qkv_dim + (size_t)head * DH;
+        const size_t c1 = col + qkv_row_of_feature(k, DH), c2 = col + qkv_row_of_feature(k + half, DH);
+        const bool is_v = head >= p.Hq + p.Hkv;
+        float4 x1 = make_float4(0.f, 0.f, 0.f, 0.f), x2 = x1;
+        float4 cs01 = make_float4(1.f, 0.f, 1.f, 0.f), cs23 = cs01;
+        float4 a1[4], a2[4];
+#pragma unroll
+        for (int s = 0; s < 4; ++s) {
+          const bool on = s < p.splits_qkv;
+          a1[s] = on ? __ldcg(reinterpret_cast<const float4*>(p.P + s * pstride + c1)) : make_float4(0.f, 0.f, 0.f, 0.f);
+          a2[s] = on ? __ldcg(reinterpret_cast<const float4*>(p.P + s * pstride + c2)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        const int seg_status = sg.ctl[CTL_STATUS];
+        const int len = sg.ctl[CTL_LEN];
+        const float ss = __ldcg(p.ssq + i) + __ldcg(p.ssq + p.n_alloc + i);
+        if (!is_v) {
+          const int pp = min(max(p.pos[i], 0), p.max_positions - 1);
+          const float4* t = reinterpret_cast<const float4*>(p.rope + (size_t)pp * half + k);
+          cs01 = t[0];
+          cs23 = t[1];
+        }
+#pragma unroll
+        for (int s = 0; s < 4; ++s) {
+          x1.x += a1[s].x; x1.y += a1[s].y; x1.z += a1[s].z; x1.w += a1[s].w;
+          x2.x += a2[s].x; x2.y += a2[s].y; x2.z += a2[s].z; x2.w += a2[s].w;
+        }
+        for (int s0 = 4; s0 < p.splits_qkv; s0 += 4) {
+#pragma unroll
+          for (int s = 0; s < 4; ++s) {
+            const bool on = s0 + s < p.splits_qkv;
+            a1[s] = on ? __ldcg(reinterpret_cast<const float4*>(p.P + (s0 + s) * pstride + c1)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            a2[s] = on ? __ldcg(reinterpret_cast<const float4*>(p.P + (s0 + s) * pstride + c2)) : make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+#pragma unroll
+          for (int s = 0; s < 4; ++s) {
+            x1.x += a1[s].x; x1.y += a1[s].y; x1.z += a1[s].z; x1.w += a1[s].w;
+            x2.x += a2[s].x; x2.y += a2[s].y; x2.z += a2[s].z; x2.w += a2[s].w;
+          }
+        }
+        if (seg_status != 0) continue;                   // nothing is written for an utterance whose tree was refused
+        const float inv = rsqrtf(ss / (float)p.d + p.eps);
+        x1.x *= inv; x1.y *= inv; x1.z *= inv; x1.w *= inv;
+        x2.x *= inv; x2.y *= inv; x2.z *= inv; x2.w *= inv;
+        const float4 r1 = make_float4(x1.x * cs01.x - x2.x * cs01.y, x1.y * cs01.z - x2.y * cs01.w,
+                                      x1.z * cs23.x - x2.z * cs23.y, x1.w * cs23.z - x2.w * cs23.w);
+        const float4 r2 = make_float4(x2.x * cs01.x + x1.x * cs01.y, x2.y * cs01.z + x1.y * cs01.w,
+                                      x2.z * cs23.x + x1.z * cs23.y, x2.w * cs23.z + x1.w * cs23.w);
+        uint32_t h1[2], l1[2], h2[2], l2[2];
+        split2_pack(r1.x, r1.y, h1[0], l1[0]);
+        split2_pack(r1.z, r1.w, h1[1], l1[1]);
+        split2_pack(r2.x, r2.y, h2[0], l2[0]);
+        split2_pack(r2.z, r2.w, h2[1], l2[1]);
+        bf16* dst;
+        size_t plane;
+        if (head < p.Hq) {
+          dst = p.Q + (size_t)i * p.q_dim + (size_t)head * DH;
+          plane = q_plane;
+        } else {
+          const int kvh = is_v ? head - p.Hq - p.Hkv : head - p.Hq;
+          const int slot = len + (i - sg.row0);
+          const int page = sg.page_table[slot / p.page_size];
+          const int off = slot % p.page_size;
+          dst = (is_v ? sg.v_pool : sg.k_pool) +
+                kv_plane_offset(layer, sg.n_pages, p.Hkv, p.page_size, DH, page, kvh, 0) + (size_t)off * DH;
+          plane = (size_t)p.page_size * DH;
+        }
+        *reinterpret_cast<uint2*>(dst + k) = make_uint2(h1[0], h1[1]);
+        *reinterpret_cast<uint2*>(dst + k + half) = make_uint2(h2[0], h2[1]);
+        *reinterpret_cast<uint2*>(dst + plane + k) = make_uint2(l1[0], l1[1]);
+        *reinterpret_cast<uint2*>(dst + plane + k + half) = make_uint2(l2[0], l2[1]);
+      }
+    };
+
+    // ---------------- attention: softmax over one key block, unnormalised partial out
+    auto attention_step = [&]() {
+      const size_t rows_alloc = (size_t)p.n_alloc * p.Hq;
+      for (int u = cta; u < p.attn_units; u += G) {
+        const int kvh = u % p.Hkv, tile_y = (u / p.Hkv) % p.row_tiles, z = u / (p.Hkv * p.row_tiles);
+        const int split = z % tab.splits;
+        const SegDev& sg = tab.seg[z / tab.splits];
+        const int node0 = tile_y * p.nodes_per_tile;
+        if (node0 >= sg.n || sg.ctl[CTL_STATUS] != 0) continue;
+        const int L = sg.ctl[CTL_LEN];
+        const int Ltot = L + sg.n;
+        const int k_begin = split * sg.chunk;
+        const int node = node0 + row / p.group;
+        const bool row_valid = row < rows_used && node < sg.n;
+        const size_t out_row = (size_t)split * rows_alloc + (size_t)(sg.row0 + node) * p.Hq + kvh * p.group + row % p.group;
+        if (k_begin >= Ltot) {                           // key block beyond the cache: an empty partial
+          if (row_valid && eg == 0) p.attML[out_row] = make_float2(-INFINITY, 0.f);
+          continue;
+        }
+        const int kc = min(sg.chunk, Ltot - k_begin);
+        const int kc_pad = (kc + 15) & ~15;
+        const int rounds = (kc_pad + ROUND - 1) / ROUND;
+        const uint32_t par = (uint32_t)(au & 1);
+        ++au;
+        const uint32_t par2 = (uint32_t)(au2 & 1);
+        if (rounds == 2) ++au2;
+        const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 256;
+        unsigned long long anc0 = 0ull, anc1 = 0ull, anc2 = 0ull, anc3 = 0ull;
+        if (row_valid) {
+          const unsigned long long* an = p.anc + (size_t)(sg.row0 + node) * 4;
+          anc0 = an[0]; anc1 = an[1]; anc2 = an[2]; anc3 = an[3];
+        }
+        auto visible_keys = [&](int base) -> uint32_t {
+          const int t0 = base - L;                      // tree slot of the chunk's first key
+          if (t0 <= -32) return 0xFFFFFFFFu;            // all 32 keys lie in the committed prefix
+          const int ts = t0 > 0 ? t0 : 0;
+          uint32_t win = 0u;                            // ancestor bits of tree slots ts .. ts + 31
+          if (ts < SPECASR_MAX_NODES) {
+            const int w = ts >> 6, sh = ts & 63;
+            const unsigned long long a = w == 0 ? anc0 : w == 1 ? anc1 : w == 2 ? anc2 : anc3;
+            const unsigned long long bq = w == 0 ? anc1 : w == 1 ? anc2 : w == 2 ? anc3 : 0ull;
+            win = (uint32_t)(sh ? (a >> sh) | (bq << (64 - sh)) : a);
+          }
+          return t0 < 0 ? ((1u << (-t0)) - 1u) | (win << (-t0)) : win;
+        };
+        auto visible32 = [&](int c0) -> uint32_t {
+          const uint32_t mine = kc - c0 >= 32 ? 0xFFFFFFFFu : (1u << (kc - c0)) - 1u;   // c0 < kc always
+          return mine & visible_keys(k_begin + c0);
+        };
+        if (ok) ok = wwait(&sc->bar_s, par);
+        float m_row = -INFINITY;
+        if (ok) {
+          tc_fence_after();
+          float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll 1
+          for (int c0 = eg * 32; c0 < kc_pad; c0 += 64) {
+            float s[32];
+            tmem_ld32(tmem_s + lane_off + c0, s);
+            const uint32_t vis = c0 < kc ? visible32(c0) : 0u;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) m4[j & 3] = fmaxf(m4[j & 3], ((vis >> j) & 1u) ? s[j] * p.scale_log2 : -INFINITY);
+          }
+          m_row = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+        }
+        sc->red_max[eg][row] = m_row;
+        worker_bar();
+        m_row = fmaxf(sc->red_max[0][row], sc->red_max[1][row]);
+        const float m_use = m_row > -INFINITY ? m_row : 0.f;      // a fully masked row gives p = 0 everywhere
+        float l2[2] = {0.f, 0.f};
+        for (int rd = 0; rd < rounds && ok; ++rd) {
+          // the P tile holds 128 keys: the second round waits until the first round's MMAs have read it
+          if (rd > 0) ok = wwait(&sc->bar_o[0], par);
+          if (!ok) break;
+          const int c_end = min(kc_pad, (rd + 1) * ROUND);
+#pragma unroll 1
+          for (int c0 = rd * ROUND + eg * 32; c0 < c_end; c0 += 64) {
+            float s[32];
+            tmem_ld32(tmem_s + lane_off + c0, s);
+            const uint32_t vis = c0 < kc ? visible32(c0) : 0u;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) s[j] = ((vis >> j) & 1u) ? exp2f(s[j] * p.scale_log2 - m_use) : 0.f;
+#pragma unroll
+            for (int gq = 0; gq < 4; ++gq) {
+              uint32_t hi[4], lo[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const int j = gq * 8 + 2 * e;
+                l2[e & 1] += s[j] + s[j + 1];
+                split2_pack(s[j], s[j + 1], hi[e], lo[e]);
+              }
+              const int c8 = ((c0 - rd * ROUND) >> 3) + gq;     // 8-key group within this round's 128 keys
+              if (rd * ROUND + c8 * 8 < kc_pad) {
+                const int off = (c8 >> 3) * SUB + row * 128 + (((c8 & 7) ^ (row & 7)) << 4);
+                *reinterpret_cast<uint4*>(As + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                *reinterpret_cast<uint4*>(As + 2 * SUB + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+              }
+            }
+          }
+          if (rd == rounds - 1 && kc < kc_pad) {
+            // value rows past the end of the cache meet p = 0, but 0 * garbage could still be NaN: clear them
+            ok = wwait(&sc->bar_v, par);
+            if (ok && eg == 0 && row < kc_pad - kc) {
+              for (int sub = 0; sub < 2 * H2; ++sub)
+                for (int i = 0; i < 8; ++i)
+                  *reinterpret_cast<uint4*>(KVs + sub * KVSUB + (kc + row) * 128 + i * 16) = make_uint4(0, 0, 0, 0);
+            }
+          }
+          if (ok) {
+            fence_proxy_async_smem();
+            mbar_arrive(&sc->bar_p[rd]);
+          }
+        }
+        sc->red_sum[eg][row] = l2[0] + l2[1];
+        if (ok) ok = rounds == 2 ? wwait(&sc->bar_o[1], par2) : wwait(&sc->bar_o[0], par);
+        // O leaves through the (now idle) K/V region so that a warp writes whole rows
+        float4* stage = reinterpret_cast<float4*>(KVs);
+        constexpr int C4 = DH / 4;
+        if (ok) {
+          tc_fence_after();
+#pragma unroll 1
+          for (int c0 = eg * 32; c0 < DH; c0 += 64) {
+            float o[32];
+            tmem_ld32(tmem_o + lane_off + c0, o);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const int c4 = (c0 >> 2) + e;
+              stage[row * C4 + (c4 ^ (row & (C4 - 1)))] = make_float4(o[4 * e], o[4 * e + 1], o[4 * e + 2], o[4 * e + 3]);
+            }
+          }
+        }
+        tc_fence_before();
+        worker_bar();
+        if (ok) {
+          const int r_base = wwarp * 16;                       // eight warps, sixteen rows each
+#pragma unroll 1
+          for (int i = 0; i < 16; ++i) {
+            const int rr = r_base + i;
+            const int nd = node0 + rr / p.group;
+            if (rr < rows_used && nd < sg.n) {
+              const size_t orow = (size_t)split * rows_alloc + (size_t)(sg.row0 + nd) * p.Hq + kvh * p.group + rr % p.group;
+              float4* dst = reinterpret_cast<float4*>(p.attO + orow * DH);
+              for (int c4 = lane; c4 < C4; c4 += 32) dst[c4] = stage[rr * C4 + (c4 ^ (rr & (C4 - 1)))];
+            }
+          }
+          if (row_valid && eg == 0) p.attML[out_row] = make_float2(m_row, sc->red_sum[0][row] + sc->red_sum[1][row]);
+        }
+        worker_bar();                                           // the staging area and red_* are free again
+      }
+    };
+
+    // ---------------- merge of the key blocks, normalisation, hi / lo split for the O projection
+    auto merge_step = [&]() {
+      const size_t rows_alloc = (size_t)p.n_alloc * p.Hq;
+      const int rows_total = p.n * p.Hq;
+      const int n_splits = tab.splits;
+      const size_t ao_plane = (size_t)p.n_alloc * p.q_dim;
+      const int c = lane * 4;
+      for (int r = cta * 8 + wwarp; r < rows_total; r += G * 8) {
+        bf16* out = p.AO + (size_t)r * DH + c;
+        const float2 none = make_float2(-INFINITY, 0.f);
+        const float2 ml0 = lane < n_splits ? __ldcg(p.attML + (size_t)lane * rows_alloc + r) : none;
+        const float2 ml1 = lane + 32 < n_splits ? __ldcg(p.attML + (size_t)(lane + 32) * rows_alloc + r) : none;
+        constexpr int B6 = 6;
+        float4 o[B6];
+#pragma unroll
+        for (int u = 0; u < B6; ++u)
+          o[u] = (u < n_splits && c < DH) ? __ldcg(reinterpret_cast<const float4*>(p.attO + ((size_t)u * rows_alloc + r) * DH + c))
+                                          : make_float4(0.f, 0.f, 0.f, 0.f);
+        float mx = fmaxf(ml0.y > 0.f ? ml0.x : -INFINITY, ml1.y > 0.f ? ml1.x : -INFINITY);
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
+        const float w0 = ml0.y > 0.f ? exp2f(ml0.x - mx) : 0.f;
+        const float w1 = ml1.y > 0.f ? exp2f(ml1.x - mx) : 0.f;
+        float den = 0.f;                                 // terms added in block order: independent of timing
+        for (int s = 0; s < n_splits; ++s) den += __shfl_sync(0xFFFFFFFFu, s < 32 ? ml0.y * w0 : ml1.y * w1, s & 31);
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int s0 = 0; s0 < n_splits; s0 += B6) {
+          if (s0 > 0) {
+#pragma unroll
+            for (int u = 0; u < B6; ++u) {
+              const int s = s0 + u;
+              o[u] = (s < n_splits && c < DH) ? __ldcg(reinterpret_cast<const float4*>(p.attO + ((size_t)s * rows_alloc + r) * DH + c))
+                                              : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+          }
+#pragma unroll
+          for (int u = 0; u < B6; ++u) {
+            const int s = s0 + u;
+            float w = __shfl_sync(0xFFFFFFFFu, s < 32 ? w0 : w1, s & 31);
+            if (s >= n_splits || !(w > 0.f)) {
+              w = 0.f;
+              o[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            acc.x += o[u].x * w; acc.y += o[u].y * w; acc.z += o[u].z * w; acc.w += o[u].w * w;
+          }
+        }
+        if (c < DH) {
+          const float rcp = 1.f / den;
+          uint32_t ph[2], pl[2];
+          split2_pack(acc.x * rcp, acc.y * rcp, ph[0], pl[0]);
+          split2_pack(acc.z * rcp, acc.w * rcp, ph[1], pl[1]);
+          *reinterpret_cast<uint2*>(out) = make_uint2(ph[0], ph[1]);
+          *reinterpret_cast<uint2*>(out + ao_plane) = make_uint2(pl[0], pl[1]);
+        }
+      }
+    };
+
+    // ================= the sequence of steps
+    const size_t stride_d = (size_t)p.n_alloc * p.d;
+    const size_t stride_qkv = (size_t)p.n_alloc * p.qkv_dim;
+    for (int l = 0; l < p.n_layers; ++l) {
+      const int base = l * ST_PER_LAYER;
+      {
+        STACK_TRACE_BEGIN();
+        if (l > 0) wait_step(base - 1);                  // the previous layer's down projection
+        norm_step(p.gains[2 * l], l > 0 ? p.splits_down : 0, stride_d);
+        arrive_step();
+        STACK_TRACE_END(SPECASR_KIND_NORM, l);
+      }
+      {
+        STACK_TRACE_BEGIN();
+        epi_partial(gemm_of(p, l, ST_QKV, cta, G), stride_qkv);
+        arrive_step();
+        STACK_TRACE_END(SPECASR_KIND_GEMM_QKV, l);
+      }
+      {
+        STACK_TRACE_BEGIN();
+        wait_step(base + ST_QKV);
+        rope_step(l);
+        arrive_step();
+        STACK_TRACE_END(SPECASR_KIND_ROPE, l);
+      }
+      {
+        STACK_TRACE_BEGIN();
+        attention_step();
+        worker_bar();
+        if (wtid == 0) {
+          __threadfence_block();
+          *(volatile int*)&sc->attn_done = l + 1;
+        }
+        arrive_step();
+        STACK_TRACE_END(SPECASR_KIND_ATTN, l);
+      }
+      {
+        STACK_TRACE_BEGIN();
+        wait_step(base + ST_ATTN);
+        merge_step();
+        arrive_step();
+        STACK_TRACE_END(SPECASR_KIND_ATTN_MERGE, l);
+      }
+      {
+        STACK_TRACE_BEGIN();
+        epi_partial(gemm_of(p, l, ST_O, cta, G), stride_d);
+        arrive_step();
+        STACK_TRACE_END(SPECASR_KIND_GEMM_O, l);
+      }
+      {
+        STACK_TRACE_BEGIN();
+        wait_step(base + ST_O);
+        norm_step(p.gains[2 * l + 1], p.splits_o, stride_d);
+        arrive_step();
+        STACK_TRACE_END(SPECASR_KIND_NORM, l);
+      }
+      {
+        STACK_TRACE_BEGIN();
+        wait_step(base + ST_NORM2);
+        load_inv();
+        epi_streamk(gemm_of(p, l, ST_GU, cta, G), true, p.epoch0 + 1 + l);
+        arrive_step();
+        STACK_TRACE_END(SPECASR_KIND_GEMM_GU, l);
+      }
+      {
+        STACK_TRACE_BEGIN();
+        epi_partial(gemm_of(p, l, ST_DOWN, cta, G), stride_d);
+        arrive_step();
+        STACK_TRACE_END(SPECASR_KIND_GEMM_DOWN, l);
+      }
+    }
+    if (p.want_head) {
+      {
+        STACK_TRACE_BEGIN();
+        wait_step(steps_total - 1);
+        norm_step(p.gains[2 * p.n_layers], p.splits_down, stride_d);
+        arrive_step();
+        STACK_TRACE_END(SPECASR_KIND_NORM, p.n_layers);
+      }
+      {
+        STACK_TRACE_BEGIN();
+        wait_step(steps_total);
+        load_inv();
+        epi_streamk(gemm_of(p, 0, -1, cta, G), false, p.epoch0 + 1 + p.n_layers);
+        STACK_TRACE_END(SPECASR_KIND_GEMM_LM, p.n_layers);
+      }
+    }
+    (void)arrived;
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (*abort) {
+    // give copies still in flight time to land before the shared memory is handed back
+    for (int i = 0; i < 64; ++i) __nanosleep(20000);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+template <int DH>
+cudaError_t launch_dh(const CUtensorMap& tmH, const CUtensorMap& tmAO, const CUtensorMap& tmA, const CUtensorMap& tmQ,
+                      const SegTable& tab, const StackParams& p, int grid, size_t smem, cudaStream_t s) {
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(k_stack<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(NUM_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeCooperative;           // all CTAs co-resident, or the launch fails
+  attr[0].val.cooperative = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, k_stack<DH>, tmH, tmAO, tmA, tmQ, tab, p);
+}
+
+}  // namespace
+
+// Shapes the fused kernel covers: tensor-core attention (head_dim 64 / 128, pages of a multiple of 16 slots),
+// up to 64 token rows (one activation box, both planes in one MMA), key-block count within one counter lane pair.
+bool fused_stack_supported(const specasr_kv* wk, int n_total, bool att_tc, int splits) {
+  const specasr_model* m = wk->m;
+  if (m->cfg.gemm_path != 0 || !att_tc || !wk->attn_tc || m->w_maps_dev == nullptr) return false;
+  if (n_total < 1 || n_total > 64) return false;
+  if (splits > kMaxAttnSplits) return false;
+  // every weight tile of a linear projection needs a CTA of its own
+  const int tiles_qkv = (m->qkv_dim + TILE_M - 1) / TILE_M, tiles_d = (m->cfg.d_model + TILE_M - 1) / TILE_M;
+  if (tiles_qkv > m->n_sm || tiles_d > m->n_sm) return false;
+  return true;
+}
+
+size_t fused_stack_sync_bytes(const specasr_model* m) {
+  return (((size_t)m->cfg.n_layers * ST_PER_LAYER + 2) * sizeof(int32_t) + 255) / 256 * 256;
+}
+
+bool launch_fused_stack(specasr_model* m, specasr_kv* wk, const SegTable& tab, int n_total, int n_max,
+                        const int32_t* ctl_shared, bool want_head, float* out_logits, cudaStream_t s) {
+  const specasr_model_config& c = m->cfg;
+  int n_pad = 16;
+  while (n_pad < n_total) n_pad <<= 1;
+  StackParams p;
+  memset(&p, 0, sizeof(p));
+  p.n_layers = c.n_layers; p.d = c.d_model; p.qkv_dim = m->qkv_dim; p.q_dim = m->q_dim;
+  p.Hq = c.n_heads; p.Hkv = c.n_kv_heads; p.ffn = c.ffn; p.vocab = c.vocab; p.page_size = c.page_size;
+  p.max_positions = c.max_positions;
+  p.eps = c.rms_eps;
+  p.scale_log2 = 1.4426950408889634f / sqrtf((float)c.head_dim);
+  p.w_maps = m->w_maps_dev;
+  p.gains = m->gains_dev;
+  p.rope = m->rope_table;
+  p.n = n_total; p.n_pad = n_pad; p.n_alloc = wk->n_alloc;
+  p.stage_bytes = W_STAGE_BYTES + KSUB * n_pad * 2 * SUB_K * 2;
+  const int epi_bytes = 2 * n_pad * 64 * 2;
+  const int attn_bytes = 4 * SUB + 2 * (c.head_dim / 64) * KVSUB;
+  int stages = (SMEM_LIMIT - (int)sizeof(StackCtl) - epi_bytes - 1024) / p.stage_bytes;
+  if (stages > MAX_STAGES) stages = MAX_STAGES;
+  p.stages = stages;
+  p.ring_bytes = stages * p.stage_bytes;
+  if (p.ring_bytes < attn_bytes) p.ring_bytes = (attn_bytes + 1023) & ~1023;
+  p.splits_qkv = gemm_tc_pick_splits(m, m->qkv_dim, c.d_model, n_pad);
+  p.splits_o = gemm_tc_pick_splits(m, c.d_model, m->q_dim, n_pad);
+  p.splits_down = gemm_tc_pick_splits(m, c.d_model, c.ffn, n_pad);
+  p.epoch0 = wk->gemm_epoch;
+  wk->gemm_epoch += c.n_layers + 1;
+  p.want_head = want_head ? 1 : 0;
+  p.group = c.n_heads / c.n_kv_heads;
+  p.nodes_per_tile = 128 / p.group;
+  p.row_tiles = (n_max + p.nodes_per_tile - 1) / p.nodes_per_tile;
+  p.attn_units = c.n_kv_heads * p.row_tiles * tab.count * tab.splits;
+  p.ctl = const_cast<int32_t*>(ctl_shared);
+  p.sync = wk->ws.sync;
+  p.X = wk->ws.X; p.P = wk->ws.P; p.fixP = wk->ws.fixP; p.fixFlag = wk->ws.fixFlag;
+  p.H = wk->ws.H; p.Q = wk->ws.Q; p.AO = wk->ws.AO; p.A = wk->ws.A;
+  p.attO = wk->ws.attO; p.attML = wk->ws.attML; p.ssq = wk->ws.ssq; p.amax = wk->ws.amax;
+  p.logits = out_logits;
+  p.pos = wk->ws.pos; p.anc = wk->ws.anc;
+#ifdef SPECASR_TRACE
+  p.tr = wk->trace;
+#endif
+  const size_t smem = (size_t)p.ring_bytes + sizeof(StackCtl) + epi_bytes + 1024;
+  int idx = 0;                                           // activation maps are indexed by log2(box rows / 16)
+  for (int b = 16; b < n_pad; b <<= 1) ++idx;
+  LaunchScope scope(wk, SPECASR_KIND_STACK, s);
+  cudaError_t e = cudaMemsetAsync(wk->ws.sync, 0, fused_stack_sync_bytes(m), s);
+  if (e == cudaSuccess) {
+    if (c.head_dim == 64) e = launch_dh<64>(wk->tm_H[idx], wk->tm_AO[idx], wk->tm_A[idx], wk->tm_Q, tab, p, m->n_sm, smem, s);
+    else e = launch_dh<128>(wk->tm_H[idx], wk->tm_AO[idx], wk->tm_A[idx], wk->tm_Q, tab, p, m->n_sm, smem, s);
+  }
+  if (e != cudaSuccess) {
+    set_error("fused layer stack launch failed: %s", cudaGetErrorString(e));
+    return false;
+  }
+  return true;
+}

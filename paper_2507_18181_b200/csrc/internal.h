@@ -63,6 +63,8 @@ struct specasr_model {
   float2* rope_table;       // [max_positions][dh/2] (cos, sin), built in fp64 on the host
   std::vector<CUtensorMap> tm_wqkv, tm_wo, tm_wgu, tm_wd;
   CUtensorMap tm_lm;
+  CUtensorMap* w_maps_dev;  // device copy for the fused layer-stack kernel: [4 * layers + 1] QKV, O, gate/up, down, ..., vocabulary
+  const float** gains_dev;  // device array [2 * layers + 1]: attention / FFN norm gains per layer, then the final norm
   int n_sm;
 };
 
@@ -83,6 +85,8 @@ struct Workspace {
   float2* attML;            // [kMaxAttnSplits][n_alloc * Hq]     (running max in log2 units, sum)
   unsigned long long* amax; // [lm_tiles][n_alloc] packed (ordered logit, ~token id) per vocab tile
   CUtensorMap* tmKV;        // [2] device copies of the K and V pool descriptors (tensor-core attention)
+  float* ssq;               // [2][n_alloc] sums of squares of the two halves of every residual row (fused stack)
+  int32_t* sync;            // arrival counters of the fused stack kernel, one per step of the call
   size_t bytes;
 };
 
@@ -237,6 +241,12 @@ bool attention_tc_plan(const specasr_model* m, int n, int total_len, int sm_budg
                        int* chunk);
 bool attention_tc_make_maps(specasr_kv* kv);
 void launch_tree_attention_tc(specasr_kv* wk, const SegTable& t, int n_max, int layer, cudaStream_t s);
+
+// ---- fused_stack.cu: the whole layer stack as one persistent kernel
+bool fused_stack_supported(const specasr_kv* wk, int n_total, bool att_tc, int splits);
+size_t fused_stack_sync_bytes(const specasr_model* m);
+bool launch_fused_stack(specasr_model* m, specasr_kv* wk, const SegTable& tab, int n_total, int n_max,
+                        const int32_t* ctl_shared, bool want_head, float* out_logits, cudaStream_t s);
 
 // ---- gemm_fma.cu / gemm_tcgen05.cu
 enum GemmEpilogue {

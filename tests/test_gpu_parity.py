@@ -490,8 +490,8 @@ kv.verify(d_t, d_p)
 torch.cuda.synchronize()
 plain = kv.out_argmax[:15].clone()
 rec = kv.trace(lambda: kv.verify(d_t, d_p))
-kinds = [B.KIND_NAMES[int(k)] for k in rec[:, 0]]
-# one launch each of prep, embedding, LM head and accept; per layer 2 norms, 4 projections, rotary, attention, merge
+kinds = [B.KIND_NAMES[int(k) & 0xFF] for k in rec[:, 0]]    # bits 8.. carry layer + 1 for the steps of the fused stack
+# one launch each of prep, embedding and accept; per layer 2 norms, 4 projections, rotary, attention, merge, then the LM head
 assert kinds.count("accept") == 1 and "gemm_lm" in kinds
 for name in ("norm", "gemm_qkv", "rope", "attn", "attn_merge", "gemm_o", "gemm_gu", "gemm_down"):
     assert name in kinds, name
