@@ -31,6 +31,8 @@
 //
 // The attention step borrows the ring's shared memory (Q / P tiles and K / V pages of one key block), so the
 // weight producer resumes when the CTA's attention units are done.
+#include <stdlib.h>
+
 #include "internal.h"
 #include "device_utils.cuh"
 #include "sm100_ptx.cuh"
@@ -85,6 +87,7 @@ struct StackParams {
   const float2* rope;
   int n, n_pad, n_alloc, stages, stage_bytes, ring_bytes;
   int splits_qkv, splits_o, splits_down, epoch0, want_head, group, nodes_per_tile, row_tiles, attn_units;
+  int lookahead;                        // weight units the L2 prefetch runs ahead of the ring loads, per CTA
   int32_t* ctl;                         // control block whose status word ends the call
   int32_t* sync;                        // [steps of the call] arrival counters, zeroed before the launch
   float* X;
@@ -127,7 +130,7 @@ struct Gemm {
   const CUtensorMap* tmW;
   int M, K, KB, tiles, splits;          // splits > 0: linear output in `splits` k-parts per tile
   int g_eff;                            // CTAs that take part
-  long long U, u0, u1;                  // all (tile, k-block) units; this CTA's range
+  int U, u0, u1;                        // all (tile, k-block) units; this CTA's range
 };
 
 __device__ __forceinline__ Gemm gemm_of(const StackParams& p, int layer, int which, int cta, int G) {
@@ -141,26 +144,34 @@ __device__ __forceinline__ Gemm gemm_of(const StackParams& p, int layer, int whi
   }
   g.KB = (g.K + KSUB * SUB_K - 1) / (KSUB * SUB_K);
   g.tiles = (g.M + TILE_M - 1) / TILE_M;
-  g.U = (long long)g.tiles * g.KB;
+  g.U = g.tiles * g.KB;
   if (g.splits > 0) {
     g.g_eff = g.tiles * g.splits;
     if (cta < g.g_eff) {
       const int tile = cta / g.splits, split = cta % g.splits;
-      g.u0 = (long long)tile * g.KB + (long long)split * g.KB / g.splits;
-      g.u1 = (long long)tile * g.KB + (long long)(split + 1) * g.KB / g.splits;
+      g.u0 = tile * g.KB + split * g.KB / g.splits;
+      g.u1 = tile * g.KB + (split + 1) * g.KB / g.splits;
     } else {
       g.u0 = g.u1 = 0;
     }
   } else {
-    g.g_eff = g.U < G ? (int)g.U : G;
+    g.g_eff = g.U < G ? g.U : G;
     if (cta < g.g_eff) {
-      g.u0 = cta * g.U / g.g_eff;
-      g.u1 = (cta + 1) * g.U / g.g_eff;
+      g.u0 = (int)((long long)cta * g.U / g.g_eff);
+      g.u1 = (int)((long long)(cta + 1) * g.U / g.g_eff);
     } else {
       g.u0 = g.u1 = 0;
     }
   }
   return g;
+}
+
+// The projection that step `st` of layer `l` runs (l == n_layers: final norm at st 0, vocabulary projection at st 1),
+// or -2 if the step is not a projection.  Every role walks the steps in one loop, so that each piece of code has a
+// single call site: the kernel's instructions are fetched again on every layer, and their size is time.
+__device__ __forceinline__ int gemm_kind_of(int l, int st, int n_layers) {
+  if (l == n_layers) return st == 1 ? -1 : -2;
+  return (st == ST_QKV || st == ST_O || st == ST_GU || st == ST_DOWN) ? st : -2;
 }
 
 // Bounded poll of a word that only grows.  Returns false when the limit ran out or the call was aborted.
@@ -208,24 +219,38 @@ __device__ __forceinline__ int seg_of_row(const SegTable& tab, int row) {
   return b;
 }
 
+// Device-side trace (build variant): worker thread 0 of every CTA appends one record per step
+// {kind | (layer + 1) << 8, start, end, time its wait for the previous steps ended} and, at a few points inside a
+// step, point records {(100 + point) | (layer + 1) << 8, now, now, 0}.
 #ifdef SPECASR_TRACE
-#define STACK_TRACE_BEGIN() const unsigned long long tr_t0_ = wtid == 0 ? global_ns() : 0ull
-#define STACK_TRACE_END(kind, layer)                                                     \
+#define STACK_TRACE_BEGIN() unsigned long long tr_t0_ = wtid == 0 ? global_ns() : 0ull, tr_mark_ = tr_t0_
+#define STACK_TRACE_MARK() do { if (wtid == 0) tr_mark_ = global_ns(); } while (0)
+#define STACK_TRACE_WRITE(code, layer, a, b, c)                                          \
   do {                                                                                   \
     if (wtid == 0 && p.tr.buf != nullptr) {                                              \
       const unsigned long long slot_ = atomicAdd(p.tr.buf, 1ull);                        \
       if (slot_ < p.tr.cap) {                                                            \
         unsigned long long* e_ = p.tr.buf + 2 + slot_ * 4;                               \
-        e_[0] = (unsigned long long)(kind) | ((unsigned long long)((layer) + 1) << 8);   \
-        e_[1] = tr_t0_;                                                                  \
-        e_[2] = global_ns();                                                             \
-        e_[3] = tr_t0_;                                                                  \
+        e_[0] = (unsigned long long)(code) | ((unsigned long long)((layer) + 1) << 8);   \
+        e_[1] = (a);                                                                     \
+        e_[2] = (b);                                                                     \
+        e_[3] = (c);                                                                     \
       }                                                                                  \
+    }                                                                                    \
+  } while (0)
+#define STACK_TRACE_END(kind, layer) STACK_TRACE_WRITE(kind, layer, tr_t0_, global_ns(), tr_mark_)
+#define STACK_TRACE_POINT(point, layer)                                                  \
+  do {                                                                                   \
+    if (wtid == 0 && p.tr.buf != nullptr && p.tr.buf[1] != 0ull) {   /* word 1 of the buffer switches points on */                               \
+      const unsigned long long now_ = global_ns();                                       \
+      STACK_TRACE_WRITE(100 + (point), layer, now_, now_, 0ull);                         \
     }                                                                                    \
   } while (0)
 #else
 #define STACK_TRACE_BEGIN()
+#define STACK_TRACE_MARK()
 #define STACK_TRACE_END(kind, layer)
+#define STACK_TRACE_POINT(point, layer)
 #endif
 
 template <int DH>
@@ -279,7 +304,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
   volatile int* abort = &sc->abort;
   int32_t* status = p.ctl + CTL_STATUS;
   const bool live = *(volatile int32_t*)status == 0;
-  const int steps_total = p.n_layers * ST_PER_LAYER;    // index of the final norm; the vocabulary projection follows
+  const int n_steps = p.n_layers * ST_PER_LAYER + (p.want_head ? 2 : 0);   // final norm and vocabulary projection last
 
   // attention geometry shared by all roles
   const int rows_used = p.nodes_per_tile * p.group;
@@ -288,29 +313,83 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
     // the call was refused before it started (shared status): nothing to do
   } else if (warp == 0 && lane == 0) {
     // =========================================================== weight producer
-    int it = 0;                                          // ring slots used so far
-    bool ok = true;
-    auto stream_weights = [&](const Gemm& g) {
-      for (long long u = g.u0; u < g.u1 && ok; ++u, ++it) {
-        const int tile = (int)(u / g.KB), kb = (int)(u % g.KB), s = it % p.stages;
-        if (!mbar_wait(&sc->empty[s], (uint32_t)((it / p.stages) & 1) ^ 1u, abort, status)) {
-          ok = false;
+    // Two cursors walk this CTA's (layer, projection, unit) list, which is fixed for the call: `ld` issues the TMA
+    // loads into the ring, `pf` runs up to p.lookahead units ahead of it and only asks for the same boxes to be
+    // brought into L2.  While the ring is full or lent to the attention step -- the stretches in which HBM would
+    // otherwise idle -- the look-ahead keeps the weights of the coming projections moving.
+    struct Cursor {
+      int l, ph;                 // layer; 0..3 = QKV, O, gate/up, down; layer == n_layers: the vocabulary projection
+      int u, u1, tile, kb, KB;   // next unit, end of the range, and the unit as (weight tile, k-block)
+      const CUtensorMap* tmW;
+      bool done;
+    };
+    auto phase_of = [&](int ph) { return ph == 0 ? ST_QKV : ph == 1 ? ST_O : ph == 2 ? ST_GU : ST_DOWN; };
+    auto settle = [&](Cursor& c) {                       // enter the next phase that has a unit for this CTA
+      while (!c.done && c.u >= c.u1) {
+        if (c.l >= p.n_layers) {
+          c.done = true;
           break;
         }
-        uint8_t* st = ring + (size_t)s * p.stage_bytes;
-        mbar_expect_tx(&sc->full[s], (uint32_t)W_STAGE_BYTES);
-        for (int q = 0; q < KSUB; ++q)                   // rows past M and columns past K read as zeros
-          tma_load_2d(st + q * W_SUB_BYTES, g.tmW, (kb * KSUB + q) * SUB_K, tile * TILE_M, &sc->full[s]);
+        if (++c.ph == 4) {
+          c.ph = 0;
+          ++c.l;
+        }
+        Gemm g;
+        if (c.l < p.n_layers) g = gemm_of(p, c.l, phase_of(c.ph), cta, G);
+        else if (p.want_head) g = gemm_of(p, 0, -1, cta, G);
+        else {
+          c.done = true;
+          break;
+        }
+        c.u = g.u0; c.u1 = g.u1; c.KB = g.KB; c.tmW = g.tmW;
+        c.tile = g.u0 / g.KB;
+        c.kb = g.u0 % g.KB;
       }
     };
-    for (int l = 0; l < p.n_layers && ok; ++l) {
-      stream_weights(gemm_of(p, l, ST_QKV, cta, G));
-      if (ok) ok = wait_smem_ge(&sc->attn_done, l + 1, abort, status);   // the attention step owns the ring meanwhile
-      if (ok) stream_weights(gemm_of(p, l, ST_O, cta, G));
-      if (ok) stream_weights(gemm_of(p, l, ST_GU, cta, G));
-      if (ok) stream_weights(gemm_of(p, l, ST_DOWN, cta, G));
+    auto advance = [&](Cursor& c) {
+      ++c.u;
+      if (++c.kb == c.KB) {
+        c.kb = 0;
+        ++c.tile;
+      }
+      if (c.u >= c.u1) settle(c);
+    };
+    Cursor ld, pf;
+    ld.l = 0; ld.ph = -1; ld.u = ld.u1 = 0; ld.tile = ld.kb = 0; ld.KB = 1; ld.tmW = nullptr; ld.done = false;
+    settle(ld);
+    pf = ld;
+    int slot = 0;                                        // next ring slot
+    uint32_t ring_par = 0u;                              // parity of the ring round in progress
+    int attn_waited = 0;                                 // attention steps whose end this thread has seen
+    bool ok = true;
+    while (!ld.done && ok) {
+      // the attention step of layer l owns the ring between that layer's QKV and O projections
+      const int need = ld.l < p.n_layers ? (ld.ph == 0 ? ld.l : ld.l + 1) : p.n_layers;
+      if (need > attn_waited) {
+        // HBM idles from here until the attention step ends: ask for the next units to be brought into L2
+        pf = ld;
+        for (int a = 0; a < p.lookahead && !pf.done; ++a) {
+          for (int q = 0; q < KSUB; ++q) tma_prefetch_2d(pf.tmW, (pf.kb * KSUB + q) * SUB_K, pf.tile * TILE_M);
+          advance(pf);
+        }
+        ok = wait_smem_ge(&sc->attn_done, need, abort, status);
+        attn_waited = need;
+        if (!ok) break;
+      }
+      if (!mbar_wait(&sc->empty[slot], ring_par ^ 1u, abort, status)) {
+        ok = false;
+        break;
+      }
+      uint8_t* st = ring + (size_t)slot * p.stage_bytes;
+      mbar_expect_tx(&sc->full[slot], (uint32_t)W_STAGE_BYTES);
+      for (int q = 0; q < KSUB; ++q)                     // rows past M and columns past K read as zeros
+        tma_load_2d(st + q * W_SUB_BYTES, ld.tmW, (ld.kb * KSUB + q) * SUB_K, ld.tile * TILE_M, &sc->full[slot]);
+      advance(ld);
+      if (++slot == p.stages) {
+        slot = 0;
+        ring_par ^= 1u;
+      }
     }
-    if (ok && p.want_head) stream_weights(gemm_of(p, 0, -1, cta, G));
   } else if (warp == 10) {
     // =========================================================== activation producer / attention producer
     int it = 0;
@@ -321,8 +400,9 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
       if (lane == 0) {
         ok = wait_word_ge(p.sync + ready_step, G, abort, status);
         fence_proxy_async_all();
-        for (long long u = g.u0; u < g.u1 && ok; ++u, ++it) {
-          const int kb = (int)(u % g.KB), s = it % p.stages;
+        int kb = g.u0 % g.KB;
+        for (int u = g.u0; u < g.u1 && ok; ++u, ++it) {
+          const int s = it % p.stages;
           if (!mbar_wait(&sc->empty[s], (uint32_t)((it / p.stages) & 1) ^ 1u, abort, status)) {
             ok = false;
             break;
@@ -331,80 +411,83 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
           mbar_expect_tx(&sc->full[s], (uint32_t)act_stage);
           for (int q = 0; q < KSUB; ++q)
             tma_load_3d(st + q * act_sub, tmAct, (kb * KSUB + q) * SUB_K, 0, 0, &sc->full[s]);
+          if (++kb == g.KB) kb = 0;
         }
       }
       ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
       it = __shfl_sync(0xFFFFFFFFu, it, 0);
     };
-    for (int l = 0; l < p.n_layers && ok; ++l) {
-      const int base = l * ST_PER_LAYER;
-      stream_acts(gemm_of(p, l, ST_QKV, cta, G), &tmH, base + ST_NORM1);
-      // ---- attention units of this CTA: lane 0 fetches Q, lane j page j of K and later of V
-      if (ok && cta < p.attn_units) {
-        if (lane == 0) {
-          ok = wait_word_ge(p.sync + base + ST_ROPE, G, abort, status);
-          fence_proxy_async_all();
+    for (int sidx = 0; sidx < n_steps && ok; ++sidx) {
+      const int l = sidx / ST_PER_LAYER, st = sidx - l * ST_PER_LAYER;
+      const int gk = gemm_kind_of(l, st, p.n_layers);
+      if (gk != -2) {
+        // the step before a projection is the one that writes its input
+        const CUtensorMap* tmAct = gk == ST_O ? &tmAO : gk == ST_DOWN ? &tmA : &tmH;
+        stream_acts(gemm_of(p, l, gk, cta, G), tmAct, sidx - 1);
+      } else if (l < p.n_layers && st == ST_ATTN) {
+        // ---- attention units of this CTA: lane 0 fetches Q, lane j page j of K and later of V
+        if (ok && cta < p.attn_units) {
+          if (lane == 0) {
+            ok = wait_word_ge(p.sync + sidx - 1, G, abort, status);
+            fence_proxy_async_all();
+          }
+          ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
         }
-        ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+        for (int u = cta; u < p.attn_units && ok; u += G) {
+          const int kvh = u % p.Hkv, tile_y = (u / p.Hkv) % p.row_tiles, z = u / (p.Hkv * p.row_tiles);
+          const int split = z % tab.splits;
+          const SegDev& sg = tab.seg[z / tab.splits];
+          const int node0 = tile_y * p.nodes_per_tile;
+          if (node0 >= sg.n || sg.ctl[CTL_STATUS] != 0) continue;
+          const int L = sg.ctl[CTL_LEN];
+          const int Ltot = L + sg.n;
+          const int k_begin = split * sg.chunk;
+          if (k_begin >= Ltot) continue;
+          const int kc = min(sg.chunk, Ltot - k_begin);
+          const int pages = (kc + p.page_size - 1) / p.page_size;
+          const uint32_t par = (uint32_t)(au & 1);
+          ++au;
+          int my_page = 0;
+          if (lane < pages) my_page = sg.page_table[split * (sg.chunk / p.page_size) + lane];
+          const uint32_t q_bytes = 2 * H2 * rows_used * 128;
+          const uint32_t kv_bytes = 2 * H2 * pages * p.page_size * 128;
+          if (lane == 0) {
+            mbar_expect_tx(&sc->bar_qk, q_bytes + kv_bytes);
+            mbar_expect_tx(&sc->bar_v, kv_bytes);
+          }
+          __syncwarp();
+          if (lane == 0) {
+            for (int plane = 0; plane < 2; ++plane)
+              for (int h = 0; h < H2; ++h)
+                tma_load_4d(As + (plane * H2 + h) * SUB, &tmQ, h * 64, kvh * p.group, sg.row0 + node0, plane, &sc->bar_qk);
+          }
+          const int c4 = l * sg.n_pages + my_page;
+          const int off = lane * p.page_size * 128;
+          if (lane < pages) {
+            for (int plane = 0; plane < 2; ++plane)
+              for (int h = 0; h < H2; ++h)
+                tma_load_5d(KVs + (plane * H2 + h) * KVSUB + off, sg.tmK, h * 64, 0, plane, kvh, c4, &sc->bar_qk);
+          }
+          // V takes K's place once the S MMAs have read K
+          ok = mbar_wait(&sc->bar_s, par, abort, status);
+          if (ok && lane < pages) {
+            for (int plane = 0; plane < 2; ++plane)
+              for (int h = 0; h < H2; ++h)
+                tma_load_5d(KVs + (plane * H2 + h) * KVSUB + off, sg.tmV, h * 64, 0, plane, kvh, c4, &sc->bar_v);
+          }
+          ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+        }
       }
-      for (int u = cta; u < p.attn_units && ok; u += G) {
-        const int kvh = u % p.Hkv, tile_y = (u / p.Hkv) % p.row_tiles, z = u / (p.Hkv * p.row_tiles);
-        const int split = z % tab.splits;
-        const SegDev& sg = tab.seg[z / tab.splits];
-        const int node0 = tile_y * p.nodes_per_tile;
-        if (node0 >= sg.n || sg.ctl[CTL_STATUS] != 0) continue;
-        const int L = sg.ctl[CTL_LEN];
-        const int Ltot = L + sg.n;
-        const int k_begin = split * sg.chunk;
-        if (k_begin >= Ltot) continue;
-        const int kc = min(sg.chunk, Ltot - k_begin);
-        const int pages = (kc + p.page_size - 1) / p.page_size;
-        const uint32_t par = (uint32_t)(au & 1);
-        ++au;
-        int my_page = 0;
-        if (lane < pages) my_page = sg.page_table[split * (sg.chunk / p.page_size) + lane];
-        const uint32_t q_bytes = 2 * H2 * rows_used * 128;
-        const uint32_t kv_bytes = 2 * H2 * pages * p.page_size * 128;
-        if (lane == 0) {
-          mbar_expect_tx(&sc->bar_qk, q_bytes + kv_bytes);
-          mbar_expect_tx(&sc->bar_v, kv_bytes);
-        }
-        __syncwarp();
-        if (lane == 0) {
-          for (int plane = 0; plane < 2; ++plane)
-            for (int h = 0; h < H2; ++h)
-              tma_load_4d(As + (plane * H2 + h) * SUB, &tmQ, h * 64, kvh * p.group, sg.row0 + node0, plane, &sc->bar_qk);
-        }
-        const int c4 = l * sg.n_pages + my_page;
-        const int off = lane * p.page_size * 128;
-        if (lane < pages) {
-          for (int plane = 0; plane < 2; ++plane)
-            for (int h = 0; h < H2; ++h)
-              tma_load_5d(KVs + (plane * H2 + h) * KVSUB + off, sg.tmK, h * 64, 0, plane, kvh, c4, &sc->bar_qk);
-        }
-        // V takes K's place once the S MMAs have read K
-        ok = mbar_wait(&sc->bar_s, par, abort, status);
-        if (ok && lane < pages) {
-          for (int plane = 0; plane < 2; ++plane)
-            for (int h = 0; h < H2; ++h)
-              tma_load_5d(KVs + (plane * H2 + h) * KVSUB + off, sg.tmV, h * 64, 0, plane, kvh, c4, &sc->bar_v);
-        }
-        ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
-      }
-      if (ok) stream_acts(gemm_of(p, l, ST_O, cta, G), &tmAO, base + ST_MERGE);
-      if (ok) stream_acts(gemm_of(p, l, ST_GU, cta, G), &tmH, base + ST_NORM2);
-      if (ok) stream_acts(gemm_of(p, l, ST_DOWN, cta, G), &tmA, base + ST_GU);
     }
-    if (ok && p.want_head) stream_acts(gemm_of(p, 0, -1, cta, G), &tmH, steps_total);
   } else if (warp == 1 && lane == 0) {
     // =========================================================== MMA issuer
     int it = 0, seg = 0, au = 0, au2 = 0;
     bool ok = true;
     const uint32_t idesc = make_idesc_bf16(2 * n_pad);
     auto run_gemm = [&](const Gemm& g) {
-      for (long long u = g.u0; u < g.u1 && ok; ++seg) {
-        const int kb0 = (int)(u % g.KB);
-        const int kb1 = (int)((g.u1 - u) < (long long)(g.KB - kb0) ? kb0 + (g.u1 - u) : g.KB);
+      for (int u = g.u0; u < g.u1 && ok; ++seg) {
+        const int kb0 = u % g.KB;
+        const int kb1 = (g.u1 - u) < (g.KB - kb0) ? kb0 + (g.u1 - u) : g.KB;
         const int b = seg & 1;
         if (!mbar_wait(&sc->acc_empty[b], (uint32_t)((seg >> 1) & 1) ^ 1u, abort, status)) {
           ok = false;
@@ -436,72 +519,73 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
         u += kb1 - kb0;
       }
     };
-    for (int l = 0; l < p.n_layers && ok; ++l) {
-      run_gemm(gemm_of(p, l, ST_QKV, cta, G));
-      // ---- attention units
-      for (int u = cta; u < p.attn_units && ok; u += G) {
-        const int tile_y = (u / p.Hkv) % p.row_tiles, z = u / (p.Hkv * p.row_tiles);
-        const int split = z % tab.splits;
-        const SegDev& sg = tab.seg[z / tab.splits];
-        if (tile_y * p.nodes_per_tile >= sg.n || sg.ctl[CTL_STATUS] != 0) continue;
-        const int Ltot = sg.ctl[CTL_LEN] + sg.n;
-        const int k_begin = split * sg.chunk;
-        if (k_begin >= Ltot) continue;
-        const int kc = min(sg.chunk, Ltot - k_begin);
-        const int kc_pad = (kc + 15) & ~15;
-        const int rounds = (kc_pad + ROUND - 1) / ROUND;
-        const uint32_t par = (uint32_t)(au & 1);
-        ++au;
-        const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 256;
-        ok = mbar_wait(&sc->bar_qk, par, abort, status);
-        if (!ok) break;
-        tc_fence_after();
-        {
-          const uint32_t idesc_s = make_idesc_bf16(kc_pad);
-          const uint32_t a0 = smem_u32(As), b0 = smem_u32(KVs);
+    for (int sidx = 0; sidx < n_steps && ok; ++sidx) {
+      const int l = sidx / ST_PER_LAYER, st = sidx - l * ST_PER_LAYER;
+      const int gk = gemm_kind_of(l, st, p.n_layers);
+      if (gk != -2) {
+        run_gemm(gemm_of(p, l, gk, cta, G));
+      } else if (l < p.n_layers && st == ST_ATTN) {
+        // ---- attention units
+        for (int u = cta; u < p.attn_units && ok; u += G) {
+          const int tile_y = (u / p.Hkv) % p.row_tiles, z = u / (p.Hkv * p.row_tiles);
+          const int split = z % tab.splits;
+          const SegDev& sg = tab.seg[z / tab.splits];
+          if (tile_y * p.nodes_per_tile >= sg.n || sg.ctl[CTL_STATUS] != 0) continue;
+          const int Ltot = sg.ctl[CTL_LEN] + sg.n;
+          const int k_begin = split * sg.chunk;
+          if (k_begin >= Ltot) continue;
+          const int kc = min(sg.chunk, Ltot - k_begin);
+          const int kc_pad = (kc + 15) & ~15;
+          const int rounds = (kc_pad + ROUND - 1) / ROUND;
+          const uint32_t par = (uint32_t)(au & 1);
+          ++au;
+          const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 256;
+          ok = mbar_wait(&sc->bar_qk, par, abort, status);
+          if (!ok) break;
+          tc_fence_after();
+          {
+            const uint32_t idesc_s = make_idesc_bf16(kc_pad);
+            const uint32_t a0 = smem_u32(As), b0 = smem_u32(KVs);
+            uint32_t acc = 0u;
+  #pragma unroll
+            for (int term = 0; term < 3; ++term) {
+              const int qp = term == 2 ? 1 : 0, kp = term == 1 ? 1 : 0;     // hi*hi, hi*lo, lo*hi
+              for (int h = 0; h < H2; ++h) {
+  #pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                  umma_bf16(tmem_s, make_smem_desc(a0 + (qp * H2 + h) * SUB + k * 32),
+                            make_smem_desc(b0 + (kp * H2 + h) * KVSUB + k * 32), idesc_s, acc);
+                  acc = 1u;
+                }
+              }
+            }
+            umma_commit(&sc->bar_s);
+          }
+          ok = mbar_wait(&sc->bar_v, par, abort, status);
+          const uint32_t idesc2 = make_idesc_bf16(DH, true);
           uint32_t acc = 0u;
-#pragma unroll
-          for (int term = 0; term < 3; ++term) {
-            const int qp = term == 2 ? 1 : 0, kp = term == 1 ? 1 : 0;     // hi*hi, hi*lo, lo*hi
-            for (int h = 0; h < H2; ++h) {
-#pragma unroll
-              for (int k = 0; k < 4; ++k) {
-                umma_bf16(tmem_s, make_smem_desc(a0 + (qp * H2 + h) * SUB + k * 32),
-                          make_smem_desc(b0 + (kp * H2 + h) * KVSUB + k * 32), idesc_s, acc);
+          for (int rd = 0; rd < rounds && ok; ++rd) {
+            const uint32_t par_r = rd == 0 ? par : (uint32_t)(au2 & 1);
+            ok = mbar_wait(&sc->bar_p[rd], par_r, abort, status);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t a0 = smem_u32(As), b0 = smem_u32(KVs);
+            const int j_end = min(kc_pad - rd * ROUND, ROUND) / 16;
+  #pragma unroll
+            for (int term = 0; term < 3; ++term) {
+              const int pp = term == 2 ? 1 : 0, vp = term == 1 ? 1 : 0;
+              for (int j = 0; j < j_end; ++j) {
+                umma_bf16(tmem_o, make_smem_desc(a0 + (pp * 2 + (j >> 2)) * SUB + (j & 3) * 32),
+                          make_smem_desc(b0 + vp * H2 * KVSUB + (rd * (ROUND / 16) + j) * 2048, KVSUB), idesc2, acc);
                 acc = 1u;
               }
             }
+            umma_commit(&sc->bar_o[rd]);
           }
-          umma_commit(&sc->bar_s);
+          if (rounds == 2) ++au2;
         }
-        ok = mbar_wait(&sc->bar_v, par, abort, status);
-        const uint32_t idesc2 = make_idesc_bf16(DH, true);
-        uint32_t acc = 0u;
-        for (int rd = 0; rd < rounds && ok; ++rd) {
-          const uint32_t par_r = rd == 0 ? par : (uint32_t)(au2 & 1);
-          ok = mbar_wait(&sc->bar_p[rd], par_r, abort, status);
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t a0 = smem_u32(As), b0 = smem_u32(KVs);
-          const int j_end = min(kc_pad - rd * ROUND, ROUND) / 16;
-#pragma unroll
-          for (int term = 0; term < 3; ++term) {
-            const int pp = term == 2 ? 1 : 0, vp = term == 1 ? 1 : 0;
-            for (int j = 0; j < j_end; ++j) {
-              umma_bf16(tmem_o, make_smem_desc(a0 + (pp * 2 + (j >> 2)) * SUB + (j & 3) * 32),
-                        make_smem_desc(b0 + vp * H2 * KVSUB + (rd * (ROUND / 16) + j) * 2048, KVSUB), idesc2, acc);
-              acc = 1u;
-            }
-          }
-          umma_commit(&sc->bar_o[rd]);
-        }
-        if (rounds == 2) ++au2;
       }
-      if (ok) run_gemm(gemm_of(p, l, ST_O, cta, G));
-      if (ok) run_gemm(gemm_of(p, l, ST_GU, cta, G));
-      if (ok) run_gemm(gemm_of(p, l, ST_DOWN, cta, G));
     }
-    if (ok && p.want_head) run_gemm(gemm_of(p, 0, -1, cta, G));
   } else if (warp >= 2 && warp < 10) {
     // =========================================================== workers
     const int wtid = threadIdx.x - 64;
@@ -514,6 +598,8 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
     bool ok = true;
     int seg = 0, au = 0, au2 = 0;
     int arrived = 0;                                     // steps this CTA has signed off
+    int cur_layer = 0;
+    (void)cur_layer;
 
     // Barriers among the workers (worker_bar) are never placed under a condition that a failed wait could make
     // differ between threads; `ok` only guards waits and memory traffic.  A wait's verdict is made uniform
@@ -627,13 +713,14 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
     };
     // linear output: fp32 partial plane `split`
     auto epi_partial = [&](const Gemm& g, size_t plane_stride) {
-      for (long long u = g.u0; u < g.u1; ++seg) {
-        const int tile = (int)(u / g.KB);
-        const int kb0 = (int)(u % g.KB);
-        const int kb1 = (int)((g.u1 - u) < (long long)(g.KB - kb0) ? kb0 + (g.u1 - u) : g.KB);
+      for (int u = g.u0; u < g.u1; ++seg) {
+        const int tile = u / g.KB;
+        const int kb0 = u % g.KB;
+        const int kb1 = (g.u1 - u) < (g.KB - kb0) ? kb0 + (g.u1 - u) : g.KB;
         u += kb1 - kb0;
         const int b = seg & 1;
         if (ok) ok = wwait_relaxed(&sc->acc_full[b], (uint32_t)((seg >> 1) & 1));
+        STACK_TRACE_POINT(10, cur_layer);
         tc_fence_after();
         if (!ok) continue;
         const uint32_t lane_addr = tmem_base + lane_off + (uint32_t)(b * acc_cols);
@@ -652,16 +739,16 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
     };
     // SiLU(gate) * up (swiglu = true) or arg-max over the vocabulary (swiglu = false), equal unit ranges
     auto epi_streamk = [&](const Gemm& g, bool swiglu, int epoch) {
-      for (long long u = g.u0; u < g.u1; ++seg) {
-        const int tile = (int)(u / g.KB);
-        const int kb0 = (int)(u % g.KB);
-        const int kb1 = (int)((g.u1 - u) < (long long)(g.KB - kb0) ? kb0 + (g.u1 - u) : g.KB);
+      for (int u = g.u0; u < g.u1; ++seg) {
+        const int tile = u / g.KB;
+        const int kb0 = u % g.KB;
+        const int kb1 = (g.u1 - u) < (g.KB - kb0) ? kb0 + (g.u1 - u) : g.KB;
         u += kb1 - kb0;
         const int b = seg & 1;
         // the CTA that holds the first k-blocks of a split tile adds what the CTAs holding the rest have parked
         int last = cta;
         if (kb0 == 0 && kb1 != g.KB)
-          while (last + 1 < g.g_eff && (last + 1) * g.U / g.g_eff < (long long)(tile + 1) * g.KB) ++last;
+          while (last + 1 < g.g_eff && (long long)(last + 1) * g.U / g.g_eff < (long long)(tile + 1) * g.KB) ++last;
         float pk0[16], pk1[16];
         auto load_parked = [&](int c0, float* f) {
 #pragma unroll
@@ -688,6 +775,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
           }
         }
         if (ok) ok = wwait_relaxed(&sc->acc_full[b], (uint32_t)((seg >> 1) & 1));
+        STACK_TRACE_POINT(kb0 != 0 ? 12 : 11, cur_layer);
         tc_fence_after();
         const uint32_t lane_addr = tmem_base + lane_off + (uint32_t)(b * acc_cols);
 
@@ -916,26 +1004,29 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
           }
           return t0 < 0 ? ((1u << (-t0)) - 1u) | (win << (-t0)) : win;
         };
-        auto visible32 = [&](int c0) -> uint32_t {
-          const uint32_t mine = kc - c0 >= 32 ? 0xFFFFFFFFu : (1u << (kc - c0)) - 1u;   // c0 < kc always
+        // bit j = key (k_begin + c0 + j) belongs to this unit's block and is visible to this row (16 keys; c0 < kc)
+        auto visible16 = [&](int c0) -> uint32_t {
+          const uint32_t mine = kc - c0 >= 16 ? 0xFFFFu : (1u << (kc - c0)) - 1u;
           return mine & visible_keys(k_begin + c0);
         };
         if (ok) ok = wwait(&sc->bar_s, par);
+        STACK_TRACE_POINT(1, cur_layer);
         float m_row = -INFINITY;
         if (ok) {
           tc_fence_after();
           float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll 1
-          for (int c0 = eg * 32; c0 < kc_pad; c0 += 64) {
-            float s[32];
-            tmem_ld32(tmem_s + lane_off + c0, s);
-            const uint32_t vis = c0 < kc ? visible32(c0) : 0u;
+          for (int c0 = eg * 16; c0 < kc_pad; c0 += 32) {        // short rolled loops: this code runs once per layer
+            float s[16];
+            tmem_ld16(tmem_s + lane_off + c0, s);
+            const uint32_t vis = c0 < kc ? visible16(c0) : 0u;
 #pragma unroll
-            for (int j = 0; j < 32; ++j) m4[j & 3] = fmaxf(m4[j & 3], ((vis >> j) & 1u) ? s[j] * p.scale_log2 : -INFINITY);
+            for (int j = 0; j < 16; ++j) m4[j & 3] = fmaxf(m4[j & 3], ((vis >> j) & 1u) ? s[j] * p.scale_log2 : -INFINITY);
           }
           m_row = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
         }
         sc->red_max[eg][row] = m_row;
+        STACK_TRACE_POINT(4, cur_layer);
         worker_bar();
         m_row = fmaxf(sc->red_max[0][row], sc->red_max[1][row]);
         const float m_use = m_row > -INFINITY ? m_row : 0.f;      // a fully masked row gives p = 0 everywhere
@@ -944,16 +1035,17 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
           // the P tile holds 128 keys: the second round waits until the first round's MMAs have read it
           if (rd > 0) ok = wwait(&sc->bar_o[0], par);
           if (!ok) break;
+          STACK_TRACE_POINT(5 + rd, cur_layer);
           const int c_end = min(kc_pad, (rd + 1) * ROUND);
 #pragma unroll 1
-          for (int c0 = rd * ROUND + eg * 32; c0 < c_end; c0 += 64) {
-            float s[32];
-            tmem_ld32(tmem_s + lane_off + c0, s);
-            const uint32_t vis = c0 < kc ? visible32(c0) : 0u;
+          for (int c0 = rd * ROUND + eg * 16; c0 < c_end; c0 += 32) {
+            float s[16];
+            tmem_ld16(tmem_s + lane_off + c0, s);
+            const uint32_t vis = c0 < kc ? visible16(c0) : 0u;
 #pragma unroll
-            for (int j = 0; j < 32; ++j) s[j] = ((vis >> j) & 1u) ? exp2f(s[j] * p.scale_log2 - m_use) : 0.f;
+            for (int j = 0; j < 16; ++j) s[j] = ((vis >> j) & 1u) ? exp2f(s[j] * p.scale_log2 - m_use) : 0.f;
 #pragma unroll
-            for (int gq = 0; gq < 4; ++gq) {
+            for (int gq = 0; gq < 2; ++gq) {
               uint32_t hi[4], lo[4];
 #pragma unroll
               for (int e = 0; e < 4; ++e) {
@@ -962,13 +1054,12 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
                 split2_pack(s[j], s[j + 1], hi[e], lo[e]);
               }
               const int c8 = ((c0 - rd * ROUND) >> 3) + gq;     // 8-key group within this round's 128 keys
-              if (rd * ROUND + c8 * 8 < kc_pad) {
-                const int off = (c8 >> 3) * SUB + row * 128 + (((c8 & 7) ^ (row & 7)) << 4);
-                *reinterpret_cast<uint4*>(As + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-                *reinterpret_cast<uint4*>(As + 2 * SUB + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-              }
+              const int off = (c8 >> 3) * SUB + row * 128 + (((c8 & 7) ^ (row & 7)) << 4);
+              *reinterpret_cast<uint4*>(As + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+              *reinterpret_cast<uint4*>(As + 2 * SUB + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
             }
           }
+          STACK_TRACE_POINT(7 + rd, cur_layer);
           if (rd == rounds - 1 && kc < kc_pad) {
             // value rows past the end of the cache meet p = 0, but 0 * garbage could still be NaN: clear them
             ok = wwait(&sc->bar_v, par);
@@ -984,7 +1075,9 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
           }
         }
         sc->red_sum[eg][row] = l2[0] + l2[1];
+        STACK_TRACE_POINT(2, cur_layer);
         if (ok) ok = rounds == 2 ? wwait(&sc->bar_o[1], par2) : wwait(&sc->bar_o[0], par);
+        STACK_TRACE_POINT(3, cur_layer);
         // O leaves through the (now idle) K/V region so that a warp writes whole rows
         float4* stage = reinterpret_cast<float4*>(KVs);
         constexpr int C4 = DH / 4;
@@ -1081,89 +1174,48 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
     // ================= the sequence of steps
     const size_t stride_d = (size_t)p.n_alloc * p.d;
     const size_t stride_qkv = (size_t)p.n_alloc * p.qkv_dim;
-    for (int l = 0; l < p.n_layers; ++l) {
-      const int base = l * ST_PER_LAYER;
-      {
-        STACK_TRACE_BEGIN();
-        if (l > 0) wait_step(base - 1);                  // the previous layer's down projection
-        norm_step(p.gains[2 * l], l > 0 ? p.splits_down : 0, stride_d);
-        arrive_step();
-        STACK_TRACE_END(SPECASR_KIND_NORM, l);
-      }
-      {
-        STACK_TRACE_BEGIN();
-        epi_partial(gemm_of(p, l, ST_QKV, cta, G), stride_qkv);
-        arrive_step();
-        STACK_TRACE_END(SPECASR_KIND_GEMM_QKV, l);
-      }
-      {
-        STACK_TRACE_BEGIN();
-        wait_step(base + ST_QKV);
-        rope_step(l);
-        arrive_step();
-        STACK_TRACE_END(SPECASR_KIND_ROPE, l);
-      }
-      {
-        STACK_TRACE_BEGIN();
+    for (int sidx = 0; sidx < n_steps; ++sidx) {
+      const int l = sidx / ST_PER_LAYER, st = sidx - l * ST_PER_LAYER;
+      const bool head = l == p.n_layers;
+      const int gk = gemm_kind_of(l, st, p.n_layers);
+      cur_layer = l;
+      int trace_kind = SPECASR_KIND_NORM;
+      (void)trace_kind;
+      STACK_TRACE_BEGIN();
+      if (gk == ST_QKV || gk == ST_O || gk == ST_DOWN) {
+        epi_partial(gemm_of(p, l, gk, cta, G), gk == ST_QKV ? stride_qkv : stride_d);
+        trace_kind = gk == ST_QKV ? SPECASR_KIND_GEMM_QKV : gk == ST_O ? SPECASR_KIND_GEMM_O : SPECASR_KIND_GEMM_DOWN;
+      } else if (gk == ST_GU || gk == -1) {
+        wait_step(sidx - 1);                             // the row sums of squares of the norm before it
+        STACK_TRACE_MARK();
+        load_inv();
+        epi_streamk(gemm_of(p, l, gk, cta, G), gk == ST_GU, p.epoch0 + 1 + l);
+        trace_kind = gk == ST_GU ? SPECASR_KIND_GEMM_GU : SPECASR_KIND_GEMM_LM;
+      } else if (st == ST_ATTN) {
         attention_step();
         worker_bar();
         if (wtid == 0) {
           __threadfence_block();
           *(volatile int*)&sc->attn_done = l + 1;
         }
-        arrive_step();
-        STACK_TRACE_END(SPECASR_KIND_ATTN, l);
+        trace_kind = SPECASR_KIND_ATTN;
+      } else {
+        if (sidx > 0) wait_step(sidx - 1);               // every other step reads what the step before it wrote
+        STACK_TRACE_MARK();
+        if (st == ST_ROPE) {
+          rope_step(l);
+          trace_kind = SPECASR_KIND_ROPE;
+        } else if (st == ST_MERGE) {
+          merge_step();
+          trace_kind = SPECASR_KIND_ATTN_MERGE;
+        } else {                                         // a norm: attention, FFN or final
+          const bool ffn = !head && st == ST_NORM2;
+          norm_step(p.gains[head ? 2 * p.n_layers : 2 * l + (ffn ? 1 : 0)],
+                    ffn ? p.splits_o : (sidx > 0 ? p.splits_down : 0), stride_d);
+        }
       }
-      {
-        STACK_TRACE_BEGIN();
-        wait_step(base + ST_ATTN);
-        merge_step();
-        arrive_step();
-        STACK_TRACE_END(SPECASR_KIND_ATTN_MERGE, l);
-      }
-      {
-        STACK_TRACE_BEGIN();
-        epi_partial(gemm_of(p, l, ST_O, cta, G), stride_d);
-        arrive_step();
-        STACK_TRACE_END(SPECASR_KIND_GEMM_O, l);
-      }
-      {
-        STACK_TRACE_BEGIN();
-        wait_step(base + ST_O);
-        norm_step(p.gains[2 * l + 1], p.splits_o, stride_d);
-        arrive_step();
-        STACK_TRACE_END(SPECASR_KIND_NORM, l);
-      }
-      {
-        STACK_TRACE_BEGIN();
-        wait_step(base + ST_NORM2);
-        load_inv();
-        epi_streamk(gemm_of(p, l, ST_GU, cta, G), true, p.epoch0 + 1 + l);
-        arrive_step();
-        STACK_TRACE_END(SPECASR_KIND_GEMM_GU, l);
-      }
-      {
-        STACK_TRACE_BEGIN();
-        epi_partial(gemm_of(p, l, ST_DOWN, cta, G), stride_d);
-        arrive_step();
-        STACK_TRACE_END(SPECASR_KIND_GEMM_DOWN, l);
-      }
-    }
-    if (p.want_head) {
-      {
-        STACK_TRACE_BEGIN();
-        wait_step(steps_total - 1);
-        norm_step(p.gains[2 * p.n_layers], p.splits_down, stride_d);
-        arrive_step();
-        STACK_TRACE_END(SPECASR_KIND_NORM, p.n_layers);
-      }
-      {
-        STACK_TRACE_BEGIN();
-        wait_step(steps_total);
-        load_inv();
-        epi_streamk(gemm_of(p, 0, -1, cta, G), false, p.epoch0 + 1 + p.n_layers);
-        STACK_TRACE_END(SPECASR_KIND_GEMM_LM, p.n_layers);
-      }
+      arrive_step();
+      STACK_TRACE_END(trace_kind, l);
     }
     (void)arrived;
   }
@@ -1219,6 +1271,18 @@ bool fused_stack_supported(const specasr_kv* wk, int n_total, bool att_tc, int s
   return true;
 }
 
+// Units (32 KB of weights each) every CTA keeps requested into L2 ahead of its ring: 16 x 148 CTAs = 78 MB, which
+// leaves room in the 126 MB L2 for the activations and the layer's K / V pages.
+static int fused_lookahead() {
+  static int v = -1;
+  if (v < 0) {
+    const char* e = getenv("SPECASR_LOOKAHEAD");
+    v = e ? atoi(e) : 16;
+    if (v < 0) v = 0;
+  }
+  return v;
+}
+
 size_t fused_stack_sync_bytes(const specasr_model* m) {
   return (((size_t)m->cfg.n_layers * ST_PER_LAYER + 2) * sizeof(int32_t) + 255) / 256 * 256;
 }
@@ -1253,6 +1317,7 @@ bool launch_fused_stack(specasr_model* m, specasr_kv* wk, const SegTable& tab, i
   p.epoch0 = wk->gemm_epoch;
   wk->gemm_epoch += c.n_layers + 1;
   p.want_head = want_head ? 1 : 0;
+  p.lookahead = fused_lookahead();
   p.group = c.n_heads / c.n_kv_heads;
   p.nodes_per_tile = 128 / p.group;
   p.row_tiles = (n_max + p.nodes_per_tile - 1) / p.nodes_per_tile;
