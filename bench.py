@@ -32,6 +32,7 @@ WORKLOADS = {
     "config1": dict(model="tiny", n_audio=64, n_text=8, n_nodes=15, levels=None, chain=False),
     # config3 cut to two layers: same kernels and launch shapes, small enough for a profiler capture
     "config3_2layers": dict(model="7b", n_layers=2, n_audio=1500, n_text=201, n_nodes=64, levels=12, chain=False),
+    "config3_4layers": dict(model="7b", n_layers=4, n_audio=1500, n_text=201, n_nodes=64, levels=12, chain=False),
     # the 13B-class shape as a second target (same tree and context as config 3)
     "config3_13b": dict(model="13b", n_audio=1500, n_text=201, n_nodes=64, levels=12, chain=False),
     # a 256-node point of the config 4 sweep cut to two layers, for a profiler capture of the large-tree regime
@@ -71,28 +72,29 @@ def algorithmic_flops(cfg, L, n):
     return 2 * n * params + 4 * n * cfg.q_dim * (L + n) * cfg.n_layers
 
 
-# DRAM traffic (read + write, MB per launch) of the projection kernel from the ncu capture summarised in
-# profiles/k_proj_config3_2layers.md: 7B shape, 64 tokens.  Valid only for the kernel source it was taken on.
-PROJ_TRAFFIC_MB = {"gemm_qkv": 51.45, "gemm_o": 34.65, "gemm_gu": 247.58, "gemm_down": 125.01, "gemm_lm": 275.95}
-PROJ_TRAFFIC_SOURCE_SHA256 = {
-    "gemm_tcgen05.cu": "821a4515b0ec6dcf6681b35259d549dae46c591a5b3d678ab23b82df97d84f86",
-    "sm100_ptx.cuh": "3a0c294121fb64b742ab3700569cef82a1922484c98acd5238167235b990940f",
+# DRAM traffic (read + write) of one launch of the fused layer-stack kernel from the ncu captures summarised in
+# profiles/k_stack_config3_cuts.md: the 2-layer and the 4-layer cut of config 3 (7B shape, 64 tokens, KV 1700).  Traffic
+# grows by a fixed amount per layer, so a full launch is the 2-layer figure plus (layers - 2) times the per-layer
+# difference.  Valid only for the kernel source it was taken on.
+STACK_TRAFFIC_MB = {"cut2": None, "cut4": None}
+STACK_TRAFFIC_SOURCE_SHA256 = {
+    "fused_stack.cu": "",
+    "sm100_ptx.cuh": "",
 }
 
 
-def proj_traffic_per_launch(wl, cfg):
-    """Average DRAM bytes per projection launch from the committed capture, or None when the capture does not
-    describe this run (another shape, or the kernel source changed since)."""
+def stack_traffic_per_launch(wl, cfg):
+    """DRAM bytes of one fused-stack launch from the committed captures, or None when they do not describe this run
+    (another shape, or the kernel source changed since)."""
     import hashlib
-    if wl.get("model") != "7b" or wl.get("n_nodes") != 64:
+    if wl.get("model") != "7b" or wl.get("n_nodes") != 64 or STACK_TRAFFIC_MB["cut2"] is None:
         return None
-    for name, want in PROJ_TRAFFIC_SOURCE_SHA256.items():
+    for name, want in STACK_TRAFFIC_SOURCE_SHA256.items():
         path = os.path.join(ROOT, "paper_2507_18181_b200", "csrc", name)
         if not os.path.exists(path) or hashlib.sha256(open(path, "rb").read()).hexdigest() != want:
             return None
-    t = PROJ_TRAFFIC_MB
-    per_layer = t["gemm_qkv"] + t["gemm_o"] + t["gemm_gu"] + t["gemm_down"]
-    return (cfg.n_layers * per_layer + t["gemm_lm"]) * 1e6 / (4 * cfg.n_layers + 1)
+    per_layer = (STACK_TRAFFIC_MB["cut4"] - STACK_TRAFFIC_MB["cut2"]) / 2.0
+    return (STACK_TRAFFIC_MB["cut2"] + (cfg.n_layers - 2) * per_layer) * 1e6
 
 
 def measured_peaks():
@@ -163,8 +165,8 @@ def oracle_sample(wl, seed=1):
     """Bounded sample of the workload for the CPU oracle: the oracle's own steps of the same verify
     call (same tree, same KV length, same shapes) run over ONE of the model's layers plus the embedding
     and vocabulary projection, each part timed; the full call is extrapolated as
-    t_globals + n_layers * t_layer + t_head.  Returns a closure that runs the sample once and returns the
-    extrapolated seconds per full call."""
+    t_globals + n_layers * t_layer + t_head.  Returns a closure that runs the sample once and returns
+    (extrapolated seconds per full call, seconds actually timed)."""
     from oracle import specasr_oracle as O
     cfg_full = model_config(wl)
     cfg = gen.get_config(wl["model"], n_layers=1)
@@ -191,7 +193,7 @@ def oracle_sample(wl, seed=1):
         logits = O.lm_logits(cfg, W, hidden)
         O.accept(tokens, parent, np.argmax(logits, axis=-1))
         t3 = time.perf_counter()
-        return (t1 - t0) + cfg_full.n_layers * (t2 - t1) + (t3 - t2)
+        return (t1 - t0) + cfg_full.n_layers * (t2 - t1) + (t3 - t2), t3 - t0
 
     desc = (f"oracle steps of verify_tree on the {wl['model']} shape, {n}-node tree, KV length {L} (seeded N(0,1) "
             f"K/V): embedding + 1 of {cfg_full.n_layers} layers + vocabulary projection + accept, full call = "
@@ -206,8 +208,9 @@ def run_reference(args, wl):
     run_once, desc = oracle_sample(wl)
     for _ in range(args.warmup):
         run_once()
-    secs = [run_once() for _ in range(args.steps)]
-    per_call = float(np.mean(secs))
+    runs = [run_once() for _ in range(args.steps)]
+    per_call = float(np.mean([r[0] for r in runs]))
+    timed = float(np.mean([r[1] for r in runs]))
     n = wl["n_nodes"]
     cores = len(os.sched_getaffinity(0))
     value = n / per_call
@@ -216,7 +219,8 @@ def run_reference(args, wl):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_call * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": args.workload, **workload_keys(wl)},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc,
+                         "extrapolated": True, "timed_seconds_per_step": timed},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line))
@@ -225,31 +229,38 @@ def run_reference(args, wl):
 # ------------------------------------------------------------------------------------------------ CUDA leg
 
 def in_flow_times(kv, step, kind_names):
-    """Per-kernel contribution to one step from the library's device-side trace: block records are grouped into
-    launches (same kind, starts close together); a launch adds (its last block's end - the latest end of all
-    launches before it).  Returns {kind name: {"launches", "us_per_step"}} or None if nothing was recorded."""
+    """Where the time of one step goes, from the library's device-side trace.  Worker thread 0 of every CTA of the
+    fused layer-stack kernel writes one record per step of the stack {kind | (layer + 1) << 8, start, end, wait end};
+    the other kernels (tree prep, embedding, accept) write one record per block.  A step of the stack is charged the
+    time from the moment the last CTA finished the step before it to the moment the last CTA finished this one.
+    Returns {name: {"launches": occurrences, "us_per_step": total}} or None if nothing was recorded."""
+    import torch
+    n_sm = torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count
     rec = kv.trace(step, capacity=1 << 18)
     if len(rec) == 0:
         return None
-    # launches of one kind lie a whole layer (or half of one) apart, blocks of one launch start within a few us of
-    # one another: cut each kind's records where consecutive starts are more than 30 us apart
-    launches = []                      # [kind, first start, last end]
-    for kind in sorted(set(int(k) for k in rec[:, 0])):
-        r = rec[rec[:, 0] == kind]
-        r = r[np.argsort(r[:, 1], kind="stable")]
-        first, last_start, end = int(r[0, 1]), int(r[0, 1]), int(r[0, 2])
-        for _, start, e, _w in r[1:]:
-            if start - last_start > 30000:
-                launches.append([kind, first, end])
-                first, end = int(start), int(e)
-            last_start = int(start)
-            end = max(end, int(e))
-        launches.append([kind, first, end])
-    launches.sort(key=lambda l: l[1])
+    kind = rec[:, 0] & 0xFF
+    layer = (rec[:, 0] >> 8).astype(np.int64) - 1
+    groups = []                                  # [name, first start, last end]
+    plain = rec[layer < 0]
+    for k in sorted(set(int(x) for x in plain[:, 0] & 0xFF)):
+        r = plain[(plain[:, 0] & 0xFF) == k]
+        groups.append([kind_names[k], int(r[:, 1].min()), int(r[:, 2].max())])
+    stack = rec[layer >= 0]
+    for l in sorted(set(int(x) for x in layer[layer >= 0])):
+        for k in sorted(set(int(x) for x in (stack[:, 0] & 0xFF)[((stack[:, 0] >> 8) - 1) == l])):
+            r = stack[((stack[:, 0] & 0xFF) == k) & (((stack[:, 0] >> 8) - 1) == l)]
+            r = r[np.argsort(r[:, 1], kind="stable")]
+            name = kind_names[k]
+            if name == "norm" and len(r) > n_sm:     # two norms per layer: the earlier half is the attention norm
+                h = len(r) // 2
+                groups.append(["norm", int(r[:h, 1].min()), int(r[:h, 2].max())])
+                r = r[h:]
+            groups.append([name, int(r[:, 1].min()), int(r[:, 2].max())])
+    groups.sort(key=lambda g: g[2])
     out = {}
-    latest = launches[0][1]
-    for kind, _, end in launches:
-        name = kind_names[kind]
+    latest = min(g[1] for g in groups)
+    for name, _, end in groups:
         d = out.setdefault(name, {"launches": 0, "us_per_step": 0.0})
         d["launches"] += 1
         d["us_per_step"] += max(0, end - latest) / 1e3
@@ -440,17 +451,25 @@ def run_ours(args, wl):
     in_flow = in_flow_from_child(args) if world == 1 and not args.no_in_flow else None
     gb = gemm_weight_bytes(cfg)
     gemm_bytes_step = cfg.n_layers * (gb["gemm_qkv"] + gb["gemm_o"] + gb["gemm_gu"] + gb["gemm_down"]) + gb["gemm_lm"]
-    gemm_ms_step = sum(ms[k] for k in gb) / prof_steps
-    gemm_launches = sum(cnt[k] for k in gb) / prof_steps
     peaks = measured_peaks()
-    achieved = gemm_bytes_step / (gemm_ms_step * 1e-3) / 1e9
-    for k in gb:
-        per = gb[k] * (cfg.n_layers if k != "gemm_lm" else 1)
-        kernels[k]["achieved_gbs"] = per / (ms[k] / prof_steps * 1e-3) / 1e9
+    ab = algorithmic_bytes(cfg, L, n)
+    if cnt.get("stack"):
+        # the whole layer stack is one persistent kernel: its algorithmic bytes are the weights it streams plus the
+        # cache rows it reads and writes, i.e. those of the step
+        dom = {"kernel": "k_stack (fused layer stack: norms, projections, rotary, attention, arg-max)",
+               "bytes": ab["total"], "ms": ms["stack"] / cnt["stack"], "traffic": stack_traffic_per_launch(wl, cfg)}
+    else:
+        gemm_ms = sum(ms[k] for k in gb)
+        gemm_n = sum(cnt[k] for k in gb)
+        dom = {"kernel": "k_proj (all projections)", "bytes": gemm_bytes_step * prof_steps / gemm_n,
+               "ms": gemm_ms / gemm_n, "traffic": None}
+        for k in gb:
+            per = gb[k] * (cfg.n_layers if k != "gemm_lm" else 1)
+            kernels[k]["achieved_gbs"] = per / (ms[k] / prof_steps * 1e-3) / 1e9
+    achieved = dom["bytes"] / (dom["ms"] * 1e-3) / 1e9
 
     ms_per_step = elapsed_ms / args.steps
     value = whole_job_rate(n, args.steps, world, elapsed_ms * 1e-3)
-    ab = algorithmic_bytes(cfg, L, n)
     fl = algorithmic_flops(cfg, L, n)
     t_roof_ms = max(ab["total"] / (peaks["hbm_gbs"] * 1e9), fl / (peaks["bf16_tflops"] * 1e12)) * 1e3
     line = {
@@ -465,11 +484,10 @@ def run_ours(args, wl):
         "step_roofline": {"algorithmic_bytes": ab["total"], "algorithmic_flops": fl, "roof_ms": t_roof_ms,
                           "frac_of_" + peaks["source"]: t_roof_ms / ms_per_step,
                           "frac_of_nominal_8TBs": (ab["total"] / 8e12 * 1e3) / ms_per_step},
-        "roofline": {"kernel": "k_gemm_tc (all projections)", "bound": "hbm", "achieved": achieved,
+        "roofline": {"kernel": dom["kernel"], "bound": "hbm", "achieved": achieved,
                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                     "peak_source": peaks["source"], "traffic": proj_traffic_per_launch(wl, cfg),
-                     "algorithmic_bytes_per_launch": gemm_bytes_step / gemm_launches,
-                     "avg_launch_ms": gemm_ms_step / gemm_launches},
+                     "peak_source": peaks["source"], "traffic": dom["traffic"],
+                     "algorithmic_bytes_per_launch": dom["bytes"], "avg_launch_ms": dom["ms"]},
         "kernels": kernels,
         "in_flow": None,
         "gpu_launches": int(launches),
@@ -480,9 +498,9 @@ def run_ours(args, wl):
     if in_flow:
         gemm_us = sum(in_flow[k]["us_per_step"] for k in gb if k in in_flow)
         line["in_flow"] = {
-            "how": "one extra step with the device-side trace on: time from the previous kernel's last block end to "
-                   "this kernel's last block end (%globaltimer), i.e. what the kernel adds to the step with the "
-                   "overlap of consecutive kernels intact",
+            "how": "one extra step with the device-side trace on: every step of the fused layer stack (and every other "
+                   "kernel) is charged the time from the end of the step before it on its last CTA to its own end "
+                   "on its last CTA (%globaltimer)",
             "us_per_launch": {k: round(v["us_per_step"] / v["launches"], 2) for k, v in in_flow.items()},
             "projections": {"us_per_step": gemm_us, "achieved_gbs": gemm_bytes_step / (gemm_us * 1e-6) / 1e9,
                             "frac_of_" + peaks["source"]: gemm_bytes_step / (gemm_us * 1e-6) / 1e9 / peaks["hbm_gbs"]},
@@ -490,13 +508,14 @@ def run_ours(args, wl):
     if world == 1 and not args.no_cpu_baseline:
         run_once, desc = oracle_sample(wl)
         run_once()
-        reps, t_start, secs = 0, time.perf_counter(), []
+        reps, t_start, runs = 0, time.perf_counter(), []
         while reps < 3 and time.perf_counter() - t_start < 25:
-            secs.append(run_once())
+            runs.append(run_once())
             reps += 1
-        per_call = float(np.mean(secs))
+        per_call = float(np.mean([r[0] for r in runs]))
         line["cpu_baseline"] = {"value": n / per_call, "unit": UNIT, "cores": len(os.sched_getaffinity(0)),
-                                "kind": "oracle", "sample": desc, "ms_per_step": per_call * 1e3}
+                                "kind": "oracle", "sample": desc, "ms_per_step": per_call * 1e3, "extrapolated": True,
+                                "timed_seconds_per_step": float(np.mean([r[1] for r in runs]))}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

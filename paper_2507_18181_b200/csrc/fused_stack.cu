@@ -31,8 +31,6 @@
 //
 // The attention step borrows the ring's shared memory (Q / P tiles and K / V pages of one key block), so the
 // weight producer resumes when the CTA's attention units are done.
-#include <stdlib.h>
-
 #include "internal.h"
 #include "device_utils.cuh"
 #include "sm100_ptx.cuh"
@@ -77,6 +75,7 @@ struct alignas(16) StackCtl {
   int abort;
   int attn_done;                        // attention steps this CTA has finished (its ring memory is free again)
   int step_ok;                          // verdict of a wait that one worker made for all of them
+  int units_done;                       // attention units the workers have finished (their shared memory is free again)
 };
 
 struct StackParams {
@@ -87,7 +86,6 @@ struct StackParams {
   const float2* rope;
   int n, n_pad, n_alloc, stages, stage_bytes, ring_bytes;
   int splits_qkv, splits_o, splits_down, epoch0, want_head, group, nodes_per_tile, row_tiles, attn_units;
-  int lookahead;                        // weight units the L2 prefetch runs ahead of the ring loads, per CTA
   int32_t* ctl;                         // control block whose status word ends the call
   int32_t* sync;                        // [steps of the call] arrival counters, zeroed before the launch
   float* X;
@@ -123,6 +121,7 @@ __device__ __forceinline__ void red_release_add(int32_t* p, int v) {
 }
 // generic-proxy accesses (ordinary loads / stores) <-> async-proxy accesses (TMA) of the same memory
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
 __device__ __forceinline__ void worker_bar() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 // One projection as this CTA sees it.
@@ -174,12 +173,21 @@ __device__ __forceinline__ int gemm_kind_of(int l, int st, int n_layers) {
   return (st == ST_QKV || st == ST_O || st == ST_GU || st == ST_DOWN) ? st : -2;
 }
 
+// The polling loops are kept out of line: the kernel has some forty waits, and its text is fetched again on every
+// layer, so a copy of the loop at each of them is paid for in instruction-cache misses.
+__device__ __noinline__ bool bar_wait(void* bar, uint32_t parity, volatile int* abort, int32_t* status) {
+  return mbar_wait(bar, parity, abort, status);
+}
+__device__ __noinline__ bool bar_wait_relaxed(void* bar, uint32_t parity, volatile int* abort, int32_t* status) {
+  return mbar_wait_relaxed(bar, parity, abort, status);
+}
+
 // Bounded poll of a word that only grows.  Returns false when the limit ran out or the call was aborted.
-__device__ __forceinline__ bool wait_word_ge(const int32_t* word, int target, volatile int* abort, int32_t* status) {
+__device__ __noinline__ bool wait_word_ge(const int32_t* word, int target, volatile int* abort, int32_t* status) {
   if (ld_acquire(word) >= target) return true;
   const unsigned long long t0 = global_ns();
   for (uint32_t it = 1;; ++it) {
-    __nanosleep(40);
+    __nanosleep(20);
     if (ld_acquire(word) >= target) return true;
     if ((it & 15u) == 0u) {
       if (*abort) return false;
@@ -195,7 +203,7 @@ __device__ __forceinline__ bool wait_word_ge(const int32_t* word, int target, vo
     }
   }
 }
-__device__ __forceinline__ bool wait_smem_ge(volatile int* word, int target, volatile int* abort, int32_t* status) {
+__device__ __noinline__ bool wait_smem_ge(volatile int* word, int target, volatile int* abort, int32_t* status) {
   if (*word >= target) return true;
   const unsigned long long t0 = global_ns();
   for (uint32_t it = 1;; ++it) {
@@ -243,7 +251,7 @@ __device__ __forceinline__ int seg_of_row(const SegTable& tab, int row) {
   do {                                                                                   \
     if (wtid == 0 && p.tr.buf != nullptr && p.tr.buf[1] != 0ull) {   /* word 1 of the buffer switches points on */                               \
       const unsigned long long now_ = global_ns();                                       \
-      STACK_TRACE_WRITE(100 + (point), layer, now_, now_, 0ull);                         \
+      STACK_TRACE_WRITE(100 + (point), layer, now_, now_, (unsigned long long)blockIdx.x);                         \
     }                                                                                    \
   } while (0)
 #else
@@ -290,6 +298,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
     mbar_init(&sc->bar_s, 1);
     sc->abort = 0;
     sc->attn_done = 0;
+    sc->units_done = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tmH);
     tma_prefetch_desc(&tmAO);
@@ -313,10 +322,10 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
     // the call was refused before it started (shared status): nothing to do
   } else if (warp == 0 && lane == 0) {
     // =========================================================== weight producer
-    // Two cursors walk this CTA's (layer, projection, unit) list, which is fixed for the call: `ld` issues the TMA
-    // loads into the ring, `pf` runs up to p.lookahead units ahead of it and only asks for the same boxes to be
-    // brought into L2.  While the ring is full or lent to the attention step -- the stretches in which HBM would
-    // otherwise idle -- the look-ahead keeps the weights of the coming projections moving.
+    // A cursor walks this CTA's (layer, projection, unit) list, which is fixed for the call, and issues the TMA loads
+    // into the ring as slots come free: weights never wait for a step, so the first tiles of the next projection
+    // are in shared memory before its input exists.  (Asking for units further ahead to be brought into L2 --
+    // continuously, or only while the attention step holds the ring -- measured slower at every depth tried.)
     struct Cursor {
       int l, ph;                 // layer; 0..3 = QKV, O, gate/up, down; layer == n_layers: the vocabulary projection
       int u, u1, tile, kb, KB;   // next unit, end of the range, and the unit as (weight tile, k-block)
@@ -354,10 +363,9 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
       }
       if (c.u >= c.u1) settle(c);
     };
-    Cursor ld, pf;
+    Cursor ld;
     ld.l = 0; ld.ph = -1; ld.u = ld.u1 = 0; ld.tile = ld.kb = 0; ld.KB = 1; ld.tmW = nullptr; ld.done = false;
     settle(ld);
-    pf = ld;
     int slot = 0;                                        // next ring slot
     uint32_t ring_par = 0u;                              // parity of the ring round in progress
     int attn_waited = 0;                                 // attention steps whose end this thread has seen
@@ -366,17 +374,11 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
       // the attention step of layer l owns the ring between that layer's QKV and O projections
       const int need = ld.l < p.n_layers ? (ld.ph == 0 ? ld.l : ld.l + 1) : p.n_layers;
       if (need > attn_waited) {
-        // HBM idles from here until the attention step ends: ask for the next units to be brought into L2
-        pf = ld;
-        for (int a = 0; a < p.lookahead && !pf.done; ++a) {
-          for (int q = 0; q < KSUB; ++q) tma_prefetch_2d(pf.tmW, (pf.kb * KSUB + q) * SUB_K, pf.tile * TILE_M);
-          advance(pf);
-        }
         ok = wait_smem_ge(&sc->attn_done, need, abort, status);
         attn_waited = need;
         if (!ok) break;
       }
-      if (!mbar_wait(&sc->empty[slot], ring_par ^ 1u, abort, status)) {
+      if (!bar_wait(&sc->empty[slot], ring_par ^ 1u, abort, status)) {
         ok = false;
         break;
       }
@@ -403,7 +405,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
         int kb = g.u0 % g.KB;
         for (int u = g.u0; u < g.u1 && ok; ++u, ++it) {
           const int s = it % p.stages;
-          if (!mbar_wait(&sc->empty[s], (uint32_t)((it / p.stages) & 1) ^ 1u, abort, status)) {
+          if (!bar_wait(&sc->empty[s], (uint32_t)((it / p.stages) & 1) ^ 1u, abort, status)) {
             ok = false;
             break;
           }
@@ -425,14 +427,10 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
         const CUtensorMap* tmAct = gk == ST_O ? &tmAO : gk == ST_DOWN ? &tmA : &tmH;
         stream_acts(gemm_of(p, l, gk, cta, G), tmAct, sidx - 1);
       } else if (l < p.n_layers && st == ST_ATTN) {
-        // ---- attention units of this CTA: lane 0 fetches Q, lane j page j of K and later of V
-        if (ok && cta < p.attn_units) {
-          if (lane == 0) {
-            ok = wait_word_ge(p.sync + sidx - 1, G, abort, status);
-            fence_proxy_async_all();
-          }
-          ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
-        }
+        // ---- attention units of this CTA: lane 0 fetches Q, lane j page j of K and later of V.
+        // (Asking for the K pages of a key block inside the committed prefix before the rotary step has finished
+        // made S ready 1.6 us earlier and the step no shorter; it was taken out again.)
+        bool rope_seen = false;
         for (int u = cta; u < p.attn_units && ok; u += G) {
           const int kvh = u % p.Hkv, tile_y = (u / p.Hkv) % p.row_tiles, z = u / (p.Hkv * p.row_tiles);
           const int split = z % tab.splits;
@@ -447,6 +445,20 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
           const int pages = (kc + p.page_size - 1) / p.page_size;
           const uint32_t par = (uint32_t)(au & 1);
           ++au;
+          auto wait_rope = [&]() {
+            if (lane == 0) {
+              ok = wait_word_ge(p.sync + sidx - 1, G, abort, status);
+              fence_proxy_async_all();
+            }
+            ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+            rope_seen = true;
+          };
+          if (!rope_seen) wait_rope();
+          // A CTA that runs several units reuses the Q / P and K / V tiles and the barriers: the next unit's loads
+          // (and the arming of its barriers) wait until the workers have stored the previous unit's output.
+          if (ok && lane == 0) ok = wait_smem_ge(&sc->units_done, au - 1, abort, status);
+          ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+          if (!ok) break;
           int my_page = 0;
           if (lane < pages) my_page = sg.page_table[split * (sg.chunk / p.page_size) + lane];
           const uint32_t q_bytes = 2 * H2 * rows_used * 128;
@@ -456,11 +468,6 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
             mbar_expect_tx(&sc->bar_v, kv_bytes);
           }
           __syncwarp();
-          if (lane == 0) {
-            for (int plane = 0; plane < 2; ++plane)
-              for (int h = 0; h < H2; ++h)
-                tma_load_4d(As + (plane * H2 + h) * SUB, &tmQ, h * 64, kvh * p.group, sg.row0 + node0, plane, &sc->bar_qk);
-          }
           const int c4 = l * sg.n_pages + my_page;
           const int off = lane * p.page_size * 128;
           if (lane < pages) {
@@ -468,8 +475,13 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
               for (int h = 0; h < H2; ++h)
                 tma_load_5d(KVs + (plane * H2 + h) * KVSUB + off, sg.tmK, h * 64, 0, plane, kvh, c4, &sc->bar_qk);
           }
+          if (lane == 0) {
+            for (int plane = 0; plane < 2; ++plane)
+              for (int h = 0; h < H2; ++h)
+                tma_load_4d(As + (plane * H2 + h) * SUB, &tmQ, h * 64, kvh * p.group, sg.row0 + node0, plane, &sc->bar_qk);
+          }
           // V takes K's place once the S MMAs have read K
-          ok = mbar_wait(&sc->bar_s, par, abort, status);
+          ok = bar_wait(&sc->bar_s, par, abort, status);
           if (ok && lane < pages) {
             for (int plane = 0; plane < 2; ++plane)
               for (int h = 0; h < H2; ++h)
@@ -489,7 +501,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
         const int kb0 = u % g.KB;
         const int kb1 = (g.u1 - u) < (g.KB - kb0) ? kb0 + (g.u1 - u) : g.KB;
         const int b = seg & 1;
-        if (!mbar_wait(&sc->acc_empty[b], (uint32_t)((seg >> 1) & 1) ^ 1u, abort, status)) {
+        if (!bar_wait(&sc->acc_empty[b], (uint32_t)((seg >> 1) & 1) ^ 1u, abort, status)) {
           ok = false;
           break;
         }
@@ -497,7 +509,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
         const uint32_t d_addr = tmem_base + (uint32_t)(b * acc_cols);
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % p.stages;
-          if (!mbar_wait(&sc->full[s], (uint32_t)((it / p.stages) & 1), abort, status)) {
+          if (!bar_wait(&sc->full[s], (uint32_t)((it / p.stages) & 1), abort, status)) {
             ok = false;
             break;
           }
@@ -540,16 +552,17 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
           const uint32_t par = (uint32_t)(au & 1);
           ++au;
           const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 256;
-          ok = mbar_wait(&sc->bar_qk, par, abort, status);
+          ok = bar_wait(&sc->bar_qk, par, abort, status);
           if (!ok) break;
           tc_fence_after();
           {
             const uint32_t idesc_s = make_idesc_bf16(kc_pad);
             const uint32_t a0 = smem_u32(As), b0 = smem_u32(KVs);
             uint32_t acc = 0u;
-  #pragma unroll
+  #pragma unroll 1
             for (int term = 0; term < 3; ++term) {
               const int qp = term == 2 ? 1 : 0, kp = term == 1 ? 1 : 0;     // hi*hi, hi*lo, lo*hi
+  #pragma unroll 1
               for (int h = 0; h < H2; ++h) {
   #pragma unroll
                 for (int k = 0; k < 4; ++k) {
@@ -561,19 +574,20 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
             }
             umma_commit(&sc->bar_s);
           }
-          ok = mbar_wait(&sc->bar_v, par, abort, status);
+          ok = bar_wait(&sc->bar_v, par, abort, status);
           const uint32_t idesc2 = make_idesc_bf16(DH, true);
           uint32_t acc = 0u;
           for (int rd = 0; rd < rounds && ok; ++rd) {
             const uint32_t par_r = rd == 0 ? par : (uint32_t)(au2 & 1);
-            ok = mbar_wait(&sc->bar_p[rd], par_r, abort, status);
+            ok = bar_wait(&sc->bar_p[rd], par_r, abort, status);
             if (!ok) break;
             tc_fence_after();
             const uint32_t a0 = smem_u32(As), b0 = smem_u32(KVs);
             const int j_end = min(kc_pad - rd * ROUND, ROUND) / 16;
-  #pragma unroll
+  #pragma unroll 1
             for (int term = 0; term < 3; ++term) {
               const int pp = term == 2 ? 1 : 0, vp = term == 1 ? 1 : 0;
+  #pragma unroll 2
               for (int j = 0; j < j_end; ++j) {
                 umma_bf16(tmem_o, make_smem_desc(a0 + (pp * 2 + (j >> 2)) * SUB + (j & 3) * 32),
                           make_smem_desc(b0 + vp * H2 * KVSUB + (rd * (ROUND / 16) + j) * 2048, KVSUB), idesc2, acc);
@@ -605,17 +619,19 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
     // differ between threads; `ok` only guards waits and memory traffic.  A wait's verdict is made uniform
     // across the warp because the TMEM loads that follow are warp-wide instructions.
     auto wwait = [&](void* bar, uint32_t parity) -> bool {
-      return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, abort, status) ? 1 : 0) != 0;
+      return __all_sync(0xFFFFFFFFu, bar_wait(bar, parity, abort, status) ? 1 : 0) != 0;
     };
     auto wwait_relaxed = [&](void* bar, uint32_t parity) -> bool {
-      return __all_sync(0xFFFFFFFFu, mbar_wait_relaxed(bar, parity, abort, status) ? 1 : 0) != 0;
+      return __all_sync(0xFFFFFFFFu, bar_wait_relaxed(bar, parity, abort, status) ? 1 : 0) != 0;
     };
     // every worker's global writes of the step are done and visible -> one arrival for the CTA
     auto arrive_step = [&]() {
-      __threadfence();
-      fence_proxy_async_all();
-      worker_bar();
-      if (wtid == 0) red_release_add(p.sync + arrived, 1);
+      worker_bar();                                      // every worker's stores of the step are issued ...
+      if (wtid == 0) {
+        __threadfence();                                 // ... and ordered before the arrival (cumulative over the barrier)
+        fence_proxy_async_global();                      // the next step may read them through TMA
+        red_release_add(p.sync + arrived, 1);
+      }
       ++arrived;
     };
     // all CTAs have signed off step `step`
@@ -653,11 +669,13 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
       const int d_part = ((d + NORM_PARTS - 1) / NORM_PARTS + 3) & ~3;
       const int items = p.n * NORM_PARTS;
       const size_t h_plane = (size_t)p.n_alloc * d;
+#pragma unroll 1
       for (int item = cta; item < items; item += G) {
         const int r = item / NORM_PARTS, part = item % NORM_PARTS;
         const int k_end = min(d, (part + 1) * d_part);
         float* x = p.X + (size_t)r * d;
         float ss = 0.f;
+#pragma unroll 1
         for (int k0 = part * d_part + wtid * 4; k0 < k_end; k0 += 2 * WORKERS * 4) {
           const int k1 = k0 + WORKERS * 4;
           const bool on1 = k1 < k_end;
@@ -665,6 +683,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
           float4 v1 = on1 ? *reinterpret_cast<const float4*>(x + k1) : make_float4(0.f, 0.f, 0.f, 0.f);
           const float4 g0 = *reinterpret_cast<const float4*>(gain + k0);
           const float4 g1 = on1 ? *reinterpret_cast<const float4*>(gain + k1) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 1
           for (int s0 = 0; s0 < n_planes; s0 += 4) {
             float4 q0[4], q1[4];
 #pragma unroll
@@ -713,6 +732,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
     };
     // linear output: fp32 partial plane `split`
     auto epi_partial = [&](const Gemm& g, size_t plane_stride) {
+#pragma unroll 1
       for (int u = g.u0; u < g.u1; ++seg) {
         const int tile = u / g.KB;
         const int kb0 = u % g.KB;
@@ -726,6 +746,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
         const uint32_t lane_addr = tmem_base + lane_off + (uint32_t)(b * acc_cols);
         float* out = p.P + (size_t)(cta % g.splits) * plane_stride;
         const int m = tile * TILE_M + row;
+#pragma unroll 1
         for (int c0 = c_first; c0 < n_pad; c0 += 32) {
           float v[16];
           load16(lane_addr, c0, v);
@@ -739,6 +760,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
     };
     // SiLU(gate) * up (swiglu = true) or arg-max over the vocabulary (swiglu = false), equal unit ranges
     auto epi_streamk = [&](const Gemm& g, bool swiglu, int epoch) {
+#pragma unroll 1
       for (int u = g.u0; u < g.u1; ++seg) {
         const int tile = u / g.KB;
         const int kb0 = u % g.KB;
@@ -754,6 +776,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
 #pragma unroll
           for (int j = 0; j < 16; ++j) f[j] = 0.f;
           if (c0 < n_pad)
+#pragma unroll 1
             for (int cc = cta + 1; cc <= last; ++cc) {
               const float* src = p.fixP + ((size_t)cc * n_pad + c0) * TILE_M + row;
 #pragma unroll
@@ -763,6 +786,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
         if (last > cta) {
           if (wtid == 0) {
             bool got = ok;
+#pragma unroll 1
             for (int cc = cta + 1; cc <= last && got; ++cc)
               got = wait_word_ge(p.fixFlag + cc, epoch, abort, status);            // flags carry the launch's epoch
             sc->step_ok = got ? 1 : 0;
@@ -783,6 +807,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
           // later k-blocks of a tile whose first k-blocks belong to an earlier CTA: park the partial sums
           float* dst = p.fixP + (size_t)cta * n_pad * TILE_M;
           if (ok) {
+#pragma unroll 1
             for (int c0 = c_first; c0 < n_pad; c0 += 32) {
               float v[16];
               load16(lane_addr, c0, v);
@@ -805,6 +830,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
           worker_bar();
         }
         if (ok) {
+#pragma unroll 1
           for (int c0 = c_first; c0 < n_pad; c0 += 32) {
             float v[16];
             load16(lane_addr, c0, v);
@@ -856,6 +882,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
             const int f0 = tile * 64;
             const int nt = p.n;
             const int chunks = 2 * nt * 8;                    // 16-byte pieces of the [2][nt][64] tile
+#pragma unroll 1
             for (int idx = wtid; idx < chunks; idx += WORKERS) {
               const int plane = idx / (nt * 8), rem = idx % (nt * 8);
               const int t = rem >> 3, ch = rem & 7;
@@ -864,6 +891,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
                     *reinterpret_cast<const uint4*>(epi_stage + (size_t)plane * n_pad * 64 + t * 64 + ch * 8);
             }
           } else {
+#pragma unroll 1
             for (int t = wtid; t < p.n; t += WORKERS) p.amax[(size_t)tile * p.n_alloc + t] = sc->key[t];
           }
           tc_fence_before();
@@ -881,6 +909,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
       const long long total = (long long)p.n * heads_all * per_head;
       const size_t pstride = (size_t)p.n_alloc * p.qkv_dim;
       const size_t q_plane = (size_t)p.n_alloc * p.q_dim;
+#pragma unroll 1
       for (long long idx = (long long)cta * WORKERS + wtid; idx < total; idx += (long long)G * WORKERS) {
         const int i = (int)(idx / (heads_all * per_head));
         const int rem = (int)(idx % (heads_all * per_head));
@@ -912,6 +941,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
           x1.x += a1[s].x; x1.y += a1[s].y; x1.z += a1[s].z; x1.w += a1[s].w;
           x2.x += a2[s].x; x2.y += a2[s].y; x2.z += a2[s].z; x2.w += a2[s].w;
         }
+#pragma unroll 1
         for (int s0 = 4; s0 < p.splits_qkv; s0 += 4) {
 #pragma unroll
           for (int s = 0; s < 4; ++s) {
@@ -962,6 +992,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
     // ---------------- attention: softmax over one key block, unnormalised partial out
     auto attention_step = [&]() {
       const size_t rows_alloc = (size_t)p.n_alloc * p.Hq;
+#pragma unroll 1
       for (int u = cta; u < p.attn_units; u += G) {
         const int kvh = u % p.Hkv, tile_y = (u / p.Hkv) % p.row_tiles, z = u / (p.Hkv * p.row_tiles);
         const int split = z % tab.splits;
@@ -1031,6 +1062,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
         m_row = fmaxf(sc->red_max[0][row], sc->red_max[1][row]);
         const float m_use = m_row > -INFINITY ? m_row : 0.f;      // a fully masked row gives p = 0 everywhere
         float l2[2] = {0.f, 0.f};
+#pragma unroll 1
         for (int rd = 0; rd < rounds && ok; ++rd) {
           // the P tile holds 128 keys: the second round waits until the first round's MMAs have read it
           if (rd > 0) ok = wwait(&sc->bar_o[0], par);
@@ -1064,7 +1096,9 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
             // value rows past the end of the cache meet p = 0, but 0 * garbage could still be NaN: clear them
             ok = wwait(&sc->bar_v, par);
             if (ok && eg == 0 && row < kc_pad - kc) {
+#pragma unroll 1
               for (int sub = 0; sub < 2 * H2; ++sub)
+#pragma unroll 1
                 for (int i = 0; i < 8; ++i)
                   *reinterpret_cast<uint4*>(KVs + sub * KVSUB + (kc + row) * 128 + i * 16) = make_uint4(0, 0, 0, 0);
             }
@@ -1095,6 +1129,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
           }
         }
         tc_fence_before();
+        STACK_TRACE_POINT(9, cur_layer);
         worker_bar();
         if (ok) {
           const int r_base = wwarp * 16;                       // eight warps, sixteen rows each
@@ -1105,12 +1140,18 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
             if (rr < rows_used && nd < sg.n) {
               const size_t orow = (size_t)split * rows_alloc + (size_t)(sg.row0 + nd) * p.Hq + kvh * p.group + rr % p.group;
               float4* dst = reinterpret_cast<float4*>(p.attO + orow * DH);
+#pragma unroll 1
               for (int c4 = lane; c4 < C4; c4 += 32) dst[c4] = stage[rr * C4 + (c4 ^ (rr & (C4 - 1)))];
             }
           }
           if (row_valid && eg == 0) p.attML[out_row] = make_float2(m_row, sc->red_sum[0][row] + sc->red_sum[1][row]);
         }
+        STACK_TRACE_POINT(13, cur_layer);
         worker_bar();                                           // the staging area and red_* are free again
+        if (wtid == 0) {
+          __threadfence_block();
+          *(volatile int*)&sc->units_done = au;                 // units this CTA has finished since the kernel began
+        }
       }
     };
 
@@ -1121,6 +1162,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
       const int n_splits = tab.splits;
       const size_t ao_plane = (size_t)p.n_alloc * p.q_dim;
       const int c = lane * 4;
+#pragma unroll 1
       for (int r = cta * 8 + wwarp; r < rows_total; r += G * 8) {
         bf16* out = p.AO + (size_t)r * DH + c;
         const float2 none = make_float2(-INFINITY, 0.f);
@@ -1138,8 +1180,10 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
         const float w0 = ml0.y > 0.f ? exp2f(ml0.x - mx) : 0.f;
         const float w1 = ml1.y > 0.f ? exp2f(ml1.x - mx) : 0.f;
         float den = 0.f;                                 // terms added in block order: independent of timing
+#pragma unroll 1
         for (int s = 0; s < n_splits; ++s) den += __shfl_sync(0xFFFFFFFFu, s < 32 ? ml0.y * w0 : ml1.y * w1, s & 31);
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 1
         for (int s0 = 0; s0 < n_splits; s0 += B6) {
           if (s0 > 0) {
 #pragma unroll
@@ -1174,6 +1218,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
     // ================= the sequence of steps
     const size_t stride_d = (size_t)p.n_alloc * p.d;
     const size_t stride_qkv = (size_t)p.n_alloc * p.qkv_dim;
+#pragma unroll 1
     for (int sidx = 0; sidx < n_steps; ++sidx) {
       const int l = sidx / ST_PER_LAYER, st = sidx - l * ST_PER_LAYER;
       const bool head = l == p.n_layers;
@@ -1224,6 +1269,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
   __syncthreads();
   if (*abort) {
     // give copies still in flight time to land before the shared memory is handed back
+#pragma unroll 1
     for (int i = 0; i < 64; ++i) __nanosleep(20000);
     __syncthreads();
   }
@@ -1271,18 +1317,6 @@ bool fused_stack_supported(const specasr_kv* wk, int n_total, bool att_tc, int s
   return true;
 }
 
-// Units (32 KB of weights each) every CTA keeps requested into L2 ahead of its ring: 16 x 148 CTAs = 78 MB, which
-// leaves room in the 126 MB L2 for the activations and the layer's K / V pages.
-static int fused_lookahead() {
-  static int v = -1;
-  if (v < 0) {
-    const char* e = getenv("SPECASR_LOOKAHEAD");
-    v = e ? atoi(e) : 16;
-    if (v < 0) v = 0;
-  }
-  return v;
-}
-
 size_t fused_stack_sync_bytes(const specasr_model* m) {
   return (((size_t)m->cfg.n_layers * ST_PER_LAYER + 2) * sizeof(int32_t) + 255) / 256 * 256;
 }
@@ -1317,7 +1351,6 @@ bool launch_fused_stack(specasr_model* m, specasr_kv* wk, const SegTable& tab, i
   p.epoch0 = wk->gemm_epoch;
   wk->gemm_epoch += c.n_layers + 1;
   p.want_head = want_head ? 1 : 0;
-  p.lookahead = fused_lookahead();
   p.group = c.n_heads / c.n_kv_heads;
   p.nodes_per_tile = 128 / p.group;
   p.row_tiles = (n_max + p.nodes_per_tile - 1) / p.nodes_per_tile;
@@ -1334,6 +1367,7 @@ bool launch_fused_stack(specasr_model* m, specasr_kv* wk, const SegTable& tab, i
 #endif
   const size_t smem = (size_t)p.ring_bytes + sizeof(StackCtl) + epi_bytes + 1024;
   int idx = 0;                                           // activation maps are indexed by log2(box rows / 16)
+#pragma unroll 1
   for (int b = 16; b < n_pad; b <<= 1) ++idx;
   LaunchScope scope(wk, SPECASR_KIND_STACK, s);
   cudaError_t e = cudaMemsetAsync(wk->ws.sync, 0, fused_stack_sync_bytes(m), s);
