@@ -390,3 +390,145 @@ def greedy_continuation(cfg, weights: Weights, cache: KVCache, root_token: int, 
         tok = int(np.argmax(logits[-1]))
         out.append(tok)
     return out
+
+
+# --------------------------------------------------------------------------- draft side (Section IV)
+#
+# The three drafting strategies of Section IV, restated as plain control flow over a "draft step"
+# callable.  They decide which tokens are proposed; they never touch what the target accepts, so the
+# lossless property of Section II-B is untouched by them.  Readings taken where the paper is silent:
+#   * "normalized logits" (Section IV-A) = softmax probability over the whole vocabulary (top2_probs);
+#   * "corresponding or adjacent positions" (Section IV-B) = position offsets 0, -1, +1, tried in that order;
+#   * a side branch of the sparse tree (Section IV-C) starts with the second-ranked token at an uncertain
+#     trunk position, is extended greedily, keeps the token on which it meets the trunk or an earlier branch
+#     and ends there; a branch also ends after `max_branch` tokens or when the node budget is used up.
+
+RECYCLE_OFFSETS = (0, -1, 1)
+
+
+def match_position(seq_tokens, seq_first_pos: int, token: int, pos: int, offsets=RECYCLE_OFFSETS,
+                   lowest_pos: int | None = None):
+    """Section IV-B, merging: does `token`, generated for position `pos`, equal the token that the
+    sequence `seq_tokens` (whose first token sits at position `seq_first_pos`) carries at the same or an
+    adjacent position?  Returns the index into seq_tokens of the first such position in the order of
+    `offsets`, or None.  Positions below `lowest_pos` are not considered."""
+    for off in offsets:
+        q = pos + off
+        if lowest_pos is not None and q < lowest_pos:
+            continue
+        i = q - seq_first_pos
+        if 0 <= i < len(seq_tokens) and int(seq_tokens[i]) == int(token):
+            return i
+    return None
+
+
+def adaptive_sequence(step_fn, root: int, max_len: int, threshold: float) -> list[int]:
+    """Section IV-A: greedy single-sequence drafting that stops after the first token whose probability
+    falls below `threshold` (that token is still proposed), or after `max_len` tokens.
+    step_fn(path) -> next-token logits [V] of the draft model after the context and `path` (path[0] = root)."""
+    path, out = [int(root)], []
+    for _ in range(max_len):
+        ids, probs = top2_probs(np.asarray(step_fn(path), dtype=F64)[None, :])
+        out.append(int(ids[0, 0]))
+        path.append(int(ids[0, 0]))
+        if probs[0, 0] < threshold:
+            break
+    return out
+
+
+def two_pass_tree(step_fn, root: int, max_len: int, threshold: float, n_nodes: int, max_branch: int) -> dict:
+    """Section IV-C, two-pass sparse-tree prediction.
+
+    Pass 1: greedy single-sequence decoding of `max_len` trunk tokens; a position whose top-1 probability
+    is below `threshold` is marked together with the second-ranked token, and decoding goes on.
+    Pass 2: at every mark, in trunk order, a branch starts with the second-ranked token as a sibling of the
+    trunk token and is extended greedily; it ends with the token that equals the trunk's (or an earlier
+    branch's) token at the corresponding or an adjacent depth, after `max_branch` tokens, or when the tree
+    has `n_nodes` nodes.  Returns tokens / parent (root = node 0, trunk = nodes 1..m in order, then the
+    branches in the order they were grown), the marks [(depth, second token)] and the depth of every node."""
+    tokens, parent, depth = [int(root)], [-1], [0]
+    path, marks = [int(root)], []
+    for j in range(1, max_len + 1):
+        if len(tokens) >= n_nodes:
+            break
+        ids, probs = top2_probs(np.asarray(step_fn(path), dtype=F64)[None, :])
+        tokens.append(int(ids[0, 0]))
+        parent.append(len(tokens) - 2)
+        depth.append(j)
+        path.append(int(ids[0, 0]))
+        if probs[0, 0] < threshold and int(ids[0, 1]) != int(ids[0, 0]):
+            marks.append((j, int(ids[0, 1])))
+    m = len(tokens) - 1                                   # trunk nodes are 1..m, trunk token at depth d is tokens[d]
+    grown = []                                            # (first depth, tokens) of the branches so far
+
+    def rejoins(tok, d):
+        if match_position(tokens[1:m + 1], 1, tok, d) is not None:
+            return True
+        return any(match_position(bt, d0, tok, d) is not None for d0, bt in grown)
+
+    for j, second in marks:
+        if len(tokens) >= n_nodes:
+            break
+        bpath = [int(root)] + tokens[1:j] + [second]
+        tokens.append(second)
+        parent.append(j - 1)                              # sibling of trunk node j
+        depth.append(j)
+        btoks = [second]
+        while not rejoins(btoks[-1], j + len(btoks) - 1) and len(btoks) < max_branch and len(tokens) < n_nodes:
+            nxt = int(np.argmax(np.asarray(step_fn(bpath), dtype=F64)))
+            tokens.append(nxt)
+            parent.append(len(tokens) - 2)
+            depth.append(j + len(btoks))
+            btoks.append(nxt)
+            bpath.append(nxt)
+        grown.append((j, btoks))
+    return {"tokens": np.asarray(tokens, np.int32), "parent": np.asarray(parent, np.int32),
+            "depth": np.asarray(depth, np.int64), "marks": marks, "trunk_len": m}
+
+
+def recycled_draft(tree_step_fn, last_accepted: int, seq1, accept_len: int, bonus: int, max_len: int,
+                   max_regen: int) -> dict:
+    """Section IV-B, draft sequence recycling after a verification round.
+
+    `seq1` is the draft sequence that was verified (trunk tokens at depths 1..m under the old root);
+    `accept_len` of them were accepted and the target emitted `bonus` for depth accept_len + 1.  The draft
+    model now decodes two sequences side by side in one masked token tree under the last accepted token:
+    sequence 1, the unaccepted tail seq1[accept_len:], which it keeps extending, and sequence 2, which starts
+    at `bonus` and regenerates what failed.  After every step the token just regenerated for depth q is
+    compared with sequence 1 at depths q, q - 1, q + 1; on a match the two sequences are merged: the next
+    draft is the regenerated tokens followed by what sequence 1 holds after the matching depth.
+
+    tree_step_fn(tokens, parent) -> logits [n, V] of the draft model over a token tree whose node 0 is
+    `last_accepted`, the last accepted token (the old root if nothing was accepted); its context is
+    everything before that token.  Returns the next draft (the tokens proposed
+    after `bonus`, at most max_len), how many regeneration steps were made and where the merge happened."""
+    seq1 = [int(t) for t in seq1]
+    a = int(accept_len)
+    tail = seq1[a:]                                       # depths a+1 .. m; tail[0] is the rejected token
+    if not tail:                                          # everything was accepted: nothing to recycle
+        return {"draft": [], "steps": 0, "merged_at": None, "regenerated": [], "extended": []}
+    regen, ext = [], []
+    merged = None
+    for step in range(max_regen):
+        # node 0 = last accepted token; chain 1 = sequence 1, chain 2 = sequence 2
+        c1 = tail + ext
+        c2 = [int(bonus)] + regen
+        tokens = [int(last_accepted)] + c1 + c2
+        parent = [-1] + [0] + list(range(1, len(c1))) + [0] + list(range(len(c1) + 1, len(c1) + len(c2)))
+        logits = np.asarray(tree_step_fn(np.asarray(tokens), np.asarray(parent)), dtype=F64)
+        ext.append(int(np.argmax(logits[len(c1)])))       # after the tip of sequence 1
+        r = int(np.argmax(logits[len(c1) + len(c2)]))     # after the tip of sequence 2
+        regen.append(r)
+        q = a + 1 + len(regen)                            # depth of the token just regenerated
+        hit = match_position(tail + ext, a + 1, r, q, lowest_pos=a + 1)
+        if hit is not None:
+            merged = a + 1 + hit
+            break
+        if len(regen) >= max_len:
+            break
+    if merged is not None:
+        reuse = (tail + ext)[merged - a:]                 # what sequence 1 holds after the matching depth
+        draft = regen + reuse
+    else:
+        draft = list(regen)
+    return {"draft": draft[:max_len], "steps": len(regen), "merged_at": merged, "regenerated": regen, "extended": ext}
