@@ -190,6 +190,28 @@ specasr_status specasr_verify_tree_batch(specasr_model* m, int32_t batch, specas
                                          int32_t* out_path, float* out_logits, int32_t* out_bonus, void* stream);
 
 /*
+ * The same verification with the draft side's quantities computed in the vocabulary projection's epilogue instead of
+ * from a materialised logits matrix: for every node the two most probable next tokens and their probabilities under
+ * the softmax over the whole vocabulary.  Run on the DRAFT model these are what Section IV reads: drafting stops where
+ * the top-1 value falls below a threshold (Section IV-A), and the second-ranked token at such a position seeds a side
+ * branch of the sparse tree (Section IV-C).
+ *   out_top2_ids   : [device] int32 [n_nodes, 2]  (ties: lower id first; -1 for an utterance whose tree was refused)
+ *   out_top2_probs : [device] fp32  [n_nodes, 2]
+ * Everything else as in specasr_verify_tree_ex / specasr_verify_tree_batch (no logits output).  Needs the fused layer
+ * stack: tensor-core attention (head_dim 64 or 128, page_size a multiple of 16) and at most 64 nodes in the call;
+ * otherwise SPECASR_ERR_UNSUPPORTED with nothing enqueued.
+ */
+specasr_status specasr_verify_tree_top2(specasr_model* m, specasr_kv* kv, const int32_t* tokens,
+                                        const int32_t* parent_idx, int32_t n_nodes, int32_t* out_argmax,
+                                        int32_t* out_accept_len, int32_t* out_path, int32_t* out_bonus,
+                                        int32_t* out_top2_ids, float* out_top2_probs, void* stream);
+specasr_status specasr_verify_tree_batch_top2(specasr_model* m, int32_t batch, specasr_kv* const* kv,
+                                              const int32_t* tokens, const int32_t* parent_idx,
+                                              const int32_t* node_offsets, int32_t* out_argmax,
+                                              int32_t* out_accept_len, int32_t* out_path, int32_t* out_bonus,
+                                              int32_t* out_top2_ids, float* out_top2_probs, void* stream);
+
+/*
  * Keep the accepted path (after a round control goes back to the draft model, Section II-B, so the cache must
  * hold exactly prefix + accepted tokens): slot L+j <- slot L+path[j] for j = 0..accept_len, all
  * layers, K and V; then L <- L + accept_len + 1.  path / accept_len are the [device] arrays a

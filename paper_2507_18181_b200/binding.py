@@ -22,7 +22,7 @@ EXPORTS = [
     "specasr_model_create", "specasr_model_destroy", "specasr_workspace_bytes", "specasr_kv_pool_bytes",
     "specasr_kv_create", "specasr_kv_destroy", "specasr_kv_length", "specasr_kv_truncate",
     "specasr_prefill_embeds", "specasr_prefill_tokens", "specasr_verify_tree", "specasr_verify_tree_ex",
-    "specasr_verify_tree_batch", "specasr_commit_kv", "specasr_poll_status", "specasr_launch_count", "specasr_last_error",
+    "specasr_verify_tree_batch", "specasr_verify_tree_top2", "specasr_verify_tree_batch_top2", "specasr_commit_kv", "specasr_poll_status", "specasr_launch_count", "specasr_last_error",
     "specasr_profile_enable", "specasr_profile_read", "specasr_trace_set", "specasr_accept_logits_static", "specasr_top2_probs",
 ]
 KIND_NAMES = ["prep", "norm", "gemm_qkv", "rope", "attn", "attn_merge", "gemm_o", "gemm_gu", "gemm_down", "gemm_lm",
@@ -79,6 +79,10 @@ def lib() -> C.CDLL:
         L.specasr_verify_tree_ex.restype = st
         L.specasr_verify_tree_batch.argtypes = [vp, i32, C.POINTER(vp), vp, vp, C.POINTER(i32), vp, vp, vp, vp, vp, vp]
         L.specasr_verify_tree_batch.restype = st
+        L.specasr_verify_tree_top2.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp]
+        L.specasr_verify_tree_top2.restype = st
+        L.specasr_verify_tree_batch_top2.argtypes = [vp, i32, C.POINTER(vp), vp, vp, C.POINTER(i32), vp, vp, vp, vp, vp, vp, vp]
+        L.specasr_verify_tree_batch_top2.restype = st
         L.specasr_commit_kv.argtypes = [vp, vp, vp, vp, vp]
         L.specasr_commit_kv.restype = st
         L.specasr_poll_status.argtypes = [vp, C.POINTER(i32), vp]
@@ -189,6 +193,26 @@ def specasr_verify_tree_batch(model: int, kv_handles, tokens: int, parent_idx: i
         raise ValueError("node_offsets needs batch + 1 entries")
     _check(lib().specasr_verify_tree_batch(model, batch, handles, tokens, parent_idx, offsets, out_argmax,
                                            out_accept_len, out_path, out_logits or None, out_bonus or None, stream))
+
+
+def specasr_verify_tree_top2(model: int, kv: int, tokens: int, parent_idx: int, n_nodes: int, out_argmax: int,
+                             out_accept_len: int, out_path: int, out_bonus: int, out_top2_ids: int, out_top2_probs: int,
+                             stream: int = 0) -> None:
+    _check(lib().specasr_verify_tree_top2(model, kv, tokens, parent_idx, n_nodes, out_argmax, out_accept_len, out_path,
+                                          out_bonus or None, out_top2_ids, out_top2_probs, stream))
+
+
+def specasr_verify_tree_batch_top2(model: int, kv_handles, tokens: int, parent_idx: int, node_offsets, out_argmax: int,
+                                   out_accept_len: int, out_path: int, out_bonus: int, out_top2_ids: int,
+                                   out_top2_probs: int, stream: int = 0) -> None:
+    batch = len(kv_handles)
+    handles = (C.c_void_p * batch)(*kv_handles)
+    offsets = (C.c_int32 * len(node_offsets))(*node_offsets)
+    if len(node_offsets) != batch + 1:
+        raise ValueError("node_offsets needs batch + 1 entries")
+    _check(lib().specasr_verify_tree_batch_top2(model, batch, handles, tokens, parent_idx, offsets, out_argmax,
+                                                out_accept_len, out_path, out_bonus or None, out_top2_ids,
+                                                out_top2_probs, stream))
 
 
 def specasr_commit_kv(model: int, kv: int, path: int, accept_len: int, stream: int = 0) -> None:

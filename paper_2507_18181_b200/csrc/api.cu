@@ -69,6 +69,8 @@ Workspace carve_workspace(const specasr_model* m, int n_alloc, void* base) {
   w.attML = (float2*)take(sizeof(float2) * kMaxAttnSplits * n_alloc * c.n_heads);
   w.amax = (unsigned long long*)take(sizeof(unsigned long long) * lm_tiles_of(m) * n_alloc);
   w.tmKV = (CUtensorMap*)take(sizeof(CUtensorMap) * 2);
+  w.sec = (unsigned long long*)take(sizeof(unsigned long long) * lm_tiles_of(m) * n_alloc);
+  w.lse = (float2*)take(sizeof(float2) * lm_tiles_of(m) * n_alloc);
   w.ssq = (float*)take(sizeof(float) * 2 * n_alloc);
   w.sync = (int32_t*)take(fused_stack_sync_bytes(m));
   w.bytes = off;
@@ -495,11 +497,11 @@ static SegDev seg_entry(const specasr_kv* u, int row0, int n) {
 // and work against its cache and control block.  With want_head the final norm, the vocabulary projection
 // and its fused per-tile argmax run as well.
 static void run_stack(specasr_model* m, specasr_kv* wk, const SegTable& tab, int n_total, int n_max, bool att_tc,
-                      const int32_t* ctl_shared, bool want_head, float* out_logits, cudaStream_t s) {
+                      const int32_t* ctl_shared, bool want_head, float* out_logits, bool want_top2, cudaStream_t s) {
   const specasr_model_config& c = m->cfg;
   const int n = n_total;
   if (fused_stack_supported(wk, n_total, att_tc, tab.splits)) {
-    launch_fused_stack(m, wk, tab, n_total, n_max, ctl_shared, want_head, out_logits, s);
+    launch_fused_stack(m, wk, tab, n_total, n_max, ctl_shared, want_head, out_logits, want_top2, s);
     return;
   }
   const int n_pad = pad_tokens(n);
@@ -579,7 +581,7 @@ static specasr_status prefill_common(specasr_model* m, specasr_kv* kv, const flo
     const SegTable tab = single_table(kv, chunk, &att_tc);
     if (embeds) launch_copy_embeds(kv, embeds + (size_t)done * m->cfg.d_model, chunk, s);
     else launch_embed_tokens(kv, tab, chunk, tokens + done, s);
-    run_stack(m, kv, tab, chunk, chunk, att_tc, kv->ws.ctl, false, nullptr, s);
+    run_stack(m, kv, tab, chunk, chunk, att_tc, kv->ws.ctl, false, nullptr, false, s);
     launch_advance_len(kv, chunk, s);
     kv->len_host += chunk;
     kv->len_upper = kv->len_host;
@@ -599,10 +601,10 @@ extern "C" specasr_status specasr_prefill_tokens(specasr_model* m, specasr_kv* k
   return prefill_common(m, kv, nullptr, tokens, n, (cudaStream_t)stream, "specasr_prefill_tokens");
 }
 
-extern "C" specasr_status specasr_verify_tree_ex(specasr_model* m, specasr_kv* kv, const int32_t* tokens,
-                                                 const int32_t* parent_idx, int32_t n_nodes, int32_t* out_argmax,
-                                                 int32_t* out_accept_len, int32_t* out_path, float* out_logits,
-                                                 int32_t* out_bonus, void* stream) {
+static specasr_status verify_tree_impl(specasr_model* m, specasr_kv* kv, const int32_t* tokens,
+                                       const int32_t* parent_idx, int32_t n_nodes, int32_t* out_argmax,
+                                       int32_t* out_accept_len, int32_t* out_path, float* out_logits,
+                                       int32_t* out_bonus, int32_t* out_top2_ids, float* out_top2_probs, void* stream) {
   if (!m || !kv || !tokens || !parent_idx || !out_argmax || !out_accept_len || !out_path) {
     set_error("specasr_verify_tree: null argument");
     return SPECASR_ERR_INVALID_ARG;
@@ -625,13 +627,40 @@ extern "C" specasr_status specasr_verify_tree_ex(specasr_model* m, specasr_kv* k
   cudaStream_t s = (cudaStream_t)stream;
   bool att_tc = false;
   const SegTable tab = single_table(kv, n_nodes, &att_tc);
+  const bool want_top2 = out_top2_ids != nullptr;
+  if (want_top2 && !fused_stack_supported(kv, n_nodes, att_tc, tab.splits)) {
+    set_error("specasr_verify_tree_top2: the top-2 epilogue needs the fused layer stack (tensor-core attention, at most "
+              "64 nodes)");
+    return SPECASR_ERR_UNSUPPORTED;
+  }
   launch_tree_prep(kv, tab, tokens, parent_idx, s);
   launch_embed_tokens(kv, tab, n_nodes, tokens, s);
-  run_stack(m, kv, tab, n_nodes, n_nodes, att_tc, kv->ws.ctl, true, out_logits, s);
+  run_stack(m, kv, tab, n_nodes, n_nodes, att_tc, kv->ws.ctl, true, out_logits, want_top2, s);
   launch_accept(kv, tab, nullptr, tokens, parent_idx, lm_tiles_of(m), out_argmax, out_accept_len, out_path, out_bonus, s);
+  if (want_top2) launch_top2_from_tiles(kv, tab, nullptr, n_nodes, lm_tiles_of(m), out_top2_ids, out_top2_probs, s);
   kv->pending_n = n_nodes;
   CUDA_TRY(cudaGetLastError());
   return SPECASR_OK;
+}
+
+extern "C" specasr_status specasr_verify_tree_ex(specasr_model* m, specasr_kv* kv, const int32_t* tokens,
+                                                 const int32_t* parent_idx, int32_t n_nodes, int32_t* out_argmax,
+                                                 int32_t* out_accept_len, int32_t* out_path, float* out_logits,
+                                                 int32_t* out_bonus, void* stream) {
+  return verify_tree_impl(m, kv, tokens, parent_idx, n_nodes, out_argmax, out_accept_len, out_path, out_logits,
+                          out_bonus, nullptr, nullptr, stream);
+}
+
+extern "C" specasr_status specasr_verify_tree_top2(specasr_model* m, specasr_kv* kv, const int32_t* tokens,
+                                                   const int32_t* parent_idx, int32_t n_nodes, int32_t* out_argmax,
+                                                   int32_t* out_accept_len, int32_t* out_path, int32_t* out_bonus,
+                                                   int32_t* out_top2_ids, float* out_top2_probs, void* stream) {
+  if (!out_top2_ids || !out_top2_probs) {
+    set_error("specasr_verify_tree_top2: null output");
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  return verify_tree_impl(m, kv, tokens, parent_idx, n_nodes, out_argmax, out_accept_len, out_path, nullptr, out_bonus,
+                          out_top2_ids, out_top2_probs, stream);
 }
 
 extern "C" specasr_status specasr_verify_tree(specasr_model* m, specasr_kv* kv, const int32_t* tokens,
@@ -643,11 +672,11 @@ extern "C" specasr_status specasr_verify_tree(specasr_model* m, specasr_kv* kv, 
 
 // Several utterances in one pass over the weights: the verification of Section II-B applied to each utterance,
 // with the norms and projections run once over all rows.
-extern "C" specasr_status specasr_verify_tree_batch(specasr_model* m, int32_t batch, specasr_kv* const* kv,
-                                                    const int32_t* tokens, const int32_t* parent_idx,
-                                                    const int32_t* node_offsets, int32_t* out_argmax,
-                                                    int32_t* out_accept_len, int32_t* out_path, float* out_logits,
-                                                    int32_t* out_bonus, void* stream) {
+static specasr_status verify_batch_impl(specasr_model* m, int32_t batch, specasr_kv* const* kv,
+                                        const int32_t* tokens, const int32_t* parent_idx,
+                                        const int32_t* node_offsets, int32_t* out_argmax,
+                                        int32_t* out_accept_len, int32_t* out_path, float* out_logits,
+                                        int32_t* out_bonus, int32_t* out_top2_ids, float* out_top2_probs, void* stream) {
   const char* who = "specasr_verify_tree_batch";
   if (!m || !kv || !tokens || !parent_idx || !node_offsets || !out_argmax || !out_accept_len || !out_path) {
     set_error("%s: null argument", who);
@@ -716,14 +745,42 @@ extern "C" specasr_status specasr_verify_tree_batch(specasr_model* m, int32_t ba
   cudaStream_t s = (cudaStream_t)stream;
   int32_t* ctl_shared = wk->ws.ctl + kCtlBatch;
   CUDA_TRY(cudaMemsetAsync(ctl_shared, 0, sizeof(int32_t) * 4, s));
+  const bool want_top2 = out_top2_ids != nullptr;
+  if (want_top2 && !fused_stack_supported(wk, total, true, tab.splits)) {
+    set_error("%s: the top-2 epilogue needs the fused layer stack (at most 64 nodes in all)", who);
+    return SPECASR_ERR_UNSUPPORTED;
+  }
   launch_tree_prep(wk, tab, tokens, parent_idx, s);
   launch_embed_tokens(wk, tab, total, tokens, s);
-  run_stack(m, wk, tab, total, n_max, true, ctl_shared, true, out_logits, s);
+  run_stack(m, wk, tab, total, n_max, true, ctl_shared, true, out_logits, want_top2, s);
   launch_accept(wk, tab, ctl_shared, tokens, parent_idx, lm_tiles_of(m), out_argmax, out_accept_len, out_path, out_bonus,
                 s);
+  if (want_top2) launch_top2_from_tiles(wk, tab, ctl_shared, total, lm_tiles_of(m), out_top2_ids, out_top2_probs, s);
   for (int b = 0; b < batch; ++b) kv[b]->pending_n = tab.seg[b].n;
   CUDA_TRY(cudaGetLastError());
   return SPECASR_OK;
+}
+
+extern "C" specasr_status specasr_verify_tree_batch(specasr_model* m, int32_t batch, specasr_kv* const* kv,
+                                                    const int32_t* tokens, const int32_t* parent_idx,
+                                                    const int32_t* node_offsets, int32_t* out_argmax,
+                                                    int32_t* out_accept_len, int32_t* out_path, float* out_logits,
+                                                    int32_t* out_bonus, void* stream) {
+  return verify_batch_impl(m, batch, kv, tokens, parent_idx, node_offsets, out_argmax, out_accept_len, out_path,
+                           out_logits, out_bonus, nullptr, nullptr, stream);
+}
+
+extern "C" specasr_status specasr_verify_tree_batch_top2(specasr_model* m, int32_t batch, specasr_kv* const* kv,
+                                                         const int32_t* tokens, const int32_t* parent_idx,
+                                                         const int32_t* node_offsets, int32_t* out_argmax,
+                                                         int32_t* out_accept_len, int32_t* out_path, int32_t* out_bonus,
+                                                         int32_t* out_top2_ids, float* out_top2_probs, void* stream) {
+  if (!out_top2_ids || !out_top2_probs) {
+    set_error("specasr_verify_tree_batch_top2: null output");
+    return SPECASR_ERR_INVALID_ARG;
+  }
+  return verify_batch_impl(m, batch, kv, tokens, parent_idx, node_offsets, out_argmax, out_accept_len, out_path, nullptr,
+                           out_bonus, out_top2_ids, out_top2_probs, stream);
 }
 
 extern "C" specasr_status specasr_commit_kv(specasr_model* m, specasr_kv* kv, const int32_t* path,

@@ -67,6 +67,8 @@ struct alignas(16) StackCtl {
   unsigned long long acc_empty[2];
   unsigned long long bar_qk, bar_v, bar_s, bar_p[2], bar_o[2];
   unsigned long long key[64];
+  unsigned long long k1q[4][64], k2q[4][64];   // per lane quadrant: best and second-best packed key of a vocabulary tile
+  float2 msq[4][64];                    // per lane quadrant: (max, sum of exp(x - max)) over the tile's rows
   float red_max[2][128];
   float red_sum[2][128];
   float inv[64];                        // 1 / rms of every token row, for the epilogue in progress
@@ -100,6 +102,8 @@ struct StackParams {
   float2* attML;
   float* ssq;                           // [NORM_PARTS][n_alloc]
   unsigned long long* amax;
+  unsigned long long* sec;              // [tiles][n_alloc] second-best packed key of every vocabulary tile, or null
+  float2* lse;                          // [tiles][n_alloc] (max, sum of exp(x - max)) of every vocabulary tile, or null
   float* logits;
   const int32_t* pos;
   const unsigned long long* anc;
@@ -871,6 +875,21 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
                 const uint32_t who = __reduce_min_sync(0xFFFFFFFFu, key == best ? (uint32_t)m : 0xFFFFFFFFu);
                 if (lane == 0 && t < p.n && best != 0u)
                   atomicMax(&sc->key[t], ((unsigned long long)best << 32) | (unsigned long long)(0xFFFFFFFFu - who));
+                if (p.sec != nullptr) {
+                  // the draft side also wants the runner-up and the softmax denominator (Sections IV-A, IV-C): second
+                  // largest key of this warp's 32 rows, and the sum of exp(x - warp max)
+                  const uint32_t key2 = (uint32_t)m != who ? key : 0u;
+                  const uint32_t sbest = __reduce_max_sync(0xFFFFFFFFu, key2);
+                  const uint32_t swho = __reduce_min_sync(0xFFFFFFFFu, key2 == sbest ? (uint32_t)m : 0xFFFFFFFFu);
+                  const uint32_t ub = (best & 0x80000000u) ? (best & 0x7FFFFFFFu) : ~best;
+                  const float vmax = __uint_as_float(ub);
+                  const float esum = warp_sum((row_ok && best != 0u) ? __expf(v[j] - vmax) : 0.f);
+                  if (lane == 0 && t < p.n) {
+                    sc->k1q[quad][t] = best != 0u ? ((unsigned long long)best << 32) | (unsigned long long)(0xFFFFFFFFu - who) : 0ull;
+                    sc->k2q[quad][t] = sbest != 0u ? ((unsigned long long)sbest << 32) | (unsigned long long)(0xFFFFFFFFu - swho) : 0ull;
+                    sc->msq[quad][t] = best != 0u ? make_float2(vmax, esum) : make_float2(-INFINITY, 0.f);
+                  }
+                }
               }
             }
           }
@@ -892,7 +911,32 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
             }
           } else {
 #pragma unroll 1
-            for (int t = wtid; t < p.n; t += WORKERS) p.amax[(size_t)tile * p.n_alloc + t] = sc->key[t];
+            for (int t = wtid; t < p.n; t += WORKERS) {
+              p.amax[(size_t)tile * p.n_alloc + t] = sc->key[t];
+              if (p.sec != nullptr) {                          // the four quadrants of the tile, in a fixed order
+                unsigned long long a = 0ull, b = 0ull;
+                float mm = -INFINITY, ss = 0.f;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                  const unsigned long long c1 = sc->k1q[q][t], c2 = sc->k2q[q][t];     // c1 > c2, all keys distinct or 0
+                  if (c1 > a) {
+                    b = a;
+                    a = c1;
+                  } else if (c1 > b) {
+                    b = c1;
+                  }
+                  if (c2 > b) b = c2;                                                   // c2 < c1 <= a
+                  const float2 ms = sc->msq[q][t];
+                  const float mx = fmaxf(mm, ms.x);
+                  if (mx > -INFINITY) {
+                    ss = ss * __expf(mm - mx) + ms.y * __expf(ms.x - mx);
+                    mm = mx;
+                  }
+                }
+                p.sec[(size_t)tile * p.n_alloc + t] = b;
+                p.lse[(size_t)tile * p.n_alloc + t] = make_float2(mm, ss);
+              }
+            }
           }
           tc_fence_before();
           mbar_arrive(&sc->acc_empty[b]);
@@ -1322,7 +1366,7 @@ size_t fused_stack_sync_bytes(const specasr_model* m) {
 }
 
 bool launch_fused_stack(specasr_model* m, specasr_kv* wk, const SegTable& tab, int n_total, int n_max,
-                        const int32_t* ctl_shared, bool want_head, float* out_logits, cudaStream_t s) {
+                        const int32_t* ctl_shared, bool want_head, float* out_logits, bool want_top2, cudaStream_t s) {
   const specasr_model_config& c = m->cfg;
   int n_pad = 16;
   while (n_pad < n_total) n_pad <<= 1;
@@ -1361,6 +1405,8 @@ bool launch_fused_stack(specasr_model* m, specasr_kv* wk, const SegTable& tab, i
   p.H = wk->ws.H; p.Q = wk->ws.Q; p.AO = wk->ws.AO; p.A = wk->ws.A;
   p.attO = wk->ws.attO; p.attML = wk->ws.attML; p.ssq = wk->ws.ssq; p.amax = wk->ws.amax;
   p.logits = out_logits;
+  p.sec = want_top2 ? wk->ws.sec : nullptr;
+  p.lse = want_top2 ? wk->ws.lse : nullptr;
   p.pos = wk->ws.pos; p.anc = wk->ws.anc;
 #ifdef SPECASR_TRACE
   p.tr = wk->trace;

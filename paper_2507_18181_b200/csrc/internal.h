@@ -85,6 +85,8 @@ struct Workspace {
   float2* attML;            // [kMaxAttnSplits][n_alloc * Hq]     (running max in log2 units, sum)
   unsigned long long* amax; // [lm_tiles][n_alloc] packed (ordered logit, ~token id) per vocab tile
   CUtensorMap* tmKV;        // [2] device copies of the K and V pool descriptors (tensor-core attention)
+  unsigned long long* sec;  // [lm_tiles][n_alloc] second-best packed key per vocabulary tile (fused stack, on request)
+  float2* lse;              // [lm_tiles][n_alloc] (max, sum of exp) per vocabulary tile (fused stack, on request)
   float* ssq;               // [2][n_alloc] sums of squares of the two halves of every residual row (fused stack)
   int32_t* sync;            // arrival counters of the fused stack kernel, one per step of the call
   size_t bytes;
@@ -246,7 +248,10 @@ void launch_tree_attention_tc(specasr_kv* wk, const SegTable& t, int n_max, int 
 bool fused_stack_supported(const specasr_kv* wk, int n_total, bool att_tc, int splits);
 size_t fused_stack_sync_bytes(const specasr_model* m);
 bool launch_fused_stack(specasr_model* m, specasr_kv* wk, const SegTable& tab, int n_total, int n_max,
-                        const int32_t* ctl_shared, bool want_head, float* out_logits, cudaStream_t s);
+                        const int32_t* ctl_shared, bool want_head, float* out_logits, bool want_top2, cudaStream_t s);
+// top2.cu: top-2 tokens and probabilities of every node from the per-tile pieces the vocabulary epilogue left
+void launch_top2_from_tiles(specasr_kv* wk, const SegTable& t, const int32_t* ctl_shared, int n_total, int n_tiles,
+                            int32_t* out_ids, float* out_probs, cudaStream_t s);
 
 // ---- gemm_fma.cu / gemm_tcgen05.cu
 enum GemmEpilogue {

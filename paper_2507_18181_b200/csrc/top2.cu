@@ -84,7 +84,75 @@ __global__ void __launch_bounds__(256) k_top2_probs(const float* __restrict__ lo
   }
 }
 
+// The same two tokens and probabilities from what the vocabulary projection's epilogue left per 128-row tile
+// (best and second-best packed key, max and sum of exp): one block per node, threads stride over the tiles.
+__global__ void __launch_bounds__(256) k_top2_from_tiles(const __grid_constant__ SegTable tab,
+                                                         const int32_t* __restrict__ ctl_shared,
+                                                         const unsigned long long* __restrict__ first,
+                                                         const unsigned long long* __restrict__ second,
+                                                         const float2* __restrict__ lse, int n_tiles, int n_alloc,
+                                                         int32_t* __restrict__ out_ids, float* __restrict__ out_probs) {
+  __shared__ Top2 s_top[8];
+  __shared__ float s_m[8], s_s[8];
+  grid_dep_launch();
+  grid_dep_wait();
+  const int node = blockIdx.x;
+  int b = 0;
+  while (b + 1 < tab.count && node >= tab.seg[b].row0 + tab.seg[b].n) ++b;
+  int32_t* ids = out_ids + (size_t)node * 2;
+  float* pr = out_probs + (size_t)node * 2;
+  if (tab.seg[b].ctl[CTL_STATUS] != 0 || (ctl_shared && ctl_shared[CTL_STATUS] != 0)) {
+    if (threadIdx.x == 0) {
+      ids[0] = ids[1] = -1;
+      pr[0] = pr[1] = 0.f;
+    }
+    return;
+  }
+  Top2 t{0ull, 0ull};
+  float m = -INFINITY, s = 0.f;
+  for (int tile = threadIdx.x; tile < n_tiles; tile += 256) {
+    top2_push(t, __ldcg(first + (size_t)tile * n_alloc + node));
+    top2_push(t, __ldcg(second + (size_t)tile * n_alloc + node));
+    const float2 ms = __ldcg(lse + (size_t)tile * n_alloc + node);
+    lse_merge(m, s, ms.x, ms.y);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const unsigned long long oa = __shfl_xor_sync(0xFFFFFFFFu, t.a, o), ob = __shfl_xor_sync(0xFFFFFFFFu, t.b, o);
+    top2_push(t, oa);
+    top2_push(t, ob);
+    const float om = __shfl_xor_sync(0xFFFFFFFFu, m, o), os = __shfl_xor_sync(0xFFFFFFFFu, s, o);
+    lse_merge(m, s, om, os);
+  }
+  const int warp = threadIdx.x >> 5;
+  if ((threadIdx.x & 31) == 0) {
+    s_top[warp] = t;
+    s_m[warp] = m;
+    s_s[warp] = s;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < 8; ++w) {
+      top2_push(t, s_top[w].a);
+      top2_push(t, s_top[w].b);
+      lse_merge(m, s, s_m[w], s_s[w]);
+    }
+    if (t.b == 0ull) t.b = t.a;                    // a one-token vocabulary
+    ids[0] = (int32_t)(0xFFFFFFFFu - (uint32_t)(t.a & 0xFFFFFFFFull));
+    ids[1] = (int32_t)(0xFFFFFFFFu - (uint32_t)(t.b & 0xFFFFFFFFull));
+    pr[0] = expf(key_value(t.a) - m) / s;
+    pr[1] = expf(key_value(t.b) - m) / s;
+  }
+}
+
 }  // namespace
+
+void launch_top2_from_tiles(specasr_kv* wk, const SegTable& t, const int32_t* ctl_shared, int n_total, int n_tiles,
+                            int32_t* out_ids, float* out_probs, cudaStream_t s) {
+  LaunchScope scope(wk, SPECASR_KIND_ACCEPT, s);
+  launch_pdl(k_top2_from_tiles, dim3(n_total), dim3(256), 0, s, t, ctl_shared, wk->ws.amax, wk->ws.sec, wk->ws.lse, n_tiles,
+             wk->n_alloc, out_ids, out_probs);
+}
 
 extern "C" specasr_status specasr_top2_probs(const float* logits, int32_t n_rows, int32_t vocab, int32_t* out_ids,
                                              float* out_probs, void* stream) {

@@ -209,3 +209,134 @@ class SpeculativeBatchLoop:
                     on_trunk += 1
                 self.draft_len[b] = min(self.draft_len[b], start[b] + on_trunk + 1)
         return [e[:n_tokens] for e in emitted]
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# Drafting strategies of Section IV on the draft model.  Control flow only: every forward pass of the draft model is
+# one tree-verification call of the library on the draft cache (the tree-masked attention is what lets two sequences
+# be decoded side by side, Section IV-B), and the top-2 tokens / probabilities come out of the vocabulary
+# projection's epilogue (specasr_verify_tree_top2).  A step re-verifies the whole uncommitted tree from its root, so
+# the draft cache itself is never advanced or rewound while drafting.
+
+RECYCLE_OFFSETS = (0, -1, 1)            # "corresponding or adjacent positions" (Section IV-B)
+
+
+def match_position(seq_tokens, seq_first_pos, token, pos, lowest_pos=None):
+    """Index into seq_tokens (whose first token sits at position seq_first_pos) of the first position among pos,
+    pos - 1, pos + 1 at which it carries `token`, or None."""
+    for off in RECYCLE_OFFSETS:
+        q = pos + off
+        if lowest_pos is not None and q < lowest_pos:
+            continue
+        i = q - seq_first_pos
+        if 0 <= i < len(seq_tokens) and int(seq_tokens[i]) == int(token):
+            return i
+    return None
+
+
+class DraftStrategies:
+    """The draft side of one utterance.  `draft_kv` holds the context up to, not including, node 0 of the trees
+    passed to it (the usual convention: the root's K/V is not in the cache yet)."""
+
+    def __init__(self, draft_kv: DeviceKV):
+        self.kv = draft_kv
+        self.device = draft_kv.model.device
+        self.forwards = 0
+
+    def tree_top2(self, tokens, parent):
+        """One forward pass of the draft model over a token tree: (ids [n, 2], probs [n, 2]) on the host."""
+        t = torch.tensor([int(x) for x in tokens], dtype=torch.int32, device=self.device)
+        p = torch.tensor([int(x) for x in parent], dtype=torch.int32, device=self.device)
+        self.kv.verify_top2(t, p)
+        self.forwards += 1
+        n = len(tokens)
+        ids = self.kv.out_top2_ids[:n].cpu().numpy()           # synchronises: the host decides how to go on
+        probs = self.kv.out_top2_probs[:n].cpu().numpy()
+        if int(ids[0, 0]) < 0:
+            raise RuntimeError(f"draft forward failed on the device (status {self.kv.status()})")
+        return ids, probs
+
+    def _chain_top2(self, path):
+        ids, probs = self.tree_top2(path, [-1] + list(range(len(path) - 1)))
+        return ids[-1], probs[-1]
+
+    def adaptive_sequence(self, root, max_len, threshold):
+        """Section IV-A: greedy drafting that stops after the first token whose probability is below the threshold."""
+        path, out = [int(root)], []
+        for _ in range(max_len):
+            ids, probs = self._chain_top2(path)
+            out.append(int(ids[0]))
+            path.append(int(ids[0]))
+            if probs[0] < threshold:
+                break
+        return out
+
+    def two_pass_tree(self, root, max_len, threshold, n_nodes, max_branch):
+        """Section IV-C: trunk by greedy decoding with uncertain positions marked, then one branch per mark that
+        starts with the second-ranked token and ends where it meets the trunk or an earlier branch."""
+        tokens, parent, depth = [int(root)], [-1], [0]
+        marks = []
+        for j in range(1, max_len + 1):
+            if len(tokens) >= n_nodes:
+                break
+            ids, probs = self._chain_top2(tokens)              # the trunk so far is a chain
+            tokens.append(int(ids[0]))
+            parent.append(len(tokens) - 2)
+            depth.append(j)
+            if probs[0] < threshold and int(ids[1]) != int(ids[0]):
+                marks.append((j, int(ids[1])))
+        m = len(tokens) - 1
+        grown = []
+
+        def rejoins(tok, d):
+            if match_position(tokens[1:m + 1], 1, tok, d) is not None:
+                return True
+            return any(match_position(bt, d0, tok, d) is not None for d0, bt in grown)
+
+        for j, second in marks:
+            if len(tokens) >= n_nodes:
+                break
+            tokens.append(second)
+            parent.append(j - 1)
+            depth.append(j)
+            btoks = [second]
+            while not rejoins(btoks[-1], j + len(btoks) - 1) and len(btoks) < max_branch and len(tokens) < n_nodes:
+                ids, _ = self.tree_top2(tokens, parent)        # the whole tree; the branch tip is its last node
+                tokens.append(int(ids[-1, 0]))
+                parent.append(len(tokens) - 2)
+                depth.append(j + len(btoks))
+                btoks.append(int(ids[-1, 0]))
+            grown.append((j, btoks))
+        return {"tokens": np.asarray(tokens, np.int32), "parent": np.asarray(parent, np.int32),
+                "depth": np.asarray(depth, np.int64), "marks": marks, "trunk_len": m}
+
+    def recycled_draft(self, last_accepted, seq1, accept_len, bonus, max_len, max_regen):
+        """Section IV-B: the unaccepted tail of the old draft (sequence 1, which keeps being extended) and the
+        regeneration from the target's token (sequence 2) are decoded side by side as two chains of one masked token
+        tree under the last accepted token; when a regenerated token equals sequence 1's token at the same or an
+        adjacent depth the sequences are merged and the rest of sequence 1 is reused."""
+        seq1 = [int(t) for t in seq1]
+        a = int(accept_len)
+        tail = seq1[a:]
+        if not tail:
+            return {"draft": [], "steps": 0, "merged_at": None, "regenerated": [], "extended": []}
+        regen, ext = [], []
+        merged = None
+        for _ in range(max_regen):
+            c1 = tail + ext
+            c2 = [int(bonus)] + regen
+            tokens = [int(last_accepted)] + c1 + c2
+            parent = [-1] + [0] + list(range(1, len(c1))) + [0] + list(range(len(c1) + 1, len(c1) + len(c2)))
+            ids, _ = self.tree_top2(tokens, parent)
+            ext.append(int(ids[len(c1), 0]))
+            r = int(ids[len(c1) + len(c2), 0])
+            regen.append(r)
+            q = a + 1 + len(regen)
+            hit = match_position(tail + ext, a + 1, r, q, lowest_pos=a + 1)
+            if hit is not None:
+                merged = a + 1 + hit
+                break
+            if len(regen) >= max_len:
+                break
+        draft = regen + (tail + ext)[merged - a:] if merged is not None else list(regen)
+        return {"draft": draft[:max_len], "steps": len(regen), "merged_at": merged, "regenerated": regen, "extended": ext}

@@ -149,6 +149,18 @@ class DeviceKV:
                                  logits.data_ptr() if logits is not None else 0, self.out_bonus.data_ptr(),
                                  self._stream())
 
+    def verify_top2(self, tokens: torch.Tensor, parent: torch.Tensor):
+        """As verify(), and the two most probable next tokens of every node with their probabilities land in
+        out_top2_ids / out_top2_probs ([n, 2] each), computed in the vocabulary projection's epilogue."""
+        n = tokens.shape[0]
+        if not hasattr(self, "out_top2_ids"):
+            self.out_top2_ids = torch.empty(self.max_nodes, 2, dtype=torch.int32, device=self.model.device)
+            self.out_top2_probs = torch.empty(self.max_nodes, 2, dtype=torch.float32, device=self.model.device)
+        B.specasr_verify_tree_top2(self.model.handle, self.handle, tokens.data_ptr(), parent.data_ptr(), n,
+                                   self.out_argmax.data_ptr(), self.out_accept.data_ptr(), self.out_path.data_ptr(),
+                                   self.out_bonus.data_ptr(), self.out_top2_ids.data_ptr(), self.out_top2_probs.data_ptr(),
+                                   self._stream())
+
     def commit(self):
         B.specasr_commit_kv(self.model.handle, self.handle, self.out_path.data_ptr(), self.out_accept.data_ptr(),
                             self._stream())
@@ -225,6 +237,18 @@ class BatchVerifier:
                                     self.out_accept.data_ptr(), self.out_path.data_ptr(),
                                     logits.data_ptr() if logits is not None else 0, self.out_bonus.data_ptr(),
                                     DeviceKV._stream())
+
+    def verify_top2(self, tokens: torch.Tensor, parent: torch.Tensor, node_offsets):
+        """As verify(), with the top-2 tokens and probabilities of every node in out_top2_ids / out_top2_probs."""
+        self.offsets = [int(o) for o in node_offsets]
+        if not hasattr(self, "out_top2_ids"):
+            total = self.kvs[0].max_nodes
+            self.out_top2_ids = torch.empty(total, 2, dtype=torch.int32, device=self.model.device)
+            self.out_top2_probs = torch.empty(total, 2, dtype=torch.float32, device=self.model.device)
+        B.specasr_verify_tree_batch_top2(self.model.handle, [kv.handle for kv in self.kvs], tokens.data_ptr(),
+                                         parent.data_ptr(), self.offsets, self.out_argmax.data_ptr(),
+                                         self.out_accept.data_ptr(), self.out_path.data_ptr(), self.out_bonus.data_ptr(),
+                                         self.out_top2_ids.data_ptr(), self.out_top2_probs.data_ptr(), DeviceKV._stream())
 
     def commit(self):
         item = self.out_path.element_size()
