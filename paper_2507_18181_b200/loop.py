@@ -139,7 +139,6 @@ class SpeculativeBatchLoop:
         `threshold` the second-ranked token becomes a one-node side branch at that position and the utterance
         stops drafting (adaptive truncation, Section IV-A, with the limited-width expansion of Section IV-C at
         the point of uncertainty); nobody drafts more than `max_len` tokens.  Returns {b: (tokens, parent)}."""
-        vocab = self.draft_kvs[0].model.cfg.vocab
         trunk = {b: [] for b in members}
         branch = {b: None for b in members}            # (depth of the parent on the trunk, token)
         cur = {b: int(roots[b]) for b in members}
@@ -149,15 +148,11 @@ class SpeculativeBatchLoop:
                 break
             bv = self._verifier(self.draft_kvs, live)
             nb = len(live)
-            if not hasattr(bv, "logits"):
-                bv.logits = torch.empty(nb, vocab, dtype=torch.float32, device=self.device)
-                bv.top_ids = torch.empty(nb, 2, dtype=torch.int32, device=self.device)
-                bv.top_probs = torch.empty(nb, 2, dtype=torch.float32, device=self.device)
             toks = torch.tensor([cur[b] for b in live], dtype=torch.int32, device=self.device)
-            bv.verify(toks, self._minus_one[:nb], list(range(nb + 1)), bv.logits)
+            # top-2 tokens and probabilities come out of the vocabulary projection's epilogue: no logits matrix is written
+            bv.verify_top2(toks, self._minus_one[:nb], list(range(nb + 1)))
             bv.commit()
-            B.specasr_top2_probs(bv.logits.data_ptr(), nb, vocab, bv.top_ids.data_ptr(), bv.top_probs.data_ptr(),
-                                 DeviceKV._stream())
+            bv.top_ids, bv.top_probs = bv.out_top2_ids[:nb], bv.out_top2_probs[:nb]
             ids = bv.top_ids.cpu().numpy()             # synchronises: the host decides who goes on
             probs = bv.top_probs.cpu().numpy()
             self.draft_steps += 1
@@ -208,6 +203,56 @@ class SpeculativeBatchLoop:
                 while on_trunk < a and int(path[on_trunk + 1]) == on_trunk + 1:
                     on_trunk += 1
                 self.draft_len[b] = min(self.draft_len[b], start[b] + on_trunk + 1)
+        return [e[:n_tokens] for e in emitted]
+
+    def decode_with_strategies(self, roots, n_tokens, strategy="two_pass", threshold=0.4, max_len=24, n_nodes=32,
+                               max_branch=4, max_regen=6):
+        """The whole method (Fig. 7): per round every utterance drafts with the draft model -- `two_pass`: a
+        two-pass sparse tree (Section IV-C); `recycle`: a single sequence that starts from the recycled remains of
+        the previous draft (Section IV-B) and is extended greedily until a token falls below the threshold or
+        max_len is reached (Section IV-A) -- then all trees are verified by the target in one batched call and the
+        accepted paths are committed.  Returns the transcripts.  `self.draft_forwards` counts draft-model passes."""
+        if self.draft_kvs is None:
+            raise ValueError("no draft caches were given")
+        emitted = [[] for _ in range(self.B)]
+        history = [[int(r)] for r in roots]
+        last = [None] * self.B                               # (trunk tokens, accept_len, last accepted token) of the last round
+        strategies = [DraftStrategies(kv) for kv in self.draft_kvs]
+        while True:
+            active = [b for b in range(self.B) if len(emitted[b]) < n_tokens]
+            if not active:
+                break
+            trees = {}
+            for b in active:
+                self.align_draft(b, history[b])              # the draft cache holds everything before the root
+                ds, root = strategies[b], history[b][-1]
+                if strategy == "two_pass":
+                    t = ds.two_pass_tree(root, max_len, threshold, n_nodes, max_branch)
+                    trees[b] = (t["tokens"], t["parent"])
+                    continue
+                trunk = []
+                if last[b] is not None and last[b][1] < len(last[b][0]):
+                    old, a, kept = last[b]
+                    kv = self.draft_kvs[b]
+                    kv.truncate(self.target_len[b] - 1)      # recycling decodes under the last accepted token
+                    trunk = ds.recycled_draft(kept, old, a, root, max_len, max_regen)["draft"]
+                    kv.prefill_tokens(torch.tensor([kept], dtype=torch.int32, device=self.device))
+                path = [root] + trunk                        # extend what was recycled, adaptively
+                while len(trunk) < max_len:
+                    ids, probs = ds._chain_top2(path)
+                    trunk.append(int(ids[0]))
+                    path.append(int(ids[0]))
+                    if probs[0] < threshold:
+                        break
+                trees[b] = (np.asarray([root] + trunk, np.int32), np.arange(-1, len(trunk), dtype=np.int32))
+            for b, (a, path, bonus) in self.verify_round(trees).items():
+                tokens = trees[b][0]
+                accepted = [int(tokens[i]) for i in path[1:]]
+                kept = accepted[-1] if accepted else history[b][-1]
+                emitted[b] += accepted + [bonus]
+                history[b] += accepted + [bonus]
+                last[b] = ([int(t) for t in tokens[1:]], a, kept) if strategy == "recycle" else None
+        self.draft_forwards = sum(ds.forwards for ds in strategies)
         return [e[:n_tokens] for e in emitted]
 
 

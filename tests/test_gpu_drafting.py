@@ -154,3 +154,42 @@ def test_recycled_draft_matches_the_oracle():
         assert want["merged_at"] is not None, name                          # the planted edit is found again
         assert want["draft"][:4] == greedy[3:7], name                       # and the recycled draft is the true continuation
     assert kv.length() == cache.length
+
+
+@pytest.mark.parametrize("strategy,same_model", [("two_pass", True), ("two_pass", False), ("recycle", True), ("recycle", False)])
+def test_whole_method_is_lossless(strategy, same_model):
+    """Draft with the strategies of Section IV, verify with the target, commit: the transcript is the target's own
+    greedy transcript (Section II-B), whatever the draft model proposes.  With the target's own weights as the draft
+    model whole trunks are accepted; with another model hardly anything is, and recycling has rejected tails to work on."""
+    from paper_2507_18181_b200.runtime import DeviceModel, DeviceKV
+    from paper_2507_18181_b200.loop import SpeculativeBatchLoop
+    cfg = gen.get_config("tiny")
+    store = gen.WeightStore(cfg, 0)
+    W = O.Weights(store, cache_layers=True)
+    target = DeviceModel(cfg, store)
+    draft = target if same_model else DeviceModel(cfg, gen.WeightStore(cfg, 5))
+    n_tokens, max_len = 16, 6
+    kvs, dkvs, roots, truth = [], [], [], []
+    for b, n_audio in enumerate((33, 58)):
+        prompt = gen.prompt_tokens(4, cfg.vocab, 0, utterance=b)
+        audio = gen.audio_prefix(n_audio, cfg.d_model, 0, utterance=b)
+        cache = O.KVCache(cfg)
+        O.prefill(cfg, W, cache, np.concatenate([audio.astype(np.float64), O.embed(W, prompt[:-1])], 0))
+        for model, lst in ((target, kvs), (draft, dkvs)):
+            kv = DeviceKV(model, max_tokens=256, max_nodes=64)
+            kv.prefill_embeds(torch.from_numpy(audio).cuda())
+            kv.prefill_tokens(torch.from_numpy(prompt[:-1].copy()).cuda())
+            lst.append(kv)
+        roots.append(int(prompt[-1]))
+        truth.append(O.greedy_continuation(cfg, W, cache, roots[-1], n_tokens + max_len + 2))
+    loop = SpeculativeBatchLoop(kvs, dkvs)
+    out = loop.decode_with_strategies(roots, n_tokens, strategy=strategy, threshold=2.0 if strategy == "two_pass" else 0.0,
+                                      max_len=max_len, n_nodes=20, max_branch=3, max_regen=3)
+    for b in range(2):
+        assert out[b] == truth[b][:n_tokens]
+        assert kvs[b].status() == 0 and dkvs[b].status() == 0 and kvs[b].length() == loop.target_len[b]
+    assert loop.draft_forwards > 0
+    if same_model:
+        assert loop.rounds <= -(-n_tokens // (max_len + 1)) + 1          # whole trunks accepted
+    else:
+        assert loop.rounds >= n_tokens // 2
