@@ -59,15 +59,17 @@ typedef struct specasr_model_config {
   int32_t d_model;
   int32_t n_heads;      /* query heads */
   int32_t n_kv_heads;   /* key/value heads; n_heads % n_kv_heads == 0 */
-  int32_t head_dim;     /* 32, 64 or 128 */
+  int32_t head_dim;     /* 64 or 128 (32 in the cross-check build variant only) */
   int32_t ffn;          /* SwiGLU inner width */
   int32_t vocab;
-  int32_t page_size;    /* tokens per KV page; a multiple of 8 (16 in the reference workload) */
+  int32_t page_size;    /* tokens per KV page; a multiple of 16, at most 208 (16 in the reference workload; any
+                           multiple of 8 in the cross-check build variant) */
   int32_t max_positions;/* length of the rotary table = largest position + 1 */
   float rms_eps;
   float rope_base;
-  int32_t gemm_path;    /* 0 = tcgen05 tensor-core projections (product path);
-                           1 = plain FMA projections, kept for cross-checking kernels on a GPU */
+  int32_t gemm_path;    /* must be 0: tcgen05 tensor-core projections.  (1 = plain FMA projections exists only in the
+                           cross-check build variant of the library, libspecasr_crosscheck.so, which the tests use
+                           to compare two engines on a GPU; the product library answers SPECASR_ERR_UNSUPPORTED.) */
   int32_t reserved[3];
 } specasr_model_config;
 
@@ -99,13 +101,22 @@ typedef struct specasr_weight_ptrs {
 typedef struct specasr_model specasr_model;
 typedef struct specasr_kv specasr_kv;
 
-/* Creates a model handle on the current CUDA device.  Fails with SPECASR_ERR_UNSUPPORTED for shapes
- * the kernels do not cover (head_dim not in {32,64,128}, d_model or ffn not a multiple of 8, ...). */
+/*
+ * Handles and bookkeeping (model / workspace / pool sizes / cache handle / length / truncate / status / launch count):
+ * no counterpart in the paper, which treats the target decoder as a black box; they exist because a C library needs
+ * somewhere to keep the borrowed weight pointers, the tensor maps and the committed length between calls.
+ *
+ * Creates a model handle on the current CUDA device.  Fails with SPECASR_ERR_UNSUPPORTED for shapes
+ * the kernels do not cover (head_dim not 64 or 128, d_model or ffn not a multiple of 8, page_size not a multiple
+ * of 16, ...).  Allocates the rotary table and a copy of the weight descriptors on the device, once.
+ */
 specasr_status specasr_model_create(const specasr_model_config* cfg, const specasr_weight_ptrs* w,
                                     specasr_model** out);
 void specasr_model_destroy(specasr_model* m);
 
-/* Bytes of [device] workspace a KV handle needs to verify trees of up to max_nodes nodes. */
+/* Bytes of [device] workspace a KV handle needs to verify trees of up to max_nodes nodes.  The library initialises
+ * the parts of it that must start in a known state (control words, flags of the projection kernels); the caller
+ * need not clear it.  (No counterpart in the paper.) */
 size_t specasr_workspace_bytes(const specasr_model* m, int32_t max_nodes);
 
 /* Bytes of ONE of the two KV pools (K and V have the same size) for n_pages pages.
@@ -124,9 +135,12 @@ specasr_status specasr_kv_create(const specasr_model* m, void* k_pool, void* v_p
                                  int32_t max_nodes, specasr_kv** out);
 void specasr_kv_destroy(specasr_kv* kv);
 
-/* Committed length in tokens, [host] out.  Synchronises `stream` if a commit is still in flight. */
+/* Committed length in tokens, [host] out.  If a commit is still in flight the host waits for the event recorded
+ * behind it (on the stream that commit was given); `stream` itself is not used.  (No counterpart in the paper.) */
 specasr_status specasr_kv_length(specasr_kv* kv, int32_t* out_len, void* stream);
-/* Rewinds (or empties) the cache to `len` <= current length.  Drops any pending verify. */
+/* Rewinds (or empties) the cache to `len` <= current length.  Drops any pending verify.  Like specasr_kv_length
+ * it first waits on the host for a commit in flight (it has to know the current length to check `len`), then
+ * enqueues the new length on `stream`.  (No counterpart in the paper.) */
 specasr_status specasr_kv_truncate(specasr_kv* kv, int32_t len, void* stream);
 
 /* Context fill (the prefill of Section II-A: audio-embedding vectors followed by prompt text), causal
@@ -223,10 +237,12 @@ specasr_status specasr_commit_kv(specasr_model* m, specasr_kv* kv, const int32_t
                                  const int32_t* accept_len, void* stream);
 
 /* Reads the device status word of the last verify/prefill on this handle ([host] out; synchronises
- * `stream`).  SPECASR_OK, SPECASR_ERR_INVALID_TREE, SPECASR_ERR_KV_CAPACITY or SPECASR_ERR_TIMEOUT. */
+ * `stream`).  SPECASR_OK, SPECASR_ERR_INVALID_TREE, SPECASR_ERR_KV_CAPACITY or SPECASR_ERR_TIMEOUT.
+ * (No counterpart in the paper: error reporting of this implementation.) */
 specasr_status specasr_poll_status(specasr_kv* kv, int32_t* out_device_status, void* stream);
 
-/* Number of kernels the library has launched on this handle so far (for launch accounting). */
+/* Number of kernels the library has launched on this handle so far (for launch accounting; no counterpart in the
+ * paper). */
 int64_t specasr_launch_count(const specasr_kv* kv);
 
 /*

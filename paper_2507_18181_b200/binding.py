@@ -7,10 +7,28 @@ anything; if the shared library is missing the import of any entry point fails l
 import ctypes as C
 import os
 
+import contextlib
+
 _HERE = os.path.dirname(os.path.abspath(__file__))
 # SPECASR_TRACE_LIB=1 selects the variant built with -DSPECASR_TRACE (specasr_trace_set records; ~2 % slower)
 TRACE_LIB = os.environ.get("SPECASR_TRACE_LIB") == "1"
 LIB_PATH = os.path.join(_HERE, "libspecasr_trace.so" if TRACE_LIB else "libspecasr.so")
+# The cross-check variant (-DSPECASR_CROSSCHECK) also carries the plain-FMA projections and attention.  It can be
+# loaded beside the product library: handles made by one library are only ever passed back to that library, which
+# `use("crosscheck")` arranges for the calls made inside it.
+VARIANT_PATHS = {"product": LIB_PATH, "crosscheck": os.path.join(_HERE, "libspecasr_crosscheck.so")}
+_current = ["product"]
+
+
+@contextlib.contextmanager
+def use(variant: str):
+    """Route the binding's calls to another build variant of the library for the duration of the block."""
+    _current.append(variant)
+    try:
+        yield
+    finally:
+        _current.pop()
+
 
 SPECASR_MAX_NODES = 256
 SPECASR_MAX_BATCH = 32
@@ -42,16 +60,17 @@ class WeightPtrs(C.Structure):
                 ("wd", C.POINTER(C.c_void_p)), ("g_attn", C.POINTER(C.c_void_p)), ("g_ffn", C.POINTER(C.c_void_p))]
 
 
-_lib = None
+_libs = {}
 
 
 def lib() -> C.CDLL:
-    global _lib
-    if _lib is None:
-        if not os.path.exists(LIB_PATH):
-            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2507_18181_b200.build` "
+    variant = _current[-1]
+    if variant not in _libs:
+        path = VARIANT_PATHS[variant]
+        if not os.path.exists(path):
+            raise RuntimeError(f"{path} is missing: build it with `python -m paper_2507_18181_b200.build` "
                                "(there is no fallback path)")
-        L = C.CDLL(LIB_PATH)
+        L = C.CDLL(path)
         vp, i32, st = C.c_void_p, C.c_int32, C.c_int
         L.specasr_model_create.argtypes = [C.POINTER(ModelConfig), C.POINTER(WeightPtrs), C.POINTER(vp)]
         L.specasr_model_create.restype = st
@@ -101,8 +120,8 @@ def lib() -> C.CDLL:
         L.specasr_top2_probs.restype = st
         L.specasr_last_error.argtypes = []
         L.specasr_last_error.restype = C.c_char_p
-        _lib = L
-    return _lib
+        _libs[variant] = L
+    return _libs[variant]
 
 
 class SpecasrError(RuntimeError):

@@ -5,9 +5,11 @@ import sys
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
-SOURCES = ["api.cu", "kernels_small.cu", "attention.cu", "attention_tc.cu", "gemm_fma.cu", "gemm_tcgen05.cu", "fused_stack.cu", "accept_static.cu", "top2.cu"]
+SOURCES = ["api.cu", "kernels_small.cu", "attention_tc.cu", "gemm_tcgen05.cu", "fused_stack.cu", "accept_static.cu", "top2.cu"]
+CROSSCHECK_SOURCES = ["gemm_fma.cu", "attention.cu"]     # the plain-FMA engine: cross-check variant only
 LIB = os.path.join(HERE, "libspecasr.so")
 LIB_TRACE = os.path.join(HERE, "libspecasr_trace.so")      # same sources with -DSPECASR_TRACE (device-side trace)
+LIB_CROSSCHECK = os.path.join(HERE, "libspecasr_crosscheck.so")   # + the plain-FMA engine (-DSPECASR_CROSSCHECK)
 
 
 def _stale(lib=None) -> bool:
@@ -20,9 +22,11 @@ def _stale(lib=None) -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False, trace: bool = False) -> str:
-    """Builds libspecasr.so, or with trace=True the variant that can record the device-side trace."""
-    lib = LIB_TRACE if trace else LIB
+def build(force: bool = False, verbose: bool = False, trace: bool = False, crosscheck: bool = False) -> str:
+    """Builds libspecasr.so, or with trace=True the variant that can record the device-side trace, or with
+    crosscheck=True the variant that also carries the plain-FMA projections and attention (a second engine used
+    by tests to cross-check the tensor-core kernels and to run shapes those do not cover)."""
+    lib = LIB_CROSSCHECK if crosscheck else (LIB_TRACE if trace else LIB)
     if not force and not _stale(lib):
         return lib
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
@@ -33,7 +37,9 @@ def build(force: bool = False, verbose: bool = False, trace: bool = False) -> st
         cmd += ["-Xptxas", "-v"]
     if trace:
         cmd += ["-DSPECASR_TRACE"]
-    cmd += [os.path.join(HERE, "csrc", s) for s in SOURCES]
+    if crosscheck:
+        cmd += ["-DSPECASR_CROSSCHECK"]
+    cmd += [os.path.join(HERE, "csrc", s) for s in SOURCES + (CROSSCHECK_SOURCES if crosscheck else [])]
     cmd += ["-o", lib, "-lcudart"]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if res.returncode != 0:

@@ -39,8 +39,14 @@ static inline int pad_tokens(int n) {
   return p;
 }
 
+// The plain-FMA projections and the plain attention kernel are a second engine kept for cross-checking kernels on a
+// GPU.  They are compiled only into the library variant built with -DSPECASR_CROSSCHECK; the product library has the
+// tensor-core path alone and refuses what that path does not cover.
 int lm_tiles_of(const specasr_model* m) {
-  return m->cfg.gemm_path == 1 ? gemm_fma_tiles(m->cfg.vocab) : gemm_tc_tiles(m->cfg.vocab);
+#ifdef SPECASR_CROSSCHECK
+  if (m->cfg.gemm_path == 1) return gemm_fma_tiles(m->cfg.vocab);
+#endif
+  return gemm_tc_tiles(m->cfg.vocab);
 }
 
 Workspace carve_workspace(const specasr_model* m, int n_alloc, void* base) {
@@ -99,6 +105,15 @@ static specasr_status model_create_impl(const specasr_model_config* cfg, const s
     set_error("specasr_model_create: unsupported shape (head_dim in {32,64,128}, d_model/ffn/page_size %% 8 == 0)");
     return SPECASR_ERR_UNSUPPORTED;
   }
+#ifndef SPECASR_CROSSCHECK
+  if (c.gemm_path != 0 || (c.head_dim != 64 && c.head_dim != 128) || c.page_size % 16 != 0 || c.page_size > 208 ||
+      c.n_heads / c.n_kv_heads > 128) {
+    set_error("specasr_model_create: this library has the tensor-core path only (gemm_path 0, head_dim 64 or 128, "
+              "page_size a multiple of 16 up to 208, at most 128 query heads per KV head); other shapes exist in the "
+              "cross-check build variant");
+    return SPECASR_ERR_UNSUPPORTED;
+  }
+#endif
   if (!w->embed || !w->lm_head || !w->g_final || !w->wqkv || !w->wo || !w->wgu || !w->wd || !w->g_attn || !w->g_ffn) {
     set_error("specasr_model_create: null weight pointer");
     return SPECASR_ERR_INVALID_ARG;
@@ -439,13 +454,15 @@ extern "C" specasr_status specasr_poll_status(specasr_kv* kv, int32_t* out_devic
 
 // ------------------------------------------------------------------------------------------------
 static void run_gemm(specasr_kv* kv, GemmArgs& a, int kind, cudaStream_t s) {
+#ifdef SPECASR_CROSSCHECK
   if (kv->m->cfg.gemm_path == 1) {
     a.splits = 1;
     launch_gemm_fma(kv, a, kind, s);
-  } else {
-    a.splits = gemm_tc_pick_splits(kv->m, a.M, a.K, a.n_pad);
-    launch_gemm_tc(kv, a, kind, s);
+    return;
   }
+#endif
+  a.splits = gemm_tc_pick_splits(kv->m, a.M, a.K, a.n_pad);
+  launch_gemm_tc(kv, a, kind, s);
 }
 
 // Key blocks of the attention over `n` nodes of one utterance; `sm_budget` is the number of SMs the launch
@@ -520,8 +537,11 @@ static void run_stack(specasr_model* m, specasr_kv* wk, const SegTable& tab, int
     a.M = m->qkv_dim; a.K = c.d_model; a.epilogue = EPI_PARTIAL;
     run_gemm(wk, a, SPECASR_KIND_GEMM_QKV, s);
     launch_rope_append(wk, tab, n, l, a.splits, s);
-    if (att_tc) launch_tree_attention_tc(wk, tab, n_max, l, s);
-    else launch_tree_attention(wk, l, n, tab.splits, s);      // single utterance only
+#ifdef SPECASR_CROSSCHECK
+    if (!att_tc) launch_tree_attention(wk, l, n, tab.splits, s);      // plain kernel, single utterance only
+    else
+#endif
+      launch_tree_attention_tc(wk, tab, n_max, l, s);
     launch_attn_merge(wk, ctl_shared, n, n_pad, tab.splits, s);
     a.W = m->wo[l]; a.tmW = tc ? &m->tm_wo[l] : nullptr; a.tmAct = wk->tm_AO; a.act = wk->ws.AO;
     a.M = c.d_model; a.K = m->q_dim; a.epilogue = EPI_PARTIAL;
@@ -576,9 +596,15 @@ static specasr_status prefill_common(specasr_model* m, specasr_kv* kv, const flo
   kv->pending_n = 0;
   for (int done = 0; done < n;) {
     const int chunk = n - done < kv->max_nodes ? n - done : kv->max_nodes;
-    launch_chain_prep(kv, chunk, s);
     bool att_tc = false;
     const SegTable tab = single_table(kv, chunk, &att_tc);
+#ifndef SPECASR_CROSSCHECK
+    if (!att_tc) {
+      set_error("%s: a cache of %d positions needs more key blocks than the workspace holds", who, kv->len_upper + chunk);
+      return SPECASR_ERR_UNSUPPORTED;
+    }
+#endif
+    launch_chain_prep(kv, chunk, s);
     if (embeds) launch_copy_embeds(kv, embeds + (size_t)done * m->cfg.d_model, chunk, s);
     else launch_embed_tokens(kv, tab, chunk, tokens + done, s);
     run_stack(m, kv, tab, chunk, chunk, att_tc, kv->ws.ctl, false, nullptr, false, s);
@@ -627,6 +653,13 @@ static specasr_status verify_tree_impl(specasr_model* m, specasr_kv* kv, const i
   cudaStream_t s = (cudaStream_t)stream;
   bool att_tc = false;
   const SegTable tab = single_table(kv, n_nodes, &att_tc);
+#ifndef SPECASR_CROSSCHECK
+  if (!att_tc) {
+    set_error("specasr_verify_tree: a cache of %d positions needs more key blocks than the workspace holds",
+              kv->len_upper + n_nodes);
+    return SPECASR_ERR_UNSUPPORTED;
+  }
+#endif
   const bool want_top2 = out_top2_ids != nullptr;
   if (want_top2 && !fused_stack_supported(kv, n_nodes, att_tc, tab.splits)) {
     set_error("specasr_verify_tree_top2: the top-2 epilogue needs the fused layer stack (tensor-core attention, at most "

@@ -45,10 +45,6 @@ struct TraceBuf {
 #define SPECASR_TRACE_MARK()
 #endif
 
-struct GemmMaps {           // TMA descriptors of one weight matrix (tcgen05 path)
-  CUtensorMap w;
-};
-
 struct specasr_model {
   specasr_model_config cfg;
   int device;
@@ -107,7 +103,7 @@ struct specasr_kv {
   int len_host;             // last length the host knows exactly
   bool len_exact;           // false while a commit's length has not been read back
   int len_upper;            // upper bound of the length
-  int32_t* pinned;          // [2] pinned host words: length, status
+  int32_t* pinned;          // [4] pinned host words: [0] length, [2] status (1 and 3 unused)
   cudaEvent_t len_event;
   bool len_event_pending;
   int64_t launches;

@@ -8,10 +8,29 @@ import torch
 from . import binding as B
 
 
+def _routed(cls):
+    """Every method of the class runs with the binding routed to the library variant the object was made with
+    (self.variant), so that handles never reach another build of the library."""
+    import functools
+    for name, fn in list(vars(cls).items()):
+        if isinstance(fn, staticmethod) or not callable(fn) or name == "__init__":
+            continue
+
+        def make(f):
+            @functools.wraps(f)
+            def wrapped(self, *a, **k):
+                with B.use(getattr(self, "variant", "product")):
+                    return f(self, *a, **k)
+            return wrapped
+        setattr(cls, name, make(fn))
+    return cls
+
+
 def _bf16_from_bits(bits: np.ndarray, device) -> torch.Tensor:
     return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(device).view(torch.bfloat16)
 
 
+@_routed
 class DeviceModel:
     """Weights of one decoder on the GPU in the layouts include/specasr.h asks for.
 
@@ -20,7 +39,19 @@ class DeviceModel:
     gains; layer -1 = embed / lm_head / g_final) and optionally map_tensors(fn, keys) for threaded draws.
     """
 
-    def __init__(self, cfg, store, page_size=16, max_positions=8192, gemm_path=0, device="cuda:0"):
+    def __init__(self, cfg, store, page_size=16, max_positions=8192, gemm_path=0, device="cuda:0", crosscheck=None):
+        """crosscheck=True loads the cross-check build variant of the library (plain-FMA projections with
+        gemm_path=1, head_dim 32, page sizes that are not a multiple of 16); by default it is chosen exactly when
+        the shape asks for something the product library does not have."""
+        if crosscheck is None:
+            crosscheck = gemm_path != 0 or cfg.head_dim not in (64, 128) or page_size % 16 != 0
+        self.variant = "crosscheck" if crosscheck else "product"
+        if crosscheck:
+            from . import build as _build
+            _build.build(crosscheck=True)
+        self._setup(cfg, store, page_size, max_positions, gemm_path, device)
+
+    def _setup(self, cfg, store, page_size, max_positions, gemm_path, device):
         self.cfg = cfg
         self.device = torch.device(device)
         torch.cuda.set_device(self.device)
@@ -86,11 +117,16 @@ class DeviceModel:
             pass
 
 
+@_routed
 class DeviceKV:
     """Paged KV cache + workspace for one utterance."""
 
     def __init__(self, model: DeviceModel, max_tokens: int, max_nodes: int = 256, shuffle_pages_seed=None,
                  poison: bool = False):
+        self.variant = model.variant
+        self._setup(model, max_tokens, max_nodes, shuffle_pages_seed, poison)
+
+    def _setup(self, model, max_tokens, max_nodes, shuffle_pages_seed, poison):
         """`poison` fills both pools and the workspace with 0xFF bytes (NaN as bf16 and fp32, -1 as int32)
         instead of zeros before the handle is created: a kernel that reads something no kernel wrote then
         produces NaN or an error instead of a silently plausible result."""
@@ -213,12 +249,14 @@ class DeviceKV:
             pass
 
 
+@_routed
 class BatchVerifier:
     """Output buffers for specasr_verify_tree_batch over a fixed list of utterances.  The first
     utterance's workspace carries the rows of all of them, so its max_nodes bounds the total."""
 
     def __init__(self, kvs):
         self.kvs = list(kvs)
+        self.variant = self.kvs[0].variant
         self.model = self.kvs[0].model
         dev = self.model.device
         total = self.kvs[0].max_nodes

@@ -170,8 +170,26 @@ def test_page_sizes_and_an_exactly_full_cache(page_size):
     assert e.value.status == B.SPECASR_ERR_KV_CAPACITY
 
 
+def test_product_library_has_one_engine():
+    """The plain-FMA projections and attention live in the cross-check build variant only: the product library
+    refuses the shapes and the switch that would need them."""
+    from paper_2507_18181_b200 import binding as B
+    from paper_2507_18181_b200.runtime import DeviceModel
+    cfg = gen.get_config("tiny")
+    store = gen.WeightStore(cfg, 0)
+    for kwargs in (dict(gemm_path=1), dict(page_size=8), dict(page_size=24)):
+        with pytest.raises(B.SpecasrError) as e:
+            DeviceModel(cfg, store, crosscheck=False, **kwargs)
+        assert e.value.status == B.SPECASR_ERR_UNSUPPORTED
+    with pytest.raises(B.SpecasrError) as e:
+        DeviceModel(gen.get_config("micro"), gen.WeightStore(gen.get_config("micro"), 0), crosscheck=False)   # head_dim 32
+    assert e.value.status == B.SPECASR_ERR_UNSUPPORTED
+    assert DeviceModel(cfg, store).variant == "product" and DeviceModel(cfg, store, gemm_path=1).variant == "crosscheck"
+
+
 def test_tensor_core_and_fma_projections_agree():
-    """Same operands, two engines: the only difference allowed is fp32 summation order."""
+    """Same operands, two engines (the second one from the cross-check build variant of the library): the only
+    difference allowed is fp32 summation order."""
     outs = []
     for path in (1, 0):
         cfg, store, model, kv = _gpu_stack("small", 3, path)
@@ -247,7 +265,7 @@ def test_node_order_does_not_matter_on_gpu():
 
 def test_error_paths_leave_state_untouched():
     from paper_2507_18181_b200 import binding as B
-    cfg, store, model, kv = _gpu_stack("micro", 0, 0, max_tokens=64, max_nodes=32)
+    cfg, store, model, kv = _gpu_stack("tiny", 0, 0, max_tokens=64, max_nodes=32)
     W, cache, prompt = _fill_both(cfg, store, kv, 20, 3, 0)
     L = kv.length()
     dev = "cuda"

@@ -13,6 +13,7 @@ import pytest
 import torch
 
 import gen
+from oracle import specasr_oracle as O
 from paper_2507_18181_b200 import binding as B
 
 pytestmark = pytest.mark.gpu
@@ -29,7 +30,7 @@ def _verify(cfg, kv, tokens, parent):
 
 def test_static_accept_matches_verify_on_two_calls_in_a_row():
     from paper_2507_18181_b200.runtime import DeviceModel, DeviceKV
-    cfg = gen.get_config("micro")
+    cfg = gen.get_config("tiny")
     model = DeviceModel(cfg, gen.WeightStore(cfg, 7))
     kv = DeviceKV(model, max_tokens=256, max_nodes=64)
     kv.prefill_embeds(torch.from_numpy(gen.audio_prefix(19, cfg.d_model, 7)).cuda())
@@ -61,6 +62,14 @@ def test_static_accept_matches_verify_on_two_calls_in_a_row():
     for tokens, parent, logits, want, outs in cases:
         for got, ref in zip(outs, want):
             assert torch.equal(got, ref)
+        # and against the oracle's accept rule applied to the arg-max of the very same logits (integer work: exact)
+        am = logits.cpu().numpy().argmax(-1)
+        ref = O.accept(tokens, parent, am)
+        n, a = len(tokens), ref["accept_len"]
+        assert np.array_equal(outs[0].cpu().numpy(), am)
+        assert int(outs[1].item()) == a and int(outs[3].item()) == ref["bonus"]
+        path = outs[2].cpu().numpy()
+        assert list(path[:a + 1]) == list(ref["path"]) and np.all(path[a + 1:] == -1)
     assert int(cases[0][3][1].item()) >= 0
     # a tree larger than the built-in array is refused on the host, with a message that names the limit
     with pytest.raises(B.SpecasrError) as e:
