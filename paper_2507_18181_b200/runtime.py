@@ -13,7 +13,7 @@ def _routed(cls):
     (self.variant), so that handles never reach another build of the library."""
     import functools
     for name, fn in list(vars(cls).items()):
-        if isinstance(fn, staticmethod) or not callable(fn) or name == "__init__":
+        if isinstance(fn, staticmethod) or not callable(fn) or name in ("__init__", "__del__"):
             continue
 
         def make(f):
