@@ -1156,40 +1156,26 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
         STACK_TRACE_POINT(2, cur_layer);
         if (ok) ok = rounds == 2 ? wwait(&sc->bar_o[1], par2) : wwait(&sc->bar_o[0], par);
         STACK_TRACE_POINT(3, cur_layer);
-        // O leaves through the (now idle) K/V region so that a warp writes whole rows
-        float4* stage = reinterpret_cast<float4*>(KVs);
-        constexpr int C4 = DH / 4;
-        if (ok) {
+        // Every thread holds 32 consecutive floats of its row per TMEM load and stores them straight to the partial
+        // output: 128 contiguous bytes per thread, whole sectors.  (Staging the tile in shared memory so that a warp
+        // writes whole rows cost two more barriers and a pass of index arithmetic, 3 us against 1.)
+        if (ok) {                                               // warp-uniform: the TMEM load is a warp-wide instruction
           tc_fence_after();
+          float4* dst = reinterpret_cast<float4*>(p.attO + out_row * DH);
 #pragma unroll 1
           for (int c0 = eg * 32; c0 < DH; c0 += 64) {
             float o[32];
             tmem_ld32(tmem_o + lane_off + c0, o);
+            if (row_valid) {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              const int c4 = (c0 >> 2) + e;
-              stage[row * C4 + (c4 ^ (row & (C4 - 1)))] = make_float4(o[4 * e], o[4 * e + 1], o[4 * e + 2], o[4 * e + 3]);
+              for (int e = 0; e < 8; ++e) dst[(c0 >> 2) + e] = make_float4(o[4 * e], o[4 * e + 1], o[4 * e + 2], o[4 * e + 3]);
             }
           }
         }
         tc_fence_before();
         STACK_TRACE_POINT(9, cur_layer);
-        worker_bar();
-        if (ok) {
-          const int r_base = wwarp * 16;                       // eight warps, sixteen rows each
-#pragma unroll 1
-          for (int i = 0; i < 16; ++i) {
-            const int rr = r_base + i;
-            const int nd = node0 + rr / p.group;
-            if (rr < rows_used && nd < sg.n) {
-              const size_t orow = (size_t)split * rows_alloc + (size_t)(sg.row0 + nd) * p.Hq + kvh * p.group + rr % p.group;
-              float4* dst = reinterpret_cast<float4*>(p.attO + orow * DH);
-#pragma unroll 1
-              for (int c4 = lane; c4 < C4; c4 += 32) dst[c4] = stage[rr * C4 + (c4 ^ (rr & (C4 - 1)))];
-            }
-          }
-          if (row_valid && eg == 0) p.attML[out_row] = make_float2(m_row, sc->red_sum[0][row] + sc->red_sum[1][row]);
-        }
+        worker_bar();                                           // both halves of every row's sum are in shared memory
+        if (ok && row_valid && eg == 0) p.attML[out_row] = make_float2(m_row, sc->red_sum[0][row] + sc->red_sum[1][row]);
         STACK_TRACE_POINT(13, cur_layer);
         worker_bar();                                           // the staging area and red_* are free again
         if (wtid == 0) {
