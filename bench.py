@@ -32,6 +32,8 @@ WORKLOADS = {
     "config1": dict(model="tiny", n_audio=64, n_text=8, n_nodes=15, levels=None, chain=False),
     # config3 cut to two layers: same kernels and launch shapes, small enough for a profiler capture
     "config3_2layers": dict(model="7b", n_layers=2, n_audio=1500, n_text=201, n_nodes=64, levels=12, chain=False),
+    "config4_kv2048": dict(model="7b", n_audio=1848, n_text=201, n_nodes=64, levels=12, chain=False),
+    "config4_n16": dict(model="7b", n_audio=1500, n_text=201, n_nodes=16, levels=None, chain=False),
     "config3_4layers": dict(model="7b", n_layers=4, n_audio=1500, n_text=201, n_nodes=64, levels=12, chain=False),
     # the 13B-class shape as a second target (same tree and context as config 3)
     "config3_13b": dict(model="13b", n_audio=1500, n_text=201, n_nodes=64, levels=12, chain=False),
@@ -73,13 +75,13 @@ def algorithmic_flops(cfg, L, n):
 
 
 # DRAM traffic (read + write) of one launch of the fused layer-stack kernel from the ncu captures summarised in
-# profiles/k_stack_config3_cuts.md: the 2-layer and the 4-layer cut of config 3 (7B shape, 64 tokens, KV 1700).  Traffic
+# profiles/k_stack_config3.md: the 2-layer and the 4-layer cut of config 3 (7B shape, 64 tokens, KV 1700).  Traffic
 # grows by a fixed amount per layer, so a full launch is the 2-layer figure plus (layers - 2) times the per-layer
 # difference.  Valid only for the kernel source it was taken on.
-STACK_TRAFFIC_MB = {"cut2": None, "cut4": None}
+STACK_TRAFFIC_MB = {"cut2": 1251.6, "cut4": 2225.4}
 STACK_TRAFFIC_SOURCE_SHA256 = {
-    "fused_stack.cu": "",
-    "sm100_ptx.cuh": "",
+    "fused_stack.cu": "8ee6378f62bba9f0ef6df8c992fcf7c1de8be589139b25a49e08df21e3fa7026",
+    "sm100_ptx.cuh": "3a0c294121fb64b742ab3700569cef82a1922484c98acd5238167235b990940f",
 }
 
 

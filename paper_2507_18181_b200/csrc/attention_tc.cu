@@ -420,6 +420,14 @@ bool attention_tc_plan(const specasr_model* m, int n, int total_len, int sm_budg
   const int fill = sm_budget / ctas;                      // blocks that still fit in one wave
   if (fill > splits) splits = fill;
   if (splits > max_splits) splits = max_splits;
+  // A cache that needs more key blocks than one wave holds: instead of a full second wave of 208-key blocks (of which
+  // only a fraction is needed), cut it into as many blocks as whole waves can take, so that every round is shorter.
+  if (splits * ctas > sm_budget && ctas <= sm_budget) {
+    const int waves = (splits * ctas + sm_budget - 1) / sm_budget;
+    int s2 = waves * sm_budget / ctas;
+    if (s2 > max_splits) s2 = max_splits;
+    if (s2 > splits) splits = s2;
+  }
   int per = (total_len + splits - 1) / splits;
   per = (per + c.page_size - 1) / c.page_size * c.page_size;
   if (per < c.page_size) per = c.page_size;
