@@ -604,7 +604,7 @@ static specasr_status prefill_common(specasr_model* m, specasr_kv* kv, const flo
       return SPECASR_ERR_UNSUPPORTED;
     }
 #endif
-    launch_chain_prep(kv, chunk, s);
+    launch_chain_prep(kv, chunk, done == 0, s);
     if (embeds) launch_copy_embeds(kv, embeds + (size_t)done * m->cfg.d_model, chunk, s);
     else launch_embed_tokens(kv, tab, chunk, tokens + done, s);
     run_stack(m, kv, tab, chunk, chunk, att_tc, kv->ws.ctl, false, nullptr, false, s);
@@ -613,6 +613,11 @@ static specasr_status prefill_common(specasr_model* m, specasr_kv* kv, const flo
     kv->len_upper = kv->len_host;
     done += chunk;
   }
+  // The device may have refused a chunk (a token id outside the vocabulary): the host learns the length the same
+  // lazy way as after a commit, so that specasr_kv_length reports what the device holds.
+  CUDA_TRY(cudaMemcpyAsync(kv->pinned, kv->ws.ctl + CTL_LEN, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+  CUDA_TRY(cudaEventRecord(kv->len_event, s));
+  kv->len_event_pending = true;           // len_host stays the optimistic value (an upper bound) until the copy lands
   CUDA_TRY(cudaGetLastError());
   return SPECASR_OK;
 }

@@ -218,7 +218,7 @@ int lm_tiles_of(const specasr_model* m);
 
 // ---- kernels_small.cu
 void launch_tree_prep(specasr_kv* wk, const SegTable& t, const int32_t* tokens, const int32_t* parent, cudaStream_t s);
-void launch_chain_prep(specasr_kv* kv, int n, cudaStream_t s);
+void launch_chain_prep(specasr_kv* kv, int n, bool first, cudaStream_t s);
 void launch_embed_tokens(specasr_kv* wk, const SegTable& t, int n_total, const int32_t* tokens, cudaStream_t s);
 void launch_copy_embeds(specasr_kv* kv, const float* embeds, int n, cudaStream_t s);
 void launch_rmsnorm_split(specasr_kv* wk, const int32_t* ctl, const float* gain, int n, int n_pad, int n_partials,

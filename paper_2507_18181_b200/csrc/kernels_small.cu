@@ -66,11 +66,14 @@ __global__ void k_tree_prep(const __grid_constant__ SegTable tab, const int32_t*
 }
 
 // Context fill: a chunk of n consecutive positions is a chain, i.e. plain causal attention.
-__global__ void k_chain_prep(int32_t* __restrict__ ctl, int n, int capacity, int32_t* __restrict__ depth,
+// Only the first chunk of a context-fill call starts from a clean status: a chunk that was refused (capacity, a
+// token id outside the vocabulary) keeps every later chunk of the same call from running on top of the gap.
+__global__ void k_chain_prep(int32_t* __restrict__ ctl, int n, int capacity, int first, int32_t* __restrict__ depth,
                              int32_t* __restrict__ pos, unsigned long long* __restrict__ anc) {
   const int i = threadIdx.x;
   grid_dep_launch();
   grid_dep_wait();
+  if (!first && ctl[CTL_STATUS] != 0) return;
   const int L = ctl[CTL_LEN];
   if (L < 0 || L + n > capacity) {
     if (i == 0) ctl[CTL_STATUS] = SPECASR_ERR_KV_CAPACITY;
@@ -100,12 +103,12 @@ void launch_tree_prep(specasr_kv* wk, const SegTable& t, const int32_t* tokens, 
              wk->ws.pos, wk->ws.anc SPECASR_TRACE_ARG(wk));
 }
 
-void launch_chain_prep(specasr_kv* kv, int n, cudaStream_t s) {
+void launch_chain_prep(specasr_kv* kv, int n, bool first, cudaStream_t s) {
   const specasr_model* m = kv->m;
   int cap = kv->max_pages * m->cfg.page_size;
   if (m->cfg.max_positions < cap) cap = m->cfg.max_positions;
   LaunchScope scope(kv, SPECASR_KIND_PREP, s);
-  launch_pdl(k_chain_prep, dim3(1), dim3(256), 0, s, kv->ws.ctl, n, cap, kv->ws.depth, kv->ws.pos, kv->ws.anc);
+  launch_pdl(k_chain_prep, dim3(1), dim3(256), 0, s, kv->ws.ctl, n, cap, first ? 1 : 0, kv->ws.depth, kv->ws.pos, kv->ws.anc);
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -315,6 +315,26 @@ def test_error_paths_leave_state_untouched():
     assert kv.length() == L
 
 
+def test_context_fill_refuses_a_token_id_outside_the_vocabulary():
+    """A prompt id >= vocab (or negative) is never turned into an address: the chunk's status word is set, the rest
+    of the call does nothing, the length does not advance, and the handle works again afterwards."""
+    from paper_2507_18181_b200 import binding as B
+    cfg, store, model, kv = _gpu_stack("tiny", 0, 0, max_tokens=128, max_nodes=32)
+    W, cache, prompt = _fill_both(cfg, store, kv, 20, 3, 0)
+    L = kv.length()
+    for bad in (cfg.vocab, -1, 2 ** 30):
+        toks = torch.tensor([5, 6, bad, 7], dtype=torch.int32, device="cuda")
+        kv.prefill_tokens(toks)
+        torch.cuda.synchronize()
+        assert kv.status() == B.SPECASR_ERR_INVALID_TREE
+        assert kv.length() == L                          # nothing of the call was appended, not even the good ids before the bad one's chunk ended
+        kv.truncate(L)                                   # clears the status
+    parent = gen.chain_tree(5)
+    tokens = gen.fill_tree_tokens(parent, cfg.vocab, seed=2, root_token=int(prompt[-1]))
+    got = _verify_gpu(cfg, kv, tokens, parent)
+    _check_against_oracle(got, O.verify_tree(cfg, W, cache, tokens, parent), tokens, parent)
+
+
 def test_single_node_tree_and_max_nodes():
     cfg, store, model, kv = _gpu_stack("micro", 1, 0, max_tokens=600, max_nodes=256)
     W, cache, prompt = _fill_both(cfg, store, kv, 10, 2, 1)
