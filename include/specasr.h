@@ -74,8 +74,14 @@ typedef struct specasr_model_config {
 } specasr_model_config;
 
 /*
- * Weights, all [device], all borrowed.  Matrices are bf16, row-major [out_features, in_features]
- * with rows 16-byte aligned (in_features % 8 == 0).  Gains are fp32.
+ * Weights, all [device], all borrowed, 16-byte aligned.  Gains are fp32.  The embedding table is bf16, row-major
+ * [vocab, d_model] (d_model % 8 == 0).  Every projection matrix W[out_features = M, in_features = K] below (and
+ * lm_head) is bf16 and TILE-PACKED: M and K are padded with zeros to multiples of 128, the padded matrix is cut
+ * into tiles of 128 rows x 64 columns, every tile is stored contiguously (row-major inside, 16 KB), and the tiles
+ * are ordered by row tile, then by column tile.  Element (m, k) therefore sits at element offset
+ *   (((m / 128) * Kt + k / 64) * 128 + m % 128) * 64 + k % 64,   Kt = 2 * ceil(K / 128),
+ * and the buffer holds ceil(M / 128) * Kt * 8192 elements.  One pipeline stage of a projection (128 rows x 128
+ * columns) is then one contiguous 32 KB run of HBM.  The logical row orders of the matrices are:
  *   wqkv[l] : [(n_heads + 2 n_kv_heads) * head_dim, d_model]  rows = all Q heads, all K heads, all V heads;
  *             within every head the rows are in rotary-paired order: stored row 32 g + 16 h + j holds
  *             feature 16 g + j + h * head_dim / 2 (0 <= j < 16, h in {0, 1}), so that a feature and its
@@ -88,7 +94,7 @@ typedef struct specasr_model_config {
  */
 typedef struct specasr_weight_ptrs {
   const void* embed;            /* [vocab, d_model] bf16 */
-  const void* lm_head;          /* [vocab, d_model] bf16 */
+  const void* lm_head;          /* [vocab, d_model] bf16, tile-packed like the projections */
   const float* g_final;         /* [d_model] */
   const void* const* wqkv;
   const void* const* wo;

@@ -8,6 +8,7 @@
 #include <new>
 
 #include "internal.h"
+#include "device_utils.cuh"
 
 // ------------------------------------------------------------------------------------------------
 static thread_local char g_err[512] = "";
@@ -185,13 +186,18 @@ static specasr_status model_create_impl(const specasr_model_config* cfg, const s
     m->tm_wo.resize(c.n_layers);
     m->tm_wgu.resize(c.n_layers);
     m->tm_wd.resize(c.n_layers);
+    // tile-packed weights: a [M, K] matrix is a stack of 128 x 64 tiles, 128 bytes per row, one box per tile
+    auto weight_map = [](CUtensorMap* map, const bf16* w, int K, uint64_t M) {
+      const uint64_t rows = ((M + 127) / 128) * (uint64_t)packed_col_tiles(K) * 128;
+      return make_tensor_map_2d(map, w, 64, rows, 64, 128);
+    };
     for (int l = 0; l < c.n_layers && ok; ++l) {
-      ok = ok && make_tensor_map_2d(&m->tm_wqkv[l], m->wqkv[l], c.d_model, m->qkv_dim, 64, 128);
-      ok = ok && make_tensor_map_2d(&m->tm_wo[l], m->wo[l], m->q_dim, c.d_model, 64, 128);
-      ok = ok && make_tensor_map_2d(&m->tm_wgu[l], m->wgu[l], c.d_model, 2 * (uint64_t)c.ffn, 64, 128);
-      ok = ok && make_tensor_map_2d(&m->tm_wd[l], m->wd[l], c.ffn, c.d_model, 64, 128);
+      ok = ok && weight_map(&m->tm_wqkv[l], m->wqkv[l], c.d_model, m->qkv_dim);
+      ok = ok && weight_map(&m->tm_wo[l], m->wo[l], m->q_dim, c.d_model);
+      ok = ok && weight_map(&m->tm_wgu[l], m->wgu[l], c.d_model, 2 * (uint64_t)c.ffn);
+      ok = ok && weight_map(&m->tm_wd[l], m->wd[l], c.ffn, c.d_model);
     }
-    ok = ok && make_tensor_map_2d(&m->tm_lm, m->lm_head, c.d_model, c.vocab, 64, 128);
+    ok = ok && weight_map(&m->tm_lm, m->lm_head, c.d_model, c.vocab);
     if (!ok) {
       cudaFree(m->rope_table);
       delete m;

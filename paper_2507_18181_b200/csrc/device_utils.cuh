@@ -50,6 +50,14 @@ __device__ __forceinline__ size_t kv_plane_offset(int layer, int n_pages, int Hk
   return ((((size_t)layer * n_pages + page) * Hkv + kvh) * 2 + plane) * (size_t)page_size * dh;
 }
 
+// Weight matrices [M, K] are stored tile-packed: 128-row x 64-column tiles, each 16 KB contiguous (row-major inside),
+// ordered [row tile][column tile]; K is padded to a multiple of 128 columns and M to a multiple of 128 rows with
+// zeros.  A pipeline stage of the projections (128 rows x 128 columns) is then one contiguous 32 KB run in HBM.
+__host__ __device__ __forceinline__ int packed_col_tiles(int K) { return 2 * ((K + 127) / 128); }
+__host__ __device__ __forceinline__ size_t packed_weight_offset(int m, int k, int K) {
+  return ((((size_t)(m >> 7) * packed_col_tiles(K) + (k >> 6)) * 128 + (m & 127)) << 6) + (k & 63);
+}
+
 // Order-preserving map of a float to an unsigned key, packed with the complement of an index so that
 // a plain unsigned max picks the largest value and, among equals, the lowest index.
 __device__ __forceinline__ unsigned long long pack_max_key(float v, uint32_t idx) {

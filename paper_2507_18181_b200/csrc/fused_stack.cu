@@ -388,8 +388,8 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
       }
       uint8_t* st = ring + (size_t)slot * p.stage_bytes;
       mbar_expect_tx(&sc->full[slot], (uint32_t)W_STAGE_BYTES);
-      for (int q = 0; q < KSUB; ++q)                     // rows past M and columns past K read as zeros
-        tma_load_2d(st + q * W_SUB_BYTES, ld.tmW, (ld.kb * KSUB + q) * SUB_K, ld.tile * TILE_M, &sc->full[slot]);
+      for (int q = 0; q < KSUB; ++q)                     // tile-packed weights: 16 KB contiguous per box, padding is zeros
+        tma_load_2d(st + q * W_SUB_BYTES, ld.tmW, 0, (ld.tile * 2 * ld.KB + ld.kb * KSUB + q) * TILE_M, &sc->full[slot]);
       advance(ld);
       if (++slot == p.stages) {
         slot = 0;

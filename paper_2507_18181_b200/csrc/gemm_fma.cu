@@ -31,7 +31,7 @@ __global__ void __launch_bounds__(256) k_gemm_fma(GemmArgs a) {
   for (int k0 = 0; k0 < a.K; k0 += BK) {
     float w[4] = {0.f, 0.f, 0.f, 0.f}, x[4] = {0.f, 0.f, 0.f, 0.f};
     if (m0 + lr < a.M && k0 + lk < a.K) {
-      const uint2 v = *reinterpret_cast<const uint2*>(a.W + (size_t)(m0 + lr) * a.K + k0 + lk);
+      const uint2 v = *reinterpret_cast<const uint2*>(a.W + packed_weight_offset(m0 + lr, k0 + lk, a.K));
       w[0] = bf16lo_to_f32(v.x); w[1] = bf16hi_to_f32(v.x);
       w[2] = bf16lo_to_f32(v.y); w[3] = bf16hi_to_f32(v.y);
     }

@@ -63,6 +63,7 @@ struct alignas(16) SharedCtl {
 
 struct TcParams {
   int M, K, n, n_pad, n_alloc, box_rows, stages, ksub, tm, n_buf, tmem_cols, KB, tiles, groups, splits, epoch;
+  int kt64;                 // 64-column tiles per row tile of the packed weight matrix
   int fold;                 // launch the FOLD instantiation: hi and lo products share the TMEM columns
   int32_t* ctl;
   float* fixP;              // [grid][tm][n_pad][128] parked partial sums (hi + lo halves added) of split tile groups
@@ -149,8 +150,8 @@ __global__ void __launch_bounds__(64 + EPI_THREADS, 1) k_proj(const __grid_const
       uint8_t* st = tiles + (size_t)s * stage_bytes;
       for (int t = 0; t < p.tm; ++t)       // rows past M read as zeros
         for (int q = 0; q < p.ksub; ++q)
-          tma_load_2d(st + (t * p.ksub + q) * W_SUB_BYTES, &tmW, (kb * p.ksub + q) * SUB_K,
-                      (group * p.tm + t) * TILE_M, &sc->full[s]);
+          tma_load_2d(st + (t * p.ksub + q) * W_SUB_BYTES, &tmW, 0,
+                      ((group * p.tm + t) * p.kt64 + kb * p.ksub + q) * TILE_M, &sc->full[s]);   // tile-packed weights
     };
     auto load_act = [&](int i) {
       const int kb = (int)((u0 + i) % KB), s = i % p.stages;
@@ -622,6 +623,7 @@ void launch_gemm_tc(specasr_kv* kv, const GemmArgs& a, int kind, cudaStream_t s)
   while (cols < p.n_buf * acc_cols) cols <<= 1;
   p.tmem_cols = cols;
   p.KB = (a.K + p.ksub * SUB_K - 1) / (p.ksub * SUB_K);
+  p.kt64 = packed_col_tiles(a.K);
   p.tiles = gemm_tc_tiles(a.M);
   p.groups = (p.tiles + p.tm - 1) / p.tm;
   p.splits = a.epilogue == EPI_PARTIAL ? a.splits : 0;

@@ -8,6 +8,16 @@ import torch
 from . import binding as B
 
 
+def pack_weight(w: "torch.Tensor") -> "torch.Tensor":
+    """[M, K] row-major bf16 -> the tile-packed layout include/specasr.h asks for: 128 x 64 tiles, each contiguous,
+    ordered [row tile][column tile], M and K padded with zeros to multiples of 128 (data movement only)."""
+    M, K = w.shape
+    Mp, Kp = -(-M // 128) * 128, -(-K // 128) * 128
+    if (Mp, Kp) != (M, K):
+        w = torch.nn.functional.pad(w, (0, Kp - K, 0, Mp - M))
+    return w.view(Mp // 128, 128, Kp // 64, 64).permute(0, 2, 1, 3).contiguous().view(-1)
+
+
 def _routed(cls):
     """Every method of the class runs with the binding routed to the library variant the object was made with
     (self.variant), so that handles never reach another build of the library."""
@@ -73,10 +83,12 @@ class DeviceModel:
                 got[(layer, name)] = torch.from_numpy(np.ascontiguousarray(arr, dtype=np.float32)).to(self.device)
             if layer >= 0 and all((layer, k) in got for k in ("wq", "wk", "wv")):
                 fused = torch.cat([got.pop((layer, k)) for k in ("wq", "wk", "wv")], dim=0)
-                got[(layer, "wqkv")] = fused[self._qkv_rows].contiguous()
+                got[(layer, "wqkv")] = pack_weight(fused[self._qkv_rows])
             if layer >= 0 and all((layer, k) in got for k in ("wg", "wu")):
                 g, u = got.pop((layer, "wg")), got.pop((layer, "wu"))
-                got[(layer, "wgu")] = torch.stack([g, u], dim=1).reshape(2 * cfg.ffn, cfg.d_model).contiguous()
+                got[(layer, "wgu")] = pack_weight(torch.stack([g, u], dim=1).reshape(2 * cfg.ffn, cfg.d_model))
+            if name in ("wo", "wd", "lm_head"):
+                got[(layer, name)] = pack_weight(got[(layer, name)])
 
         keys = [(-1, n) for n in ("embed", "lm_head", "g_final")]
         for l in range(L):
