@@ -42,9 +42,21 @@ namespace {
 constexpr int TILE_M = 128;
 constexpr int SUB_K = 64;               // bf16 elements = 128 bytes = one swizzle row
 constexpr int UMMA_K = 16;
-constexpr int KSUB = 2;                 // 64-wide k sub-blocks per ring stage (256 contiguous bytes per weight row)
+#ifndef STACK_TM
+#define STACK_TM 1
+#endif
+#ifndef STACK_KSUB
+#define STACK_KSUB 2
+#endif
+// A ring stage holds TM weight tiles (128 rows each) of KSUB 64-wide k sub-blocks and ONE activation block that all
+// of them multiply.  One tile of two sub-blocks (32 KB of weights, contiguous in the tile-packed layout) is what is
+// built.  A tile pair of one sub-block (TM 2, KSUB 1) halves the activation bytes that cross from L2 into shared
+// memory per weight byte, but doubles the k-parts and parked partial sums; it measured 7 % slower at 64 tokens and
+// at 16, and leaving the activation loads out altogether shortens the call by 5 % only: they are not what bounds it.
+constexpr int TM = STACK_TM;
+constexpr int KSUB = STACK_KSUB;
 constexpr int W_SUB_BYTES = TILE_M * SUB_K * 2;
-constexpr int W_STAGE_BYTES = KSUB * W_SUB_BYTES;
+constexpr int W_STAGE_BYTES = TM * KSUB * W_SUB_BYTES;
 constexpr int MAX_STAGES = 6;
 constexpr int SMEM_LIMIT = 227 * 1024;
 constexpr int WORKERS = 256;            // warps 2..9
@@ -131,9 +143,9 @@ __device__ __forceinline__ void worker_bar() { asm volatile("bar.sync 1, 256;" :
 // One projection as this CTA sees it.
 struct Gemm {
   const CUtensorMap* tmW;
-  int M, K, KB, tiles, splits;          // splits > 0: linear output in `splits` k-parts per tile
+  int M, K, KB, Kt, tiles, groups, splits;   // tiles of 128 rows in groups of TM; splits > 0: linear output in `splits` k-parts per group
   int g_eff;                            // CTAs that take part
-  int U, u0, u1;                        // all (tile, k-block) units; this CTA's range
+  int U, u0, u1;                        // all (tile group, k-block) units; this CTA's range
 };
 
 __device__ __forceinline__ Gemm gemm_of(const StackParams& p, int layer, int which, int cta, int G) {
@@ -146,10 +158,12 @@ __device__ __forceinline__ Gemm gemm_of(const StackParams& p, int layer, int whi
     default: g.M = p.vocab; g.K = p.d; g.splits = 0; g.tmW = p.w_maps + 4 * p.n_layers; break;      // vocabulary
   }
   g.KB = (g.K + KSUB * SUB_K - 1) / (KSUB * SUB_K);
+  g.Kt = packed_col_tiles(g.K);
   g.tiles = (g.M + TILE_M - 1) / TILE_M;
-  g.U = g.tiles * g.KB;
+  g.groups = (g.tiles + TM - 1) / TM;
+  g.U = g.groups * g.KB;
   if (g.splits > 0) {
-    g.g_eff = g.tiles * g.splits;
+    g.g_eff = g.groups * g.splits;
     if (cta < g.g_eff) {
       const int tile = cta / g.splits, split = cta % g.splits;
       g.u0 = tile * g.KB + split * g.KB / g.splits;
@@ -332,7 +346,8 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
     // continuously, or only while the attention step holds the ring -- measured slower at every depth tried.)
     struct Cursor {
       int l, ph;                 // layer; 0..3 = QKV, O, gate/up, down; layer == n_layers: the vocabulary projection
-      int u, u1, tile, kb, KB;   // next unit, end of the range, and the unit as (weight tile, k-block)
+      int u, u1, tile, kb, KB;   // next unit, end of the range, and the unit as (weight tile group, k-block)
+      int Kt, tiles;             // 64-wide column tiles per row tile of the packed matrix; its row tiles
       const CUtensorMap* tmW;
       bool done;
     };
@@ -354,7 +369,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
           c.done = true;
           break;
         }
-        c.u = g.u0; c.u1 = g.u1; c.KB = g.KB; c.tmW = g.tmW;
+        c.u = g.u0; c.u1 = g.u1; c.KB = g.KB; c.tmW = g.tmW; c.Kt = g.Kt; c.tiles = g.tiles;
         c.tile = g.u0 / g.KB;
         c.kb = g.u0 % g.KB;
       }
@@ -368,7 +383,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
       if (c.u >= c.u1) settle(c);
     };
     Cursor ld;
-    ld.l = 0; ld.ph = -1; ld.u = ld.u1 = 0; ld.tile = ld.kb = 0; ld.KB = 1; ld.tmW = nullptr; ld.done = false;
+    ld.l = 0; ld.ph = -1; ld.u = ld.u1 = 0; ld.tile = ld.kb = 0; ld.KB = 1; ld.Kt = 2; ld.tiles = 1; ld.tmW = nullptr; ld.done = false;
     settle(ld);
     int slot = 0;                                        // next ring slot
     uint32_t ring_par = 0u;                              // parity of the ring round in progress
@@ -388,8 +403,13 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
       }
       uint8_t* st = ring + (size_t)slot * p.stage_bytes;
       mbar_expect_tx(&sc->full[slot], (uint32_t)W_STAGE_BYTES);
-      for (int q = 0; q < KSUB; ++q)                     // tile-packed weights: 16 KB contiguous per box, padding is zeros
-        tma_load_2d(st + q * W_SUB_BYTES, ld.tmW, 0, (ld.tile * 2 * ld.KB + ld.kb * KSUB + q) * TILE_M, &sc->full[slot]);
+      for (int t = 0; t < TM; ++t) {                     // tile-packed weights: 16 KB contiguous per box, padding is zeros
+        // a group past the last row tile reads that tile again (its accumulator is never looked at)
+        const int tile = min(ld.tile * TM + t, ld.tiles - 1);
+        for (int q = 0; q < KSUB; ++q)
+          tma_load_2d(st + (t * KSUB + q) * W_SUB_BYTES, ld.tmW, 0, (tile * ld.Kt + ld.kb * KSUB + q) * TILE_M,
+                      &sc->full[slot]);
+      }
       advance(ld);
       if (++slot == p.stages) {
         slot = 0;
@@ -510,7 +530,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
           break;
         }
         tc_fence_after();
-        const uint32_t d_addr = tmem_base + (uint32_t)(b * acc_cols);
+        const uint32_t d_addr = tmem_base + (uint32_t)(b * TM * acc_cols);
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % p.stages;
           if (!bar_wait(&sc->full[s], (uint32_t)((it / p.stages) & 1), abort, status)) {
@@ -518,15 +538,18 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
             break;
           }
           tc_fence_after();
-          const uint32_t w_addr = smem_u32(ring + (size_t)s * p.stage_bytes);
-          const uint32_t act_addr = w_addr + W_STAGE_BYTES;
+          const uint32_t w_lo = smem_desc_lo(smem_u32(ring + (size_t)s * p.stage_bytes));
+          const uint32_t act_lo = w_lo + (W_STAGE_BYTES >> 4);
 #pragma unroll
-          for (int q = 0; q < KSUB; ++q) {
+          for (int t = 0; t < TM; ++t) {
 #pragma unroll
-            for (int k = 0; k < SUB_K / UMMA_K; ++k) {
-              const uint32_t acc = (kb > kb0 || q > 0 || k > 0) ? 1u : 0u;
-              umma_bf16(d_addr, make_smem_desc(w_addr + q * W_SUB_BYTES + k * UMMA_K * 2),
-                        make_smem_desc(act_addr + q * act_sub + k * UMMA_K * 2), idesc, acc);
+            for (int q = 0; q < KSUB; ++q) {
+#pragma unroll
+              for (int k = 0; k < SUB_K / UMMA_K; ++k) {
+                const uint32_t acc = (q > 0 || k > 0) ? 1u : (kb > kb0 ? 1u : 0u);
+                umma_bf16_lo(d_addr + (uint32_t)(t * acc_cols), w_lo + (((t * KSUB + q) * W_SUB_BYTES + k * UMMA_K * 2) >> 4),
+                             act_lo + ((q * act_sub + k * UMMA_K * 2) >> 4), idesc, acc);
+              }
             }
           }
           umma_commit(&sc->empty[s]);                    // arrives once these MMAs have read the stage
@@ -561,19 +584,16 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
           tc_fence_after();
           {
             const uint32_t idesc_s = make_idesc_bf16(kc_pad);
-            const uint32_t a0 = smem_u32(As), b0 = smem_u32(KVs);
-            uint32_t acc = 0u;
-  #pragma unroll 1
-            for (int term = 0; term < 3; ++term) {
+            const uint32_t a_lo = smem_desc_lo(smem_u32(As)), b_lo = smem_desc_lo(smem_u32(KVs));
+  #pragma unroll
+            for (int term = 0; term < 3; ++term) {       // straight-line: a few instructions per MMA
               const int qp = term == 2 ? 1 : 0, kp = term == 1 ? 1 : 0;     // hi*hi, hi*lo, lo*hi
-  #pragma unroll 1
+  #pragma unroll
               for (int h = 0; h < H2; ++h) {
   #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                  umma_bf16(tmem_s, make_smem_desc(a0 + (qp * H2 + h) * SUB + k * 32),
-                            make_smem_desc(b0 + (kp * H2 + h) * KVSUB + k * 32), idesc_s, acc);
-                  acc = 1u;
-                }
+                for (int k = 0; k < 4; ++k)
+                  umma_bf16_lo(tmem_s, a_lo + (((qp * H2 + h) * SUB + k * 32) >> 4),
+                               b_lo + (((kp * H2 + h) * KVSUB + k * 32) >> 4), idesc_s, (term | h | k) ? 1u : 0u);
               }
             }
             umma_commit(&sc->bar_s);
@@ -586,16 +606,19 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
             ok = bar_wait(&sc->bar_p[rd], par_r, abort, status);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t a0 = smem_u32(As), b0 = smem_u32(KVs);
+            const uint32_t a_lo = smem_desc_lo(smem_u32(As));
+            const uint32_t b_lo = smem_desc_lo(smem_u32(KVs), KVSUB) + (uint32_t)((rd * (ROUND / 16) * 2048) >> 4);
             const int j_end = min(kc_pad - rd * ROUND, ROUND) / 16;
-  #pragma unroll 1
+  #pragma unroll
             for (int term = 0; term < 3; ++term) {
               const int pp = term == 2 ? 1 : 0, vp = term == 1 ? 1 : 0;
-  #pragma unroll 2
-              for (int j = 0; j < j_end; ++j) {
-                umma_bf16(tmem_o, make_smem_desc(a0 + (pp * 2 + (j >> 2)) * SUB + (j & 3) * 32),
-                          make_smem_desc(b0 + vp * H2 * KVSUB + (rd * (ROUND / 16) + j) * 2048, KVSUB), idesc2, acc);
-                acc = 1u;
+  #pragma unroll
+              for (int j = 0; j < ROUND / 16; ++j) {
+                if (j < j_end) {
+                  umma_bf16_lo(tmem_o, a_lo + (((pp * 2 + (j >> 2)) * SUB + (j & 3) * 32) >> 4),
+                               b_lo + ((vp * H2 * KVSUB + j * 2048) >> 4), idesc2, acc);
+                  acc = 1u;
+                }
               }
             }
             umma_commit(&sc->bar_o[rd]);
@@ -738,7 +761,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
     auto epi_partial = [&](const Gemm& g, size_t plane_stride) {
 #pragma unroll 1
       for (int u = g.u0; u < g.u1; ++seg) {
-        const int tile = u / g.KB;
+        const int grp = u / g.KB;
         const int kb0 = u % g.KB;
         const int kb1 = (g.u1 - u) < (g.KB - kb0) ? kb0 + (g.u1 - u) : g.KB;
         u += kb1 - kb0;
@@ -747,16 +770,19 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
         STACK_TRACE_POINT(10, cur_layer);
         tc_fence_after();
         if (!ok) continue;
-        const uint32_t lane_addr = tmem_base + lane_off + (uint32_t)(b * acc_cols);
         float* out = p.P + (size_t)(cta % g.splits) * plane_stride;
-        const int m = tile * TILE_M + row;
 #pragma unroll 1
-        for (int c0 = c_first; c0 < n_pad; c0 += 32) {
-          float v[16];
-          load16(lane_addr, c0, v);
+        for (int t = 0; t < TM; ++t) {
+          const uint32_t lane_addr = tmem_base + lane_off + (uint32_t)((b * TM + t) * acc_cols);
+          const int m = (grp * TM + t) * TILE_M + row;
+#pragma unroll 1
+          for (int c0 = c_first; c0 < n_pad; c0 += 32) {
+            float v[16];
+            load16(lane_addr, c0, v);
 #pragma unroll
-          for (int j = 0; j < 16; ++j)
-            if (c0 + j < p.n && m < g.M) out[(size_t)(c0 + j) * g.M + m] = v[j];
+            for (int j = 0; j < 16; ++j)
+              if (c0 + j < p.n && m < g.M) out[(size_t)(c0 + j) * g.M + m] = v[j];
+          }
         }
         tc_fence_before();
         mbar_arrive(&sc->acc_empty[b]);
@@ -766,23 +792,23 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
     auto epi_streamk = [&](const Gemm& g, bool swiglu, int epoch) {
 #pragma unroll 1
       for (int u = g.u0; u < g.u1; ++seg) {
-        const int tile = u / g.KB;
+        const int grp = u / g.KB;
         const int kb0 = u % g.KB;
         const int kb1 = (g.u1 - u) < (g.KB - kb0) ? kb0 + (g.u1 - u) : g.KB;
         u += kb1 - kb0;
         const int b = seg & 1;
-        // the CTA that holds the first k-blocks of a split tile adds what the CTAs holding the rest have parked
+        // the CTA that holds the first k-blocks of a split tile group adds what the CTAs holding the rest have parked
         int last = cta;
         if (kb0 == 0 && kb1 != g.KB)
-          while (last + 1 < g.g_eff && (long long)(last + 1) * g.U / g.g_eff < (long long)(tile + 1) * g.KB) ++last;
+          while (last + 1 < g.g_eff && (long long)(last + 1) * g.U / g.g_eff < (long long)(grp + 1) * g.KB) ++last;
         float pk0[16], pk1[16];
-        auto load_parked = [&](int c0, float* f) {
+        auto load_parked = [&](int t, int c0, float* f) {
 #pragma unroll
           for (int j = 0; j < 16; ++j) f[j] = 0.f;
           if (c0 < n_pad)
 #pragma unroll 1
             for (int cc = cta + 1; cc <= last; ++cc) {
-              const float* src = p.fixP + ((size_t)cc * n_pad + c0) * TILE_M + row;
+              const float* src = p.fixP + (((size_t)cc * TM + t) * n_pad + c0) * TILE_M + row;
 #pragma unroll
               for (int j = 0; j < 16; ++j) f[j] += __ldcg(src + j * TILE_M);
             }
@@ -797,26 +823,26 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
           }
           worker_bar();
           ok = ok && sc->step_ok != 0;
-          if (ok) {
-            load_parked(c_first, pk0);
-            load_parked(c_first + 32, pk1);
-          }
         }
         if (ok) ok = wwait_relaxed(&sc->acc_full[b], (uint32_t)((seg >> 1) & 1));
         STACK_TRACE_POINT(kb0 != 0 ? 12 : 11, cur_layer);
         tc_fence_after();
-        const uint32_t lane_addr = tmem_base + lane_off + (uint32_t)(b * acc_cols);
+        const uint32_t lane_base = tmem_base + lane_off + (uint32_t)(b * TM * acc_cols);
 
         if (kb0 != 0) {
-          // later k-blocks of a tile whose first k-blocks belong to an earlier CTA: park the partial sums
-          float* dst = p.fixP + (size_t)cta * n_pad * TILE_M;
+          // later k-blocks of a group whose first k-blocks belong to an earlier CTA: park the partial sums
+          float* dst = p.fixP + (size_t)cta * TM * n_pad * TILE_M;
           if (ok) {
 #pragma unroll 1
-            for (int c0 = c_first; c0 < n_pad; c0 += 32) {
-              float v[16];
-              load16(lane_addr, c0, v);
+            for (int t = 0; t < TM; ++t) {
+              if ((grp * TM + t) >= g.tiles) break;
+#pragma unroll 1
+              for (int c0 = c_first; c0 < n_pad; c0 += 32) {
+                float v[16];
+                load16(lane_base + (uint32_t)(t * acc_cols), c0, v);
 #pragma unroll
-              for (int j = 0; j < 16; ++j) dst[(size_t)(c0 + j) * TILE_M + row] = v[j];
+                for (int j = 0; j < 16; ++j) dst[((size_t)t * n_pad + c0 + j) * TILE_M + row] = v[j];
+              }
             }
             tc_fence_before();
             mbar_arrive(&sc->acc_empty[b]);
@@ -827,6 +853,15 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
           continue;
         }
 
+#pragma unroll 1
+        for (int t = 0; t < TM; ++t) {
+        const int tile = grp * TM + t;
+        if (tile >= g.tiles) break;
+        const uint32_t lane_addr = lane_base + (uint32_t)(t * acc_cols);
+        if (last > cta && ok) {
+          load_parked(t, c_first, pk0);
+          load_parked(t, c_first + 32, pk1);
+        }
         const int m = tile * TILE_M + row;
         const bool row_ok = m < g.M;
         if (!swiglu) {
@@ -938,10 +973,13 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
               }
             }
           }
+        }
+        worker_bar();
+        }
+        if (ok) {
           tc_fence_before();
           mbar_arrive(&sc->acc_empty[b]);
         }
-        worker_bar();
       }
     };
 
@@ -1342,8 +1380,9 @@ bool fused_stack_supported(const specasr_kv* wk, int n_total, bool att_tc, int s
   if (n_total < 1 || n_total > 64) return false;
   if (splits > kMaxAttnSplits) return false;
   // every weight tile of a linear projection needs a CTA of its own
-  const int tiles_qkv = (m->qkv_dim + TILE_M - 1) / TILE_M, tiles_d = (m->cfg.d_model + TILE_M - 1) / TILE_M;
-  if (tiles_qkv > m->n_sm || tiles_d > m->n_sm) return false;
+  const int groups_qkv = (m->qkv_dim + TM * TILE_M - 1) / (TM * TILE_M);
+  const int groups_d = (m->cfg.d_model + TM * TILE_M - 1) / (TM * TILE_M);
+  if (groups_qkv > m->n_sm || groups_d > m->n_sm) return false;
   return true;
 }
 
@@ -1375,9 +1414,18 @@ bool launch_fused_stack(specasr_model* m, specasr_kv* wk, const SegTable& tab, i
   p.stages = stages;
   p.ring_bytes = stages * p.stage_bytes;
   if (p.ring_bytes < attn_bytes) p.ring_bytes = (attn_bytes + 1023) & ~1023;
-  p.splits_qkv = gemm_tc_pick_splits(m, m->qkv_dim, c.d_model, n_pad);
-  p.splits_o = gemm_tc_pick_splits(m, c.d_model, m->q_dim, n_pad);
-  p.splits_down = gemm_tc_pick_splits(m, c.d_model, c.ffn, n_pad);
+  // k parts of the linear projections: tile groups * parts should just fill the SMs
+  auto pick_splits = [&](int M, int K) {
+    const int groups = (M + TM * TILE_M - 1) / (TM * TILE_M);
+    const int KB = (K + KSUB * SUB_K - 1) / (KSUB * SUB_K);
+    int sp = m->n_sm / groups;
+    if (sp > kMaxSplitK) sp = kMaxSplitK;
+    if (sp > KB) sp = KB;
+    return sp < 1 ? 1 : sp;
+  };
+  p.splits_qkv = pick_splits(m->qkv_dim, c.d_model);
+  p.splits_o = pick_splits(c.d_model, m->q_dim);
+  p.splits_down = pick_splits(c.d_model, c.ffn);
   p.epoch0 = wk->gemm_epoch;
   wk->gemm_epoch += c.n_layers + 1;
   p.want_head = want_head ? 1 : 0;

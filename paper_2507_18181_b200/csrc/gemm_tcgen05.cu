@@ -209,19 +209,17 @@ __global__ void __launch_bounds__(64 + EPI_THREADS, 1) k_proj(const __grid_const
           const uint32_t act_addr = w_addr + w_bytes;
           for (int t = 0; t < p.tm; ++t) {
             for (int q = 0; q < p.ksub; ++q) {
-              const uint32_t a_addr = w_addr + (t * p.ksub + q) * W_SUB_BYTES;
+              const uint32_t a_lo = smem_desc_lo(w_addr + (t * p.ksub + q) * W_SUB_BYTES);
               for (int jb = 0; jb < n_blocks; ++jb) {
                 const uint32_t b_addr = act_addr + q * act_sub + (uint32_t)(jb * 2 * p.box_rows * SUB_K * 2);
                 const uint32_t d_addr = d_base + (uint32_t)(t * tile_cols + jb * (FOLD ? 1 : 2) * p.box_rows);
-                const uint32_t lo_addr = b_addr + (uint32_t)(p.box_rows * SUB_K * 2);   // lo rows follow the hi rows
+                const uint32_t b_lo = smem_desc_lo(b_addr);
+                const uint32_t lo_lo = smem_desc_lo(b_addr + (uint32_t)(p.box_rows * SUB_K * 2));   // lo rows follow the hi rows
 #pragma unroll
                 for (int k = 0; k < SUB_K / UMMA_K; ++k) {
-                  const uint32_t acc = (kb > kb0 || q > 0 || k > 0) ? 1u : 0u;
-                  umma_bf16(d_addr, make_smem_desc(a_addr + k * UMMA_K * 2), make_smem_desc(b_addr + k * UMMA_K * 2),
-                            idesc, acc);
-                  if (FOLD)
-                    umma_bf16(d_addr, make_smem_desc(a_addr + k * UMMA_K * 2), make_smem_desc(lo_addr + k * UMMA_K * 2),
-                              idesc, 1u);
+                  const uint32_t acc = k > 0 ? 1u : ((kb > kb0 || q > 0) ? 1u : 0u);
+                  umma_bf16_lo(d_addr, a_lo + ((k * UMMA_K * 2) >> 4), b_lo + ((k * UMMA_K * 2) >> 4), idesc, acc);
+                  if (FOLD) umma_bf16_lo(d_addr, a_lo + ((k * UMMA_K * 2) >> 4), lo_lo + ((k * UMMA_K * 2) >> 4), idesc, 1u);
                 }
               }
             }
