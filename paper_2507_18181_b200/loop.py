@@ -43,24 +43,57 @@ class SpeculativeBatchLoop:
             self._verifiers[key] = BatchVerifier([kvs[b] for b in members])
         return self._verifiers[key]
 
-    def run_draft(self, feeds):
+    def run_draft(self, feeds, missing=None):
         """feeds: {b: tokens} -- tokens the draft model of utterance b consumes this round, one per autoregressive step.
         Step j runs every utterance that still has a token left as one batched call of single-node trees and
         appends that token's K/V to its draft cache.  (The proposer supplies the draft tokens, so the draft
-        model's own arg-max is not read back.)"""
+        model's own arg-max is not read back.)  missing: {b: committed tokens the draft cache has not seen yet}
+        (pending_alignment); they ride in front of the utterance's first token as one chain, all utterances in the
+        same batched call, instead of one call per utterance before the round."""
         if self.draft_kvs is None:
             return
+        missing = missing or {}
         steps = max((len(f) for f in feeds.values()), default=0)
+        if any(len(m) > 0 for m in missing.values()):
+            steps = max(steps, 1)
         for j in range(steps):
-            members = [b for b in sorted(feeds) if len(feeds[b]) > j]
+            if j == 0:
+                chains = {b: [int(t) for t in missing.get(b, [])] + [int(t) for t in feeds[b][:1]] for b in sorted(feeds)}
+                members = [b for b in sorted(feeds) if chains[b]]
+            else:
+                chains = {b: [int(feeds[b][j])] for b in sorted(feeds) if len(feeds[b]) > j}
+                members = sorted(chains)
+            if not members:
+                continue
             bv = self._verifier(self.draft_kvs, members)
-            toks = torch.tensor([int(feeds[b][j]) for b in members], dtype=torch.int32, device=self.device)
-            bv.verify(toks, self._minus_one[:len(members)], list(range(len(members) + 1)))
-            bv.commit()
-            for b in members:
-                self.draft_len[b] += 1
-                self.draft_dev_len[b] += 1
+            sizes = [len(chains[b]) for b in members]
+            if max(sizes) == 1:
+                toks = torch.tensor([chains[b][0] for b in members], dtype=torch.int32, device=self.device)
+                bv.verify(toks, self._minus_one[:len(members)], list(range(len(members) + 1)))
+                bv.commit()
+            else:
+                toks = torch.tensor([t for b in members for t in chains[b]], dtype=torch.int32, device=self.device)
+                par = torch.tensor([i - 1 for n in sizes for i in range(n)], dtype=torch.int32, device=self.device)
+                bv.verify(toks, par, [0] + list(np.cumsum(sizes)))
+                bv.commit_chains()
+            for b, n in zip(members, sizes):
+                self.draft_len[b] += n
+                self.draft_dev_len[b] += n
             self.draft_steps += 1
+
+    def pending_alignment(self, b, committed_tokens):
+        """As align_draft, but the committed tokens the draft cache has not seen are returned (for run_draft to put in
+        front of the utterance's first draft token) instead of being fed in a call of their own."""
+        if self.draft_kvs is None:
+            return []
+        want = self.target_len[b]
+        have = min(self.draft_len[b], want)
+        if self.draft_dev_len[b] != have:
+            self.draft_kvs[b].truncate(have)
+        self.draft_len[b] = self.draft_dev_len[b] = have
+        if have == want:
+            return []
+        return [int(t) for t in committed_tokens[len(committed_tokens) - 1 - (want - have):len(committed_tokens) - 1]]
 
     def align_draft(self, b, committed_tokens):
         """Brings utterance b's draft cache to the target's committed length (everything but the next root, which
@@ -116,14 +149,14 @@ class SpeculativeBatchLoop:
             active = [b for b in range(self.B) if len(emitted[b]) < n_tokens]
             if not active:
                 break
-            trees, feeds = {}, {}
+            trees, feeds, missing = {}, {}, {}
             for b in active:
                 tokens, parent, feed = proposer.propose(b, emitted[b])
                 assert int(tokens[0]) == history[b][-1]
                 trees[b] = (tokens, parent)
                 feeds[b] = feed
-                self.align_draft(b, history[b])
-            self.run_draft(feeds)
+                missing[b] = self.pending_alignment(b, history[b])
+            self.run_draft(feeds, missing)
             for b, (a, path, bonus) in self.verify_round(trees).items():
                 accepted = [int(trees[b][0][i]) for i in path[1:]]
                 emitted[b] += accepted + [bonus]

@@ -305,3 +305,15 @@ class BatchVerifier:
         for b, kv in enumerate(self.kvs):
             B.specasr_commit_kv(self.model.handle, kv.handle, self.out_path.data_ptr() + item * self.offsets[b],
                                 self.out_accept.data_ptr() + item * b, DeviceKV._stream())
+
+    def commit_chains(self):
+        """After a verify() whose trees were chains: keeps every node of every chain (the caller's own choice of
+        path, which specasr_commit_kv allows), whatever the model's arg-max said.  Used to feed known tokens."""
+        sizes = [self.offsets[b + 1] - self.offsets[b] for b in range(len(self.kvs))]
+        path = torch.tensor([i for n in sizes for i in range(n)], dtype=torch.int32, device=self.model.device)
+        accept = torch.tensor([n - 1 for n in sizes], dtype=torch.int32, device=self.model.device)
+        item = path.element_size()
+        for b, kv in enumerate(self.kvs):
+            B.specasr_commit_kv(self.model.handle, kv.handle, path.data_ptr() + item * self.offsets[b],
+                                accept.data_ptr() + item * b, DeviceKV._stream())
+        self._chain_commit = (path, accept)              # alive until the stream has run the copies
