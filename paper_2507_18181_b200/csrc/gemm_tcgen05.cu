@@ -148,7 +148,7 @@ __global__ void __launch_bounds__(64 + EPI_THREADS, 1) k_proj(const __grid_const
       const long long u = u0 + i;
       const int group = (int)(u / KB), kb = (int)(u % KB), s = i % p.stages;
       uint8_t* st = tiles + (size_t)s * stage_bytes;
-      for (int t = 0; t < p.tm; ++t)       // rows past M read as zeros
+      for (int t = 0; t < p.tm; ++t)       // rows past M are the zero padding of the packed matrix
         for (int q = 0; q < p.ksub; ++q)
           tma_load_2d(st + (t * p.ksub + q) * W_SUB_BYTES, &tmW, 0,
                       ((group * p.tm + t) * p.kt64 + kb * p.ksub + q) * TILE_M, &sc->full[s]);   // tile-packed weights
@@ -581,7 +581,7 @@ static void tc_shape(int n_pad, int* tm, int* ksub) {
   // but leaves only two 96 KB stages at 256 tokens, and the step is bound by the latency of a stage, not by
   // bandwidth (256 tokens, gate/up: 175 us with pairs, 144 us without).
   *tm = 1;
-  *ksub = n_pad <= 64 ? 2 : 1;                    // 256 contiguous bytes per weight row keep DRAM pages busy
+  *ksub = n_pad <= 64 ? 2 : 1;                    // two 16 KB tiles of the packed matrix per stage: 32 KB contiguous
 }
 
 // Number of k parts of the linear projections: tile groups * parts should just fill the SMs.
