@@ -42,3 +42,20 @@ def test_host_side_argument_errors_need_no_gpu():
     assert lib.specasr_commit_kv(None, None, None, None, None) == binding.SPECASR_ERR_INVALID_ARG
     n = ctypes.c_int32()
     assert lib.specasr_kv_length(None, ctypes.byref(n), None) == binding.SPECASR_ERR_INVALID_ARG
+
+
+def test_pack_weight_follows_the_offset_formula_of_the_header():
+    """The tile-packed weight layout (include/specasr.h): element (m, k) of a [M, K] matrix sits at
+    (((m / 128) * Kt + k / 64) * 128 + m % 128) * 64 + k % 64 with Kt = 2 * ceil(K / 128); padding reads as zero."""
+    import torch
+    from paper_2507_18181_b200.runtime import pack_weight
+    for M, K in ((128, 128), (200, 72), (384, 320), (96, 64)):
+        w = torch.arange(1, M * K + 1, dtype=torch.float32).reshape(M, K)
+        packed = pack_weight(w)
+        Kt = 2 * -(-K // 128)
+        assert packed.numel() == -(-M // 128) * Kt * 128 * 64
+        m = torch.arange(M)[:, None].expand(M, K)
+        k = torch.arange(K)[None, :].expand(M, K)
+        off = (((m // 128) * Kt + k // 64) * 128 + m % 128) * 64 + k % 64
+        assert torch.equal(packed[off.reshape(-1)], w.reshape(-1))
+        assert float(packed.sum()) == float(w.sum())          # everything else is padding
