@@ -284,7 +284,7 @@ __global__ void __launch_bounds__(64 + SOFTMAX_THREADS, 1) k_tree_attention_tc(c
         tmem_ld32(tmem_s + lane_off + c0, s);
         const uint32_t vis = visible32(c0);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) s[j] = ((vis >> j) & 1u) ? exp2f(s[j] * p.scale_log2 - m_use) : 0.f;
+        for (int j = 0; j < 32; ++j) s[j] = ((vis >> j) & 1u) ? fast_exp2(s[j] * p.scale_log2 - m_use) : 0.f;
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
           uint32_t hi[4], lo[4];

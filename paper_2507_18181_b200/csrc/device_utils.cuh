@@ -12,6 +12,15 @@ __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bflo
   lo = __float2bfloat16_rn(x - __bfloat162float(hi));
 }
 
+// 2^x by the special-function unit alone (relative error about 2^-22, denormal results flushed to zero).  exp2f()
+// wraps the same instruction in range handling that the soft-max does not need (its arguments are <= 0 and a result
+// below 2^-126 is as good as zero) and that made up a tenth of the attention step.
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 // Two values -> packed (hi0, hi1) and (lo0, lo1) words, element 0 in the low half; one packed
 // conversion per plane.
 __device__ __forceinline__ void split2_pack(float a, float b, uint32_t& hi, uint32_t& lo) {

@@ -1157,7 +1157,7 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
             tmem_ld16(tmem_s + lane_off + c0, s);
             const uint32_t vis = c0 < kc ? visible16(c0) : 0u;
 #pragma unroll
-            for (int j = 0; j < 16; ++j) s[j] = ((vis >> j) & 1u) ? exp2f(s[j] * p.scale_log2 - m_use) : 0.f;
+            for (int j = 0; j < 16; ++j) s[j] = ((vis >> j) & 1u) ? fast_exp2(s[j] * p.scale_log2 - m_use) : 0.f;
 #pragma unroll
             for (int gq = 0; gq < 2; ++gq) {
               uint32_t hi[4], lo[4];
