@@ -78,9 +78,9 @@ def algorithmic_flops(cfg, L, n):
 # profiles/k_stack_config3.md: the 2-layer and the 4-layer cut of config 3 (7B shape, 64 tokens, KV 1700).  Traffic
 # grows by a fixed amount per layer, so a full launch is the 2-layer figure plus (layers - 2) times the per-layer
 # difference.  Valid only for the kernel source it was taken on.
-STACK_TRAFFIC_MB = {"cut2": 1252.4, "cut4": 2225.7}
+STACK_TRAFFIC_MB = {"cut2": 1252.6, "cut4": 2228.0}
 STACK_TRAFFIC_SOURCE_SHA256 = {
-    "fused_stack.cu": "bf3d8def0e13740d9a950a56c5cbeb0bc6ddd283ee8b97a140ff7e0a0f4c91d1",
+    "fused_stack.cu": "077073dfca1a59de599181e079301eaf000d98cb0b6fb51e392c4d8b4cd71ab5",
     "sm100_ptx.cuh": "f811f56641d5fa39c0c575ce57fecebd5da4265ce577e5678d955814594e3f4d",
     "device_utils.cuh": "a35abef135a039a872df2c3961d941f9636495b6918adef1293a236f9905c175",
 }

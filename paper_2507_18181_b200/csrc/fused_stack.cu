@@ -1236,10 +1236,10 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
         const float2 none = make_float2(-INFINITY, 0.f);
         const float2 ml0 = lane < n_splits ? __ldcg(p.attML + (size_t)lane * rows_alloc + r) : none;
         const float2 ml1 = lane + 32 < n_splits ? __ldcg(p.attML + (size_t)(lane + 32) * rows_alloc + r) : none;
-        constexpr int B6 = 6;
-        float4 o[B6];
+        constexpr int MB = 10;                        // partial outputs in flight per round trip to L2 (config 3 has 9 key blocks)
+        float4 o[MB];
 #pragma unroll
-        for (int u = 0; u < B6; ++u)
+        for (int u = 0; u < MB; ++u)
           o[u] = (u < n_splits && c < DH) ? __ldcg(reinterpret_cast<const float4*>(p.attO + ((size_t)u * rows_alloc + r) * DH + c))
                                           : make_float4(0.f, 0.f, 0.f, 0.f);
         float mx = fmaxf(ml0.y > 0.f ? ml0.x : -INFINITY, ml1.y > 0.f ? ml1.x : -INFINITY);
@@ -1252,17 +1252,17 @@ k_stack(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtenso
         for (int s = 0; s < n_splits; ++s) den += __shfl_sync(0xFFFFFFFFu, s < 32 ? ml0.y * w0 : ml1.y * w1, s & 31);
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 1
-        for (int s0 = 0; s0 < n_splits; s0 += B6) {
+        for (int s0 = 0; s0 < n_splits; s0 += MB) {
           if (s0 > 0) {
 #pragma unroll
-            for (int u = 0; u < B6; ++u) {
+            for (int u = 0; u < MB; ++u) {
               const int s = s0 + u;
               o[u] = (s < n_splits && c < DH) ? __ldcg(reinterpret_cast<const float4*>(p.attO + ((size_t)s * rows_alloc + r) * DH + c))
                                               : make_float4(0.f, 0.f, 0.f, 0.f);
             }
           }
 #pragma unroll
-          for (int u = 0; u < B6; ++u) {
+          for (int u = 0; u < MB; ++u) {
             const int s = s0 + u;
             float w = __shfl_sync(0xFFFFFFFFu, s < 32 ? w0 : w1, s & 31);
             if (s >= n_splits || !(w > 0.f)) {
